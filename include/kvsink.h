@@ -1,0 +1,160 @@
+/*
+ * libkvsink -- KVSink quantized-KV-cache hot path for NVIDIA B200 (sm_100a).
+ *
+ * C ABI.  Every pointer documented "device" must point to CUDA device memory owned by the caller;
+ * "host" pointers are ordinary host memory.  The library allocates no device memory, keeps no global
+ * state, launches all work asynchronously on the caller's stream and never synchronises, except in
+ * kvsink_read_status.  Every entry point returns 0 (KVSINK_OK) or a negative KVSINK_ERR_* code; argument
+ * errors are detected on the host before anything is launched.  Nothing traps or spins on the device.
+ *
+ * Citations are to arXiv 2508.04257 ("KVSink"): Eq. 3 / Eq. 7 (attention, split into sink and non-sink
+ * sums), Eq. 6 (cache append), Eq. 8-11 (asymmetric n-bit quantization, Appendix C), Algorithm 1
+ * (prefill with KVSink: sink exclusion and top-k sink prediction), Section 4.3 (the prediction rule).
+ */
+#ifndef KVSINK_H_
+#define KVSINK_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define KVSINK_OK 0
+#define KVSINK_ERR_BAD_ARG (-1)      /* NULL / misaligned pointer, negative size, inconsistent strides */
+#define KVSINK_ERR_BAD_CONFIG (-2)   /* a kvsink_config field is out of range */
+#define KVSINK_ERR_UNSUPPORTED (-3)  /* a valid request this build has no kernel for */
+#define KVSINK_ERR_WORKSPACE (-4)    /* workspace missing or too small */
+#define KVSINK_ERR_SEQ_OVERFLOW (-5) /* seq_len + T > max_seq */
+#define KVSINK_ERR_SINK_OVERFLOW (-6)
+#define KVSINK_ERR_CUDA (-7)         /* a CUDA runtime call failed (launch, attribute, copy) */
+#define KVSINK_ERR_TIMEOUT (-8)
+
+/* Bits of the device status word (kvsink_cache.status, read with kvsink_read_status). */
+#define KVSINK_STATUS_SINK_MISMATCH 1 /* a token whose mask bit is set was not found in sink_pos */
+
+/* Tokens per packed tile. */
+#define KVSINK_TILE 16
+
+/*
+ * Problem description (Algorithm 1 "Parameters", plus the quantizer of Appendix C).
+ *   batch, n_q_heads, n_kv_heads, head_dim, hidden : B, Hq, Hkv, D, d.  Hq % Hkv == 0, D in {64,128}.
+ *   bits     : n of Eq. 8 (2, 3 or 4; 3 needs D == 128).
+ *   group    : G.  Keys are quantized per channel over groups of G consecutive tokens; values per token
+ *              over groups of min(G, D) consecutive channels.  G % 16 == 0, D % min(G,D) == 0.
+ *   max_seq  : capacity of the cache in tokens, a multiple of G.
+ *   topk     : k of Algorithm 1.  pfn_n: N of Preserve-First-N.  Sink capacity per sequence = topk + pfn_n.
+ *   channels : the pre-identified outlier channel(s) c of Section 4.3 (indices into hidden);
+ *              n_channels == 0 means "all d channels".
+ */
+typedef struct kvsink_config {
+    int32_t batch, n_q_heads, n_kv_heads, head_dim, hidden;
+    int32_t bits, group, max_seq, topk, pfn_n;
+    int32_t n_channels;
+    int32_t channels[8];
+} kvsink_config;
+
+/*
+ * One layer's cache.  All pointers are device pointers, 16-byte aligned, caller-allocated with the sizes
+ * kvsink_cache_sizes reports and zero-filled before first use.  u = b * Hkv + h is the (sequence, KV head) unit.
+ *   k_codes, v_codes : packed codes, [u][max_seq/16][tile_bytes]; one tile = 16 tokens x D channels.  A K tile
+ *                      is a stack of D/16 matrices [16 tokens x 16 channels], a V tile a stack of D/16 matrices
+ *                      [16 channels x 16 tokens]; element (row, col) of matrix m lives in lane
+ *                      4*(row%8) + (col%8)/2, pair slot s = 4*m + row/8 + 2*(col/8), half e = col%2 (the
+ *                      m16n8k16 A-operand ownership).  2 bit: lane word s/8, bits [16e+2k, +2) with k = s%8.
+ *                      4 bit: lane word s/4, bits [16e+4k, +4) with k = s%4.  3 bit: low two bits as 2 bit,
+ *                      high bit in a second section, word (s/8)/2, bit 16e + 4*(k/2) + 2*(1-(s/8)%2) + k%2.
+ *                      A section of n words per lane is stored as planes of up to four words per lane
+ *                      (plane p = words [4p, 4p+4)), lane l's words of a plane of width w at word w*l.
+ *   k_scale, k_zero  : float [u][max_seq/G][D]   -- scale, zero of Eq. 10-11 per channel per token group.
+ *   v_scale, v_zero  : float [u][max_seq][D/Gv]  -- per token per channel group, Gv = min(G, D).
+ *   k_tail           : fp16 [u][G][D]; row p % G holds the key of token p until its group is complete.
+ *   sink_k, sink_v   : fp16 [u][capacity][D]; slot j holds the exact rows of token sink_pos[b][j].
+ *   sink_bitmask     : uint32 [B][ceil(max_seq/32)]; bit p%32 of word p/32 is set iff token p is a sink.
+ *   sink_pos         : int32 [B][capacity] ascending, -1 beyond sink_count[b].  sink_count: int32 [B].
+ *                      The three sink arrays may be shared by the caches of all layers.
+ *   status           : int32 [1], OR of KVSINK_STATUS_* bits raised by kernels.
+ *   seq_len          : tokens in the cache (host field, the same for every sequence); advanced by
+ *                      kvsink_quantize_append.
+ * Fields of tokens that were never appended are unspecified.
+ */
+typedef struct kvsink_cache {
+    uint8_t *k_codes, *v_codes;
+    float *k_scale, *k_zero, *v_scale, *v_zero;
+    void *k_tail;
+    void *sink_k, *sink_v;
+    uint32_t *sink_bitmask;
+    int32_t *sink_pos, *sink_count;
+    int32_t *status;
+    int32_t seq_len;
+} kvsink_cache;
+
+typedef struct kvsink_sizes {
+    int64_t k_codes_bytes, v_codes_bytes;   /* each of k_codes, v_codes */
+    int64_t k_param_floats, v_param_floats; /* floats in each of scale and zero */
+    int64_t k_tail_halfs, sink_halfs;       /* fp16 elements; sink_halfs for each of sink_k, sink_v */
+    int64_t bitmask_words, sink_pos_ints;
+    int64_t predict_workspace_bytes;        /* for kvsink_predict_sinks with S == max_seq */
+    int64_t decode_workspace_bytes;         /* for kvsink_decode_attention */
+    int32_t sink_capacity, v_group, v_groups_per_row, tile_bytes;
+} kvsink_sizes;
+
+/*
+ * Buffer sizes for a configuration (host only, no CUDA call).  With scale/zero and the position index left
+ * out, k_codes_bytes + v_codes_bytes per layer and 2 * D * Hkv * 2 bytes per preserved token per layer are
+ * the "KV cache memory" columns of the paper's efficiency table (Appendix F).
+ */
+int kvsink_cache_sizes(const kvsink_config *cfg, kvsink_sizes *out);
+
+/*
+ * Sink-token prediction (Algorithm 1, the branch taken at the emergence layer; Section 4.3 items (1)-(4)).
+ * score[b][i] = max over the listed channels of |hidden[b][i][c]|; per sequence the k = topk tokens of
+ * largest score are selected, ties going to the lower index; the first pfn_n tokens are OR'd in.
+ *   hidden     device, fp16, element (b, i, c) at hidden + b*stride_b + i*stride_s + c (strides in elements).
+ *   S          tokens per sequence, 0 <= S <= max_seq.
+ *   bitmask    device out, uint32 [B][ceil(max_seq/32)], every word rewritten.
+ *   sink_pos   device out, int32 [B][topk+pfn_n], ascending, -1 padded.   sink_count  device out, int32 [B].
+ *   workspace  device scratch of at least kvsink_sizes.predict_workspace_bytes, 16-byte aligned.
+ */
+int kvsink_predict_sinks(const kvsink_config *cfg, const void *hidden, int32_t S, int64_t stride_b, int64_t stride_s,
+                         uint32_t *bitmask, int32_t *sink_pos, int32_t *sink_count, void *workspace,
+                         size_t workspace_bytes, void *cuda_stream);
+
+/*
+ * Append T tokens per sequence to the cache (Eq. 6) and quantize them (Eq. 8-11) with sink exclusion
+ * (Algorithm 1, the two "quantize" statements): tokens whose mask bit is set keep exact fp16 K and V rows in
+ * the side buffer and take no part in any group's min/max; every other value is coded as
+ * clamp(rint(x/scale) + zero, 0, 2^bits - 1) with scale = (max-min)/(2^bits-1), zero = -rint(min/scale) in
+ * IEEE binary32 (a constant group takes scale = |min|, or 1 when min is 0; a group of sink tokens only takes
+ * scale = zero = 0).  Values are coded on arrival; a key waits in k_tail until its G-token group is complete.
+ *   k_new, v_new  device, fp16, element (b, h, t, c) at base + b*stride_b + h*stride_h + t*stride_t + c;
+ *                 strides in elements, multiples of 8; both tensors share the strides.
+ *   T             T == 1 at any time; T > 1 only while seq_len is a multiple of G (for instance the prefill).
+ * On success cache->seq_len (host) is advanced by T.
+ */
+int kvsink_quantize_append(const kvsink_config *cfg, kvsink_cache *cache, const void *k_new, const void *v_new, int32_t T,
+                           int64_t stride_b, int64_t stride_h, int64_t stride_t, void *cuda_stream);
+
+/*
+ * Single-token decode attention over the whole cache (Eq. 3 with Eq. 7's split): for query head hq, KV head
+ * hq / (Hq/Hkv), scores q.k/sqrt(D) over all seq_len tokens under one softmax, where a token's K and V are
+ * the fp16 side-buffer rows if it is a sink, else the dequantised codes scale*(code - zero) (K from k_tail
+ * while its group is incomplete).  Accumulation is fp32.
+ *   q          device, fp16 [B][Hq][D] contiguous.      out  device, float [B][Hq][D].
+ *   lse        device, float [B][Hq] or NULL: natural log of the sum of exp of the scaled scores.
+ *   workspace  device scratch of at least kvsink_sizes.decode_workspace_bytes, 16-byte aligned.
+ */
+int kvsink_decode_attention(const kvsink_config *cfg, const kvsink_cache *cache, const void *q, float *out, float *lse,
+                            void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/* Copies the device status word to *host_status and waits for the stream (the only call that synchronises). */
+int kvsink_read_status(const kvsink_cache *cache, int32_t *host_status, void *cuda_stream);
+
+/* Static text for a status code. */
+const char *kvsink_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* KVSINK_H_ */

@@ -1,0 +1,559 @@
+/*
+ * KVSink reference oracle -- TEST INFRASTRUCTURE ONLY.
+ *
+ * A plain, slow, sequential CPU restatement of the KVSink hot path (sink-token prediction,
+ * asymmetric group quantization with sink exclusion, packed KV cache with an fp16 side buffer,
+ * single-token decode attention).  It exists so that the CUDA library can be checked against
+ * something obviously correct.  It shares no code with the CUDA path, is never linked into the
+ * product, and must only be called from tests, the smoke check and the CPU-baseline leg of the
+ * benchmark.
+ *
+ * Every function cites the passage of the paper (arXiv 2508.04257) it follows:
+ *   Eq. 3        softmax attention                         (Section 2)
+ *   Eq. 6        KV-cache append                           (Section 2)
+ *   Eq. 7        attention split into sink / non-sink sums (Section 4.2)
+ *   Eq. 8-11     asymmetric n-bit integer quantization     (Appendix C)
+ *   Algorithm 1  prefill with KVSink (sink exclusion, top-k sink prediction) (Appendix G)
+ *   Section 4.3  items (1)-(4): top-k on a pre-identified outlier channel, once, at prefill
+ *
+ * Pins (see tests/test_oracle_*.py): Table 4 memory columns (closed form), |x - x'| <= scale/2,
+ * exact rational re-derivation of codes, bit-exact round trip of sink / first-N rows, planted
+ * outliers, brute-force sort for top-k, textbook fp64 softmax attention on the dequantised
+ * tensors, Eq. 7 log-sum-exp merge identity, and the published m16n8k16 A-fragment ownership
+ * table for the physical code order.
+ *
+ * Parity unpinned: none of the arithmetic.  The physical order of codes inside a 16-token tile is a
+ * design choice the paper does not fix; it is pinned only against the published tensor-core
+ * fragment table and by pack/unpack identity.
+ *
+ * Floating point: quantization parameters and codes follow Eq. 8-11 in IEEE binary32 with
+ * round-to-nearest-even and no fused multiply-add (build with -ffp-contract=off); attention is
+ * evaluated in binary64.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+#define KVO_OK 0
+#define KVO_ERR_BAD_ARG (-1)
+#define KVO_ERR_BAD_CONFIG (-2)
+#define KVO_ERR_SEQ_OVERFLOW (-5)
+
+#define KVO_TILE 16
+
+typedef struct {
+    int32_t batch, n_q_heads, n_kv_heads, head_dim, hidden;
+    int32_t bits, group, max_seq, topk, pfn_n;
+    int32_t n_channels;
+    int32_t channels[8];
+} kvo_config;
+
+typedef struct {
+    uint8_t *k_codes, *v_codes;
+    float *k_scale, *k_zero, *v_scale, *v_zero;
+    uint16_t *k_tail;
+    uint16_t *sink_k, *sink_v;
+    uint32_t *sink_bitmask;
+    int32_t *sink_pos, *sink_count;
+    int32_t seq_len;
+} kvo_cache;
+
+typedef struct {
+    int64_t k_codes_bytes, v_codes_bytes;    /* per cache (one layer) */
+    int64_t k_param_floats, v_param_floats;  /* floats in EACH of scale and zero */
+    int64_t k_tail_halfs, sink_halfs;        /* fp16 elements; sink_halfs is for EACH of sink_k, sink_v */
+    int64_t bitmask_words, sink_pos_ints;
+    int32_t sink_capacity, v_group, v_groups_per_row, tile_bytes;
+} kvo_sizes;
+
+/* Threads the independent-unit loops run on (1 when built without OpenMP). */
+int kvo_num_threads(void)
+{
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
+void kvo_set_num_threads(int n)
+{
+#ifdef _OPENMP
+    if (n > 0) omp_set_num_threads(n);
+#else
+    (void)n;
+#endif
+}
+
+/* ---------- binary16 <-> binary32 (exact widening) ---------- */
+static float half_to_float(uint16_t h)
+{
+    uint32_t sign = (uint32_t)(h >> 15) << 31;
+    uint32_t ex = (h >> 10) & 0x1f;
+    uint32_t man = h & 0x3ff;
+    uint32_t bits;
+    if (ex == 0) {
+        if (man == 0) {
+            bits = sign;
+        } else { /* subnormal: man * 2^-24 */
+            float f = (float)man * 5.9604644775390625e-08f;
+            memcpy(&bits, &f, 4);
+            bits |= sign;
+        }
+    } else if (ex == 31) {
+        bits = sign | 0x7f800000u | (man << 13);
+    } else {
+        bits = sign | ((ex + 112) << 23) | (man << 13);
+    }
+    float out;
+    memcpy(&out, &bits, 4);
+    return out;
+}
+
+/* ---------- sizes: Table 4 memory columns are codes_bytes and sink row bytes ---------- */
+static int check_config(const kvo_config *c)
+{
+    if (!c) return KVO_ERR_BAD_ARG;
+    if (c->batch < 1 || c->n_kv_heads < 1 || c->n_q_heads < 1) return KVO_ERR_BAD_CONFIG;
+    if (c->n_q_heads % c->n_kv_heads) return KVO_ERR_BAD_CONFIG;
+    if (c->head_dim < 16 || c->head_dim % 16) return KVO_ERR_BAD_CONFIG;
+    if (c->bits < 2 || c->bits > 4) return KVO_ERR_BAD_CONFIG;
+    if (c->bits == 3 && c->head_dim % 64) return KVO_ERR_BAD_CONFIG;
+    if (c->group < 16 || c->group % 16) return KVO_ERR_BAD_CONFIG;
+    if (c->max_seq < c->group || c->max_seq % c->group) return KVO_ERR_BAD_CONFIG;
+    if (c->topk < 0 || c->pfn_n < 0) return KVO_ERR_BAD_CONFIG;
+    if (c->n_channels < 0 || c->n_channels > 8) return KVO_ERR_BAD_CONFIG;
+    int gv = c->group < c->head_dim ? c->group : c->head_dim;
+    if (c->head_dim % gv) return KVO_ERR_BAD_CONFIG;
+    return KVO_OK;
+}
+
+static int v_group_of(const kvo_config *c) { return c->group < c->head_dim ? c->group : c->head_dim; }
+static int sink_cap_of(const kvo_config *c) { return c->topk + c->pfn_n; }
+
+int kvo_cache_sizes(const kvo_config *c, kvo_sizes *s)
+{
+    int rc = check_config(c);
+    if (rc) return rc;
+    if (!s) return KVO_ERR_BAD_ARG;
+    int64_t units = (int64_t)c->batch * c->n_kv_heads;
+    int gv = v_group_of(c);
+    s->v_group = gv;
+    s->v_groups_per_row = c->head_dim / gv;
+    s->tile_bytes = KVO_TILE * c->head_dim * c->bits / 8;
+    s->k_codes_bytes = units * c->max_seq * c->head_dim * c->bits / 8;
+    s->v_codes_bytes = s->k_codes_bytes;
+    s->k_param_floats = units * (c->max_seq / c->group) * c->head_dim;
+    s->v_param_floats = units * c->max_seq * s->v_groups_per_row;
+    s->k_tail_halfs = units * c->group * c->head_dim;
+    s->sink_capacity = sink_cap_of(c);
+    s->sink_halfs = units * s->sink_capacity * c->head_dim;
+    s->bitmask_words = (int64_t)c->batch * ((c->max_seq + 31) / 32);
+    s->sink_pos_ints = (int64_t)c->batch * s->sink_capacity;
+    return KVO_OK;
+}
+
+/* ---------- physical order of codes inside a 16-token tile ----------
+ * A tile of K is a stack of head_dim/16 matrices [16 tokens x 16 channels]; a tile of V is a stack
+ * of head_dim/16 matrices [16 channels x 16 tokens].  Matrix element (row, col) of matrix m belongs
+ * to "lane" 4*(row%8) + (col%8)/2, pair slot r = row/8 + 2*(col/8), half e = col%2 -- the
+ * ownership table of the 16x16 A operand of the m16n8k16 tensor-core instruction.  Lane words are
+ * little-endian 32-bit; slot s = 4*m + r.
+ *   2 bit: word s/8, field k = s%8 at bit 16e + 2k.
+ *   4 bit: word s/4, field k = s%4 at bit 16e + 4k.
+ *   3 bit: the low two bits as in 2 bit ("lo" section); the high bit in a "hi" section with one
+ *          word per two lo words: hi word (s/8)/2, bit 16e + 4*(k/2) + 2*(1 - (s/8)%2) + k%2.
+ * A section of n words per lane is stored as planes of up to four words per lane: plane p holds
+ * words [4p, min(4p+4, n)); a plane of width u puts lane l's words at word offset u*l.
+ */
+static int section_word_offset(int n_words, int lane, int i)
+{
+    int off = 0, p = i / 4;
+    for (int pp = 0; pp < p; ++pp) {
+        int u = n_words - 4 * pp;
+        if (u > 4) u = 4;
+        off += 32 * u;
+    }
+    int u = n_words - 4 * p;
+    if (u > 4) u = 4;
+    return off + u * lane + (i - 4 * p);
+}
+
+/* Writes / reads the b-bit code of matrix element (m,row,col) in a tile of `tile_words`. */
+static void tile_put(uint32_t *tile, int D, int bits, int m, int row, int col, uint32_t code)
+{
+    int lane = 4 * (row % 8) + (col % 8) / 2;
+    int r = row / 8 + 2 * (col / 8);
+    int e = col % 2;
+    int s = 4 * m + r;
+    if (bits == 2) {
+        int n = D / 32, i = s / 8, k = s % 8;
+        uint32_t *w = &tile[section_word_offset(n, lane, i)];
+        int sh = 16 * e + 2 * k;
+        *w = (*w & ~(3u << sh)) | ((code & 3u) << sh);
+    } else if (bits == 4) {
+        int n = D / 16, i = s / 4, k = s % 4;
+        uint32_t *w = &tile[section_word_offset(n, lane, i)];
+        int sh = 16 * e + 4 * k;
+        *w = (*w & ~(15u << sh)) | ((code & 15u) << sh);
+    } else {
+        int nlo = D / 32, nhi = D / 64, i = s / 8, k = s % 8;
+        uint32_t *w = &tile[section_word_offset(nlo, lane, i)];
+        int sh = 16 * e + 2 * k;
+        *w = (*w & ~(3u << sh)) | ((code & 3u) << sh);
+        uint32_t *h = &tile[32 * nlo + section_word_offset(nhi, lane, i / 2)];
+        int hb = 16 * e + 4 * (k / 2) + 2 * (1 - (i % 2)) + (k % 2);
+        *h = (*h & ~(1u << hb)) | (((code >> 2) & 1u) << hb);
+    }
+}
+
+static uint32_t tile_get(const uint32_t *tile, int D, int bits, int m, int row, int col)
+{
+    int lane = 4 * (row % 8) + (col % 8) / 2;
+    int r = row / 8 + 2 * (col / 8);
+    int e = col % 2;
+    int s = 4 * m + r;
+    if (bits == 2) {
+        int n = D / 32, i = s / 8, k = s % 8;
+        return (tile[section_word_offset(n, lane, i)] >> (16 * e + 2 * k)) & 3u;
+    } else if (bits == 4) {
+        int n = D / 16, i = s / 4, k = s % 4;
+        return (tile[section_word_offset(n, lane, i)] >> (16 * e + 4 * k)) & 15u;
+    } else {
+        int nlo = D / 32, nhi = D / 64, i = s / 8, k = s % 8;
+        uint32_t lo = (tile[section_word_offset(nlo, lane, i)] >> (16 * e + 2 * k)) & 3u;
+        int hb = 16 * e + 4 * (k / 2) + 2 * (1 - (i % 2)) + (k % 2);
+        uint32_t hi = (tile[32 * nlo + section_word_offset(nhi, lane, i / 2)] >> hb) & 1u;
+        return lo | (hi << 2);
+    }
+}
+
+static uint32_t *tile_ptr(uint8_t *codes, const kvo_config *c, int b, int h, int token)
+{
+    int64_t row_bytes = (int64_t)c->head_dim * c->bits / 8;
+    int64_t unit = ((int64_t)b * c->n_kv_heads + h) * c->max_seq * row_bytes;
+    return (uint32_t *)(codes + unit + (int64_t)(token / KVO_TILE) * KVO_TILE * row_bytes);
+}
+
+static void k_code_put(uint8_t *codes, const kvo_config *c, int b, int h, int token, int ch, uint32_t code)
+{
+    tile_put(tile_ptr(codes, c, b, h, token), c->head_dim, c->bits, ch / 16, token % 16, ch % 16, code);
+}
+static uint32_t k_code_get(const uint8_t *codes, const kvo_config *c, int b, int h, int token, int ch)
+{
+    return tile_get(tile_ptr((uint8_t *)codes, c, b, h, token), c->head_dim, c->bits, ch / 16, token % 16, ch % 16);
+}
+static void v_code_put(uint8_t *codes, const kvo_config *c, int b, int h, int token, int ch, uint32_t code)
+{
+    tile_put(tile_ptr(codes, c, b, h, token), c->head_dim, c->bits, ch / 16, ch % 16, token % 16, code);
+}
+static uint32_t v_code_get(const uint8_t *codes, const kvo_config *c, int b, int h, int token, int ch)
+{
+    return tile_get(tile_ptr((uint8_t *)codes, c, b, h, token), c->head_dim, c->bits, ch / 16, ch % 16, token % 16);
+}
+
+/* Logical codes of every token < seq (int8, [B,Hkv,seq,D]); kind 0 = K, 1 = V. */
+int kvo_unpack_codes(const kvo_config *c, const uint8_t *codes, int kind, int seq, int8_t *out)
+{
+    int rc = check_config(c);
+    if (rc) return rc;
+    for (int b = 0; b < c->batch; ++b)
+        for (int h = 0; h < c->n_kv_heads; ++h)
+            for (int t = 0; t < seq; ++t)
+                for (int ch = 0; ch < c->head_dim; ++ch) {
+                    uint32_t v = kind ? v_code_get(codes, c, b, h, t, ch) : k_code_get(codes, c, b, h, t, ch);
+                    out[(((int64_t)b * c->n_kv_heads + h) * seq + t) * c->head_dim + ch] = (int8_t)v;
+                }
+    return KVO_OK;
+}
+
+/* ---------- sink mask ---------- */
+static int mask_bit(const uint32_t *bitmask, const kvo_config *c, int b, int pos)
+{
+    int words = (c->max_seq + 31) / 32;
+    return (bitmask[(int64_t)b * words + pos / 32] >> (pos % 32)) & 1u;
+}
+
+typedef struct { float score; int32_t idx; } scored;
+static int by_score_desc_then_index(const void *pa, const void *pb)
+{
+    const scored *a = (const scored *)pa, *b = (const scored *)pb;
+    if (a->score > b->score) return -1;
+    if (a->score < b->score) return 1;
+    return (a->idx > b->idx) - (a->idx < b->idx);
+}
+
+/*
+ * Algorithm 1, the two statements under "if l = l_E", and Section 4.3 items (1)-(4):
+ * S_sink = token indices of Top-k |H[i,c]|.  With several listed channels the score of a token is
+ * the largest |H[i,c]| over them; with none listed it is the largest over all d channels.
+ * Ties go to the lower token index.  The first pfn_n tokens are OR'd in (Preserve-First-N).
+ * Outputs: bitmask (bit i%32 of word i/32, row of ceil(max_seq/32) words per sequence, rewritten
+ * in full), ascending positions, and their count.
+ */
+int kvo_predict_sinks(const kvo_config *c, const uint16_t *hidden, int32_t S, int64_t stride_b, int64_t stride_s,
+                      uint32_t *bitmask, int32_t *sink_pos, int32_t *sink_count)
+{
+    int rc = check_config(c);
+    if (rc) return rc;
+    if (!hidden || !bitmask || !sink_pos || !sink_count || S < 0 || S > c->max_seq) return KVO_ERR_BAD_ARG;
+    for (int i = 0; i < c->n_channels; ++i)
+        if (c->channels[i] < 0 || c->channels[i] >= c->hidden) return KVO_ERR_BAD_CONFIG;
+    int words = (c->max_seq + 31) / 32;
+    int cap = sink_cap_of(c);
+    scored *sc = (scored *)malloc(sizeof(scored) * (size_t)(S > 0 ? S : 1));
+    for (int b = 0; b < c->batch; ++b) {
+        uint32_t *bm = bitmask + (int64_t)b * words;
+        memset(bm, 0, sizeof(uint32_t) * (size_t)words);
+        for (int i = 0; i < S; ++i) {
+            const uint16_t *row = hidden + b * stride_b + i * stride_s;
+            float best = 0.0f;
+            if (c->n_channels == 0) {
+                for (int ch = 0; ch < c->hidden; ++ch) {
+                    float a = fabsf(half_to_float(row[ch]));
+                    if (a > best) best = a;
+                }
+            } else {
+                for (int j = 0; j < c->n_channels; ++j) {
+                    float a = fabsf(half_to_float(row[c->channels[j]]));
+                    if (a > best) best = a;
+                }
+            }
+            sc[i].score = best;
+            sc[i].idx = i;
+        }
+        qsort(sc, (size_t)S, sizeof(scored), by_score_desc_then_index);
+        int k = c->topk < S ? c->topk : S;
+        for (int j = 0; j < k; ++j) bm[sc[j].idx / 32] |= 1u << (sc[j].idx % 32);
+        int n = c->pfn_n < S ? c->pfn_n : S;
+        for (int i = 0; i < n; ++i) bm[i / 32] |= 1u << (i % 32);
+        int cnt = 0;
+        for (int i = 0; i < S; ++i)
+            if ((bm[i / 32] >> (i % 32)) & 1u) sink_pos[(int64_t)b * cap + cnt++] = i;
+        for (int j = cnt; j < cap; ++j) sink_pos[(int64_t)b * cap + j] = -1;
+        sink_count[b] = cnt;
+    }
+    free(sc);
+    return KVO_OK;
+}
+
+/* ---------- Eq. 8-11 on one group ----------
+ * x: the group's values; member[j] != 0 marks the values that take part (non-sink tokens).
+ * scale = (max - min) / (2^n - 1)                     Eq. 10 (no clipping: plain min / max)
+ * zero  = -round(min / scale)                         Eq. 11
+ * Q     = clamp(round(x / scale) + zero, 0, 2^n - 1)  Eq. 8
+ * round = to nearest, ties to even.  A group whose members are all equal takes scale = |min|
+ * (1 if min is 0) so that it reproduces itself; a group without members takes scale = zero = 0.
+ * Non-members get code 0.
+ */
+void kvo_quantize_group(const float *x, const uint8_t *member, int n, int bits, float *scale_out, float *zero_out,
+                        int32_t *codes)
+{
+    const float qmax = (float)((1 << bits) - 1);
+    int any = 0;
+    float mn = 0.0f, mx = 0.0f;
+    for (int j = 0; j < n; ++j) {
+        if (!member[j]) continue;
+        if (!any) { mn = mx = x[j]; any = 1; }
+        else { if (x[j] < mn) mn = x[j]; if (x[j] > mx) mx = x[j]; }
+    }
+    if (!any) {
+        *scale_out = 0.0f;
+        *zero_out = 0.0f;
+        for (int j = 0; j < n; ++j) codes[j] = 0;
+        return;
+    }
+    float r = mx - mn;
+    float scale;
+    if (r == 0.0f) scale = (mn == 0.0f) ? 1.0f : fabsf(mn);
+    else scale = r / qmax;
+    float zero = 0.0f - rintf(mn / scale);
+    for (int j = 0; j < n; ++j) {
+        if (!member[j]) { codes[j] = 0; continue; }
+        float q = rintf(x[j] / scale) + zero;
+        q = fminf(fmaxf(q, 0.0f), qmax);
+        codes[j] = (int32_t)q;
+    }
+    *scale_out = scale;
+    *zero_out = zero;
+}
+
+/* Eq. 9: X' = scale * (Q - zero), in binary32. */
+static float dequant(float scale, float zero, uint32_t code) { return scale * ((float)code - zero); }
+
+/* ---------- append (Eq. 6) with sink exclusion (Algorithm 1, the two "quantize" statements) ----------
+ * Tokens are appended one by one at positions seq_len, seq_len+1, ...  For the token at position p of
+ * sequence b (all KV heads alike):
+ *   - if bit p of the sink mask is set, its K and V rows are copied bit for bit into the side buffer at
+ *     slot = rank of p in sink_pos[b]; its packed V codes and V parameters are 0;
+ *   - otherwise V is quantized per token, one group per v_group channels (Eq. 8-11), and stored;
+ *   - its K row goes to k_tail[p % group]; when p completes a group of `group` tokens, that group is
+ *     quantized per channel over its non-sink tokens (Eq. 8-11) and stored; sink tokens get code 0.
+ * new tokens: fp16 [B, Hkv, T, D] with element strides stride_b, stride_h, stride_t (D contiguous).
+ */
+int kvo_quantize_append(const kvo_config *c, kvo_cache *cache, const uint16_t *k_new, const uint16_t *v_new, int32_t T,
+                        int64_t stride_b, int64_t stride_h, int64_t stride_t)
+{
+    int rc = check_config(c);
+    if (rc) return rc;
+    if (!cache || !k_new || !v_new || T < 0) return KVO_ERR_BAD_ARG;
+    if (cache->seq_len < 0 || (int64_t)cache->seq_len + T > c->max_seq) return KVO_ERR_SEQ_OVERFLOW;
+    const int D = c->head_dim, G = c->group, gv = v_group_of(c), ngv = D / gv, cap = sink_cap_of(c);
+    const int Hk = c->n_kv_heads;
+    const int buf = G > D ? G : D;
+    int bad = 0;
+    /* (sequence, KV head) units are independent; the loop over them may run on several threads */
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int64_t unit = 0; unit < (int64_t)c->batch * Hk; ++unit) {
+        const int b = (int)(unit / Hk), h = (int)(unit % Hk);
+        float *xs = (float *)malloc(sizeof(float) * (size_t)buf);
+        uint8_t *mem = (uint8_t *)malloc((size_t)buf);
+        int32_t *codes = (int32_t *)malloc(sizeof(int32_t) * (size_t)buf);
+        uint16_t *tail = cache->k_tail + unit * G * D;
+        for (int i = 0; i < T; ++i) {
+            int p = cache->seq_len + i;
+            const uint16_t *krow = k_new + b * stride_b + h * stride_h + i * stride_t;
+            const uint16_t *vrow = v_new + b * stride_b + h * stride_h + i * stride_t;
+            int sink = mask_bit(cache->sink_bitmask, c, b, p);
+            if (sink) {
+                int slot = -1;
+                for (int j = 0; j < cache->sink_count[b]; ++j)
+                    if (cache->sink_pos[(int64_t)b * cap + j] == p) slot = j;
+                if (slot < 0) {
+#pragma omp atomic write
+                    bad = 1;
+                    continue;
+                }
+                memcpy(cache->sink_k + (unit * cap + slot) * D, krow, sizeof(uint16_t) * (size_t)D);
+                memcpy(cache->sink_v + (unit * cap + slot) * D, vrow, sizeof(uint16_t) * (size_t)D);
+            }
+            /* V: per token */
+            for (int j = 0; j < ngv; ++j) {
+                float sc = 0.0f, ze = 0.0f;
+                for (int e = 0; e < gv; ++e) { xs[e] = half_to_float(vrow[j * gv + e]); mem[e] = (uint8_t)!sink; }
+                kvo_quantize_group(xs, mem, gv, c->bits, &sc, &ze, codes);
+                cache->v_scale[(unit * c->max_seq + p) * ngv + j] = sc;
+                cache->v_zero[(unit * c->max_seq + p) * ngv + j] = ze;
+                for (int e = 0; e < gv; ++e) v_code_put(cache->v_codes, c, b, h, p, j * gv + e, (uint32_t)codes[e]);
+            }
+            /* K: tail, then per channel when the group is complete */
+            memcpy(tail + (int64_t)(p % G) * D, krow, sizeof(uint16_t) * (size_t)D);
+            if ((p + 1) % G == 0) {
+                int g = p / G;
+                for (int ch = 0; ch < D; ++ch) {
+                    float sc = 0.0f, ze = 0.0f;
+                    for (int t = 0; t < G; ++t) {
+                        xs[t] = half_to_float(tail[(int64_t)t * D + ch]);
+                        mem[t] = (uint8_t)!mask_bit(cache->sink_bitmask, c, b, g * G + t);
+                    }
+                    kvo_quantize_group(xs, mem, G, c->bits, &sc, &ze, codes);
+                    cache->k_scale[(unit * (c->max_seq / G) + g) * D + ch] = sc;
+                    cache->k_zero[(unit * (c->max_seq / G) + g) * D + ch] = ze;
+                    for (int t = 0; t < G; ++t) k_code_put(cache->k_codes, c, b, h, g * G + t, ch, (uint32_t)codes[t]);
+                }
+            }
+        }
+        free(xs); free(mem); free(codes);
+    }
+    if (bad) return KVO_ERR_BAD_ARG;
+    cache->seq_len += T;
+    return KVO_OK;
+}
+
+/* ---------- the K and V row that attention sees for token p (Eq. 7: sink rows exact, the rest dequantised) ---------- */
+static int sink_slot(const kvo_config *c, const kvo_cache *cache, int b, int p)
+{
+    int cap = sink_cap_of(c);
+    for (int j = 0; j < cache->sink_count[b]; ++j)
+        if (cache->sink_pos[(int64_t)b * cap + j] == p) return j;
+    return -1;
+}
+
+static void kv_row(const kvo_config *c, const kvo_cache *cache, int b, int h, int p, double *krow, double *vrow)
+{
+    const int D = c->head_dim, G = c->group, gv = v_group_of(c), ngv = D / gv, cap = sink_cap_of(c);
+    int64_t unit = (int64_t)b * c->n_kv_heads + h;
+    int n_body = (cache->seq_len / G) * G;
+    if (mask_bit(cache->sink_bitmask, c, b, p)) {
+        int slot = sink_slot(c, cache, b, p);
+        for (int ch = 0; ch < D; ++ch) {
+            krow[ch] = slot < 0 ? NAN : (double)half_to_float(cache->sink_k[(unit * cap + slot) * D + ch]);
+            vrow[ch] = slot < 0 ? NAN : (double)half_to_float(cache->sink_v[(unit * cap + slot) * D + ch]);
+        }
+        return;
+    }
+    for (int ch = 0; ch < D; ++ch) {
+        if (p >= n_body) {
+            krow[ch] = (double)half_to_float(cache->k_tail[(unit * G + p % G) * D + ch]);
+        } else {
+            int64_t pi = (unit * (c->max_seq / G) + p / G) * D + ch;
+            krow[ch] = (double)dequant(cache->k_scale[pi], cache->k_zero[pi], k_code_get(cache->k_codes, c, b, h, p, ch));
+        }
+        int64_t vi = (unit * c->max_seq + p) * ngv + ch / gv;
+        vrow[ch] = (double)dequant(cache->v_scale[vi], cache->v_zero[vi], v_code_get(cache->v_codes, c, b, h, p, ch));
+    }
+}
+
+/* Dense K', V' (binary64, [B,Hkv,seq_len,D]) exactly as attention consumes them. */
+int kvo_dequant_dense(const kvo_config *c, const kvo_cache *cache, double *kd, double *vd)
+{
+    int rc = check_config(c);
+    if (rc) return rc;
+    const int D = c->head_dim, n = cache->seq_len;
+    for (int b = 0; b < c->batch; ++b)
+        for (int h = 0; h < c->n_kv_heads; ++h)
+            for (int p = 0; p < n; ++p) {
+                int64_t o = ((((int64_t)b * c->n_kv_heads + h) * n) + p) * D;
+                kv_row(c, cache, b, h, p, kd + o, vd + o);
+            }
+    return KVO_OK;
+}
+
+/*
+ * Eq. 3 for one query token per head, over every cached token, with Eq. 7's split: the token's K and V
+ * are the fp16 side-buffer rows if it is a sink, else the dequantised codes (K from the fp16 tail while
+ * its group is incomplete).  Query head hq reads KV head hq / (Hq/Hkv).  Scores are scaled by 1/sqrt(D),
+ * there is no mask (a decode query sees the whole cache).  binary64 throughout.
+ * out [B,Hq,D], lse [B,Hq] (natural-log sum of exp of the scaled scores) may be NULL.
+ */
+int kvo_decode_attention(const kvo_config *c, const kvo_cache *cache, const uint16_t *q, double *out, double *lse)
+{
+    int rc = check_config(c);
+    if (rc) return rc;
+    if (!cache || !q || !out) return KVO_ERR_BAD_ARG;
+    const int D = c->head_dim, n = cache->seq_len, rep = c->n_q_heads / c->n_kv_heads;
+    /* (sequence, query head) pairs are independent; the loop over them may run on several threads */
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int64_t bh = 0; bh < (int64_t)c->batch * c->n_q_heads; ++bh) {
+        const int b = (int)(bh / c->n_q_heads), hq = (int)(bh % c->n_q_heads);
+        double *krow = (double *)malloc(sizeof(double) * (size_t)D);
+        double *vrow = (double *)malloc(sizeof(double) * (size_t)D);
+        double *s = (double *)malloc(sizeof(double) * (size_t)(n > 0 ? n : 1));
+        int h = hq / rep;
+        const uint16_t *qv = q + ((int64_t)b * c->n_q_heads + hq) * D;
+        double *o = out + ((int64_t)b * c->n_q_heads + hq) * D;
+        double mx = -INFINITY;
+        for (int p = 0; p < n; ++p) {
+            kv_row(c, cache, b, h, p, krow, vrow);
+            double acc = 0.0;
+            for (int ch = 0; ch < D; ++ch) acc += (double)half_to_float(qv[ch]) * krow[ch];
+            s[p] = acc / sqrt((double)D);
+            if (s[p] > mx) mx = s[p];
+        }
+        double den = 0.0;
+        for (int ch = 0; ch < D; ++ch) o[ch] = 0.0;
+        for (int p = 0; p < n; ++p) {
+            double w = exp(s[p] - mx);
+            den += w;
+            kv_row(c, cache, b, h, p, krow, vrow);
+            for (int ch = 0; ch < D; ++ch) o[ch] += w * vrow[ch];
+        }
+        for (int ch = 0; ch < D; ++ch) o[ch] = n > 0 ? o[ch] / den : 0.0;
+        if (lse) lse[(int64_t)b * c->n_q_heads + hq] = n > 0 ? mx + log(den) : -INFINITY;
+        free(krow); free(vrow); free(s);
+    }
+    return KVO_OK;
+}
