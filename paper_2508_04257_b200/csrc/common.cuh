@@ -1,0 +1,103 @@
+// Shared definitions for the libkvsink kernels (device + host).
+#pragma once
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/kvsink.h"
+
+namespace kvsink {
+
+// Derived, validated problem parameters passed to kernels by value.
+struct Params {
+    int B, Hq, Hkv, D, hidden;
+    int bits, G, max_seq, topk, pfn_n, cap;
+    int Gv, NGv;        // value channel-group size and groups per row
+    int rep;            // query heads per KV head
+    int tile_bytes;     // bytes of one packed 16-token tile
+    int row_bytes;      // D * bits / 8
+    int mask_words;     // bitmask words per sequence
+    int n_channels;
+    int channels[8];
+};
+
+// ---- physical order of codes inside a 16-token tile (see kvsink.h, kvsink_cache) ----
+// Word i of lane `lane` inside a section of n words per lane stored as planes of up to four words per lane.
+__host__ __device__ inline int section_word_offset(int n, int lane, int i)
+{
+    int off = 0, p = i >> 2;
+    for (int pp = 0; pp < p; ++pp) {
+        int u = n - 4 * pp;
+        off += 32 * (u > 4 ? 4 : u);
+    }
+    int u = n - 4 * p;
+    if (u > 4) u = 4;
+    return off + u * lane + (i - 4 * p);
+}
+
+// Inverse: physical word offset inside a section -> (lane, i).
+__host__ __device__ inline void section_word_owner(int n, int off, int *lane, int *i)
+{
+    int p = 0;
+    for (;;) {
+        int u = n - 4 * p;
+        if (u > 4) u = 4;
+        if (off < 32 * u) {
+            *lane = off / u;
+            *i = 4 * p + off % u;
+            return;
+        }
+        off -= 32 * u;
+        ++p;
+    }
+}
+
+__device__ __forceinline__ uint32_t smem_addr(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ float warp_sum(float v)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+// Eq. 10-11 for one group from its exact fp16 extremes; all operations IEEE binary32, round to nearest even.
+// any == false (no member) gives scale = zero = 0.
+__device__ __forceinline__ void group_params(bool any, float mn, float mx, float qmax, float *scale, float *zero)
+{
+    if (!any) {
+        *scale = 0.0f;
+        *zero = 0.0f;
+        return;
+    }
+    float r = __fsub_rn(mx, mn);
+    float s;
+    if (r == 0.0f) s = (mn == 0.0f) ? 1.0f : fabsf(mn);
+    else s = __fdiv_rn(r, qmax);
+    *scale = s;
+    *zero = __fsub_rn(0.0f, rintf(__fdiv_rn(mn, s)));
+}
+
+// Eq. 8 for one value (exact form: IEEE division, rint, clamp).
+__device__ __forceinline__ uint32_t code_exact(float x, float scale, float zero, float qmax)
+{
+    float q = __fadd_rn(rintf(__fdiv_rn(x, scale)), zero);
+    q = fminf(fmaxf(q, 0.0f), qmax);
+    return (uint32_t)(int)q;
+}
+
+__device__ __forceinline__ bool mask_bit(const uint32_t *__restrict__ bm, int pos) { return (bm[pos >> 5] >> (pos & 31)) & 1u; }
+
+// Launchers implemented in the kernel translation units; all return a KVSINK_* code.
+int launch_predict_sinks(const Params &p, const __half *hidden, int S, int64_t stride_b, int64_t stride_s, uint32_t *bitmask,
+                         int32_t *sink_pos, int32_t *sink_count, void *workspace, cudaStream_t st);
+int launch_quantize_groups(const Params &p, const kvsink_cache &c, const __half *k_src, const __half *v_src, int first_token,
+                           int n_groups, int64_t sb, int64_t sh, int64_t stt, bool do_v_and_sinks, cudaStream_t st);
+int launch_quantize_tokens(const Params &p, const kvsink_cache &c, const __half *k_src, const __half *v_src, int src_offset,
+                           int first_token, int n_tokens, int64_t sb, int64_t sh, int64_t stt, cudaStream_t st);
+int launch_decode(const Params &p, const kvsink_cache &c, const __half *q, float *out, float *lse, void *workspace,
+                  size_t workspace_bytes, cudaStream_t st);
+size_t decode_workspace_bytes(const Params &p);
+size_t predict_workspace_bytes(const Params &p);
+
+}  // namespace kvsink

@@ -1,0 +1,171 @@
+// Sink-token prediction: per-token outlier score, exact per-sequence top-k with index tie-break,
+// Preserve-First-N, bitmask + ascending position list (Algorithm 1 at the emergence layer; Section 4.3).
+#include "common.cuh"
+
+namespace kvsink {
+
+struct ChannelList {
+    int n;
+    int c[8];
+};
+
+// score = max over listed channels of |H| as the 15-bit magnitude pattern of the fp16 value (order-preserving).
+__global__ void sink_score_listed(const uint16_t *__restrict__ H, int S, int64_t sb, int64_t ss, ChannelList cl,
+                                  uint16_t *__restrict__ score, int score_stride)
+{
+    int i = blockIdx.x * blockDim.x + threadIdx.x;
+    int b = blockIdx.y;
+    if (i >= S) return;
+    const uint16_t *row = H + b * sb + i * ss;
+    unsigned best = 0;
+#pragma unroll 1
+    for (int j = 0; j < cl.n; ++j) {
+        unsigned a = __ldg(row + cl.c[j]) & 0x7fffu;
+        best = a > best ? a : best;
+    }
+    score[(size_t)b * score_stride + i] = (uint16_t)best;
+}
+
+// All d channels: one warp per token.
+__global__ void sink_score_all(const uint16_t *__restrict__ H, int S, int d, int64_t sb, int64_t ss,
+                               uint16_t *__restrict__ score, int score_stride)
+{
+    int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+    int b = blockIdx.y;
+    if (warp >= S) return;
+    const uint16_t *row = H + b * sb + warp * ss;
+    unsigned best = 0;
+    for (int c = lane; c < d; c += 32) {
+        unsigned a = __ldg(row + c) & 0x7fffu;
+        best = a > best ? a : best;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        unsigned x = __shfl_xor_sync(0xffffffffu, best, o);
+        best = x > best ? x : best;
+    }
+    if (lane == 0) score[(size_t)b * score_stride + warp] = (uint16_t)best;
+}
+
+constexpr int SEL_THREADS = 1024;
+
+// Exclusive prefix count of `flag` over the block in thread order; *total = number of set flags.
+__device__ __forceinline__ int block_excl_count(bool flag, int *total, unsigned *warp_tot)
+{
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    unsigned bal = __ballot_sync(0xffffffffu, flag);
+    int within = __popc(bal & ((1u << lane) - 1u));
+    if (lane == 0) warp_tot[w] = __popc(bal);
+    __syncthreads();
+    unsigned v = warp_tot[lane];
+    unsigned incl = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        unsigned x = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += x;
+    }
+    int before = (int)__shfl_sync(0xffffffffu, incl - v, w);
+    *total = (int)__shfl_sync(0xffffffffu, incl, 31);
+    __syncthreads();
+    return before + within;
+}
+
+// One block per sequence: 2-pass radix select of the k-th largest 16-bit score, then an ordered pass that
+// breaks ties by index, ORs the first N tokens in and emits mask words and ascending positions.
+__global__ void __launch_bounds__(SEL_THREADS)
+sink_select(const uint16_t *__restrict__ score, int score_stride, int S, int k, int N, int mask_words, int cap,
+            uint32_t *__restrict__ bitmask, int32_t *__restrict__ sink_pos, int32_t *__restrict__ sink_count)
+{
+    __shared__ unsigned hist[256];
+    __shared__ unsigned warp_tot[32];
+    __shared__ int s_hi, s_need, s_vstar, s_r;
+    const int b = blockIdx.x, tid = threadIdx.x;
+    const uint16_t *sc = score + (size_t)b * score_stride;
+    const int kk = k < S ? k : S;
+    int vstar = 0x10000, r = 0;   // no score exceeds 0x10000: no top-k selection when kk == 0
+    if (kk > 0) {
+        if (tid < 256) hist[tid] = 0;
+        __syncthreads();
+        for (int i = tid; i < S; i += SEL_THREADS) atomicAdd(&hist[sc[i] >> 8], 1u);
+        __syncthreads();
+        if (tid == 0) {
+            int cum = 0, bin = 255;
+            for (; bin > 0; --bin) {
+                if (cum + (int)hist[bin] >= kk) break;
+                cum += (int)hist[bin];
+            }
+            s_hi = bin;
+            s_need = kk - cum;
+        }
+        __syncthreads();
+        const int hi = s_hi;
+        if (tid < 256) hist[tid] = 0;
+        __syncthreads();
+        for (int i = tid; i < S; i += SEL_THREADS) {
+            unsigned v = sc[i];
+            if ((int)(v >> 8) == hi) atomicAdd(&hist[v & 0xffu], 1u);
+        }
+        __syncthreads();
+        if (tid == 0) {
+            int cum = 0, bin = 255, need = s_need;
+            for (; bin > 0; --bin) {
+                if (cum + (int)hist[bin] >= need) break;
+                cum += (int)hist[bin];
+            }
+            s_vstar = (hi << 8) | bin;
+            s_r = need - cum;
+        }
+        __syncthreads();
+        vstar = s_vstar;
+        r = s_r;
+    }
+    int run_eq = 0, run_sel = 0;
+    const int S_round = (S + SEL_THREADS - 1) / SEL_THREADS * SEL_THREADS;
+    for (int base = 0; base < S_round; base += SEL_THREADS) {
+        const int i = base + tid;
+        const int key = i < S ? (int)sc[i] : -1;
+        const bool gt = key > vstar, eq = key == vstar;
+        int tot_eq;
+        const int eq_rank = run_eq + block_excl_count(eq, &tot_eq, warp_tot);
+        const bool sel = i < S && (i < N || gt || (eq && eq_rank < r));
+        const unsigned word = __ballot_sync(0xffffffffu, sel);
+        if ((tid & 31) == 0 && (i >> 5) < mask_words) bitmask[(size_t)b * mask_words + (i >> 5)] = word;
+        int tot_sel;
+        const int rank = run_sel + block_excl_count(sel, &tot_sel, warp_tot);
+        if (sel && rank < cap) sink_pos[(size_t)b * cap + rank] = i;
+        run_eq += tot_eq;
+        run_sel += tot_sel;
+    }
+    for (int w = S_round / 32 + tid; w < mask_words; w += SEL_THREADS) bitmask[(size_t)b * mask_words + w] = 0u;
+    for (int j = run_sel + tid; j < cap; j += SEL_THREADS) sink_pos[(size_t)b * cap + j] = -1;
+    if (tid == 0) sink_count[b] = run_sel < cap ? run_sel : cap;
+}
+
+size_t predict_workspace_bytes(const Params &p)
+{
+    size_t stride = ((size_t)p.max_seq + 7) / 8 * 8;
+    return (size_t)p.B * stride * sizeof(uint16_t) + 16;
+}
+
+int launch_predict_sinks(const Params &p, const __half *hidden, int S, int64_t sb, int64_t ss, uint32_t *bitmask, int32_t *sink_pos,
+                         int32_t *sink_count, void *workspace, cudaStream_t st)
+{
+    uint16_t *score = (uint16_t *)workspace;
+    const int stride = (p.max_seq + 7) / 8 * 8;
+    if (S > 0) {
+        if (p.n_channels > 0) {
+            ChannelList cl;
+            cl.n = p.n_channels;
+            for (int i = 0; i < 8; ++i) cl.c[i] = p.channels[i];
+            dim3 grid((S + 255) / 256, p.B);
+            sink_score_listed<<<grid, 256, 0, st>>>((const uint16_t *)hidden, S, sb, ss, cl, score, stride);
+        } else {
+            dim3 grid((S + 7) / 8, p.B);
+            sink_score_all<<<grid, 256, 0, st>>>((const uint16_t *)hidden, S, p.hidden, sb, ss, score, stride);
+        }
+    }
+    sink_select<<<p.B, SEL_THREADS, 0, st>>>(score, stride, S, p.topk, p.pfn_n, p.mask_words, p.cap, bitmask, sink_pos, sink_count);
+    return cudaGetLastError() == cudaSuccess ? KVSINK_OK : KVSINK_ERR_CUDA;
+}
+
+}  // namespace kvsink

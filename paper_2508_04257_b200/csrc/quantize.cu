@@ -1,0 +1,316 @@
+// Asymmetric group quantization (Eq. 8-11) with sink exclusion (Algorithm 1), bit-packing into the tile
+// layout, side-buffer compaction of sink rows, and the append path (Eq. 6).
+#include "common.cuh"
+
+namespace kvsink {
+
+// Slot of position `pos` in the ascending list sink_pos[0..count), or -1.
+__device__ __forceinline__ int find_slot(const int32_t *__restrict__ sink_pos, int count, int pos)
+{
+    int lo = 0, hi = count - 1;
+    while (lo <= hi) {
+        int mid = (lo + hi) >> 1;
+        int v = sink_pos[mid];
+        if (v == pos) return mid;
+        if (v < pos) lo = mid + 1;
+        else hi = mid - 1;
+    }
+    return -1;
+}
+
+// Matrix element (m, row, col) held in pair slot s, half e of `lane`.
+__device__ __forceinline__ void slot_to_elem(int lane, int s, int e, int *m, int *row, int *col)
+{
+    const int g = lane >> 2, t = lane & 3, r = s & 3;
+    *m = s >> 2;
+    *row = g + 8 * (r & 1);
+    *col = 2 * t + e + 8 * (r >> 1);
+}
+
+// Assemble one physical word of a tile; get(m,row,col) supplies the code of a matrix element and `word`
+// indexes the tile's 32-bit words in memory order.
+template <typename Get>
+__device__ __forceinline__ uint32_t assemble_word(int bits, int D, int word, Get get)
+{
+    uint32_t out = 0;
+    int lane, i, m, row, col;
+    if (bits == 2 || bits == 4) {
+        const int n = D * bits / 64, fields = 16 / bits;   // fields per half word: 8 or 4
+        section_word_owner(n, word, &lane, &i);
+        for (int k = 0; k < fields; ++k)
+            for (int e = 0; e < 2; ++e) {
+                slot_to_elem(lane, fields * i + k, e, &m, &row, &col);
+                out |= (get(m, row, col) & ((1u << bits) - 1u)) << (16 * e + bits * k);
+            }
+    } else {
+        const int nlo = D / 32, nhi = D / 64;
+        if (word < 32 * nlo) {
+            section_word_owner(nlo, word, &lane, &i);
+            for (int k = 0; k < 8; ++k)
+                for (int e = 0; e < 2; ++e) {
+                    slot_to_elem(lane, 8 * i + k, e, &m, &row, &col);
+                    out |= (get(m, row, col) & 3u) << (16 * e + 2 * k);
+                }
+        } else {
+            int j;
+            section_word_owner(nhi, word - 32 * nlo, &lane, &j);
+            for (int w = 0; w < 2; ++w)
+                for (int k = 0; k < 8; ++k)
+                    for (int e = 0; e < 2; ++e) {
+                        slot_to_elem(lane, 8 * (2 * j + w) + k, e, &m, &row, &col);
+                        out |= ((get(m, row, col) >> 2) & 1u) << (16 * e + 4 * (k >> 1) + 2 * (1 - w) + (k & 1));
+                    }
+        }
+    }
+    return out;
+}
+
+// ---------------------------------------------------------------------------------------------------------
+// Whole groups: one block per (token group, KV head, sequence).  Keys per channel over the group's non-sink
+// tokens, values per token, sink rows to the side buffer.
+// ---------------------------------------------------------------------------------------------------------
+constexpr int QG_THREADS = 256;
+
+__global__ void __launch_bounds__(QG_THREADS)
+quantize_groups_kernel(Params p, kvsink_cache c, const __half *__restrict__ k_src, const __half *__restrict__ v_src,
+                       int first_token, int64_t sb, int64_t sh, int64_t stt, int do_v_and_sinks)
+{
+    extern __shared__ __align__(16) unsigned char smem[];
+    const int D = p.D, G = p.G, RS = D + 8;      // padded row stride in halves
+    __half *Kt = (__half *)smem;                  // [G][RS]
+    __half *Vt = Kt + (size_t)G * RS;             // [G][RS]
+    uint8_t *kcode = (uint8_t *)(Vt + (size_t)G * RS);   // [G][D]
+    uint8_t *vcode = kcode + (size_t)G * D;               // [G][D]
+    float *ks = (float *)(vcode + (size_t)G * D);         // [D] scale
+    float *kz = ks + D;                                   // [D] zero
+    float *vs = kz + D;                                   // [G][NGv]
+    float *vz = vs + G * p.NGv;
+    uint8_t *flag = (uint8_t *)(vz + G * p.NGv);          // [G] sink flags
+
+    const int tid = threadIdx.x;
+    const int grp = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
+    const int64_t unit = (int64_t)b * p.Hkv + h;
+    const int p0 = first_token + grp * G;         // absolute position of the group's first token
+    const int gidx = p0 / G;
+    const float qmax = (float)((1 << p.bits) - 1);
+    const uint32_t *bm = c.sink_bitmask + (size_t)b * p.mask_words;
+
+    // load the tiles (16-byte chunks)
+    const int chunks = D / 8;
+    const __half *kbase = k_src + b * sb + h * sh + (int64_t)(grp * G) * stt;
+    const __half *vbase = v_src + b * sb + h * sh + (int64_t)(grp * G) * stt;
+    for (int idx = tid; idx < G * chunks; idx += QG_THREADS) {
+        int t = idx / chunks, ch = (idx % chunks) * 8;
+        *(uint4 *)(Kt + (size_t)t * RS + ch) = __ldg((const uint4 *)(kbase + (int64_t)t * stt + ch));
+        if (do_v_and_sinks) *(uint4 *)(Vt + (size_t)t * RS + ch) = __ldg((const uint4 *)(vbase + (int64_t)t * stt + ch));
+    }
+    for (int t = tid; t < G; t += QG_THREADS) flag[t] = mask_bit(bm, p0 + t) ? 1 : 0;
+    __syncthreads();
+
+    // key parameters: one thread per channel
+    for (int ch = tid; ch < D; ch += QG_THREADS) {
+        bool any = false;
+        float mn = 0.f, mx = 0.f;
+        for (int t = 0; t < G; ++t) {
+            if (flag[t]) continue;
+            float x = __half2float(Kt[(size_t)t * RS + ch]);
+            if (!any) { mn = mx = x; any = true; }
+            else { mn = fminf(mn, x); mx = fmaxf(mx, x); }
+        }
+        float s, z;
+        group_params(any, mn, mx, qmax, &s, &z);
+        ks[ch] = s;
+        kz[ch] = z;
+        size_t o = ((size_t)unit * (p.max_seq / G) + gidx) * D + ch;
+        c.k_scale[o] = s;
+        c.k_zero[o] = z;
+    }
+    // value parameters: one thread per (token, channel group)
+    if (do_v_and_sinks) {
+        for (int it = tid; it < G * p.NGv; it += QG_THREADS) {
+            int t = it / p.NGv, j = it % p.NGv;
+            float s = 0.f, z = 0.f;
+            if (!flag[t]) {
+                const __half *row = Vt + (size_t)t * RS + j * p.Gv;
+                float mn = __half2float(row[0]), mx = mn;
+                for (int e = 1; e < p.Gv; ++e) {
+                    float x = __half2float(row[e]);
+                    mn = fminf(mn, x);
+                    mx = fmaxf(mx, x);
+                }
+                group_params(true, mn, mx, qmax, &s, &z);
+            }
+            vs[it] = s;
+            vz[it] = z;
+            size_t o = ((size_t)unit * p.max_seq + p0 + t) * p.NGv + j;
+            c.v_scale[o] = s;
+            c.v_zero[o] = z;
+        }
+    }
+    __syncthreads();
+
+    // codes
+    for (int idx = tid; idx < G * D; idx += QG_THREADS) {
+        int t = idx / D, ch = idx % D;
+        uint32_t kc = 0, vc = 0;
+        if (!flag[t]) {
+            kc = code_exact(__half2float(Kt[(size_t)t * RS + ch]), ks[ch], kz[ch], qmax);
+            if (do_v_and_sinks) {
+                int j = ch / p.Gv;
+                vc = code_exact(__half2float(Vt[(size_t)t * RS + ch]), vs[t * p.NGv + j], vz[t * p.NGv + j], qmax);
+            }
+        }
+        kcode[idx] = (uint8_t)kc;
+        vcode[idx] = (uint8_t)vc;
+    }
+    __syncthreads();
+
+    // pack: the group's tiles are contiguous in memory; one thread per 32-bit word
+    const int tile_words = p.tile_bytes / 4, n_tiles = G / KVSINK_TILE;
+    uint32_t *kout = (uint32_t *)(c.k_codes + (size_t)unit * p.max_seq * p.row_bytes + (size_t)(p0 / KVSINK_TILE) * p.tile_bytes);
+    uint32_t *vout = (uint32_t *)(c.v_codes + (size_t)unit * p.max_seq * p.row_bytes + (size_t)(p0 / KVSINK_TILE) * p.tile_bytes);
+    for (int idx = tid; idx < n_tiles * tile_words; idx += QG_THREADS) {
+        int tile = idx / tile_words, word = idx % tile_words;
+        const uint8_t *kc = kcode + (size_t)tile * KVSINK_TILE * D;
+        kout[idx] = assemble_word(p.bits, D, word, [&](int m, int row, int col) { return (uint32_t)kc[row * D + 16 * m + col]; });
+        if (do_v_and_sinks) {
+            const uint8_t *vc = vcode + (size_t)tile * KVSINK_TILE * D;
+            vout[idx] = assemble_word(p.bits, D, word, [&](int m, int row, int col) { return (uint32_t)vc[col * D + 16 * m + row]; });
+        }
+    }
+
+    // sink rows: exact fp16 copies into the side buffer at the rank of their position
+    if (do_v_and_sinks) {
+        const int count = min(c.sink_count[b], p.cap);
+        for (int t = 0; t < G; ++t) {
+            if (!flag[t]) continue;
+            int slot = find_slot(c.sink_pos + (size_t)b * p.cap, count, p0 + t);
+            if (slot < 0) {
+                if (tid == 0) atomicOr(c.status, KVSINK_STATUS_SINK_MISMATCH);
+                continue;
+            }
+            __half *dk = (__half *)c.sink_k + ((size_t)unit * p.cap + slot) * D;
+            __half *dv = (__half *)c.sink_v + ((size_t)unit * p.cap + slot) * D;
+            for (int ch = tid; ch < chunks; ch += QG_THREADS) {
+                *(uint4 *)(dk + ch * 8) = *(const uint4 *)(Kt + (size_t)t * RS + ch * 8);
+                *(uint4 *)(dv + ch * 8) = *(const uint4 *)(Vt + (size_t)t * RS + ch * 8);
+            }
+        }
+    }
+}
+
+static size_t groups_smem_bytes(const Params &p)
+{
+    size_t RS = p.D + 8;
+    return 2 * (size_t)p.G * RS * 2 + 2 * (size_t)p.G * p.D + 2 * (size_t)p.D * 4 + 2 * (size_t)p.G * p.NGv * 4 + p.G + 16;
+}
+
+int launch_quantize_groups(const Params &p, const kvsink_cache &c, const __half *k_src, const __half *v_src, int first_token,
+                           int n_groups, int64_t sb, int64_t sh, int64_t stt, bool do_v_and_sinks, cudaStream_t st)
+{
+    if (n_groups <= 0) return KVSINK_OK;
+    size_t smem = groups_smem_bytes(p);
+    if (smem > 227 * 1024) return KVSINK_ERR_UNSUPPORTED;
+    if (cudaFuncSetAttribute(quantize_groups_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+        return KVSINK_ERR_CUDA;
+    dim3 grid(n_groups, p.Hkv, p.B);
+    quantize_groups_kernel<<<grid, QG_THREADS, smem, st>>>(p, c, k_src, v_src, first_token, sb, sh, stt, do_v_and_sinks ? 1 : 0);
+    return cudaGetLastError() == cudaSuccess ? KVSINK_OK : KVSINK_ERR_CUDA;
+}
+
+// ---------------------------------------------------------------------------------------------------------
+// Single tokens (decode-time append, and the remainder of a prefill that does not fill a group): values are
+// quantized per token and inserted into their tile, keys go to the fp16 tail, sink rows to the side buffer.
+// One block per (tile touched, KV head, sequence).
+// ---------------------------------------------------------------------------------------------------------
+constexpr int QT_THREADS = 128;
+
+__global__ void __launch_bounds__(QT_THREADS)
+quantize_tokens_kernel(Params p, kvsink_cache c, const __half *__restrict__ k_src, const __half *__restrict__ v_src, int src_offset,
+                       int first_token, int n_tokens, int64_t sb, int64_t sh, int64_t stt)
+{
+    __shared__ uint8_t vcode[KVSINK_TILE * 128];
+    __shared__ uint8_t present[KVSINK_TILE];
+    const int D = p.D, G = p.G;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int h = blockIdx.y, b = blockIdx.z;
+    const int64_t unit = (int64_t)b * p.Hkv + h;
+    const int tile = first_token / KVSINK_TILE + blockIdx.x;
+    const int t_lo = max(first_token, tile * KVSINK_TILE), t_hi = min(first_token + n_tokens, (tile + 1) * KVSINK_TILE);
+    const float qmax = (float)((1 << p.bits) - 1);
+    const uint32_t *bm = c.sink_bitmask + (size_t)b * p.mask_words;
+    if (tid < KVSINK_TILE) present[tid] = (tile * KVSINK_TILE + tid >= t_lo && tile * KVSINK_TILE + tid < t_hi) ? 1 : 0;
+
+    const int cpl = D / 32;   // channels per lane (2 or 4)
+    for (int pos = t_lo + warp; pos < t_hi; pos += QT_THREADS / 32) {
+        const int64_t src = b * sb + h * sh + (int64_t)(src_offset + pos - first_token) * stt;
+        const bool sink = mask_bit(bm, pos);
+        float x[4];
+        __half kx[4], vx[4];
+        for (int e = 0; e < cpl; ++e) {
+            vx[e] = v_src[src + lane * cpl + e];
+            x[e] = __half2float(vx[e]);
+            kx[e] = k_src[src + lane * cpl + e];
+        }
+        // key row -> tail
+        __half *tail = (__half *)c.k_tail + ((size_t)unit * G + pos % G) * D;
+        for (int e = 0; e < cpl; ++e) tail[lane * cpl + e] = kx[e];
+        if (sink) {
+            const int count = min(c.sink_count[b], p.cap);
+            int slot = find_slot(c.sink_pos + (size_t)b * p.cap, count, pos);
+            if (slot < 0) {
+                if (lane == 0) atomicOr(c.status, KVSINK_STATUS_SINK_MISMATCH);
+            } else {
+                __half *dk = (__half *)c.sink_k + ((size_t)unit * p.cap + slot) * D;
+                __half *dv = (__half *)c.sink_v + ((size_t)unit * p.cap + slot) * D;
+                for (int e = 0; e < cpl; ++e) {
+                    dk[lane * cpl + e] = kx[e];
+                    dv[lane * cpl + e] = vx[e];
+                }
+            }
+        }
+        // value row: min / max over the lanes of each channel group
+        float mn = x[0], mx = x[0];
+        for (int e = 1; e < cpl; ++e) { mn = fminf(mn, x[e]); mx = fmaxf(mx, x[e]); }
+        const int lanes_per_group = p.Gv / cpl;
+        for (int o = 1; o < lanes_per_group; o <<= 1) {
+            mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, o));
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+        }
+        float s, z;
+        group_params(!sink, mn, mx, qmax, &s, &z);
+        const int j = lane / lanes_per_group;
+        if (lane % lanes_per_group == 0) {
+            size_t o = ((size_t)unit * p.max_seq + pos) * p.NGv + j;
+            c.v_scale[o] = s;
+            c.v_zero[o] = z;
+        }
+        for (int e = 0; e < cpl; ++e)
+            vcode[(pos % KVSINK_TILE) * D + lane * cpl + e] = sink ? 0 : (uint8_t)code_exact(x[e], s, z, qmax);
+    }
+    __syncthreads();
+
+    // insert the new tokens' fields into the tile; fields of other tokens keep their bits
+    const int tile_words = p.tile_bytes / 4;
+    uint32_t *vout = (uint32_t *)(c.v_codes + (size_t)unit * p.max_seq * p.row_bytes + (size_t)tile * p.tile_bytes);
+    const bool fresh = (t_lo % KVSINK_TILE) == 0;   // no earlier token lives in this tile
+    for (int word = tid; word < tile_words; word += QT_THREADS) {
+        uint32_t keep = fresh ? 0u : vout[word];
+        uint32_t newbits = assemble_word(p.bits, D, word, [&](int m, int row, int col) {
+            return present[col] ? (uint32_t)vcode[col * D + 16 * m + row] : 0u; });
+        uint32_t fieldmask = assemble_word(p.bits, D, word, [&](int m, int row, int col) { return present[col] ? 0xffu : 0u; });
+        vout[word] = (keep & ~fieldmask) | newbits;
+    }
+}
+
+int launch_quantize_tokens(const Params &p, const kvsink_cache &c, const __half *k_src, const __half *v_src, int src_offset,
+                           int first_token, int n_tokens, int64_t sb, int64_t sh, int64_t stt, cudaStream_t st)
+{
+    if (n_tokens <= 0) return KVSINK_OK;
+    int tiles = (first_token + n_tokens - 1) / KVSINK_TILE - first_token / KVSINK_TILE + 1;
+    dim3 grid(tiles, p.Hkv, p.B);
+    quantize_tokens_kernel<<<grid, QT_THREADS, 0, st>>>(p, c, k_src, v_src, src_offset, first_token, n_tokens, sb, sh, stt);
+    return cudaGetLastError() == cudaSuccess ? KVSINK_OK : KVSINK_ERR_CUDA;
+}
+
+}  // namespace kvsink
