@@ -1,0 +1,162 @@
+// C-ABI entry points of libkvsink: argument validation on the host, then kernel launches on the caller's stream.
+#include "common.cuh"
+
+using namespace kvsink;
+
+static int derive(const kvsink_config *cfg, Params *p)
+{
+    if (!cfg) return KVSINK_ERR_BAD_ARG;
+    if (cfg->batch < 1 || cfg->n_kv_heads < 1 || cfg->n_q_heads < 1 || cfg->hidden < 1) return KVSINK_ERR_BAD_CONFIG;
+    if (cfg->n_q_heads % cfg->n_kv_heads) return KVSINK_ERR_BAD_CONFIG;
+    if (cfg->bits < 2 || cfg->bits > 4) return KVSINK_ERR_BAD_CONFIG;
+    if (cfg->group < 16 || cfg->group % 16) return KVSINK_ERR_BAD_CONFIG;
+    if (cfg->max_seq < cfg->group || cfg->max_seq % cfg->group) return KVSINK_ERR_BAD_CONFIG;
+    if (cfg->topk < 0 || cfg->pfn_n < 0) return KVSINK_ERR_BAD_CONFIG;
+    if (cfg->n_channels < 0 || cfg->n_channels > 8) return KVSINK_ERR_BAD_CONFIG;
+    for (int i = 0; i < cfg->n_channels; ++i)
+        if (cfg->channels[i] < 0 || cfg->channels[i] >= cfg->hidden) return KVSINK_ERR_BAD_CONFIG;
+    if (cfg->head_dim < 16 || cfg->head_dim % 16) return KVSINK_ERR_BAD_CONFIG;
+    if (cfg->head_dim != 64 && cfg->head_dim != 128) return KVSINK_ERR_UNSUPPORTED;
+    if (cfg->bits == 3 && cfg->head_dim != 128) return KVSINK_ERR_UNSUPPORTED;
+    const int gv = cfg->group < cfg->head_dim ? cfg->group : cfg->head_dim;
+    if (cfg->head_dim % gv) return KVSINK_ERR_BAD_CONFIG;
+    if (cfg->head_dim / gv > 4) return KVSINK_ERR_UNSUPPORTED;
+    p->B = cfg->batch; p->Hq = cfg->n_q_heads; p->Hkv = cfg->n_kv_heads; p->D = cfg->head_dim; p->hidden = cfg->hidden;
+    p->bits = cfg->bits; p->G = cfg->group; p->max_seq = cfg->max_seq; p->topk = cfg->topk; p->pfn_n = cfg->pfn_n;
+    p->cap = cfg->topk + cfg->pfn_n;
+    p->Gv = gv; p->NGv = cfg->head_dim / gv;
+    p->rep = cfg->n_q_heads / cfg->n_kv_heads;
+    p->row_bytes = cfg->head_dim * cfg->bits / 8;
+    p->tile_bytes = KVSINK_TILE * p->row_bytes;
+    p->mask_words = (cfg->max_seq + 31) / 32;
+    p->n_channels = cfg->n_channels;
+    for (int i = 0; i < 8; ++i) p->channels[i] = cfg->channels[i];
+    return KVSINK_OK;
+}
+
+static bool aligned16(const void *ptr) { return ptr && ((uintptr_t)ptr & 15u) == 0; }
+
+static int check_cache(const kvsink_cache *c, const Params &p)
+{
+    if (!c) return KVSINK_ERR_BAD_ARG;
+    if (!aligned16(c->k_codes) || !aligned16(c->v_codes) || !aligned16(c->k_scale) || !aligned16(c->k_zero) ||
+        !aligned16(c->v_scale) || !aligned16(c->v_zero) || !aligned16(c->k_tail) || !aligned16(c->sink_bitmask) || !c->sink_count ||
+        !c->status)
+        return KVSINK_ERR_BAD_ARG;
+    if (p.cap > 0 && (!aligned16(c->sink_k) || !aligned16(c->sink_v) || !c->sink_pos)) return KVSINK_ERR_BAD_ARG;
+    if (c->seq_len < 0 || c->seq_len > p.max_seq) return KVSINK_ERR_BAD_ARG;
+    return KVSINK_OK;
+}
+
+extern "C" int kvsink_cache_sizes(const kvsink_config *cfg, kvsink_sizes *out)
+{
+    Params p;
+    int rc = derive(cfg, &p);
+    if (rc) return rc;
+    if (!out) return KVSINK_ERR_BAD_ARG;
+    const int64_t units = (int64_t)p.B * p.Hkv;
+    out->k_codes_bytes = units * p.max_seq * p.row_bytes;
+    out->v_codes_bytes = out->k_codes_bytes;
+    out->k_param_floats = units * (p.max_seq / p.G) * p.D;
+    out->v_param_floats = units * p.max_seq * p.NGv;
+    out->k_tail_halfs = units * p.G * p.D;
+    out->sink_halfs = units * p.cap * p.D;
+    out->bitmask_words = (int64_t)p.B * p.mask_words;
+    out->sink_pos_ints = (int64_t)p.B * p.cap;
+    out->predict_workspace_bytes = (int64_t)predict_workspace_bytes(p);
+    out->decode_workspace_bytes = (int64_t)decode_workspace_bytes(p);
+    out->sink_capacity = p.cap;
+    out->v_group = p.Gv;
+    out->v_groups_per_row = p.NGv;
+    out->tile_bytes = p.tile_bytes;
+    return KVSINK_OK;
+}
+
+extern "C" int kvsink_predict_sinks(const kvsink_config *cfg, const void *hidden, int32_t S, int64_t stride_b, int64_t stride_s,
+                                    uint32_t *bitmask, int32_t *sink_pos, int32_t *sink_count, void *workspace,
+                                    size_t workspace_bytes, void *cuda_stream)
+{
+    Params p;
+    int rc = derive(cfg, &p);
+    if (rc) return rc;
+    if (!hidden || !bitmask || !sink_count || (p.cap > 0 && !sink_pos)) return KVSINK_ERR_BAD_ARG;
+    if (S < 0 || S > p.max_seq || stride_s < p.hidden || stride_b < 0) return KVSINK_ERR_BAD_ARG;
+    if (!aligned16(workspace) || workspace_bytes < predict_workspace_bytes(p)) return KVSINK_ERR_WORKSPACE;
+    return launch_predict_sinks(p, (const __half *)hidden, S, stride_b, stride_s, bitmask, sink_pos, sink_count, workspace,
+                                (cudaStream_t)cuda_stream);
+}
+
+extern "C" int kvsink_quantize_append(const kvsink_config *cfg, kvsink_cache *cache, const void *k_new, const void *v_new, int32_t T,
+                                      int64_t stride_b, int64_t stride_h, int64_t stride_t, void *cuda_stream)
+{
+    Params p;
+    int rc = derive(cfg, &p);
+    if (rc) return rc;
+    rc = check_cache(cache, p);
+    if (rc) return rc;
+    if (T < 0) return KVSINK_ERR_BAD_ARG;
+    if (T == 0) return KVSINK_OK;
+    if (!aligned16(k_new) || !aligned16(v_new)) return KVSINK_ERR_BAD_ARG;
+    if (stride_t < p.D || (stride_t % 8) || (stride_h % 8) || (stride_b % 8) || stride_h < 0 || stride_b < 0) return KVSINK_ERR_BAD_ARG;
+    if ((int64_t)cache->seq_len + T > p.max_seq) return KVSINK_ERR_SEQ_OVERFLOW;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    const int S0 = cache->seq_len, G = p.G;
+    const __half *k = (const __half *)k_new, *v = (const __half *)v_new;
+    if (T > 1 && (S0 % G) != 0) return KVSINK_ERR_UNSUPPORTED;
+    if (S0 % G == 0 && T >= G) {
+        const int n_groups = T / G;
+        rc = launch_quantize_groups(p, *cache, k, v, S0, n_groups, stride_b, stride_h, stride_t, true, st);
+        if (rc) return rc;
+        rc = launch_quantize_tokens(p, *cache, k, v, n_groups * G, S0 + n_groups * G, T - n_groups * G, stride_b, stride_h, stride_t, st);
+        if (rc) return rc;
+    } else {
+        rc = launch_quantize_tokens(p, *cache, k, v, 0, S0, T, stride_b, stride_h, stride_t, st);
+        if (rc) return rc;
+        if ((S0 + T) % G == 0) {
+            // the open group is complete: quantize its keys per channel from the fp16 tail
+            rc = launch_quantize_groups(p, *cache, (const __half *)cache->k_tail, (const __half *)cache->k_tail, S0 + T - G, 1,
+                                        (int64_t)p.Hkv * G * p.D, (int64_t)G * p.D, p.D, false, st);
+            if (rc) return rc;
+        }
+    }
+    cache->seq_len = S0 + T;
+    return KVSINK_OK;
+}
+
+extern "C" int kvsink_decode_attention(const kvsink_config *cfg, const kvsink_cache *cache, const void *q, float *out, float *lse,
+                                       void *workspace, size_t workspace_bytes, void *cuda_stream)
+{
+    Params p;
+    int rc = derive(cfg, &p);
+    if (rc) return rc;
+    rc = check_cache(cache, p);
+    if (rc) return rc;
+    if (!aligned16(q) || !aligned16(out)) return KVSINK_ERR_BAD_ARG;
+    if (!aligned16(workspace)) return KVSINK_ERR_WORKSPACE;
+    return launch_decode(p, *cache, (const __half *)q, out, lse, workspace, workspace_bytes, (cudaStream_t)cuda_stream);
+}
+
+extern "C" int kvsink_read_status(const kvsink_cache *cache, int32_t *host_status, void *cuda_stream)
+{
+    if (!cache || !cache->status || !host_status) return KVSINK_ERR_BAD_ARG;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    if (cudaMemcpyAsync(host_status, cache->status, sizeof(int32_t), cudaMemcpyDeviceToHost, st) != cudaSuccess) return KVSINK_ERR_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return KVSINK_ERR_CUDA;
+    return KVSINK_OK;
+}
+
+extern "C" const char *kvsink_strerror(int code)
+{
+    switch (code) {
+    case KVSINK_OK: return "ok";
+    case KVSINK_ERR_BAD_ARG: return "bad argument (null or misaligned pointer, negative size, bad stride)";
+    case KVSINK_ERR_BAD_CONFIG: return "configuration field out of range";
+    case KVSINK_ERR_UNSUPPORTED: return "valid request without a kernel in this build";
+    case KVSINK_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+    case KVSINK_ERR_SEQ_OVERFLOW: return "appending would exceed max_seq";
+    case KVSINK_ERR_SINK_OVERFLOW: return "more sink tokens than the side buffer holds";
+    case KVSINK_ERR_CUDA: return "a CUDA runtime call failed";
+    case KVSINK_ERR_TIMEOUT: return "a bounded device wait ran out";
+    default: return "unknown status";
+    }
+}

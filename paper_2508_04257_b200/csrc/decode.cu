@@ -1,0 +1,501 @@
+// Single-token decode attention over the packed cache (Eq. 3 with Eq. 7's split into sink and non-sink sums).
+//
+// A packed tile is the register image of the m16n8k16 A operand, so a lane's 128-bit load IS its fragment.
+// Codes are never converted: a b-bit field masked in place is an fp16 subnormal (code * 2^k * 2^-24), which the
+// tensor core multiplies exactly; the power-of-two position factors are folded into the B operand (column half)
+// and into the fp32 epilogue (row half).
+//   scores   S[token, head] = sum_c code[token, c] * (q[head, c] * scale[c]) - sum_c q*scale*zero      (keys)
+//   outputs  O[c, head]     = sum_t code[c, t] * (p[t, head] * scale[t])  - sum_t p*scale*zero         (values)
+// with M = 16 tokens (keys) or 16 channels (values), N = 8 query heads of one KV head, fp32 accumulation.
+// Each warp streams whole key groups of one (sequence, KV head) unit; sequence splits are merged by a second
+// kernel.  Sink tokens are masked out of the packed stream and added from the fp16 side buffer under the same
+// softmax; keys of the open group come from the fp16 tail.
+#include "common.cuh"
+
+namespace kvsink {
+
+constexpr int DEC_WARPS = 4;
+constexpr int DEC_THREADS = DEC_WARPS * 32;
+constexpr float M_INIT = -1.0e30f;
+
+__device__ __forceinline__ float ex2(float x)
+{
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+__device__ __forceinline__ void mma16816(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1)
+{
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+
+__device__ __forceinline__ uint32_t movm_trans(uint32_t v)
+{
+    uint32_t o;
+    asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(o) : "r"(v));
+    return o;
+}
+
+__device__ __forceinline__ uint32_t pack_half2(float lo, float hi)
+{
+    __half2 h = __floats2half2_rn(lo, hi);
+    return *reinterpret_cast<uint32_t *>(&h);
+}
+
+template <int BITS, int D>
+struct Geo {
+    static constexpr int W = D * BITS / 64;                  // 32-bit words per lane per tile
+    static constexpr int NLO = (BITS == 3) ? D / 32 : W;     // words per lane in the first section
+    static constexpr int NHI = (BITS == 3) ? D / 64 : 0;
+    static constexpr int NM = D / 16;                        // 16x16 matrices per tile
+    // value of a masked field = code * ROWF^(row half) * COLF^(col half) * 2^-24
+    static constexpr float ROWF = (BITS == 2) ? 4.f : (BITS == 3 ? 1.f : 16.f);
+    static constexpr float COLF = (BITS == 4) ? 1.f : 16.f;
+};
+
+// A lane's words of one tile: section planes of up to four words per lane.
+template <int N>
+__device__ __forceinline__ void load_section(const uint32_t *__restrict__ sec, int lane, uint32_t *w)
+{
+#pragma unroll
+    for (int p = 0; p * 4 < N; ++p) {
+        const int u = (N - 4 * p) > 4 ? 4 : (N - 4 * p);
+        const uint32_t *src = sec + u * lane;
+        if (u == 4) {
+            uint4 v = __ldg((const uint4 *)src);
+            w[4 * p] = v.x; w[4 * p + 1] = v.y; w[4 * p + 2] = v.z; w[4 * p + 3] = v.w;
+        } else if (u == 2) {
+            uint2 v = __ldg((const uint2 *)src);
+            w[4 * p] = v.x; w[4 * p + 1] = v.y;
+        } else {
+#pragma unroll
+            for (int i = 0; i < u; ++i) w[4 * p + i] = __ldg(src + i);
+        }
+        sec += 32 * u;
+    }
+}
+
+template <int BITS, int D>
+__device__ __forceinline__ void load_tile(const uint32_t *__restrict__ tile, int lane, uint32_t (&w)[Geo<BITS, D>::W])
+{
+    using G_ = Geo<BITS, D>;
+    load_section<G_::NLO>(tile, lane, w);
+    if constexpr (BITS == 3) load_section<G_::NHI>(tile + 32 * G_::NLO, lane, w + G_::NLO);
+}
+
+// Masked fields of a lane's words as the A registers of the tile's NM matrices.
+template <int BITS, int D>
+__device__ __forceinline__ void tile_frags(const uint32_t (&w)[Geo<BITS, D>::W], uint32_t (&a)[Geo<BITS, D>::NM][4])
+{
+    using G_ = Geo<BITS, D>;
+    if constexpr (BITS == 2) {
+#pragma unroll
+        for (int i = 0; i < G_::W; ++i) {
+            const uint32_t x = w[i], y = x >> 8;
+            a[2 * i][0] = x & 0x00030003u; a[2 * i][1] = x & 0x000c000cu; a[2 * i][2] = x & 0x00300030u; a[2 * i][3] = x & 0x00c000c0u;
+            a[2 * i + 1][0] = y & 0x00030003u; a[2 * i + 1][1] = y & 0x000c000cu; a[2 * i + 1][2] = y & 0x00300030u; a[2 * i + 1][3] = y & 0x00c000c0u;
+        }
+    } else if constexpr (BITS == 4) {
+#pragma unroll
+        for (int i = 0; i < G_::W; ++i) {
+            const uint32_t x = w[i], y = x >> 8;
+            a[i][0] = x & 0x000f000fu; a[i][1] = x & 0x00f000f0u; a[i][2] = y & 0x000f000fu; a[i][3] = y & 0x00f000f0u;
+        }
+    } else {
+#pragma unroll
+        for (int i = 0; i < G_::NLO; ++i) {
+            const uint32_t x = w[i];
+            const uint32_t hh = (i & 1) ? (w[G_::NLO + i / 2] << 2) : w[G_::NLO + i / 2];
+            const uint32_t me = (x & 0x33333333u) | (hh & 0xccccccccu);                 // even fields, 3 bits at 4j
+            const uint32_t mo = ((x >> 2) & 0x33333333u) | ((hh >> 1) & 0xccccccccu);   // odd fields
+            const uint32_t me8 = me >> 8, mo8 = mo >> 8;
+            a[2 * i][0] = me & 0x00070007u; a[2 * i][1] = mo & 0x00070007u; a[2 * i][2] = me & 0x00700070u; a[2 * i][3] = mo & 0x00700070u;
+            a[2 * i + 1][0] = me8 & 0x00070007u; a[2 * i + 1][1] = mo8 & 0x00070007u; a[2 * i + 1][2] = me8 & 0x00700070u; a[2 * i + 1][3] = mo8 & 0x00700070u;
+        }
+    }
+}
+
+template <int BITS, int D>
+__global__ void __launch_bounds__(DEC_THREADS)
+decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__restrict__ out, float *__restrict__ lse,
+              float *__restrict__ part_ws, int nsplit, int groups_per_split, int qchunks, int seq_len)
+{
+    using G_ = Geo<BITS, D>;
+    constexpr int NM = G_::NM, W = G_::W;
+    constexpr float LOG2E = 1.4426950408889634f;
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    float *qs = (float *)smem_raw;                                   // [8][D] q * log2e/sqrt(D) * 2^4
+    __half *q16 = (__half *)(qs + 8 * D);                            // [8][D] q as given
+    __half *Bs_all = q16 + 8 * D;                                    // [warps][8][D] key B operand of the current group
+    float *part = (float *)(Bs_all + DEC_WARPS * 8 * D);             // [2*warps][nq][D+2]
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = lane >> 2, t = lane & 3;
+    const int split = blockIdx.x, h = blockIdx.y / qchunks, qc = blockIdx.y % qchunks, b = blockIdx.z;
+    const int nq = min(8, p.rep - 8 * qc), hq0 = h * p.rep + 8 * qc;
+    const int64_t unit = (int64_t)b * p.Hkv + h;
+    const int G = p.G, n = seq_len, n_groups = n / G, n_body = n_groups * G;
+    const int NGv = p.NGv, mpg = p.Gv / 16;                          // value matrices per channel group
+    const uint32_t *bm = c.sink_bitmask + (size_t)b * p.mask_words;
+    const float qscale = LOG2E * rsqrtf((float)D);
+
+    for (int i = tid; i < 8 * D; i += DEC_THREADS) {
+        const int qh = i / D, ch = i % D;
+        __half v = qh < nq ? q[((size_t)b * p.Hq + hq0 + qh) * D + ch] : __float2half(0.f);
+        q16[i] = v;
+        qs[i] = __half2float(v) * qscale * 16.f;
+    }
+    __syncthreads();
+
+    const int PS = D + 2;                                            // partial record: o[D], m, l
+    float *my_part = part + (size_t)(2 * warp) * nq * PS;
+
+    // ---------------- sink rows (fp16 side buffer), plain fp32 arithmetic ----------------
+    {
+        constexpr int CPL = D / 32;
+        float ms[8], ls[8], os[8][CPL];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            ms[i] = M_INIT; ls[i] = 0.f;
+#pragma unroll
+            for (int e = 0; e < CPL; ++e) os[i][e] = 0.f;
+        }
+        const int count = min(c.sink_count[b], p.cap);
+        const int worker = split * DEC_WARPS + warp, nworkers = nsplit * DEC_WARPS;
+        for (int j = worker; j < count; j += nworkers) {
+            const int pos = c.sink_pos[(size_t)b * p.cap + j];
+            if (pos < 0 || pos >= n) continue;
+            const __half *kr = (const __half *)c.sink_k + ((size_t)unit * p.cap + j) * D + lane * CPL;
+            const __half *vr = (const __half *)c.sink_v + ((size_t)unit * p.cap + j) * D + lane * CPL;
+            float kf[CPL], vf[CPL];
+#pragma unroll
+            for (int e = 0; e < CPL; ++e) { kf[e] = __half2float(kr[e]); vf[e] = __half2float(vr[e]); }
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                if (i < nq) {
+                    float d = 0.f;
+#pragma unroll
+                    for (int e = 0; e < CPL; ++e) d += qs[i * D + lane * CPL + e] * kf[e];
+                    const float s = warp_sum(d) * 0.0625f;
+                    const float mnew = fmaxf(ms[i], s);
+                    const float corr = ex2(ms[i] - mnew), pp = ex2(s - mnew);
+                    ls[i] = ls[i] * corr + pp;
+#pragma unroll
+                    for (int e = 0; e < CPL; ++e) os[i][e] = os[i][e] * corr + pp * vf[e];
+                    ms[i] = mnew;
+                }
+            }
+        }
+        float *sp = my_part + (size_t)nq * PS;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            if (i < nq) {
+#pragma unroll
+                for (int e = 0; e < CPL; ++e) sp[i * PS + lane * CPL + e] = os[i][e];
+                if (lane == 0) { sp[i * PS + D] = ms[i]; sp[i * PS + D + 1] = ls[i]; }
+            }
+        }
+    }
+
+    // ---------------- packed stream ----------------
+    float m_run[2] = {M_INIT, M_INIT}, l_run[2] = {0.f, 0.f};
+    float O[NM][4];
+    float bv[4][2];                       // sum p*scale*zero per value channel group and head pair
+#pragma unroll
+    for (int m = 0; m < NM; ++m)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) O[m][i] = 0.f;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) bv[j][0] = bv[j][1] = 0.f;
+
+    __half *Bs = Bs_all + (size_t)warp * 8 * D;
+    const uint8_t *kc_base = c.k_codes + (size_t)unit * p.max_seq * p.row_bytes;
+    const uint8_t *vc_base = c.v_codes + (size_t)unit * p.max_seq * p.row_bytes;
+    const float *vs_base = c.v_scale + (size_t)unit * p.max_seq * NGv;
+    const float *vz_base = c.v_zero + (size_t)unit * p.max_seq * NGv;
+
+    // One 16-token tile: scores in s[4] (log2 units, -inf where the token does not take part) -> softmax -> values.
+    auto tile_values = [&](int T, float (&s)[4], bool v0, bool v1) {
+        float tm0 = fmaxf(s[0], s[2]), tm1 = fmaxf(s[1], s[3]);
+#pragma unroll
+        for (int o = 4; o < 32; o <<= 1) {
+            tm0 = fmaxf(tm0, __shfl_xor_sync(0xffffffffu, tm0, o));
+            tm1 = fmaxf(tm1, __shfl_xor_sync(0xffffffffu, tm1, o));
+        }
+        const float mn0 = fmaxf(m_run[0], tm0), mn1 = fmaxf(m_run[1], tm1);
+        if (__any_sync(0xffffffffu, mn0 > m_run[0] || mn1 > m_run[1])) {
+            const float c0 = ex2(m_run[0] - mn0), c1 = ex2(m_run[1] - mn1);
+            l_run[0] *= c0; l_run[1] *= c1;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) { bv[j][0] *= c0; bv[j][1] *= c1; }
+#pragma unroll
+            for (int m = 0; m < NM; ++m) { O[m][0] *= c0; O[m][2] *= c0; O[m][1] *= c1; O[m][3] *= c1; }
+            m_run[0] = mn0; m_run[1] = mn1;
+        }
+        const float p0 = ex2(s[0] - mn0), p1 = ex2(s[1] - mn1), p2 = ex2(s[2] - mn0), p3 = ex2(s[3] - mn1);
+        l_run[0] += p0 + p2;
+        l_run[1] += p1 + p3;
+        uint32_t vw[W];
+        load_tile<BITS, D>((const uint32_t *)(vc_base + (size_t)T * p.tile_bytes), lane, vw);
+        uint32_t va[NM][4];
+        tile_frags<BITS, D>(vw, va);
+        const int tok0 = T * KVSINK_TILE + g, tok1 = tok0 + 8;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            if (j < NGv) {
+                const float sv0 = v0 ? __ldg(vs_base + (size_t)tok0 * NGv + j) : 0.f, zv0 = v0 ? __ldg(vz_base + (size_t)tok0 * NGv + j) : 0.f;
+                const float sv1 = v1 ? __ldg(vs_base + (size_t)tok1 * NGv + j) : 0.f, zv1 = v1 ? __ldg(vz_base + (size_t)tok1 * NGv + j) : 0.f;
+                const float w0 = p0 * sv0, w1 = p1 * sv0, w2 = p2 * sv1, w3 = p3 * sv1;
+                bv[j][0] += w0 * zv0 + w2 * zv1;
+                bv[j][1] += w1 * zv0 + w3 * zv1;
+                const uint32_t b0 = movm_trans(pack_half2(w0 * 16.f, w1 * 16.f));
+                const uint32_t b1 = movm_trans(pack_half2(w2 * (16.f / G_::COLF), w3 * (16.f / G_::COLF)));
+#pragma unroll
+                for (int m = 0; m < NM; ++m)
+                    if (m / mpg == j) mma16816(O[m], va[m], b0, b1);
+            }
+        }
+    };
+
+    // ---- complete key groups of this split ----
+    const int g_begin = split * groups_per_split, g_end = min(n_groups, g_begin + groups_per_split);
+    for (int grp = g_begin + warp; grp < g_end; grp += DEC_WARPS) {
+        // B operand of the group: fp16(q * scale) per channel and head, column half pre-divided by COLF;
+        // bias = sum_c fp16(q*scale) * zero with the same rounded factor.
+        float bias[2] = {0.f, 0.f};
+        {
+            constexpr int CPL = D / 32;
+            const float *sc = c.k_scale + ((size_t)unit * (p.max_seq / G) + grp) * D + lane * CPL;
+            const float *ze = c.k_zero + ((size_t)unit * (p.max_seq / G) + grp) * D + lane * CPL;
+            float scv[CPL], zev[CPL];
+#pragma unroll
+            for (int e = 0; e < CPL; ++e) { scv[e] = __ldg(sc + e); zev[e] = __ldg(ze + e); }
+            __syncwarp();
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                if (i < nq) {
+                    float bsum = 0.f;
+#pragma unroll
+                    for (int e = 0; e < CPL; ++e) {
+                        const int ch = lane * CPL + e;
+                        __half hb = __float2half_rn(fminf(fmaxf(qs[i * D + ch] * scv[e], -60000.f), 60000.f));
+                        bsum += __half2float(hb) * zev[e];
+                        if ((ch & 8) && G_::COLF != 1.f) hb = __hmul(hb, __float2half(1.f / G_::COLF));
+                        Bs[i * D + ch] = hb;
+                    }
+                    bsum = warp_sum(bsum) * 0.0625f;
+                    if (i == 2 * t) bias[0] = bsum;
+                    if (i == 2 * t + 1) bias[1] = bsum;
+                }
+            }
+            __syncwarp();
+        }
+        uint32_t bk[NM][2];
+#pragma unroll
+        for (int m = 0; m < NM; ++m) {
+            bk[m][0] = g < nq ? *(const uint32_t *)(Bs + g * D + 16 * m + 2 * t) : 0u;
+            bk[m][1] = g < nq ? *(const uint32_t *)(Bs + g * D + 16 * m + 2 * t + 8) : 0u;
+        }
+        const int T0 = grp * (G / KVSINK_TILE);
+        for (int T = T0; T < T0 + G / KVSINK_TILE; ++T) {
+            uint32_t kw[W];
+            load_tile<BITS, D>((const uint32_t *)(kc_base + (size_t)T * p.tile_bytes), lane, kw);
+            uint32_t ka[NM][4];
+            tile_frags<BITS, D>(kw, ka);
+            float acc[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+            for (int m = 0; m < NM; ++m) mma16816(acc, ka[m], bk[m][0], bk[m][1]);
+            constexpr float KS0 = 1048576.f, KS1 = 1048576.f / G_::ROWF;
+            float s[4] = {acc[0] * KS0 - bias[0], acc[1] * KS0 - bias[1], acc[2] * KS1 - bias[0], acc[3] * KS1 - bias[1]};
+            const uint32_t mask16 = (bm[T >> 1] >> (16 * (T & 1))) & 0xffffu;
+            bool v0 = true, v1 = true;
+            if (mask16) {
+                v0 = !((mask16 >> g) & 1u);
+                v1 = !((mask16 >> (g + 8)) & 1u);
+                if (!v0) s[0] = s[1] = -INFINITY;
+                if (!v1) s[2] = s[3] = -INFINITY;
+            }
+            tile_values(T, s, v0, v1);
+        }
+    }
+
+    // ---- tokens of the open group: keys from the fp16 tail (last split only) ----
+    if (split == nsplit - 1) {
+        const __half *tail = (const __half *)c.k_tail + (size_t)unit * G * D;
+        const int T_begin = n_body / KVSINK_TILE, T_end = (n + KVSINK_TILE - 1) / KVSINK_TILE;
+        for (int T = T_begin + warp; T < T_end; T += DEC_WARPS) {
+            const int tok0 = T * KVSINK_TILE + g, tok1 = tok0 + 8;
+            const bool in0 = tok0 < n, in1 = tok1 < n;
+            const __half *r0 = tail + (size_t)(tok0 % G) * D, *r1 = tail + (size_t)(tok1 % G) * D;
+            float acc[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+            for (int m = 0; m < NM; ++m) {
+                uint32_t a[4];
+                a[0] = in0 ? *(const uint32_t *)(r0 + 16 * m + 2 * t) : 0u;
+                a[1] = in1 ? *(const uint32_t *)(r1 + 16 * m + 2 * t) : 0u;
+                a[2] = in0 ? *(const uint32_t *)(r0 + 16 * m + 2 * t + 8) : 0u;
+                a[3] = in1 ? *(const uint32_t *)(r1 + 16 * m + 2 * t + 8) : 0u;
+                const uint32_t b0 = *(const uint32_t *)(q16 + g * D + 16 * m + 2 * t);
+                const uint32_t b1 = *(const uint32_t *)(q16 + g * D + 16 * m + 2 * t + 8);
+                mma16816(acc, a, b0, b1);
+            }
+            const bool v0 = in0 && !mask_bit(bm, in0 ? tok0 : 0), v1 = in1 && !mask_bit(bm, in1 ? tok1 : 0);
+            float s[4] = {v0 ? acc[0] * qscale : -INFINITY, v0 ? acc[1] * qscale : -INFINITY,
+                          v1 ? acc[2] * qscale : -INFINITY, v1 ? acc[3] * qscale : -INFINITY};
+            tile_values(T, s, v0, v1);
+        }
+    }
+
+    // ---- this warp's packed partial: finish the reductions over the token lanes, convert units ----
+#pragma unroll
+    for (int o = 4; o < 32; o <<= 1) {
+        l_run[0] += __shfl_xor_sync(0xffffffffu, l_run[0], o);
+        l_run[1] += __shfl_xor_sync(0xffffffffu, l_run[1], o);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            bv[j][0] += __shfl_xor_sync(0xffffffffu, bv[j][0], o);
+            bv[j][1] += __shfl_xor_sync(0xffffffffu, bv[j][1], o);
+        }
+    }
+#pragma unroll
+    for (int m = 0; m < NM; ++m) {
+        const int j = m / mpg;
+        float bj0 = 0.f, bj1 = 0.f;
+#pragma unroll
+        for (int jj = 0; jj < 4; ++jj)
+            if (jj == j) { bj0 = bv[jj][0]; bj1 = bv[jj][1]; }
+        constexpr float OS0 = 1048576.f, OS1 = 1048576.f / G_::ROWF;
+        const int ch0 = 16 * m + g, ch1 = ch0 + 8;
+        if (2 * t < nq) {
+            my_part[(2 * t) * PS + ch0] = O[m][0] * OS0 - bj0;
+            my_part[(2 * t) * PS + ch1] = O[m][2] * OS1 - bj0;
+        }
+        if (2 * t + 1 < nq) {
+            my_part[(2 * t + 1) * PS + ch0] = O[m][1] * OS0 - bj1;
+            my_part[(2 * t + 1) * PS + ch1] = O[m][3] * OS1 - bj1;
+        }
+    }
+    if (g == 0) {
+        if (2 * t < nq) { my_part[(2 * t) * PS + D] = m_run[0]; my_part[(2 * t) * PS + D + 1] = l_run[0]; }
+        if (2 * t + 1 < nq) { my_part[(2 * t + 1) * PS + D] = m_run[1]; my_part[(2 * t + 1) * PS + D + 1] = l_run[1]; }
+    }
+    __syncthreads();
+
+    // ---- merge the block's partials; write the result or this split's partial ----
+    for (int idx = tid; idx < nq * D; idx += DEC_THREADS) {
+        const int qh = idx / D, ch = idx % D;
+        float M = M_INIT;
+        for (int w = 0; w < 2 * DEC_WARPS; ++w) M = fmaxf(M, part[((size_t)w * nq + qh) * PS + D]);
+        float acc = 0.f, L = 0.f;
+        for (int w = 0; w < 2 * DEC_WARPS; ++w) {
+            const float *pr = part + ((size_t)w * nq + qh) * PS;
+            const float f = ex2(pr[D] - M);
+            acc += pr[ch] * f;
+            L += pr[D + 1] * f;
+        }
+        const size_t oq = (size_t)b * p.Hq + hq0 + qh;
+        if (nsplit == 1) {
+            out[oq * D + ch] = L > 0.f ? acc / L : 0.f;
+            if (lse && ch == 0) lse[oq] = L > 0.f ? (M + log2f(L)) * 0.6931471805599453f : -INFINITY;
+        } else {
+            float *wsr = part_ws + (oq * nsplit + split) * PS;
+            wsr[ch] = acc;
+            if (ch == 0) { wsr[D] = M; wsr[D + 1] = L; }
+        }
+    }
+}
+
+// Merge of the sequence splits: one block per (sequence, query head), one thread per channel.
+__global__ void decode_merge_kernel(const float *__restrict__ part_ws, int nsplit, int D, float *__restrict__ out, float *__restrict__ lse)
+{
+    const int PS = D + 2;
+    const size_t oq = blockIdx.x;
+    const int ch = threadIdx.x;
+    const float *base = part_ws + oq * nsplit * PS;
+    float M = M_INIT;
+    for (int s = 0; s < nsplit; ++s) M = fmaxf(M, base[(size_t)s * PS + D]);
+    float acc = 0.f, L = 0.f;
+    for (int s = 0; s < nsplit; ++s) {
+        const float f = ex2(base[(size_t)s * PS + D] - M);
+        acc += base[(size_t)s * PS + ch] * f;
+        L += base[(size_t)s * PS + D + 1] * f;
+    }
+    out[oq * D + ch] = L > 0.f ? acc / L : 0.f;
+    if (lse && ch == 0) lse[oq] = L > 0.f ? (M + log2f(L)) * 0.6931471805599453f : -INFINITY;
+}
+
+// ---- host side ----
+constexpr int DEC_SLOTS = 148 * 4;   // resident blocks the split heuristic plans for
+
+static int max_splits(const Params &p)
+{
+    const int qchunks = (p.rep + 7) / 8;
+    const long units = (long)p.B * p.Hkv * qchunks;
+    long ns = (2L * DEC_SLOTS + units - 1) / units;
+    const long mg = p.max_seq / p.G;
+    if (ns > mg) ns = mg;
+    return (int)(ns < 1 ? 1 : ns);
+}
+
+static int choose_splits(const Params &p, int n_groups)
+{
+    const int qchunks = (p.rep + 7) / 8;
+    const long units = (long)p.B * p.Hkv * qchunks;
+    const int ns_max = max_splits(p) < n_groups ? max_splits(p) : (n_groups > 0 ? n_groups : 1);
+    int best = 1;
+    double best_cost = 1e300;
+    for (int ns = 1; ns <= ns_max; ++ns) {
+        const long waves = (units * ns + DEC_SLOTS - 1) / DEC_SLOTS;
+        const int per_block = (n_groups + ns - 1) / ns;
+        const int per_warp = (per_block + DEC_WARPS - 1) / DEC_WARPS;
+        const double cost = (double)waves * (per_warp + 0.5);
+        if (cost < best_cost - 1e-9) { best_cost = cost; best = ns; }
+    }
+    return best;
+}
+
+size_t decode_workspace_bytes(const Params &p)
+{
+    return (size_t)p.B * p.Hq * max_splits(p) * (p.D + 2) * sizeof(float) + 16;
+}
+
+template <int BITS, int D>
+static int launch_decode_t(const Params &p, const kvsink_cache &c, const __half *q, float *out, float *lse, float *ws, cudaStream_t st)
+{
+    const int n_groups = c.seq_len / p.G;
+    const int nsplit = choose_splits(p, n_groups);
+    const int gps = n_groups > 0 ? (n_groups + nsplit - 1) / nsplit : 0;
+    const int qchunks = (p.rep + 7) / 8;
+    const int nq_max = p.rep < 8 ? p.rep : 8;
+    const size_t smem = 8 * D * 4 + 8 * D * 2 + (size_t)DEC_WARPS * 8 * D * 2 + (size_t)2 * DEC_WARPS * nq_max * (D + 2) * 4;
+    auto kern = decode_kernel<BITS, D>;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return KVSINK_ERR_CUDA;
+    dim3 grid(nsplit, p.Hkv * qchunks, p.B);
+    kern<<<grid, DEC_THREADS, smem, st>>>(p, c, q, out, lse, ws, nsplit, gps, qchunks, c.seq_len);
+    if (cudaGetLastError() != cudaSuccess) return KVSINK_ERR_CUDA;
+    if (nsplit > 1) {
+        decode_merge_kernel<<<p.B * p.Hq, D, 0, st>>>(ws, nsplit, D, out, lse);
+        if (cudaGetLastError() != cudaSuccess) return KVSINK_ERR_CUDA;
+    }
+    return KVSINK_OK;
+}
+
+int launch_decode(const Params &p, const kvsink_cache &c, const __half *q, float *out, float *lse, void *workspace,
+                  size_t workspace_bytes, cudaStream_t st)
+{
+    if (workspace_bytes < decode_workspace_bytes(p)) return KVSINK_ERR_WORKSPACE;
+    float *ws = (float *)workspace;
+    if (p.D == 128) {
+        if (p.bits == 2) return launch_decode_t<2, 128>(p, c, q, out, lse, ws, st);
+        if (p.bits == 3) return launch_decode_t<3, 128>(p, c, q, out, lse, ws, st);
+        if (p.bits == 4) return launch_decode_t<4, 128>(p, c, q, out, lse, ws, st);
+    } else if (p.D == 64) {
+        if (p.bits == 2) return launch_decode_t<2, 64>(p, c, q, out, lse, ws, st);
+        if (p.bits == 4) return launch_decode_t<4, 64>(p, c, q, out, lse, ws, st);
+    }
+    return KVSINK_ERR_UNSUPPORTED;
+}
+
+}  // namespace kvsink
