@@ -45,6 +45,18 @@ __device__ __forceinline__ uint32_t pack_half2(float lo, float hi)
     return *reinterpret_cast<uint32_t *>(&h);
 }
 
+// floor(log2(x)) of a positive normal float; -127 for zero and subnormals.
+__device__ __forceinline__ int floor_log2(float x) { return (int)((__float_as_uint(x) >> 23) & 0xffu) - 127; }
+// 2^e for -126 <= e <= 127.
+__device__ __forceinline__ float pow2i(int e) { return __uint_as_float((uint32_t)(e + 127) << 23); }
+
+__device__ __forceinline__ float warp_max(float v)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+    return v;
+}
+
 template <int BITS, int D>
 struct Geo {
     static constexpr int W = D * BITS / 64;                  // 32-bit words per lane per tile
@@ -127,7 +139,7 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
     constexpr int NM = G_::NM, W = G_::W;
     constexpr float LOG2E = 1.4426950408889634f;
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    float *qs = (float *)smem_raw;                                   // [8][D] q * log2e/sqrt(D) * 2^4
+    float *qs = (float *)smem_raw;                                   // [8][D] q * log2e/sqrt(D)
     __half *q16 = (__half *)(qs + 8 * D);                            // [8][D] q as given
     __half *Bs_all = q16 + 8 * D;                                    // [warps][8][D] key B operand of the current group
     float *part = (float *)(Bs_all + DEC_WARPS * 8 * D);             // [2*warps][nq][D+2]
@@ -145,7 +157,7 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
         const int qh = i / D, ch = i % D;
         __half v = qh < nq ? q[((size_t)b * p.Hq + hq0 + qh) * D + ch] : __float2half(0.f);
         q16[i] = v;
-        qs[i] = __half2float(v) * qscale * 16.f;
+        qs[i] = __half2float(v) * qscale;
     }
     __syncthreads();
 
@@ -178,7 +190,7 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
                     float d = 0.f;
 #pragma unroll
                     for (int e = 0; e < CPL; ++e) d += qs[i * D + lane * CPL + e] * kf[e];
-                    const float s = warp_sum(d) * 0.0625f;
+                    const float s = warp_sum(d);
                     const float mnew = fmaxf(ms[i], s);
                     const float corr = ex2(ms[i] - mnew), pp = ex2(s - mnew);
                     ls[i] = ls[i] * corr + pp;
@@ -203,6 +215,8 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
     float m_run[2] = {M_INIT, M_INIT}, l_run[2] = {0.f, 0.f};
     float O[NM][4];
     float bv[4][2];                       // sum p*scale*zero per value channel group and head pair
+    int ev = 60;                          // the value B operand is p * scale * 2^ev; lowered so that it fits fp16
+    float evf = pow2i(60);
 #pragma unroll
     for (int m = 0; m < NM; ++m)
 #pragma unroll
@@ -250,12 +264,30 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
                 const float w0 = p0 * sv0, w1 = p1 * sv0, w2 = p2 * sv1, w3 = p3 * sv1;
                 bv[j][0] += w0 * zv0 + w2 * zv1;
                 bv[j][1] += w1 * zv0 + w3 * zv1;
-                const uint32_t b0 = movm_trans(pack_half2(w0 * 16.f, w1 * 16.f));
-                const uint32_t b1 = movm_trans(pack_half2(w2 * (16.f / G_::COLF), w3 * (16.f / G_::COLF)));
+                const uint32_t b0 = movm_trans(pack_half2(w0 * evf, w1 * evf));
+                const uint32_t b1 = movm_trans(pack_half2(w2 * (evf / G_::COLF), w3 * (evf / G_::COLF)));
 #pragma unroll
                 for (int m = 0; m < NM; ++m)
                     if (m / mpg == j) mma16816(O[m], va[m], b0, b1);
             }
+        }
+    };
+
+    // Before a span of tokens is consumed: make sure p * scale * 2^ev stays below 2^13 for every value scale in it.
+    auto fit_value_scale = [&](int tok_begin, int tok_end) {
+        float mx = 0.f;
+        for (int i = tok_begin * NGv + lane; i < tok_end * NGv; i += 32) mx = fmaxf(mx, fabsf(__ldg(vs_base + i)));
+        mx = warp_max(mx);
+        int need = 12 - floor_log2(mx);
+        need = need > 60 ? 60 : (need < -60 ? -60 : need);
+        if (need < ev) {
+            const float f = pow2i(need - ev);
+#pragma unroll
+            for (int m = 0; m < NM; ++m)
+#pragma unroll
+                for (int i = 0; i < 4; ++i) O[m][i] *= f;
+            ev = need;
+            evf = pow2i(ev);
         }
     };
 
@@ -264,7 +296,7 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
     for (int grp = g_begin + warp; grp < g_end; grp += DEC_WARPS) {
         // B operand of the group: fp16(q * scale) per channel and head, column half pre-divided by COLF;
         // bias = sum_c fp16(q*scale) * zero with the same rounded factor.
-        float bias[2] = {0.f, 0.f};
+        float bias[2] = {0.f, 0.f}, ksc[2] = {0.f, 0.f};
         {
             constexpr int CPL = D / 32;
             const float *sc = c.k_scale + ((size_t)unit * (p.max_seq / G) + grp) * D + lane * CPL;
@@ -276,18 +308,25 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
                 if (i < nq) {
+                    float v[CPL], amax = 0.f;
+#pragma unroll
+                    for (int e = 0; e < CPL; ++e) { v[e] = qs[i * D + lane * CPL + e] * scv[e]; amax = fmaxf(amax, fabsf(v[e])); }
+                    amax = warp_max(amax);
+                    int sh = 13 - floor_log2(amax);                 // largest factor lands in [2^13, 2^14)
+                    sh = sh > 60 ? 60 : (sh < -60 ? -60 : sh);
+                    const float f = pow2i(sh);
                     float bsum = 0.f;
 #pragma unroll
                     for (int e = 0; e < CPL; ++e) {
                         const int ch = lane * CPL + e;
-                        __half hb = __float2half_rn(fminf(fmaxf(qs[i * D + ch] * scv[e], -60000.f), 60000.f));
+                        __half hb = __float2half_rn(v[e] * f);
                         bsum += __half2float(hb) * zev[e];
                         if ((ch & 8) && G_::COLF != 1.f) hb = __hmul(hb, __float2half(1.f / G_::COLF));
                         Bs[i * D + ch] = hb;
                     }
-                    bsum = warp_sum(bsum) * 0.0625f;
-                    if (i == 2 * t) bias[0] = bsum;
-                    if (i == 2 * t + 1) bias[1] = bsum;
+                    bsum = warp_sum(bsum) * pow2i(-sh);
+                    if (i == 2 * t) { bias[0] = bsum; ksc[0] = pow2i(24 - sh); }
+                    if (i == 2 * t + 1) { bias[1] = bsum; ksc[1] = pow2i(24 - sh); }
                 }
             }
             __syncwarp();
@@ -298,6 +337,7 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
             bk[m][0] = g < nq ? *(const uint32_t *)(Bs + g * D + 16 * m + 2 * t) : 0u;
             bk[m][1] = g < nq ? *(const uint32_t *)(Bs + g * D + 16 * m + 2 * t + 8) : 0u;
         }
+        fit_value_scale(grp * G, grp * G + G);
         const int T0 = grp * (G / KVSINK_TILE);
         for (int T = T0; T < T0 + G / KVSINK_TILE; ++T) {
             uint32_t kw[W];
@@ -307,8 +347,9 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
             float acc[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
             for (int m = 0; m < NM; ++m) mma16816(acc, ka[m], bk[m][0], bk[m][1]);
-            constexpr float KS0 = 1048576.f, KS1 = 1048576.f / G_::ROWF;
-            float s[4] = {acc[0] * KS0 - bias[0], acc[1] * KS0 - bias[1], acc[2] * KS1 - bias[0], acc[3] * KS1 - bias[1]};
+            constexpr float R1 = 1.f / G_::ROWF;
+            float s[4] = {acc[0] * ksc[0] - bias[0], acc[1] * ksc[1] - bias[1], acc[2] * (ksc[0] * R1) - bias[0],
+                          acc[3] * (ksc[1] * R1) - bias[1]};
             const uint32_t mask16 = (bm[T >> 1] >> (16 * (T & 1))) & 0xffffu;
             bool v0 = true, v1 = true;
             if (mask16) {
@@ -326,6 +367,7 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
         const __half *tail = (const __half *)c.k_tail + (size_t)unit * G * D;
         const int T_begin = n_body / KVSINK_TILE, T_end = (n + KVSINK_TILE - 1) / KVSINK_TILE;
         for (int T = T_begin + warp; T < T_end; T += DEC_WARPS) {
+            fit_value_scale(T * KVSINK_TILE, min(n, (T + 1) * KVSINK_TILE));
             const int tok0 = T * KVSINK_TILE + g, tok1 = tok0 + 8;
             const bool in0 = tok0 < n, in1 = tok1 < n;
             const __half *r0 = tail + (size_t)(tok0 % G) * D, *r1 = tail + (size_t)(tok1 % G) * D;
@@ -366,7 +408,7 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
 #pragma unroll
         for (int jj = 0; jj < 4; ++jj)
             if (jj == j) { bj0 = bv[jj][0]; bj1 = bv[jj][1]; }
-        constexpr float OS0 = 1048576.f, OS1 = 1048576.f / G_::ROWF;
+        const float OS0 = pow2i(24 - ev), OS1 = OS0 / G_::ROWF;
         const int ch0 = 16 * m + g, ch1 = ch0 + 8;
         if (2 * t < nq) {
             my_part[(2 * t) * PS + ch0] = O[m][0] * OS0 - bj0;

@@ -87,11 +87,11 @@ def _randn_half(shape, gen: torch.Generator, device, chunk_rows: int = 1 << 14) 
 
 
 def sink_positions(wl: Workload) -> np.ndarray:
-    """Planted sink tokens per sequence, int64 [B, topk] ascending; token 0 is always one of them."""
+    """Planted sink tokens per sequence, int64 [B, min(topk, S)] ascending; token 0 is always one of them."""
     rng = np.random.default_rng(wl.seed ^ 0xA11CE)
-    out = np.zeros((wl.batch, max(wl.topk, 0)), np.int64)
+    out = np.zeros((wl.batch, max(min(wl.topk, wl.seq), 0)), np.int64)
     for b in range(wl.batch):
-        k = wl.topk
+        k = min(wl.topk, wl.seq)
         if k <= 0:
             continue
         chosen = {0}
