@@ -30,6 +30,10 @@ extern "C" {
 #define KVSINK_ERR_SINK_OVERFLOW (-6)
 #define KVSINK_ERR_CUDA (-7)         /* a CUDA runtime call failed (launch, attribute, copy) */
 #define KVSINK_ERR_TIMEOUT (-8)
+#define KVSINK_ERR_STATIC_SCRATCH (-9) /* kvsink_decode_attention_static: the built-in scratch array is too small */
+
+/* Size of the scratch array built into the library for kvsink_decode_attention_static (4 MiB per GPU). */
+#define KVSINK_STATIC_SCRATCH_BYTES (4 * 1024 * 1024)
 
 /* Bits of the device status word (kvsink_cache.status, read with kvsink_read_status). */
 #define KVSINK_STATUS_SINK_MISMATCH 1 /* a token whose mask bit is set was not found in sink_pos */
@@ -147,6 +151,32 @@ int kvsink_quantize_append(const kvsink_config *cfg, kvsink_cache *cache, const 
  */
 int kvsink_decode_attention(const kvsink_config *cfg, const kvsink_cache *cache, const void *q, float *out, float *lse,
                             void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/*
+ * kvsink_decode_attention for callers that cannot allocate device memory.  (No counterpart in the paper: this is
+ * a deployment convenience of this library.)
+ *
+ * Some hosts of this code may not call cudaMalloc at all: a plug-in that runs inside another engine's memory
+ * plan, a real-time loop that forbids allocation after start-up, a process that was handed a fixed set of
+ * buffers.  They can provide q, the cache and out (they own those anyway) but have nowhere to get the
+ * split-partial workspace from.  This entry point computes exactly what kvsink_decode_attention computes, with
+ * the same kernels, and keeps the partials in an array of KVSINK_STATIC_SCRATCH_BYTES that is part of the
+ * library image: every GPU on which the library is loaded holds that memory until the process exits.  It calls
+ * no cudaMalloc / cudaFree and no allocating library routine.
+ *
+ *   - Arguments are those of kvsink_decode_attention without workspace / workspace_bytes.
+ *   - Limit: kvsink_sizes.decode_workspace_bytes of the configuration must not exceed
+ *     KVSINK_STATIC_SCRATCH_BYTES, otherwise KVSINK_ERR_STATIC_SCRATCH is returned and nothing is launched
+ *     (use kvsink_decode_attention with your own workspace then).
+ *   - The first call on each device looks up the array's device address (a CUDA runtime query, made with that
+ *     device current, no allocation).  Make that first call outside of any stream capture.
+ *   - All calls on a device share the one array, which keeps whatever the previous call left in it.  Nothing in
+ *     it has to start at zero -- each call overwrites every record it later reads -- but two calls whose kernels
+ *     overlap on the GPU (different streams, no ordering between them) race on it and corrupt each other's
+ *     result.  Calls on one stream, or otherwise ordered, are safe.
+ */
+int kvsink_decode_attention_static(const kvsink_config *cfg, const kvsink_cache *cache, const void *q, float *out, float *lse,
+                                   void *cuda_stream);
 
 /* Copies the device status word to *host_status and waits for the stream (the only call that synchronises). */
 int kvsink_read_status(const kvsink_cache *cache, int32_t *host_status, void *cuda_stream);

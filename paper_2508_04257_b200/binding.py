@@ -16,7 +16,8 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _LIB_PATH = os.path.join(_HERE, "libkvsink.so")
 
 EXPORTS = ("kvsink_cache_sizes", "kvsink_predict_sinks", "kvsink_quantize_append", "kvsink_decode_attention",
-           "kvsink_read_status", "kvsink_strerror")
+           "kvsink_decode_attention_static", "kvsink_read_status", "kvsink_strerror")
+STATIC_SCRATCH_BYTES = 4 * 1024 * 1024
 
 
 class KvsinkError(RuntimeError):
@@ -173,6 +174,23 @@ def decode_attention(cfg: Config, cache: KVCache, q: torch.Tensor, out: Optional
                                        C.c_size_t(workspace.numel()), _stream())
     if rc:
         raise KvsinkError(rc, "kvsink_decode_attention")
+    return out, lse
+
+
+def decode_attention_static(cfg: Config, cache: KVCache, q: torch.Tensor, out: torch.Tensor, lse: Optional[torch.Tensor] = None):
+    """kvsink_decode_attention_static: decode attention for callers that may not allocate device memory.
+
+    Same result as decode_attention, but the split partials go to a 4 MiB array built into the library instead of
+    a workspace tensor, and this wrapper allocates nothing either: `out` (fp32 [B,Hq,D]) and, if wanted, `lse`
+    (fp32 [B,Hq]) must be passed in.  Raises KvsinkError(-9) when the configuration needs more scratch than the
+    built-in array holds.  Calls that may overlap on the GPU must not share a device (they share the array).
+    """
+    assert q.is_cuda and q.dtype == torch.float16 and q.is_contiguous()
+    assert out.is_cuda and out.dtype == torch.float32 and out.is_contiguous()
+    cc = cache.c()
+    rc = lib().kvsink_decode_attention_static(C.byref(cfg.c()), C.byref(cc), _ptr(q), _ptr(out), _ptr(lse), _stream())
+    if rc:
+        raise KvsinkError(rc, "kvsink_decode_attention_static")
     return out, lse
 
 

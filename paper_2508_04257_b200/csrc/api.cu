@@ -136,6 +136,19 @@ extern "C" int kvsink_decode_attention(const kvsink_config *cfg, const kvsink_ca
     return launch_decode(p, *cache, (const __half *)q, out, lse, workspace, workspace_bytes, (cudaStream_t)cuda_stream);
 }
 
+extern "C" int kvsink_decode_attention_static(const kvsink_config *cfg, const kvsink_cache *cache, const void *q, float *out,
+                                              float *lse, void *cuda_stream)
+{
+    Params p;
+    int rc = derive(cfg, &p);
+    if (rc) return rc;
+    if (decode_workspace_bytes(p) > (size_t)KVSINK_STATIC_SCRATCH_BYTES) return KVSINK_ERR_STATIC_SCRATCH;
+    rc = check_cache(cache, p);
+    if (rc) return rc;
+    if (!aligned16(q) || !aligned16(out)) return KVSINK_ERR_BAD_ARG;
+    return launch_decode_static(p, *cache, (const __half *)q, out, lse, (cudaStream_t)cuda_stream);
+}
+
 extern "C" int kvsink_read_status(const kvsink_cache *cache, int32_t *host_status, void *cuda_stream)
 {
     if (!cache || !cache->status || !host_status) return KVSINK_ERR_BAD_ARG;
@@ -157,6 +170,9 @@ extern "C" const char *kvsink_strerror(int code)
     case KVSINK_ERR_SINK_OVERFLOW: return "more sink tokens than the side buffer holds";
     case KVSINK_ERR_CUDA: return "a CUDA runtime call failed";
     case KVSINK_ERR_TIMEOUT: return "a bounded device wait ran out";
+    case KVSINK_ERR_STATIC_SCRATCH:
+        return "this configuration needs more split scratch than the library's built-in array holds "
+               "(KVSINK_STATIC_SCRATCH_BYTES); use kvsink_decode_attention with a caller workspace";
     default: return "unknown status";
     }
 }

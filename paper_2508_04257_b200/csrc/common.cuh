@@ -97,6 +97,7 @@ int launch_quantize_tokens(const Params &p, const kvsink_cache &c, const __half 
                            int first_token, int n_tokens, int64_t sb, int64_t sh, int64_t stt, cudaStream_t st);
 int launch_decode(const Params &p, const kvsink_cache &c, const __half *q, float *out, float *lse, void *workspace,
                   size_t workspace_bytes, cudaStream_t st);
+int launch_decode_static(const Params &p, const kvsink_cache &c, const __half *q, float *out, float *lse, cudaStream_t st);
 size_t decode_workspace_bytes(const Params &p);
 size_t predict_workspace_bytes(const Params &p);
 

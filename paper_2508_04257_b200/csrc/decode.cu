@@ -10,6 +10,8 @@
 // Each warp streams whole key groups of one (sequence, KV head) unit; sequence splits are merged by a second
 // kernel.  Sink tokens are masked out of the packed stream and added from the fp16 side buffer under the same
 // softmax; keys of the open group come from the fp16 tail.
+#include <mutex>
+
 #include "common.cuh"
 
 namespace kvsink {
@@ -538,6 +540,34 @@ int launch_decode(const Params &p, const kvsink_cache &c, const __half *q, float
         if (p.bits == 4) return launch_decode_t<4, 64>(p, c, q, out, lse, ws, st);
     }
     return KVSINK_ERR_UNSUPPORTED;
+}
+
+// ---------------------------------------------------------------------------------------------------------
+// Decode attention without caller-provided scratch: the split partials live in a fixed array inside the library
+// image.  Every GPU that loads the library holds these KVSINK_STATIC_SCRATCH_BYTES until the process exits.
+// ---------------------------------------------------------------------------------------------------------
+static __device__ __align__(256) unsigned char g_decode_scratch[KVSINK_STATIC_SCRATCH_BYTES];
+
+// In host code `g_decode_scratch` is only a handle for the runtime, not a device address; the address is looked
+// up once per device (with that device current) and cached.
+static void *g_scratch_ptr[64];
+static bool g_scratch_known[64];
+static std::mutex g_scratch_mutex;
+
+int launch_decode_static(const Params &p, const kvsink_cache &c, const __half *q, float *out, float *lse, cudaStream_t st)
+{
+    if (decode_workspace_bytes(p) > (size_t)KVSINK_STATIC_SCRATCH_BYTES) return KVSINK_ERR_STATIC_SCRATCH;
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return KVSINK_ERR_CUDA;
+    std::lock_guard<std::mutex> guard(g_scratch_mutex);
+    if (!g_scratch_known[dev]) {
+        void *ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_decode_scratch) != cudaSuccess || ptr == nullptr) return KVSINK_ERR_CUDA;
+        g_scratch_ptr[dev] = ptr;
+        g_scratch_known[dev] = true;
+    }
+    // No clearing is needed: the split kernel writes every partial record the merge kernel reads.
+    return launch_decode(p, c, q, out, lse, g_scratch_ptr[dev], (size_t)KVSINK_STATIC_SCRATCH_BYTES, st);
 }
 
 }  // namespace kvsink
