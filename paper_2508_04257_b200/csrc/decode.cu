@@ -143,8 +143,9 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
     extern __shared__ __align__(16) unsigned char smem_raw[];
     float *qs = (float *)smem_raw;                                   // [8][D] q * log2e/sqrt(D)
     __half *q16 = (__half *)(qs + 8 * D);                            // [8][D] q as given
-    __half *Bs_all = q16 + 8 * D;                                    // [warps][8][D] key B operand of the current group
-    float *part = (float *)(Bs_all + DEC_WARPS * 8 * D);             // [2*warps][nq][D+2]
+    constexpr int BST = D + 8;                                       // padded row stride of the B tables (bank spread)
+    __half *Bs_all = q16 + 8 * D;                                    // [warps][2][8][BST] key B operand (hi, lo) of the group
+    float *part = (float *)(Bs_all + DEC_WARPS * 2 * 8 * BST);       // [2*warps][nq][D+2]
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = lane >> 2, t = lane & 3;
     const int split = blockIdx.x, h = blockIdx.y / qchunks, qc = blockIdx.y % qchunks, b = blockIdx.z;
@@ -226,7 +227,7 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
 #pragma unroll
     for (int j = 0; j < 4; ++j) bv[j][0] = bv[j][1] = 0.f;
 
-    __half *Bs = Bs_all + (size_t)warp * 8 * D;
+    __half *Bs = Bs_all + (size_t)warp * 2 * 8 * BST, *Bl = Bs + 8 * BST;
     const uint8_t *kc_base = c.k_codes + (size_t)unit * p.max_seq * p.row_bytes;
     const uint8_t *vc_base = c.v_codes + (size_t)unit * p.max_seq * p.row_bytes;
     const float *vs_base = c.v_scale + (size_t)unit * p.max_seq * NGv;
@@ -299,6 +300,7 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
         // B operand of the group: fp16(q * scale) per channel and head, column half pre-divided by COLF;
         // bias = sum_c fp16(q*scale) * zero with the same rounded factor.
         float bias[2] = {0.f, 0.f}, ksc[2] = {0.f, 0.f};
+        uint32_t need_lo = 0;     // bit m: matrix m also gets the low half of the split factor (warp-uniform)
         {
             constexpr int CPL = D / 32;
             const float *sc = c.k_scale + ((size_t)unit * (p.max_seq / G) + grp) * D + lane * CPL;
@@ -318,14 +320,29 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
                     sh = sh > 60 ? 60 : (sh < -60 ? -60 : sh);
                     const float f = pow2i(sh);
                     float bsum = 0.f;
+                    bool big = false;
 #pragma unroll
                     for (int e = 0; e < CPL; ++e) {
                         const int ch = lane * CPL + e;
-                        __half hb = __float2half_rn(v[e] * f);
-                        bsum += __half2float(hb) * zev[e];
-                        if ((ch & 8) && G_::COLF != 1.f) hb = __hmul(hb, __float2half(1.f / G_::COLF));
-                        Bs[i * D + ch] = hb;
+                        const float vf = v[e] * f;
+                        __half hb = __float2half_rn(vf);
+                        // fp16 keeps 11 bits of the factor; where that could move a score by more than ~4e-4
+                        // (factor * largest |code - zero| * 2^-12) the rounding residual is kept as a second factor
+                        __half lb = __float2half_rn(vf - __half2float(hb));
+                        big |= fabsf(v[e]) * (fabsf(zev[e]) + (float)((1 << BITS) - 1)) > 1.6f;
+                        bsum += (__half2float(hb) + __half2float(lb)) * zev[e];
+                        if ((ch & 8) && G_::COLF != 1.f) {
+                            hb = __hmul(hb, __float2half(1.f / G_::COLF));
+                            lb = __hmul(lb, __float2half(1.f / G_::COLF));
+                        }
+                        Bs[i * BST + ch] = hb;
+                        Bl[i * BST + ch] = lb;
                     }
+                    const uint32_t bal = __ballot_sync(0xffffffffu, big);
+                    constexpr int LPM = 16 / CPL;     // lanes per 16-channel matrix
+#pragma unroll
+                    for (int m = 0; m < NM; ++m)
+                        if ((bal >> (LPM * m)) & ((1u << LPM) - 1u)) need_lo |= 1u << m;
                     bsum = warp_sum(bsum) * pow2i(-sh);
                     if (i == 2 * t) { bias[0] = bsum; ksc[0] = pow2i(24 - sh); }
                     if (i == 2 * t + 1) { bias[1] = bsum; ksc[1] = pow2i(24 - sh); }
@@ -336,8 +353,8 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
         uint32_t bk[NM][2];
 #pragma unroll
         for (int m = 0; m < NM; ++m) {
-            bk[m][0] = g < nq ? *(const uint32_t *)(Bs + g * D + 16 * m + 2 * t) : 0u;
-            bk[m][1] = g < nq ? *(const uint32_t *)(Bs + g * D + 16 * m + 2 * t + 8) : 0u;
+            bk[m][0] = g < nq ? *(const uint32_t *)(Bs + g * BST + 16 * m + 2 * t) : 0u;
+            bk[m][1] = g < nq ? *(const uint32_t *)(Bs + g * BST + 16 * m + 2 * t + 8) : 0u;
         }
         fit_value_scale(grp * G, grp * G + G);
         const int T0 = grp * (G / KVSINK_TILE);
@@ -348,7 +365,14 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
             tile_frags<BITS, D>(kw, ka);
             float acc[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-            for (int m = 0; m < NM; ++m) mma16816(acc, ka[m], bk[m][0], bk[m][1]);
+            for (int m = 0; m < NM; ++m) {
+                mma16816(acc, ka[m], bk[m][0], bk[m][1]);
+                if (need_lo & (1u << m)) {
+                    const uint32_t l0 = g < nq ? *(const uint32_t *)(Bl + g * BST + 16 * m + 2 * t) : 0u;
+                    const uint32_t l1 = g < nq ? *(const uint32_t *)(Bl + g * BST + 16 * m + 2 * t + 8) : 0u;
+                    mma16816(acc, ka[m], l0, l1);
+                }
+            }
             constexpr float R1 = 1.f / G_::ROWF;
             float s[4] = {acc[0] * ksc[0] - bias[0], acc[1] * ksc[1] - bias[1], acc[2] * (ksc[0] * R1) - bias[0],
                           acc[3] * (ksc[1] * R1) - bias[1]};
@@ -513,7 +537,7 @@ static int launch_decode_t(const Params &p, const kvsink_cache &c, const __half 
     const int gps = n_groups > 0 ? (n_groups + nsplit - 1) / nsplit : 0;
     const int qchunks = (p.rep + 7) / 8;
     const int nq_max = p.rep < 8 ? p.rep : 8;
-    const size_t smem = 8 * D * 4 + 8 * D * 2 + (size_t)DEC_WARPS * 8 * D * 2 + (size_t)2 * DEC_WARPS * nq_max * (D + 2) * 4;
+    const size_t smem = 8 * D * 4 + 8 * D * 2 + (size_t)DEC_WARPS * 2 * 8 * (D + 8) * 2 + (size_t)2 * DEC_WARPS * nq_max * (D + 2) * 4;
     auto kern = decode_kernel<BITS, D>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return KVSINK_ERR_CUDA;
     dim3 grid(nsplit, p.Hkv * qchunks, p.B);
