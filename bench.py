@@ -195,6 +195,8 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=dev)
 
     wl = synth.WORKLOADS[args.workload].scaled(seed=synth.WORKLOADS[args.workload].seed + 7919 * rank)
+    if args.batch > 0:
+        wl = wl.scaled(batch=args.batch)
     L = args.instances
     cfg = kv.Config(wl.batch, wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.hidden, wl.bits, wl.group, wl.max_seq, wl.topk, wl.pfn_n,
                     wl.channels)
@@ -350,6 +352,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="llama2_7b_layer", choices=sorted(synth.WORKLOADS))
     ap.add_argument("--instances", type=int, default=4, help="layer-shaped instances per step")
+    ap.add_argument("--batch", type=int, default=0, help="override the workload's batch (profiling a smaller case)")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--cpu-heads", type=int, default=32, help="KV heads in the CPU-oracle sample (0 = skip)")
     ap.add_argument("--ref-heads", type=int, default=4, help="KV heads per step of --impl reference")

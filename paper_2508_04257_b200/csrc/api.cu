@@ -34,6 +34,15 @@ static int derive(const kvsink_config *cfg, Params *p)
     return KVSINK_OK;
 }
 
+// Whole groups: the streaming kernel where the shape has one, else the generic kernel.
+static int quantize_groups(const Params &p, const kvsink_cache &c, const __half *k, const __half *v, int first_token, int n_groups,
+                           int64_t sb, int64_t sh, int64_t stt, bool do_v_and_sinks, cudaStream_t st)
+{
+    int rc = launch_quantize_groups_fast(p, c, k, v, first_token, n_groups, sb, sh, stt, do_v_and_sinks, st);
+    if (rc != KVSINK_ERR_UNSUPPORTED) return rc;
+    return launch_quantize_groups(p, c, k, v, first_token, n_groups, sb, sh, stt, do_v_and_sinks, st);
+}
+
 static bool aligned16(const void *ptr) { return ptr && ((uintptr_t)ptr & 15u) == 0; }
 
 static int check_cache(const kvsink_cache *c, const Params &p)
@@ -105,7 +114,7 @@ extern "C" int kvsink_quantize_append(const kvsink_config *cfg, kvsink_cache *ca
     if (T > 1 && (S0 % G) != 0) return KVSINK_ERR_UNSUPPORTED;
     if (S0 % G == 0 && T >= G) {
         const int n_groups = T / G;
-        rc = launch_quantize_groups(p, *cache, k, v, S0, n_groups, stride_b, stride_h, stride_t, true, st);
+        rc = quantize_groups(p, *cache, k, v, S0, n_groups, stride_b, stride_h, stride_t, true, st);
         if (rc) return rc;
         rc = launch_quantize_tokens(p, *cache, k, v, n_groups * G, S0 + n_groups * G, T - n_groups * G, stride_b, stride_h, stride_t, st);
         if (rc) return rc;
@@ -114,7 +123,7 @@ extern "C" int kvsink_quantize_append(const kvsink_config *cfg, kvsink_cache *ca
         if (rc) return rc;
         if ((S0 + T) % G == 0) {
             // the open group is complete: quantize its keys per channel from the fp16 tail
-            rc = launch_quantize_groups(p, *cache, (const __half *)cache->k_tail, (const __half *)cache->k_tail, S0 + T - G, 1,
+            rc = quantize_groups(p, *cache, (const __half *)cache->k_tail, (const __half *)cache->k_tail, S0 + T - G, 1,
                                         (int64_t)p.Hkv * G * p.D, (int64_t)G * p.D, p.D, false, st);
             if (rc) return rc;
         }
