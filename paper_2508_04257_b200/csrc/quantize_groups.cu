@@ -36,27 +36,29 @@ __device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], const void *
 
 // Per channel (keys) or per (token, channel group) (values): what the fast coder needs.
 struct __align__(16) Coder {
-    float r_lo, r_hi;   // 1/scale nudged down / up; +inf forces the exact path
+    float r_lo, r_hi;   // 1/scale nudged down / up; r_lo = +inf forces the exact path
     float magic;        // M + zero
-    float ymax;         // M + zero clamp: M + qmax
+    float pad;
 };
 
-__device__ __forceinline__ Coder make_coder(float scale, float zero, float absmax, float qmax)
+// mn, mx: the group's extremes.  The fast coder is used only where it is provably exact: |x/scale| and |zero| far
+// below 2^22 (integer-in-mantissa), and the top code cannot exceed qmax (so no clamp is needed).
+__device__ __forceinline__ Coder make_coder(float scale, float zero, float mn, float mx, float qmax)
 {
     Coder c;
+    c.pad = 0.f;
     if (scale == 0.f) {   // no member, or sink token: code 0
         c.r_lo = c.r_hi = 0.f;
         c.magic = MAGIC;
-        c.ymax = MAGIC + qmax;
         return c;
     }
     const float r = __frcp_rn(scale);
-    // the integer-in-mantissa trick needs |x/scale| and |zero| well below 2^22
-    const bool ok = absmax * r < 2097152.f && fabsf(zero) < 2097152.f && r < 3.0e38f;
+    const float absmax = fmaxf(fabsf(mn), fabsf(mx));
+    const bool top_fits = __fadd_rn(rintf(__fdiv_rn(mx, scale)), zero) <= qmax;
+    const bool ok = absmax * r < 2097152.f && fabsf(zero) < 2097152.f && r < 3.0e38f && top_fits;
     c.r_lo = ok ? __fmul_rn(r, 1.f - 2.384185791015625e-07f) : __int_as_float(0x7f800000);
     c.r_hi = ok ? __fmul_rn(r, 1.f + 2.384185791015625e-07f) : r;
     c.magic = MAGIC + (ok ? zero : 0.f);
-    c.ymax = MAGIC + qmax;
     return c;
 }
 
@@ -68,13 +70,12 @@ __device__ __forceinline__ uint32_t code_pair(uint32_t h2, const Coder &c0, cons
     const float a0 = fmaf(x.x, c0.r_lo, c0.magic), b0 = fmaf(x.x, c0.r_hi, c0.magic);
     const float a1 = fmaf(x.y, c1.r_lo, c1.magic), b1 = fmaf(x.y, c1.r_hi, c1.magic);
     differ |= (__float_as_uint(a0) ^ __float_as_uint(b0)) | (__float_as_uint(a1) ^ __float_as_uint(b1));
-    const uint32_t u0 = __float_as_uint(fminf(a0, c0.ymax)), u1 = __float_as_uint(fminf(a1, c1.ymax));
-    // low halves of u0 and u1 (the bit pattern of 1.5 * 2^23 has a zero low half); the mask only matters for rows that are discarded
-    return __byte_perm(u0, u1, 0x5410) & (((1u << BITS) - 1u) * 0x00010001u);
+    // low halves of the two results (the bit pattern of 1.5 * 2^23 has a zero low half)
+    return __byte_perm(__float_as_uint(a0), __float_as_uint(a1), 0x5410);
 }
 
 template <int BITS>
-__device__ __forceinline__ uint32_t code_pair_exact(uint32_t h2, float s0, float z0, float s1, float z1)
+__device__ __noinline__ uint32_t code_pair_exact(uint32_t h2, float s0, float z0, float s1, float z1)
 {
     const float2 x = __half22float2(*reinterpret_cast<const __half2 *>(&h2));
     const float qmax = (float)((1 << BITS) - 1);
@@ -110,7 +111,66 @@ template <> struct RowMask<2> { static constexpr uint32_t LO = 0x00330033u, HI =
 template <> struct RowMask<4> { static constexpr uint32_t LO = 0x0f0f0f0fu, HI = 0u; };
 template <> struct RowMask<3> { static constexpr uint32_t LO = 0x00330033u, HI = 0x00110011u; };
 
-template <int BITS, int D>
+// Codes of one value tile (16 tokens x D channels) in the tile's register layout, written to `tile` (shared memory).
+// The lane's four tokens are 2*t4, 2*t4+1, 2*t4+8, 2*t4+9.  Returns (warp-uniform) whether any lane's fast result
+// is not certain; with EXACT those matrices are recomputed with the IEEE division.
+template <int BITS, int D, int NGv, bool EXACT>
+__device__ __forceinline__ bool encode_v_tile(const __half *Xt, const Coder *coder, const float *xscale, const float *xzero, int T,
+                                              int lane, uint32_t *tile)
+{
+    constexpr int W = D * BITS / 64;
+    constexpr int NLO = (BITS == 3) ? D / 32 : W, NHI = (BITS == 3) ? D / 64 : 0;
+    constexpr int mpg = (D / NGv) / 16;      // matrices per channel group
+    const int t4 = lane & 3, mj = lane >> 3, rr = lane & 7;
+    const int tok = 16 * T + rr + 8 * (mj >> 1), tk0 = 16 * T + 2 * t4;
+    const __half *rowp = Xt + (size_t)tok * D;
+    const int sw = tok & 7;
+    uint32_t wl[NLO], wh[NHI > 0 ? NHI : 1], differ_all = 0;
+#pragma unroll
+    for (int i = 0; i < NLO; ++i) wl[i] = 0;
+#pragma unroll
+    for (int i = 0; i < (NHI > 0 ? NHI : 1); ++i) wh[i] = 0;
+#pragma unroll
+    for (int jg = 0; jg < NGv; ++jg) {
+        Coder vc[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) vc[q] = coder[(tk0 + (q & 1) + 8 * (q >> 1)) * NGv + jg];
+#pragma unroll
+        for (int mi = 0; mi < mpg; ++mi) {
+            const int m = jg * mpg + mi;
+            uint32_t a[4], pc[4], differ = 0;
+            ldmatrix_x4_trans(a, rowp + (((2 * m + (mj & 1)) ^ sw) * 8));
+#pragma unroll
+            for (int r = 0; r < 4; ++r) pc[r] = code_pair<BITS>(a[r], vc[2 * (r >> 1)], vc[2 * (r >> 1) + 1], differ);
+            if (EXACT && differ) {
+#pragma unroll
+                for (int r = 0; r < 4; ++r) {
+                    const int i0 = (tk0 + 8 * (r >> 1)) * NGv + jg;
+                    pc[r] = code_pair_exact<BITS>(a[r], xscale[i0], xzero[i0], xscale[i0 + NGv], xzero[i0 + NGv]);
+                }
+            }
+            differ_all |= differ;
+            uint32_t lo, hi;
+            pack_matrix<BITS>(pc, m, &lo, &hi);
+            if constexpr (BITS == 4) {
+                wl[m] = lo;
+            } else {
+                wl[m >> 1] |= lo << (8 * (m & 1));
+                if constexpr (BITS == 3) wh[m >> 2] |= hi;
+            }
+        }
+    }
+    if (!EXACT && __any_sync(0xffffffffu, differ_all != 0)) return true;
+#pragma unroll
+    for (int i = 0; i < NLO; ++i) tile[section_word_offset(NLO, lane, i)] = wl[i];
+    if constexpr (BITS == 3) {
+#pragma unroll
+        for (int i = 0; i < NHI; ++i) tile[32 * NLO + section_word_offset(NHI, lane, i)] = wh[i];
+    }
+    return false;
+}
+
+template <int BITS, int D, int NGv>
 __global__ void __launch_bounds__(QF_THREADS, 3)
 quantize_groups_fast(Params p, kvsink_cache c, const __half *__restrict__ k_src, const __half *__restrict__ v_src, int first_token,
                      int n_groups, int64_t sb, int64_t sh, int64_t stt, int kinds)
@@ -122,7 +182,8 @@ quantize_groups_fast(Params p, kvsink_cache c, const __half *__restrict__ k_src,
     constexpr int NLO = (BITS == 3) ? D / 32 : W, NHI = (BITS == 3) ? D / 64 : 0;
     constexpr int TILE_WORDS = 32 * W;
     const float qmax = (float)((1 << BITS) - 1);
-    const int G = p.G, NGv = p.NGv, Gv = p.Gv, n_tiles = G / KVSINK_TILE;
+    constexpr int Gv = D / NGv;
+    const int G = p.G, n_tiles = G / KVSINK_TILE;
 
     extern __shared__ __align__(128) unsigned char smem[];
     __half *Xbuf = (__half *)smem;                                 // [2][G][D] swizzled 16-byte chunks (double buffer)
@@ -150,9 +211,12 @@ quantize_groups_fast(Params p, kvsink_cache c, const __half *__restrict__ k_src,
         decode_item(item, &b, &h, &grp, &kind);
         const __half *xbase = (kind == 0 ? k_src : v_src) + b * sb + h * sh + (int64_t)(grp * G) * stt;
         __half *Xt = Xbuf + (size_t)buf * G * D;
-        for (int idx = tid; idx < G * CH; idx += QF_THREADS) {
-            const int t = idx / CH, ch = idx % CH;
-            cp_async16(Xt + (size_t)t * D + (ch ^ (t & 7)) * 8, xbase + (int64_t)t * stt + ch * 8);
+        {
+            constexpr int RPI = QF_THREADS / CH;          // rows per iteration (a multiple of 8, so t & 7 is fixed)
+            const int ch = tid % CH, t0 = tid / CH;
+            const __half *src = xbase + (int64_t)t0 * stt + ch * 8;
+            __half *dst = Xt + (size_t)t0 * D + (ch ^ (t0 & 7)) * 8;
+            for (int t = t0; t < G; t += RPI, src += (int64_t)RPI * stt, dst += (size_t)RPI * D) cp_async16(dst, src);
         }
         if (tid < n_tiles) {
             const int tok = first_token + grp * G + tid * KVSINK_TILE;   // multiple of 16
@@ -229,7 +293,7 @@ quantize_groups_fast(Params p, kvsink_cache c, const __half *__restrict__ k_src,
                 group_params(any, mn, mx, qmax, &s, &z);
                 xscale[ch] = s;
                 xzero[ch] = z;
-                coder[ch] = make_coder(s, z, fmaxf(fabsf(mn), fabsf(mx)), qmax);
+                coder[ch] = make_coder(s, z, mn, mx, qmax);
                 const size_t o = ((size_t)unit * (p.max_seq / G) + p0 / G) * D + ch;
                 c.k_scale[o] = s;
                 c.k_zero[o] = z;
@@ -255,7 +319,8 @@ quantize_groups_fast(Params p, kvsink_cache c, const __half *__restrict__ k_src,
                     ldmatrix_x4(a, Xt + (size_t)tok * D + ((chunk ^ (tok & 7)) * 8));
 #pragma unroll
                     for (int r = 0; r < 4; ++r) pc[r] = code_pair<BITS>(a[r], kc[2 * (r >> 1)], kc[2 * (r >> 1) + 1], differ);
-                    if (differ) {
+                    const uint32_t m16 = tm[T];
+                    if (differ | m16) {   // rare: a value too close to a rounding tie, or a tile with sink tokens
 #pragma unroll
                         for (int r = 0; r < 4; ++r) {
                             const int ch = 16 * m + 2 * t4 + 8 * (r >> 1);
@@ -264,7 +329,6 @@ quantize_groups_fast(Params p, kvsink_cache c, const __half *__restrict__ k_src,
                     }
                     uint32_t lo, hi;
                     pack_matrix<BITS>(pc, m, &lo, &hi);
-                    const uint32_t m16 = tm[T];
                     if (m16) {   // sink tokens keep code 0 in the packed stream
                         uint32_t keep = 0xffffffffu, keeph = 0xffffffffu;
                         const int hsh = 8 * (m & 1) + 2 * (1 - ((m >> 1) & 1));
@@ -309,10 +373,10 @@ quantize_groups_fast(Params p, kvsink_cache c, const __half *__restrict__ k_src,
             }
             __syncthreads();
             {
-                const int spg = Gv / 32;     // sets per channel group
+                constexpr int spg = Gv / 32;     // sets per channel group
                 for (int i2 = tid; i2 < G * NGv; i2 += QF_THREADS) {
                     const int t = i2 / NGv, j = i2 % NGv;
-                    float s = 0.f, z = 0.f, amax = 0.f;
+                    float s = 0.f, z = 0.f, gmn = 0.f, gmx = 0.f;
                     if (!is_sink(t)) {
                         __half lo = __ushort_as_half(0x7C00), hi = __ushort_as_half(0xFC00);
                         for (int q = 0; q < spg; ++q) {
@@ -320,68 +384,26 @@ quantize_groups_fast(Params p, kvsink_cache c, const __half *__restrict__ k_src,
                             lo = __hmin(lo, __ushort_as_half((unsigned short)(v & 0xffffu)));
                             hi = __hmax(hi, __ushort_as_half((unsigned short)(v >> 16)));
                         }
-                        const float mn = __half2float(lo), mx = __half2float(hi);
-                        group_params(true, mn, mx, qmax, &s, &z);
-                        amax = fmaxf(fabsf(mn), fabsf(mx));
+                        gmn = __half2float(lo);
+                        gmx = __half2float(hi);
+                        group_params(true, gmn, gmx, qmax, &s, &z);
                     }
                     xscale[i2] = s;
                     xzero[i2] = z;
-                    coder[i2] = make_coder(s, z, amax, qmax);
+                    coder[i2] = make_coder(s, z, gmn, gmx, qmax);
                     const size_t o = ((size_t)unit * p.max_seq + p0 + t) * NGv + j;
                     c.v_scale[o] = s;
                     c.v_zero[o] = z;
                 }
             }
             __syncthreads();
-            // ---- codes: a warp takes whole tiles; the lane's four tokens are 2*t4, 2*t4+1, 2*t4+8, 2*t4+9 ----
-            {
-                const int mpg = Gv / 16;
-                const int row_in_tile = rr + 8 * (mj >> 1);
-                for (int T = warp; T < n_tiles; T += QF_WARPS) {
-                    uint32_t wl[NLO > 0 ? NLO : 1], wh[NHI > 0 ? NHI : 1];
-#pragma unroll
-                    for (int i = 0; i < NLO; ++i) wl[i] = 0;
-#pragma unroll
-                    for (int i = 0; i < (NHI > 0 ? NHI : 1); ++i) wh[i] = 0;
-                    Coder vc[4];
-                    const int tok = 16 * T + row_in_tile;
-                    const int tk0 = 16 * T + 2 * t4;
-#pragma unroll
-                    for (int m = 0; m < NM; ++m) {
-                        if (m % 2 == 0 && (m == 0 || (m / mpg) != ((m - 2) / mpg))) {   // new channel group (groups hold >= 2 matrices)
-                            const int jg = m / mpg;
-#pragma unroll
-                            for (int q = 0; q < 4; ++q) vc[q] = coder[(tk0 + (q & 1) + 8 * (q >> 1)) * NGv + jg];
-                        }
-                        uint32_t a[4], pc[4], differ = 0;
-                        const int chunk = 2 * m + (mj & 1);
-                        ldmatrix_x4_trans(a, Xt + (size_t)tok * D + ((chunk ^ (tok & 7)) * 8));
-#pragma unroll
-                        for (int r = 0; r < 4; ++r) pc[r] = code_pair<BITS>(a[r], vc[2 * (r >> 1)], vc[2 * (r >> 1) + 1], differ);
-                        if (differ) {
-#pragma unroll
-                            for (int r = 0; r < 4; ++r) {
-                                const int i0 = (tk0 + 8 * (r >> 1)) * NGv + m / mpg;
-                                pc[r] = code_pair_exact<BITS>(a[r], xscale[i0], xzero[i0], xscale[i0 + NGv], xzero[i0 + NGv]);
-                            }
-                        }
-                        uint32_t lo, hi;
-                        pack_matrix<BITS>(pc, m, &lo, &hi);
-                        if constexpr (BITS == 4) {
-                            wl[m] = lo;
-                        } else {
-                            wl[m >> 1] |= lo << (8 * (m & 1));
-                            if constexpr (BITS == 3) wh[m >> 2] |= hi;
-                        }
-                    }
-                    uint32_t *tile = xout + (size_t)T * TILE_WORDS;
-#pragma unroll
-                    for (int i = 0; i < NLO; ++i) tile[section_word_offset(NLO, lane, i)] = wl[i];
-                    if constexpr (BITS == 3) {
-#pragma unroll
-                        for (int i = 0; i < NHI; ++i) tile[32 * NLO + section_word_offset(NHI, lane, i)] = wh[i];
-                    }
-                }
+            // ---- codes: a warp takes whole tiles ----
+            for (int T = warp; T < n_tiles; T += QF_WARPS) {
+                uint32_t *tile = xout + (size_t)T * TILE_WORDS;
+                // everything through the fast coder; if any lane saw a value too close to a rounding tie (rare), the whole
+                // warp repeats the tile with the exact division where a lane's matrix needs it
+                if (encode_v_tile<BITS, D, NGv, false>(Xt, coder, xscale, xzero, T, lane, tile))
+                    encode_v_tile<BITS, D, NGv, true>(Xt, coder, xscale, xzero, T, lane, tile);
             }
         }
         __syncthreads();
@@ -424,18 +446,18 @@ quantize_groups_fast(Params p, kvsink_cache c, const __half *__restrict__ k_src,
     }
 }
 
-template <int BITS, int D>
-static int launch_fast(const Params &p, const kvsink_cache &c, const __half *k_src, const __half *v_src, int first_token, int n_groups,
-                       int64_t sb, int64_t sh, int64_t stt, bool do_v, cudaStream_t st)
+template <int BITS, int D, int NGV>
+static int launch_fast_n(const Params &p, const kvsink_cache &c, const __half *k_src, const __half *v_src, int first_token, int n_groups,
+                         int64_t sb, int64_t sh, int64_t stt, bool do_v, cudaStream_t st)
 {
     const int G = p.G, n_tiles = G / KVSINK_TILE;
     constexpr int W = D * BITS / 64;
-    const size_t max_coders = (size_t)(D > G * p.NGv ? D : G * p.NGv);
+    const size_t max_coders = (size_t)(D > G * NGV ? D : G * NGV);
     size_t stat_words = (size_t)(QF_WARPS * D > G * (D / 32) ? QF_WARPS * D : G * (D / 32));
     if (stat_words < (size_t)n_tiles * 32 * W) stat_words = (size_t)n_tiles * 32 * W;
     const size_t smem = 2 * (size_t)G * D * 2 + max_coders * (16 + 8) + stat_words * 4 + 2 * (size_t)n_tiles * 4 + 16;
     if (smem > 227 * 1024) return KVSINK_ERR_UNSUPPORTED;
-    auto kern = quantize_groups_fast<BITS, D>;
+    auto kern = quantize_groups_fast<BITS, D, NGV>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return KVSINK_ERR_CUDA;
     const int kinds = do_v ? 2 : 1;
     const long n_items = (long)p.B * p.Hkv * n_groups * kinds;
@@ -446,6 +468,17 @@ static int launch_fast(const Params &p, const kvsink_cache &c, const __half *k_s
     if (blocks > n_items) blocks = n_items;
     kern<<<(unsigned)blocks, QF_THREADS, smem, st>>>(p, c, k_src, v_src, first_token, n_groups, sb, sh, stt, kinds);
     return cudaGetLastError() == cudaSuccess ? KVSINK_OK : KVSINK_ERR_CUDA;
+}
+
+template <int BITS, int D>
+static int launch_fast(const Params &p, const kvsink_cache &c, const __half *k_src, const __half *v_src, int first_token, int n_groups,
+                       int64_t sb, int64_t sh, int64_t stt, bool do_v, cudaStream_t st)
+{
+    if (p.NGv == 1) return launch_fast_n<BITS, D, 1>(p, c, k_src, v_src, first_token, n_groups, sb, sh, stt, do_v, st);
+    if (p.NGv == 2) return launch_fast_n<BITS, D, 2>(p, c, k_src, v_src, first_token, n_groups, sb, sh, stt, do_v, st);
+    if constexpr (D == 128)
+        if (p.NGv == 4) return launch_fast_n<BITS, D, 4>(p, c, k_src, v_src, first_token, n_groups, sb, sh, stt, do_v, st);
+    return KVSINK_ERR_UNSUPPORTED;
 }
 
 // Returns KVSINK_ERR_UNSUPPORTED when the shape has no streaming kernel (the caller then uses the generic one).
