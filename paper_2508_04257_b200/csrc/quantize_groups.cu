@@ -104,12 +104,6 @@ __device__ __forceinline__ void pack_matrix(const uint32_t (&pc)[4], int m, uint
     }
 }
 
-// Field masks of matrix row g (pair slots r = 0, 2) in the forms pack_matrix returns, before placement.
-template <int BITS> struct RowMask;
-template <> struct RowMask<2> { static constexpr uint32_t LO = 0x00330033u, HI = 0u; };
-template <> struct RowMask<4> { static constexpr uint32_t LO = 0x0f0f0f0fu, HI = 0u; };
-template <> struct RowMask<3> { static constexpr uint32_t LO = 0x00330033u, HI = 0x00110011u; };
-
 // Reduces the lane's pairwise extremes over the eight lanes that hold the other rows (lane bits 2..4).
 __device__ __forceinline__ void reduce_rows(__half2 &mn, __half2 &mx)
 {
@@ -156,15 +150,26 @@ quantize_groups_stream(Params p, kvsink_cache c, const __half *__restrict__ k_sr
     WarpScratch &scr = scr_all[warp];
     const long n_items = (long)p.B * p.Hkv * n_groups * kinds;
 
-    auto decode_item = [&](long item, int *b, int *h, int *grp, int *kind) {
-        *kind = (int)(item % kinds); item /= kinds;
-        *grp = (int)(item % n_groups); item /= n_groups;
-        *h = (int)(item % p.Hkv);
-        *b = (int)(item / p.Hkv);
+    // item -> (kind, group, head, sequence) as mixed-radix digits; advancing by gridDim.x is a digit-wise add with carry
+    struct ItemPos { int kind, grp, h, b; };
+    auto decode_item = [&](long item) {
+        ItemPos q;
+        q.kind = (int)(item % kinds); item /= kinds;
+        q.grp = (int)(item % n_groups); item /= n_groups;
+        q.h = (int)(item % p.Hkv);
+        q.b = (int)(item / p.Hkv);
+        return q;
     };
-    auto stage = [&](long item, int buf) {
-        int b, h, grp, kind;
-        decode_item(item, &b, &h, &grp, &kind);
+    const ItemPos step = decode_item((long)gridDim.x);
+    auto advance = [&](ItemPos q) {
+        q.kind += step.kind; int cy = q.kind >= kinds; q.kind -= cy ? kinds : 0;
+        q.grp += step.grp + cy; cy = q.grp >= n_groups; q.grp -= cy ? n_groups : 0;
+        q.h += step.h + cy; cy = q.h >= p.Hkv; q.h -= cy ? p.Hkv : 0;
+        q.b += step.b + cy;
+        return q;
+    };
+    auto stage = [&](const ItemPos &q, int buf) {
+        const int b = q.b, h = q.h, grp = q.grp, kind = q.kind;
         const __half *xbase = (kind == 0 ? k_src : v_src) + b * sb + h * sh + (int64_t)(grp * G) * stt;
         __half *Xt = Xbuf + (size_t)buf * G * D;
         constexpr int RPI = THREADS / CH;             // rows per iteration: 16, so (t & 7) is the same every iteration
@@ -181,18 +186,20 @@ quantize_groups_stream(Params p, kvsink_cache c, const __half *__restrict__ k_sr
     };
 
     long item = blockIdx.x;
-    if (item < n_items) stage(item, 0);
+    ItemPos cur = decode_item(item);
+    if (item < n_items) stage(cur, 0);
     for (int it = 0; item < n_items; item += gridDim.x, ++it) {
         const int buf = it & 1;
+        const ItemPos nxt = advance(cur);
         if (item + gridDim.x < n_items) {
-            stage(item + gridDim.x, buf ^ 1);
+            stage(nxt, buf ^ 1);
             asm volatile("cp.async.wait_group 1;" ::: "memory");
         } else {
             asm volatile("cp.async.wait_group 0;" ::: "memory");
         }
         __syncthreads();   // the item's tile is in shared memory; everyone is done with the previous item's xout
-        int b, h, grp, kind;
-        decode_item(item, &b, &h, &grp, &kind);
+        const int b = cur.b, h = cur.h, grp = cur.grp, kind = cur.kind;
+        cur = nxt;
         const __half *Xt = Xbuf + (size_t)buf * G * D;
         const uint32_t *tm = tmask + buf * NT;
         const int64_t unit = (int64_t)b * p.Hkv + h;
@@ -257,17 +264,12 @@ quantize_groups_stream(Params p, kvsink_cache c, const __half *__restrict__ k_sr
                         const float2 z0 = scr.sz[4 * t4 + 2 * (r >> 1)], z1 = scr.sz[4 * t4 + 2 * (r >> 1) + 1];
                         pc[r] = code_pair_exact<BITS>(a[T][r], z0.x, z0.y, z1.x, z1.y);
                     }
+                    // sink tokens keep code 0 in the packed stream: pair slots 0, 2 are row g, slots 1, 3 row g + 8
+                    if ((m16 >> g) & 1u) pc[0] = pc[2] = 0;
+                    if ((m16 >> (g + 8)) & 1u) pc[1] = pc[3] = 0;
                 }
                 uint32_t lo, hi;
                 pack_matrix<BITS>(pc, m, &lo, &hi);
-                if (m16) {   // sink tokens keep code 0 in the packed stream
-                    uint32_t keep = 0xffffffffu, keeph = 0xffffffffu;
-                    const int hsh = 8 * (m & 1) + 2 * (1 - ((m >> 1) & 1));
-                    if ((m16 >> g) & 1u) { keep &= ~RowMask<BITS>::LO; keeph &= ~(RowMask<BITS>::HI << hsh); }
-                    if ((m16 >> (g + 8)) & 1u) { keep &= ~(RowMask<BITS>::LO << (BITS == 4 ? 4 : 2)); keeph &= ~(RowMask<BITS>::HI << (hsh + 1)); }
-                    lo &= keep;
-                    hi &= keeph;
-                }
                 uint32_t *tile = xout + T * TILE_WORDS;
                 if constexpr (BITS == 4) {
                     tile[lo_word] = lo;
