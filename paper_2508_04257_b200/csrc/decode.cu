@@ -132,8 +132,8 @@ __device__ __forceinline__ void tile_frags(const uint32_t (&w)[Geo<BITS, D>::W],
     }
 }
 
-template <int BITS, int D>
-__global__ void __launch_bounds__(DEC_THREADS)
+template <int BITS, int D, int NGv>
+__global__ void __launch_bounds__(DEC_THREADS, 4)
 decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__restrict__ out, float *__restrict__ lse,
               float *__restrict__ part_ws, int nsplit, int groups_per_split, int qchunks, int seq_len)
 {
@@ -152,7 +152,7 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
     const int nq = min(8, p.rep - 8 * qc), hq0 = h * p.rep + 8 * qc;
     const int64_t unit = (int64_t)b * p.Hkv + h;
     const int G = p.G, n = seq_len, n_groups = n / G, n_body = n_groups * G;
-    const int NGv = p.NGv, mpg = p.Gv / 16;                          // value matrices per channel group
+    constexpr int mpg = (D / NGv) / 16;                              // value matrices per channel group
     const uint32_t *bm = c.sink_bitmask + (size_t)b * p.mask_words;
     const float qscale = LOG2E * rsqrtf((float)D);
 
@@ -217,7 +217,7 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
     // ---------------- packed stream ----------------
     float m_run[2] = {M_INIT, M_INIT}, l_run[2] = {0.f, 0.f};
     float O[NM][4];
-    float bv[4][2];                       // sum p*scale*zero per value channel group and head pair
+    float bv[NGv][2];                     // sum p*scale*zero per value channel group and head pair
     int ev = 60;                          // the value B operand is p * scale * 2^ev; lowered so that it fits fp16
     float evf = pow2i(60);
 #pragma unroll
@@ -225,7 +225,7 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
 #pragma unroll
         for (int i = 0; i < 4; ++i) O[m][i] = 0.f;
 #pragma unroll
-    for (int j = 0; j < 4; ++j) bv[j][0] = bv[j][1] = 0.f;
+    for (int j = 0; j < NGv; ++j) bv[j][0] = bv[j][1] = 0.f;
 
     __half *Bs = Bs_all + (size_t)warp * 2 * 8 * BST, *Bl = Bs + 8 * BST;
     const uint8_t *kc_base = c.k_codes + (size_t)unit * p.max_seq * p.row_bytes;
@@ -233,8 +233,28 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
     const float *vs_base = c.v_scale + (size_t)unit * p.max_seq * NGv;
     const float *vz_base = c.v_zero + (size_t)unit * p.max_seq * NGv;
 
+    // What a warp needs from memory for one 16-token tile of the packed stream (prefetched one tile ahead).
+    struct TileIn {
+        uint32_t kw[W], vw[W];
+        float sv0[NGv], zv0[NGv], sv1[NGv], zv1[NGv];   // value scale / zero of tokens g and g+8
+        uint32_t mask16;
+    };
+    auto load_tile_in = [&](TileIn &ti, int T) {
+        load_tile<BITS, D>((const uint32_t *)(kc_base + (size_t)T * p.tile_bytes), lane, ti.kw);
+        load_tile<BITS, D>((const uint32_t *)(vc_base + (size_t)T * p.tile_bytes), lane, ti.vw);
+        const float *s0 = vs_base + (size_t)(T * KVSINK_TILE + g) * NGv, *z0 = vz_base + (size_t)(T * KVSINK_TILE + g) * NGv;
+#pragma unroll
+        for (int j = 0; j < NGv; ++j) {
+            ti.sv0[j] = __ldg(s0 + j); ti.zv0[j] = __ldg(z0 + j);
+            ti.sv1[j] = __ldg(s0 + 8 * NGv + j); ti.zv1[j] = __ldg(z0 + 8 * NGv + j);
+        }
+        ti.mask16 = (__ldg(bm + (T >> 1)) >> (16 * (T & 1))) & 0xffffu;
+    };
+
     // One 16-token tile: scores in s[4] (log2 units, -inf where the token does not take part) -> softmax -> values.
-    auto tile_values = [&](int T, float (&s)[4], bool v0, bool v1) {
+    // Tokens that do not take part must come with finite (or zeroed) value parameters.
+    auto tile_values = [&](float (&s)[4], const uint32_t (&vw)[W], const float (&sv0)[NGv], const float (&zv0)[NGv],
+                           const float (&sv1)[NGv], const float (&zv1)[NGv]) {
         float tm0 = fmaxf(s[0], s[2]), tm1 = fmaxf(s[1], s[3]);
 #pragma unroll
         for (int o = 4; o < 32; o <<= 1) {
@@ -246,7 +266,7 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
             const float c0 = ex2(m_run[0] - mn0), c1 = ex2(m_run[1] - mn1);
             l_run[0] *= c0; l_run[1] *= c1;
 #pragma unroll
-            for (int j = 0; j < 4; ++j) { bv[j][0] *= c0; bv[j][1] *= c1; }
+            for (int j = 0; j < NGv; ++j) { bv[j][0] *= c0; bv[j][1] *= c1; }
 #pragma unroll
             for (int m = 0; m < NM; ++m) { O[m][0] *= c0; O[m][2] *= c0; O[m][1] *= c1; O[m][3] *= c1; }
             m_run[0] = mn0; m_run[1] = mn1;
@@ -254,25 +274,17 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
         const float p0 = ex2(s[0] - mn0), p1 = ex2(s[1] - mn1), p2 = ex2(s[2] - mn0), p3 = ex2(s[3] - mn1);
         l_run[0] += p0 + p2;
         l_run[1] += p1 + p3;
-        uint32_t vw[W];
-        load_tile<BITS, D>((const uint32_t *)(vc_base + (size_t)T * p.tile_bytes), lane, vw);
         uint32_t va[NM][4];
         tile_frags<BITS, D>(vw, va);
-        const int tok0 = T * KVSINK_TILE + g, tok1 = tok0 + 8;
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            if (j < NGv) {
-                const float sv0 = v0 ? __ldg(vs_base + (size_t)tok0 * NGv + j) : 0.f, zv0 = v0 ? __ldg(vz_base + (size_t)tok0 * NGv + j) : 0.f;
-                const float sv1 = v1 ? __ldg(vs_base + (size_t)tok1 * NGv + j) : 0.f, zv1 = v1 ? __ldg(vz_base + (size_t)tok1 * NGv + j) : 0.f;
-                const float w0 = p0 * sv0, w1 = p1 * sv0, w2 = p2 * sv1, w3 = p3 * sv1;
-                bv[j][0] += w0 * zv0 + w2 * zv1;
-                bv[j][1] += w1 * zv0 + w3 * zv1;
-                const uint32_t b0 = movm_trans(pack_half2(w0 * evf, w1 * evf));
-                const uint32_t b1 = movm_trans(pack_half2(w2 * (evf / G_::COLF), w3 * (evf / G_::COLF)));
+        for (int j = 0; j < NGv; ++j) {
+            const float w0 = p0 * sv0[j], w1 = p1 * sv0[j], w2 = p2 * sv1[j], w3 = p3 * sv1[j];
+            bv[j][0] += w0 * zv0[j] + w2 * zv1[j];
+            bv[j][1] += w1 * zv0[j] + w3 * zv1[j];
+            const uint32_t b0 = movm_trans(pack_half2(w0 * evf, w1 * evf));
+            const uint32_t b1 = movm_trans(pack_half2(w2 * (evf / G_::COLF), w3 * (evf / G_::COLF)));
 #pragma unroll
-                for (int m = 0; m < NM; ++m)
-                    if (m / mpg == j) mma16816(O[m], va[m], b0, b1);
-            }
+            for (int mi = 0; mi < mpg; ++mi) mma16816(O[j * mpg + mi], va[j * mpg + mi], b0, b1);
         }
     };
 
@@ -294,15 +306,20 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
         }
     };
 
-    // ---- complete key groups of this split ----
+    // ---- complete key groups of this split: warp w takes groups g_begin + w, + DEC_WARPS, ... ----
     const int g_begin = split * groups_per_split, g_end = min(n_groups, g_begin + groups_per_split);
-    for (int grp = g_begin + warp; grp < g_end; grp += DEC_WARPS) {
-        // B operand of the group: fp16(q * scale) per channel and head, column half pre-divided by COLF;
-        // bias = sum_c fp16(q*scale) * zero with the same rounded factor.
+    const int TPG = G / KVSINK_TILE;
+    TileIn nxt;
+    int grp = g_begin + warp;
+    if (grp < g_end) load_tile_in(nxt, grp * TPG);
+    for (; grp < g_end; grp += DEC_WARPS) {
+        // B operand of the group: fp16(q * scale * 2^sh) per channel and head (sh puts the largest factor of the head
+        // in [2^13, 2^14)), column half pre-divided by COLF; bias = sum_c of the same rounded factors * zero.
         float bias[2] = {0.f, 0.f}, ksc[2] = {0.f, 0.f};
         uint32_t need_lo = 0;     // bit m: matrix m also gets the low half of the split factor (warp-uniform)
         {
             constexpr int CPL = D / 32;
+            constexpr float QMAX = (float)((1 << BITS) - 1);
             const float *sc = c.k_scale + ((size_t)unit * (p.max_seq / G) + grp) * D + lane * CPL;
             const float *ze = c.k_zero + ((size_t)unit * (p.max_seq / G) + grp) * D + lane * CPL;
             float scv[CPL], zev[CPL];
@@ -316,7 +333,7 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
 #pragma unroll
                     for (int e = 0; e < CPL; ++e) { v[e] = qs[i * D + lane * CPL + e] * scv[e]; amax = fmaxf(amax, fabsf(v[e])); }
                     amax = warp_max(amax);
-                    int sh = 13 - floor_log2(amax);                 // largest factor lands in [2^13, 2^14)
+                    int sh = 13 - floor_log2(amax);
                     sh = sh > 60 ? 60 : (sh < -60 ? -60 : sh);
                     const float f = pow2i(sh);
                     float bsum = 0.f;
@@ -329,7 +346,7 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
                         // fp16 keeps 11 bits of the factor; where that could move a score by more than ~4e-4
                         // (factor * largest |code - zero| * 2^-12) the rounding residual is kept as a second factor
                         __half lb = __float2half_rn(vf - __half2float(hb));
-                        big |= fabsf(v[e]) * (fabsf(zev[e]) + (float)((1 << BITS) - 1)) > 1.6f;
+                        big |= fabsf(v[e]) * fmaxf(fabsf(zev[e]), fabsf(QMAX - zev[e])) > 1.6f;
                         bsum += (__half2float(hb) + __half2float(lb)) * zev[e];
                         if ((ch & 8) && G_::COLF != 1.f) {
                             hb = __hmul(hb, __float2half(1.f / G_::COLF));
@@ -357,34 +374,38 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
             bk[m][1] = g < nq ? *(const uint32_t *)(Bs + g * BST + 16 * m + 2 * t + 8) : 0u;
         }
         fit_value_scale(grp * G, grp * G + G);
-        const int T0 = grp * (G / KVSINK_TILE);
-        for (int T = T0; T < T0 + G / KVSINK_TILE; ++T) {
-            uint32_t kw[W];
-            load_tile<BITS, D>((const uint32_t *)(kc_base + (size_t)T * p.tile_bytes), lane, kw);
+        constexpr float R1 = 1.f / G_::ROWF;
+        const float ks0 = ksc[0], ks1 = ksc[1], ks0r = ksc[0] * R1, ks1r = ksc[1] * R1;
+        for (int i = 0; i < TPG; ++i) {
+            const TileIn cur = nxt;
+            {   // prefetch the warp's next tile (possibly the first tile of its next group)
+                const bool last = i + 1 == TPG;
+                const int Tn = last ? (grp + DEC_WARPS) * TPG : grp * TPG + i + 1;
+                if (!last || grp + DEC_WARPS < g_end) load_tile_in(nxt, Tn);
+            }
             uint32_t ka[NM][4];
-            tile_frags<BITS, D>(kw, ka);
+            tile_frags<BITS, D>(cur.kw, ka);
             float acc[4] = {0.f, 0.f, 0.f, 0.f};
+            if (need_lo == 0) {
 #pragma unroll
-            for (int m = 0; m < NM; ++m) {
-                mma16816(acc, ka[m], bk[m][0], bk[m][1]);
-                if (need_lo & (1u << m)) {
-                    const uint32_t l0 = g < nq ? *(const uint32_t *)(Bl + g * BST + 16 * m + 2 * t) : 0u;
-                    const uint32_t l1 = g < nq ? *(const uint32_t *)(Bl + g * BST + 16 * m + 2 * t + 8) : 0u;
-                    mma16816(acc, ka[m], l0, l1);
+                for (int m = 0; m < NM; ++m) mma16816(acc, ka[m], bk[m][0], bk[m][1]);
+            } else {
+#pragma unroll
+                for (int m = 0; m < NM; ++m) {
+                    mma16816(acc, ka[m], bk[m][0], bk[m][1]);
+                    if (need_lo & (1u << m)) {
+                        const uint32_t l0 = g < nq ? *(const uint32_t *)(Bl + g * BST + 16 * m + 2 * t) : 0u;
+                        const uint32_t l1 = g < nq ? *(const uint32_t *)(Bl + g * BST + 16 * m + 2 * t + 8) : 0u;
+                        mma16816(acc, ka[m], l0, l1);
+                    }
                 }
             }
-            constexpr float R1 = 1.f / G_::ROWF;
-            float s[4] = {acc[0] * ksc[0] - bias[0], acc[1] * ksc[1] - bias[1], acc[2] * (ksc[0] * R1) - bias[0],
-                          acc[3] * (ksc[1] * R1) - bias[1]};
-            const uint32_t mask16 = (bm[T >> 1] >> (16 * (T & 1))) & 0xffffu;
-            bool v0 = true, v1 = true;
-            if (mask16) {
-                v0 = !((mask16 >> g) & 1u);
-                v1 = !((mask16 >> (g + 8)) & 1u);
-                if (!v0) s[0] = s[1] = -INFINITY;
-                if (!v1) s[2] = s[3] = -INFINITY;
+            float s[4] = {acc[0] * ks0 - bias[0], acc[1] * ks1 - bias[1], acc[2] * ks0r - bias[0], acc[3] * ks1r - bias[1]};
+            if (cur.mask16) {   // sink tokens are not part of the packed stream (their value parameters are zero)
+                if ((cur.mask16 >> g) & 1u) s[0] = s[1] = -INFINITY;
+                if ((cur.mask16 >> (g + 8)) & 1u) s[2] = s[3] = -INFINITY;
             }
-            tile_values(T, s, v0, v1);
+            tile_values(s, cur.vw, cur.sv0, cur.zv0, cur.sv1, cur.zv1);
         }
     }
 
@@ -412,7 +433,15 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
             const bool v0 = in0 && !mask_bit(bm, in0 ? tok0 : 0), v1 = in1 && !mask_bit(bm, in1 ? tok1 : 0);
             float s[4] = {v0 ? acc[0] * qscale : -INFINITY, v0 ? acc[1] * qscale : -INFINITY,
                           v1 ? acc[2] * qscale : -INFINITY, v1 ? acc[3] * qscale : -INFINITY};
-            tile_values(T, s, v0, v1);
+            uint32_t vw[W];
+            load_tile<BITS, D>((const uint32_t *)(vc_base + (size_t)T * p.tile_bytes), lane, vw);
+            float sv0[NGv], zv0[NGv], sv1[NGv], zv1[NGv];
+#pragma unroll
+            for (int j = 0; j < NGv; ++j) {   // tokens beyond the sequence have no parameters yet
+                sv0[j] = v0 ? __ldg(vs_base + (size_t)tok0 * NGv + j) : 0.f; zv0[j] = v0 ? __ldg(vz_base + (size_t)tok0 * NGv + j) : 0.f;
+                sv1[j] = v1 ? __ldg(vs_base + (size_t)tok1 * NGv + j) : 0.f; zv1[j] = v1 ? __ldg(vz_base + (size_t)tok1 * NGv + j) : 0.f;
+            }
+            tile_values(s, vw, sv0, zv0, sv1, zv1);
         }
     }
 
@@ -422,18 +451,14 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
         l_run[0] += __shfl_xor_sync(0xffffffffu, l_run[0], o);
         l_run[1] += __shfl_xor_sync(0xffffffffu, l_run[1], o);
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
+        for (int j = 0; j < NGv; ++j) {
             bv[j][0] += __shfl_xor_sync(0xffffffffu, bv[j][0], o);
             bv[j][1] += __shfl_xor_sync(0xffffffffu, bv[j][1], o);
         }
     }
 #pragma unroll
     for (int m = 0; m < NM; ++m) {
-        const int j = m / mpg;
-        float bj0 = 0.f, bj1 = 0.f;
-#pragma unroll
-        for (int jj = 0; jj < 4; ++jj)
-            if (jj == j) { bj0 = bv[jj][0]; bj1 = bv[jj][1]; }
+        const float bj0 = bv[m / mpg][0], bj1 = bv[m / mpg][1];
         const float OS0 = pow2i(24 - ev), OS1 = OS0 / G_::ROWF;
         const int ch0 = 16 * m + g, ch1 = ch0 + 8;
         if (2 * t < nq) {
@@ -529,8 +554,8 @@ size_t decode_workspace_bytes(const Params &p)
     return (size_t)p.B * p.Hq * max_splits(p) * (p.D + 2) * sizeof(float) + 16;
 }
 
-template <int BITS, int D>
-static int launch_decode_t(const Params &p, const kvsink_cache &c, const __half *q, float *out, float *lse, float *ws, cudaStream_t st)
+template <int BITS, int D, int NGV>
+static int launch_decode_n(const Params &p, const kvsink_cache &c, const __half *q, float *out, float *lse, float *ws, cudaStream_t st)
 {
     const int n_groups = c.seq_len / p.G;
     const int nsplit = choose_splits(p, n_groups);
@@ -538,7 +563,7 @@ static int launch_decode_t(const Params &p, const kvsink_cache &c, const __half 
     const int qchunks = (p.rep + 7) / 8;
     const int nq_max = p.rep < 8 ? p.rep : 8;
     const size_t smem = 8 * D * 4 + 8 * D * 2 + (size_t)DEC_WARPS * 2 * 8 * (D + 8) * 2 + (size_t)2 * DEC_WARPS * nq_max * (D + 2) * 4;
-    auto kern = decode_kernel<BITS, D>;
+    auto kern = decode_kernel<BITS, D, NGV>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return KVSINK_ERR_CUDA;
     dim3 grid(nsplit, p.Hkv * qchunks, p.B);
     kern<<<grid, DEC_THREADS, smem, st>>>(p, c, q, out, lse, ws, nsplit, gps, qchunks, c.seq_len);
@@ -548,6 +573,15 @@ static int launch_decode_t(const Params &p, const kvsink_cache &c, const __half 
         if (cudaGetLastError() != cudaSuccess) return KVSINK_ERR_CUDA;
     }
     return KVSINK_OK;
+}
+
+template <int BITS, int D>
+static int launch_decode_t(const Params &p, const kvsink_cache &c, const __half *q, float *out, float *lse, float *ws, cudaStream_t st)
+{
+    if (p.NGv == 1) return launch_decode_n<BITS, D, 1>(p, c, q, out, lse, ws, st);
+    if (p.NGv == 2) return launch_decode_n<BITS, D, 2>(p, c, q, out, lse, ws, st);
+    if (p.NGv == 4) return launch_decode_n<BITS, D, 4>(p, c, q, out, lse, ws, st);
+    return KVSINK_ERR_UNSUPPORTED;
 }
 
 int launch_decode(const Params &p, const kvsink_cache &c, const __half *q, float *out, float *lse, void *workspace,
