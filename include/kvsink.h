@@ -37,6 +37,7 @@ extern "C" {
 
 /* Bits of the device status word (kvsink_cache.status, read with kvsink_read_status). */
 #define KVSINK_STATUS_SINK_MISMATCH 1 /* a token whose mask bit is set was not found in sink_pos */
+#define KVSINK_STATUS_TIMEOUT 2       /* a bounded wait for a shared-memory bulk copy ran out; the result is invalid */
 
 /* Tokens per packed tile. */
 #define KVSINK_TILE 16

@@ -23,7 +23,11 @@ def build(force: bool = False, verbose: bool = False) -> str:
     if force or _stale():
         nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
         cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-o", LIB] + [os.path.join(CSRC, s) for s in SOURCES]
-        subprocess.run(cmd, check=True)
+        r = subprocess.run(cmd)
+        if r.returncode != 0:
+            if os.path.exists(LIB):
+                os.remove(LIB)      # never leave a stale library behind a failed build
+            raise RuntimeError(f"nvcc failed with status {r.returncode}")
     return LIB
 
 

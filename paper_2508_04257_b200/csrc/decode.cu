@@ -92,6 +92,36 @@ __device__ __forceinline__ void load_section(const uint32_t *__restrict__ sec, i
     }
 }
 
+// The same from a tile image in shared memory.
+template <int N>
+__device__ __forceinline__ void load_section_shared(const uint32_t *sec, int lane, uint32_t *w)
+{
+#pragma unroll
+    for (int p = 0; p * 4 < N; ++p) {
+        const int u = (N - 4 * p) > 4 ? 4 : (N - 4 * p);
+        const uint32_t *src = sec + u * lane;
+        if (u == 4) {
+            uint4 v = *(const uint4 *)src;
+            w[4 * p] = v.x; w[4 * p + 1] = v.y; w[4 * p + 2] = v.z; w[4 * p + 3] = v.w;
+        } else if (u == 2) {
+            uint2 v = *(const uint2 *)src;
+            w[4 * p] = v.x; w[4 * p + 1] = v.y;
+        } else {
+#pragma unroll
+            for (int i = 0; i < u; ++i) w[4 * p + i] = src[i];
+        }
+        sec += 32 * u;
+    }
+}
+
+template <int BITS, int D>
+__device__ __forceinline__ void load_tile_shared(const uint32_t *tile, int lane, uint32_t (&w)[Geo<BITS, D>::W])
+{
+    using G_ = Geo<BITS, D>;
+    load_section_shared<G_::NLO>(tile, lane, w);
+    if constexpr (BITS == 3) load_section_shared<G_::NHI>(tile + 32 * G_::NLO, lane, w + G_::NLO);
+}
+
 template <int BITS, int D>
 __device__ __forceinline__ void load_tile(const uint32_t *__restrict__ tile, int lane, uint32_t (&w)[Geo<BITS, D>::W])
 {
@@ -132,29 +162,79 @@ __device__ __forceinline__ void tile_frags(const uint32_t (&w)[Geo<BITS, D>::W],
     }
 }
 
+// ---- per-warp bulk-copy ring (TMA, cp.async.bulk) ----
+__device__ __forceinline__ void mbar_init(uint64_t *bar, unsigned count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t *bar, unsigned bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, unsigned parity)
+{
+    unsigned ok;
+    asm volatile("{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
+                 : "=r"(ok) : "r"(smem_addr(bar)), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Global -> shared bulk copy; addresses and size are multiples of 16 bytes; completion is counted on `bar`.
+__device__ __forceinline__ void bulk_g2s(void *dst, const void *src, unsigned bytes, uint64_t *bar)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(smem_addr(dst)), "l"(src), "r"(bytes), "r"(smem_addr(bar)) : "memory");
+}
+
+constexpr int DEC_WAIT_LIMIT = 1 << 22;   // polls of a full-barrier before a warp gives up (far beyond any real latency)
+
+// Shared-memory plan of a decode block, shared by the kernel and the launcher.
+template <int BITS, int D, int NGv>
+struct DecodePlan {
+    static constexpr int W = D * BITS / 64, TILE_BYTES = 128 * W;
+    static constexpr int BST = D + 8;                 // padded row stride of the key B tables (bank spread)
+    __host__ __device__ static int chunk_tiles(int tpg) { return (tpg % 2 == 0) ? 2 : 1; }
+    __host__ __device__ static int slot_bytes(int ct) { return ct * (2 * TILE_BYTES + 2 * 16 * NGv * 4); }
+    __host__ __device__ static int slots(int ct) { int n = 9216 / slot_bytes(ct); return n < 2 ? 2 : (n > 4 ? 4 : n); }
+    __host__ __device__ static size_t bytes(int nq, int tpg)
+    {
+        const int ct = chunk_tiles(tpg);
+        size_t ring = (size_t)DEC_WARPS * slots(ct) * slot_bytes(ct);
+        size_t part = (size_t)2 * DEC_WARPS * nq * (D + 2) * 4;
+        size_t fixed = 8 * D * 4 + 8 * D * 2 + (size_t)DEC_WARPS * 2 * nq * BST * 2 + DEC_WARPS * 4 * 8;
+        fixed = (fixed + 127) / 128 * 128;
+        return fixed + (ring > part ? ring : part);
+    }
+};
+
 template <int BITS, int D, int NGv>
 __global__ void __launch_bounds__(DEC_THREADS, 4)
 decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__restrict__ out, float *__restrict__ lse,
               float *__restrict__ part_ws, int nsplit, int groups_per_split, int qchunks, int seq_len)
 {
     using G_ = Geo<BITS, D>;
-    constexpr int NM = G_::NM, W = G_::W;
+    using Plan = DecodePlan<BITS, D, NGv>;
+    constexpr int NM = G_::NM, W = G_::W, BST = Plan::BST, TILE_WORDS = 32 * W;
+    constexpr int mpg = (D / NGv) / 16;                              // value matrices per channel group
     constexpr float LOG2E = 1.4426950408889634f;
-    extern __shared__ __align__(16) unsigned char smem_raw[];
-    float *qs = (float *)smem_raw;                                   // [8][D] q * log2e/sqrt(D)
-    __half *q16 = (__half *)(qs + 8 * D);                            // [8][D] q as given
-    constexpr int BST = D + 8;                                       // padded row stride of the B tables (bank spread)
-    __half *Bs_all = q16 + 8 * D;                                    // [warps][2][8][BST] key B operand (hi, lo) of the group
-    float *part = (float *)(Bs_all + DEC_WARPS * 2 * 8 * BST);       // [2*warps][nq][D+2]
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = lane >> 2, t = lane & 3;
     const int split = blockIdx.x, h = blockIdx.y / qchunks, qc = blockIdx.y % qchunks, b = blockIdx.z;
     const int nq = min(8, p.rep - 8 * qc), hq0 = h * p.rep + 8 * qc;
     const int64_t unit = (int64_t)b * p.Hkv + h;
     const int G = p.G, n = seq_len, n_groups = n / G, n_body = n_groups * G;
-    constexpr int mpg = (D / NGv) / 16;                              // value matrices per channel group
+    const int TPG = G / KVSINK_TILE, CT = Plan::chunk_tiles(TPG), CPG = TPG / CT;   // tiles per group, tiles per chunk, chunks per group
+    const int NSLOT = Plan::slots(CT), SLOT_BYTES = Plan::slot_bytes(CT);
     const uint32_t *bm = c.sink_bitmask + (size_t)b * p.mask_words;
     const float qscale = LOG2E * rsqrtf((float)D);
+
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    float *qs = (float *)smem_raw;                                   // [8][D] q * log2e/sqrt(D)
+    __half *q16 = (__half *)(qs + 8 * D);                            // [8][D] q as given
+    __half *Bs_all = q16 + 8 * D;                                    // [warps][2][nq][BST] key B operand (hi, lo) of the group
+    uint64_t *bars = (uint64_t *)(Bs_all + (size_t)DEC_WARPS * 2 * nq * BST);   // [warps][4] full barriers of the ring slots
+    const size_t fixed = ((size_t)((unsigned char *)(bars + DEC_WARPS * 4) - smem_raw) + 127) / 128 * 128;
+    unsigned char *ring_all = smem_raw + fixed;                      // [warps][NSLOT][SLOT_BYTES]; later reused for the partials
+    float *part = (float *)ring_all;                                 // [2*warps][nq][D+2]
 
     for (int i = tid; i < 8 * D; i += DEC_THREADS) {
         const int qh = i / D, ch = i % D;
@@ -162,57 +242,14 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
         q16[i] = v;
         qs[i] = __half2float(v) * qscale;
     }
+    uint64_t *my_bars = bars + warp * 4;
+    if (lane == 0) {
+        for (int i = 0; i < 4; ++i) mbar_init(&my_bars[i], 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
     __syncthreads();
 
     const int PS = D + 2;                                            // partial record: o[D], m, l
-    float *my_part = part + (size_t)(2 * warp) * nq * PS;
-
-    // ---------------- sink rows (fp16 side buffer), plain fp32 arithmetic ----------------
-    {
-        constexpr int CPL = D / 32;
-        float ms[8], ls[8], os[8][CPL];
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            ms[i] = M_INIT; ls[i] = 0.f;
-#pragma unroll
-            for (int e = 0; e < CPL; ++e) os[i][e] = 0.f;
-        }
-        const int count = min(c.sink_count[b], p.cap);
-        const int worker = split * DEC_WARPS + warp, nworkers = nsplit * DEC_WARPS;
-        for (int j = worker; j < count; j += nworkers) {
-            const int pos = c.sink_pos[(size_t)b * p.cap + j];
-            if (pos < 0 || pos >= n) continue;
-            const __half *kr = (const __half *)c.sink_k + ((size_t)unit * p.cap + j) * D + lane * CPL;
-            const __half *vr = (const __half *)c.sink_v + ((size_t)unit * p.cap + j) * D + lane * CPL;
-            float kf[CPL], vf[CPL];
-#pragma unroll
-            for (int e = 0; e < CPL; ++e) { kf[e] = __half2float(kr[e]); vf[e] = __half2float(vr[e]); }
-#pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                if (i < nq) {
-                    float d = 0.f;
-#pragma unroll
-                    for (int e = 0; e < CPL; ++e) d += qs[i * D + lane * CPL + e] * kf[e];
-                    const float s = warp_sum(d);
-                    const float mnew = fmaxf(ms[i], s);
-                    const float corr = ex2(ms[i] - mnew), pp = ex2(s - mnew);
-                    ls[i] = ls[i] * corr + pp;
-#pragma unroll
-                    for (int e = 0; e < CPL; ++e) os[i][e] = os[i][e] * corr + pp * vf[e];
-                    ms[i] = mnew;
-                }
-            }
-        }
-        float *sp = my_part + (size_t)nq * PS;
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            if (i < nq) {
-#pragma unroll
-                for (int e = 0; e < CPL; ++e) sp[i * PS + lane * CPL + e] = os[i][e];
-                if (lane == 0) { sp[i * PS + D] = ms[i]; sp[i * PS + D + 1] = ls[i]; }
-            }
-        }
-    }
 
     // ---------------- packed stream ----------------
     float m_run[2] = {M_INIT, M_INIT}, l_run[2] = {0.f, 0.f};
@@ -227,35 +264,34 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
 #pragma unroll
     for (int j = 0; j < NGv; ++j) bv[j][0] = bv[j][1] = 0.f;
 
-    __half *Bs = Bs_all + (size_t)warp * 2 * 8 * BST, *Bl = Bs + 8 * BST;
+    __half *Bs = Bs_all + (size_t)warp * 2 * nq * BST, *Bl = Bs + (size_t)nq * BST;
     const uint8_t *kc_base = c.k_codes + (size_t)unit * p.max_seq * p.row_bytes;
     const uint8_t *vc_base = c.v_codes + (size_t)unit * p.max_seq * p.row_bytes;
     const float *vs_base = c.v_scale + (size_t)unit * p.max_seq * NGv;
     const float *vz_base = c.v_zero + (size_t)unit * p.max_seq * NGv;
 
-    // What a warp needs from memory for one 16-token tile of the packed stream (prefetched one tile ahead).
-    struct TileIn {
-        uint32_t kw[W], vw[W];
-        float sv0[NGv], zv0[NGv], sv1[NGv], zv1[NGv];   // value scale / zero of tokens g and g+8
-        uint32_t mask16;
-    };
-    auto load_tile_in = [&](TileIn &ti, int T) {
-        load_tile<BITS, D>((const uint32_t *)(kc_base + (size_t)T * p.tile_bytes), lane, ti.kw);
-        load_tile<BITS, D>((const uint32_t *)(vc_base + (size_t)T * p.tile_bytes), lane, ti.vw);
-        const float *s0 = vs_base + (size_t)(T * KVSINK_TILE + g) * NGv, *z0 = vz_base + (size_t)(T * KVSINK_TILE + g) * NGv;
+    // Lowers ev so that p * scale * 2^ev stays below 2^13 for a warp-wide maximum scale mx.
+    auto fit_value_scale = [&](float mx) {
+        mx = warp_max(mx);
+        int need = 12 - floor_log2(mx);
+        need = need > 60 ? 60 : (need < -60 ? -60 : need);
+        if (need < ev) {
+            const float f = pow2i(need - ev);
 #pragma unroll
-        for (int j = 0; j < NGv; ++j) {
-            ti.sv0[j] = __ldg(s0 + j); ti.zv0[j] = __ldg(z0 + j);
-            ti.sv1[j] = __ldg(s0 + 8 * NGv + j); ti.zv1[j] = __ldg(z0 + 8 * NGv + j);
+            for (int m = 0; m < NM; ++m)
+#pragma unroll
+                for (int i = 0; i < 4; ++i) O[m][i] *= f;
+            ev = need;
+            evf = pow2i(ev);
         }
-        ti.mask16 = (__ldg(bm + (T >> 1)) >> (16 * (T & 1))) & 0xffffu;
     };
 
-    // One 16-token tile: scores in s[4] (log2 units, -inf where the token does not take part) -> softmax -> values.
-    // Tokens that do not take part must come with finite (or zeroed) value parameters.
-    auto tile_values = [&](float (&s)[4], const uint32_t (&vw)[W], const float (&sv0)[NGv], const float (&zv0)[NGv],
-                           const float (&sv1)[NGv], const float (&zv1)[NGv]) {
-        float tm0 = fmaxf(s[0], s[2]), tm1 = fmaxf(s[1], s[3]);
+    // Softmax update for NT tiles at once (scores in log2 units, -inf where a token does not take part), then the
+    // value products.  vw / sv / zv: the tiles' value words and the (scale, zero) of tokens g and g+8 of each tile.
+    auto softmax_values = [&](const int NT, float (&s)[2][4], const uint32_t (&vw)[2][W], const float (&sv)[2][2][NGv],
+                              const float (&zv)[2][2][NGv]) {
+        float tm0 = fmaxf(s[0][0], s[0][2]), tm1 = fmaxf(s[0][1], s[0][3]);
+        if (NT == 2) { tm0 = fmaxf(tm0, fmaxf(s[1][0], s[1][2])); tm1 = fmaxf(tm1, fmaxf(s[1][1], s[1][3])); }
 #pragma unroll
         for (int o = 4; o < 32; o <<= 1) {
             tm0 = fmaxf(tm0, __shfl_xor_sync(0xffffffffu, tm0, o));
@@ -271,48 +307,51 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
             for (int m = 0; m < NM; ++m) { O[m][0] *= c0; O[m][2] *= c0; O[m][1] *= c1; O[m][3] *= c1; }
             m_run[0] = mn0; m_run[1] = mn1;
         }
-        const float p0 = ex2(s[0] - mn0), p1 = ex2(s[1] - mn1), p2 = ex2(s[2] - mn0), p3 = ex2(s[3] - mn1);
-        l_run[0] += p0 + p2;
-        l_run[1] += p1 + p3;
-        uint32_t va[NM][4];
-        tile_frags<BITS, D>(vw, va);
 #pragma unroll
-        for (int j = 0; j < NGv; ++j) {
-            const float w0 = p0 * sv0[j], w1 = p1 * sv0[j], w2 = p2 * sv1[j], w3 = p3 * sv1[j];
-            bv[j][0] += w0 * zv0[j] + w2 * zv1[j];
-            bv[j][1] += w1 * zv0[j] + w3 * zv1[j];
-            const uint32_t b0 = movm_trans(pack_half2(w0 * evf, w1 * evf));
-            const uint32_t b1 = movm_trans(pack_half2(w2 * (evf / G_::COLF), w3 * (evf / G_::COLF)));
+        for (int k = 0; k < 2; ++k) {
+            if (k >= NT) break;
+            const float p0 = ex2(s[k][0] - mn0), p1 = ex2(s[k][1] - mn1), p2 = ex2(s[k][2] - mn0), p3 = ex2(s[k][3] - mn1);
+            l_run[0] += p0 + p2;
+            l_run[1] += p1 + p3;
+            uint32_t va[NM][4];
+            tile_frags<BITS, D>(vw[k], va);
 #pragma unroll
-            for (int mi = 0; mi < mpg; ++mi) mma16816(O[j * mpg + mi], va[j * mpg + mi], b0, b1);
+            for (int j = 0; j < NGv; ++j) {
+                const float w0 = p0 * sv[k][0][j], w1 = p1 * sv[k][0][j], w2 = p2 * sv[k][1][j], w3 = p3 * sv[k][1][j];
+                bv[j][0] += w0 * zv[k][0][j] + w2 * zv[k][1][j];
+                bv[j][1] += w1 * zv[k][0][j] + w3 * zv[k][1][j];
+                const uint32_t b0 = movm_trans(pack_half2(w0 * evf, w1 * evf));
+                const uint32_t b1 = movm_trans(pack_half2(w2 * (evf / G_::COLF), w3 * (evf / G_::COLF)));
+#pragma unroll
+                for (int mi = 0; mi < mpg; ++mi) mma16816(O[j * mpg + mi], va[j * mpg + mi], b0, b1);
+            }
         }
     };
 
-    // Before a span of tokens is consumed: make sure p * scale * 2^ev stays below 2^13 for every value scale in it.
-    auto fit_value_scale = [&](int tok_begin, int tok_end) {
-        float mx = 0.f;
-        for (int i = tok_begin * NGv + lane; i < tok_end * NGv; i += 32) mx = fmaxf(mx, fabsf(__ldg(vs_base + i)));
-        mx = warp_max(mx);
-        int need = 12 - floor_log2(mx);
-        need = need > 60 ? 60 : (need < -60 ? -60 : need);
-        if (need < ev) {
-            const float f = pow2i(need - ev);
-#pragma unroll
-            for (int m = 0; m < NM; ++m)
-#pragma unroll
-                for (int i = 0; i < 4; ++i) O[m][i] *= f;
-            ev = need;
-            evf = pow2i(ev);
-        }
-    };
-
-    // ---- complete key groups of this split: warp w takes groups g_begin + w, + DEC_WARPS, ... ----
+    // ---- complete key groups of this split: warp w takes groups g_begin + w, + DEC_WARPS, ...; its chunks (CT tiles
+    //      each) arrive through a ring of NSLOT bulk-copy slots, issued NSLOT - 1 chunks ahead by lane 0 ----
     const int g_begin = split * groups_per_split, g_end = min(n_groups, g_begin + groups_per_split);
-    const int TPG = G / KVSINK_TILE;
-    TileIn nxt;
-    int grp = g_begin + warp;
-    if (grp < g_end) load_tile_in(nxt, grp * TPG);
-    for (; grp < g_end; grp += DEC_WARPS) {
+    const int my_groups = g_begin + warp < g_end ? (g_end - g_begin - warp + DEC_WARPS - 1) / DEC_WARPS : 0;
+    const int my_chunks = my_groups * CPG;
+    unsigned char *ring = ring_all + (size_t)warp * NSLOT * SLOT_BYTES;
+    const int KV_BYTES = CT * Plan::TILE_BYTES, SZ_BYTES = CT * 16 * NGv * 4;
+    auto issue_chunk = [&](int ci) {      // lane 0 only
+        const int grp = g_begin + warp + (ci / CPG) * DEC_WARPS;
+        const int T0 = grp * TPG + (ci % CPG) * CT;
+        const int slot = ci % NSLOT;
+        unsigned char *dst = ring + (size_t)slot * SLOT_BYTES;
+        mbar_expect_tx(&my_bars[slot], 2 * KV_BYTES + 2 * SZ_BYTES);
+        bulk_g2s(dst, kc_base + (size_t)T0 * Plan::TILE_BYTES, KV_BYTES, &my_bars[slot]);
+        bulk_g2s(dst + KV_BYTES, vc_base + (size_t)T0 * Plan::TILE_BYTES, KV_BYTES, &my_bars[slot]);
+        bulk_g2s(dst + 2 * KV_BYTES, vs_base + (size_t)T0 * 16 * NGv, SZ_BYTES, &my_bars[slot]);
+        bulk_g2s(dst + 2 * KV_BYTES + SZ_BYTES, vz_base + (size_t)T0 * 16 * NGv, SZ_BYTES, &my_bars[slot]);
+    };
+    if (lane == 0)
+        for (int ci = 0; ci < NSLOT - 1 && ci < my_chunks; ++ci) issue_chunk(ci);
+    bool stream_ok = true;
+
+    for (int gi = 0; gi < my_groups && stream_ok; ++gi) {
+        const int grp = g_begin + warp + gi * DEC_WARPS;
         // B operand of the group: fp16(q * scale * 2^sh) per channel and head (sh puts the largest factor of the head
         // in [2^13, 2^14)), column half pre-divided by COLF; bias = sum_c of the same rounded factors * zero.
         float bias[2] = {0.f, 0.f}, ksc[2] = {0.f, 0.f};
@@ -373,39 +412,77 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
             bk[m][0] = g < nq ? *(const uint32_t *)(Bs + g * BST + 16 * m + 2 * t) : 0u;
             bk[m][1] = g < nq ? *(const uint32_t *)(Bs + g * BST + 16 * m + 2 * t + 8) : 0u;
         }
-        fit_value_scale(grp * G, grp * G + G);
         constexpr float R1 = 1.f / G_::ROWF;
         const float ks0 = ksc[0], ks1 = ksc[1], ks0r = ksc[0] * R1, ks1r = ksc[1] * R1;
-        for (int i = 0; i < TPG; ++i) {
-            const TileIn cur = nxt;
-            {   // prefetch the warp's next tile (possibly the first tile of its next group)
-                const bool last = i + 1 == TPG;
-                const int Tn = last ? (grp + DEC_WARPS) * TPG : grp * TPG + i + 1;
-                if (!last || grp + DEC_WARPS < g_end) load_tile_in(nxt, Tn);
+
+        for (int cj = 0; cj < CPG; ++cj) {
+            const int ci = gi * CPG + cj, slot = ci % NSLOT;
+            // refill the slot freed by the previous chunk, then wait for this chunk's bytes
+            __syncwarp();
+            if (lane == 0 && ci + NSLOT - 1 < my_chunks) issue_chunk(ci + NSLOT - 1);
+            {
+                const unsigned parity = (unsigned)(ci / NSLOT) & 1u;
+                int polls = 0;
+                while (!mbar_try_wait(&my_bars[slot], parity)) {
+                    if (++polls > DEC_WAIT_LIMIT) { stream_ok = false; break; }
+                }
+                stream_ok = __all_sync(0xffffffffu, stream_ok);
+                if (!stream_ok) {
+                    if (lane == 0) atomicOr(c.status, KVSINK_STATUS_TIMEOUT);
+                    break;
+                }
             }
-            uint32_t ka[NM][4];
-            tile_frags<BITS, D>(cur.kw, ka);
-            float acc[4] = {0.f, 0.f, 0.f, 0.f};
-            if (need_lo == 0) {
+            const unsigned char *sl = ring + (size_t)slot * SLOT_BYTES;
+            const float *ssv = (const float *)(sl + 2 * KV_BYTES), *szv = (const float *)(sl + 2 * KV_BYTES + SZ_BYTES);
+            // largest value scale of the chunk (one float per lane and pass)
+            {
+                float mx = 0.f;
+                for (int i = lane; i < CT * 16 * NGv; i += 32) mx = fmaxf(mx, fabsf(ssv[i]));
+                fit_value_scale(mx);
+            }
+            const int T0 = grp * TPG + cj * CT;
+            const uint32_t mword = __ldg(bm + (T0 >> 1));
+            float s[2][4];
+            uint32_t vw[2][W];
+            float sv[2][2][NGv], zv[2][2][NGv];
 #pragma unroll
-                for (int m = 0; m < NM; ++m) mma16816(acc, ka[m], bk[m][0], bk[m][1]);
-            } else {
+            for (int k = 0; k < 2; ++k) {
+                if (k < CT) {
+                    uint32_t kw[W];
+                    load_tile_shared<BITS, D>((const uint32_t *)sl + k * TILE_WORDS, lane, kw);
+                    load_tile_shared<BITS, D>((const uint32_t *)(sl + KV_BYTES) + k * TILE_WORDS, lane, vw[k]);
 #pragma unroll
-                for (int m = 0; m < NM; ++m) {
-                    mma16816(acc, ka[m], bk[m][0], bk[m][1]);
-                    if (need_lo & (1u << m)) {
-                        const uint32_t l0 = g < nq ? *(const uint32_t *)(Bl + g * BST + 16 * m + 2 * t) : 0u;
-                        const uint32_t l1 = g < nq ? *(const uint32_t *)(Bl + g * BST + 16 * m + 2 * t + 8) : 0u;
-                        mma16816(acc, ka[m], l0, l1);
+                    for (int j = 0; j < NGv; ++j) {
+                        sv[k][0][j] = ssv[(k * 16 + g) * NGv + j]; zv[k][0][j] = szv[(k * 16 + g) * NGv + j];
+                        sv[k][1][j] = ssv[(k * 16 + g + 8) * NGv + j]; zv[k][1][j] = szv[(k * 16 + g + 8) * NGv + j];
+                    }
+                    uint32_t ka[NM][4];
+                    tile_frags<BITS, D>(kw, ka);
+                    float acc[4] = {0.f, 0.f, 0.f, 0.f};
+                    if (need_lo == 0) {
+#pragma unroll
+                        for (int m = 0; m < NM; ++m) mma16816(acc, ka[m], bk[m][0], bk[m][1]);
+                    } else {
+#pragma unroll
+                        for (int m = 0; m < NM; ++m) {
+                            mma16816(acc, ka[m], bk[m][0], bk[m][1]);
+                            if (need_lo & (1u << m)) {
+                                const uint32_t l0 = g < nq ? *(const uint32_t *)(Bl + g * BST + 16 * m + 2 * t) : 0u;
+                                const uint32_t l1 = g < nq ? *(const uint32_t *)(Bl + g * BST + 16 * m + 2 * t + 8) : 0u;
+                                mma16816(acc, ka[m], l0, l1);
+                            }
+                        }
+                    }
+                    s[k][0] = acc[0] * ks0 - bias[0]; s[k][1] = acc[1] * ks1 - bias[1];
+                    s[k][2] = acc[2] * ks0r - bias[0]; s[k][3] = acc[3] * ks1r - bias[1];
+                    const uint32_t mask16 = (mword >> (16 * ((T0 + k) & 1))) & 0xffffu;
+                    if (mask16) {   // sink tokens are not part of the packed stream (their value parameters are zero)
+                        if ((mask16 >> g) & 1u) s[k][0] = s[k][1] = -INFINITY;
+                        if ((mask16 >> (g + 8)) & 1u) s[k][2] = s[k][3] = -INFINITY;
                     }
                 }
             }
-            float s[4] = {acc[0] * ks0 - bias[0], acc[1] * ks1 - bias[1], acc[2] * ks0r - bias[0], acc[3] * ks1r - bias[1]};
-            if (cur.mask16) {   // sink tokens are not part of the packed stream (their value parameters are zero)
-                if ((cur.mask16 >> g) & 1u) s[0] = s[1] = -INFINITY;
-                if ((cur.mask16 >> (g + 8)) & 1u) s[2] = s[3] = -INFINITY;
-            }
-            tile_values(s, cur.vw, cur.sv0, cur.zv0, cur.sv1, cur.zv1);
+            softmax_values(CT, s, vw, sv, zv);
         }
     }
 
@@ -414,7 +491,6 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
         const __half *tail = (const __half *)c.k_tail + (size_t)unit * G * D;
         const int T_begin = n_body / KVSINK_TILE, T_end = (n + KVSINK_TILE - 1) / KVSINK_TILE;
         for (int T = T_begin + warp; T < T_end; T += DEC_WARPS) {
-            fit_value_scale(T * KVSINK_TILE, min(n, (T + 1) * KVSINK_TILE));
             const int tok0 = T * KVSINK_TILE + g, tok1 = tok0 + 8;
             const bool in0 = tok0 < n, in1 = tok1 < n;
             const __half *r0 = tail + (size_t)(tok0 % G) * D, *r1 = tail + (size_t)(tok1 % G) * D;
@@ -431,17 +507,21 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
                 mma16816(acc, a, b0, b1);
             }
             const bool v0 = in0 && !mask_bit(bm, in0 ? tok0 : 0), v1 = in1 && !mask_bit(bm, in1 ? tok1 : 0);
-            float s[4] = {v0 ? acc[0] * qscale : -INFINITY, v0 ? acc[1] * qscale : -INFINITY,
-                          v1 ? acc[2] * qscale : -INFINITY, v1 ? acc[3] * qscale : -INFINITY};
-            uint32_t vw[W];
-            load_tile<BITS, D>((const uint32_t *)(vc_base + (size_t)T * p.tile_bytes), lane, vw);
-            float sv0[NGv], zv0[NGv], sv1[NGv], zv1[NGv];
+            float s[2][4];
+            s[0][0] = v0 ? acc[0] * qscale : -INFINITY; s[0][1] = v0 ? acc[1] * qscale : -INFINITY;
+            s[0][2] = v1 ? acc[2] * qscale : -INFINITY; s[0][3] = v1 ? acc[3] * qscale : -INFINITY;
+            uint32_t vw[2][W];
+            load_tile<BITS, D>((const uint32_t *)(vc_base + (size_t)T * p.tile_bytes), lane, vw[0]);
+            float sv[2][2][NGv], zv[2][2][NGv];
+            float mx = 0.f;
 #pragma unroll
             for (int j = 0; j < NGv; ++j) {   // tokens beyond the sequence have no parameters yet
-                sv0[j] = v0 ? __ldg(vs_base + (size_t)tok0 * NGv + j) : 0.f; zv0[j] = v0 ? __ldg(vz_base + (size_t)tok0 * NGv + j) : 0.f;
-                sv1[j] = v1 ? __ldg(vs_base + (size_t)tok1 * NGv + j) : 0.f; zv1[j] = v1 ? __ldg(vz_base + (size_t)tok1 * NGv + j) : 0.f;
+                sv[0][0][j] = v0 ? __ldg(vs_base + (size_t)tok0 * NGv + j) : 0.f; zv[0][0][j] = v0 ? __ldg(vz_base + (size_t)tok0 * NGv + j) : 0.f;
+                sv[0][1][j] = v1 ? __ldg(vs_base + (size_t)tok1 * NGv + j) : 0.f; zv[0][1][j] = v1 ? __ldg(vz_base + (size_t)tok1 * NGv + j) : 0.f;
+                mx = fmaxf(mx, fmaxf(fabsf(sv[0][0][j]), fabsf(sv[0][1][j])));
             }
-            tile_values(s, vw, sv0, zv0, sv1, zv1);
+            fit_value_scale(mx);
+            softmax_values(1, s, vw, sv, zv);
         }
     }
 
@@ -456,6 +536,8 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
             bv[j][1] += __shfl_xor_sync(0xffffffffu, bv[j][1], o);
         }
     }
+    __syncthreads();   // every warp has drained its ring: the space now holds the block's partials
+    float *my_part = part + (size_t)(2 * warp) * nq * PS;
 #pragma unroll
     for (int m = 0; m < NM; ++m) {
         const float bj0 = bv[m / mpg][0], bj1 = bv[m / mpg][1];
@@ -473,6 +555,53 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
     if (g == 0) {
         if (2 * t < nq) { my_part[(2 * t) * PS + D] = m_run[0]; my_part[(2 * t) * PS + D + 1] = l_run[0]; }
         if (2 * t + 1 < nq) { my_part[(2 * t + 1) * PS + D] = m_run[1]; my_part[(2 * t + 1) * PS + D + 1] = l_run[1]; }
+    }
+
+    // ---------------- sink rows (fp16 side buffer), plain fp32 arithmetic, spread over all warps of all splits ----------------
+    {
+        constexpr int CPL = D / 32;
+        float ms[8], ls[8], os[8][CPL];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            ms[i] = M_INIT; ls[i] = 0.f;
+#pragma unroll
+            for (int e = 0; e < CPL; ++e) os[i][e] = 0.f;
+        }
+        const int count = min(c.sink_count[b], p.cap);
+        const int worker = split * DEC_WARPS + warp, nworkers = nsplit * DEC_WARPS;
+        for (int j = worker; j < count; j += nworkers) {
+            const int pos = c.sink_pos[(size_t)b * p.cap + j];
+            if (pos < 0 || pos >= n) continue;
+            const __half *kr = (const __half *)c.sink_k + ((size_t)unit * p.cap + j) * D + lane * CPL;
+            const __half *vr = (const __half *)c.sink_v + ((size_t)unit * p.cap + j) * D + lane * CPL;
+            float kf[CPL], vf[CPL];
+#pragma unroll
+            for (int e = 0; e < CPL; ++e) { kf[e] = __half2float(kr[e]); vf[e] = __half2float(vr[e]); }
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                if (i < nq) {
+                    float d = 0.f;
+#pragma unroll
+                    for (int e = 0; e < CPL; ++e) d += qs[i * D + lane * CPL + e] * kf[e];
+                    const float sc = warp_sum(d);
+                    const float mnew = fmaxf(ms[i], sc);
+                    const float corr = ex2(ms[i] - mnew), pp = ex2(sc - mnew);
+                    ls[i] = ls[i] * corr + pp;
+#pragma unroll
+                    for (int e = 0; e < CPL; ++e) os[i][e] = os[i][e] * corr + pp * vf[e];
+                    ms[i] = mnew;
+                }
+            }
+        }
+        float *sp = my_part + (size_t)nq * PS;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            if (i < nq) {
+#pragma unroll
+                for (int e = 0; e < CPL; ++e) sp[i * PS + lane * CPL + e] = os[i][e];
+                if (lane == 0) { sp[i * PS + D] = ms[i]; sp[i * PS + D + 1] = ls[i]; }
+            }
+        }
     }
     __syncthreads();
 
@@ -562,7 +691,7 @@ static int launch_decode_n(const Params &p, const kvsink_cache &c, const __half 
     const int gps = n_groups > 0 ? (n_groups + nsplit - 1) / nsplit : 0;
     const int qchunks = (p.rep + 7) / 8;
     const int nq_max = p.rep < 8 ? p.rep : 8;
-    const size_t smem = 8 * D * 4 + 8 * D * 2 + (size_t)DEC_WARPS * 2 * 8 * (D + 8) * 2 + (size_t)2 * DEC_WARPS * nq_max * (D + 2) * 4;
+    const size_t smem = DecodePlan<BITS, D, NGV>::bytes(nq_max, p.G / KVSINK_TILE);
     auto kern = decode_kernel<BITS, D, NGV>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return KVSINK_ERR_CUDA;
     dim3 grid(nsplit, p.Hkv * qchunks, p.B);
