@@ -187,43 +187,49 @@ __device__ __forceinline__ void bulk_g2s(void *dst, const void *src, unsigned by
 
 constexpr int DEC_WAIT_LIMIT = 1 << 22;   // polls of a full-barrier before a warp gives up (far beyond any real latency)
 
-// Shared-memory plan of a decode block, shared by the kernel and the launcher.
-template <int BITS, int D, int NGv>
+// Shared-memory plan of a decode block, shared by the kernel and the launcher.  CT = tiles per ring chunk.
+template <int BITS, int D, int NGv, int CT>
 struct DecodePlan {
     static constexpr int W = D * BITS / 64, TILE_BYTES = 128 * W;
-    static constexpr int BST = D + 8;                 // padded row stride of the key B tables (bank spread)
-    __host__ __device__ static int chunk_tiles(int tpg) { return (tpg % 2 == 0) ? 2 : 1; }
-    __host__ __device__ static int slot_bytes(int ct) { return ct * (2 * TILE_BYTES + 2 * 16 * NGv * 4); }
-    __host__ __device__ static int slots(int ct) { int n = 9216 / slot_bytes(ct); return n < 2 ? 2 : (n > 4 ? 4 : n); }
-    __host__ __device__ static size_t bytes(int nq, int tpg)
+    static constexpr int BST = D + 8;                                   // padded row stride of the key B tables (bank spread)
+    static constexpr int KV_BYTES = CT * TILE_BYTES, SZ_BYTES = CT * 16 * NGv * 4;
+    static constexpr int SLOT_BYTES = 2 * KV_BYTES + 2 * SZ_BYTES;      // K words, V words, V scales, V zeros of CT tiles
+    static constexpr int NSLOT = (9216 / SLOT_BYTES >= 4) ? 4 : 2;      // power of two
+    static constexpr int KP_BYTES = 2 * D * 4;                          // key scale + zero of one group
+    static constexpr int WARP_RING = NSLOT * SLOT_BYTES + 2 * KP_BYTES;
+    __host__ __device__ static size_t fixed_bytes(int nq)
     {
-        const int ct = chunk_tiles(tpg);
-        size_t ring = (size_t)DEC_WARPS * slots(ct) * slot_bytes(ct);
-        size_t part = (size_t)2 * DEC_WARPS * nq * (D + 2) * 4;
-        size_t fixed = 8 * D * 4 + 8 * D * 2 + (size_t)DEC_WARPS * 2 * nq * BST * 2 + DEC_WARPS * 4 * 8;
-        fixed = (fixed + 127) / 128 * 128;
-        return fixed + (ring > part ? ring : part);
+        size_t f = 8 * D * 4 + 8 * D * 2 + (size_t)DEC_WARPS * 2 * nq * BST * 2 + DEC_WARPS * 8 * 8;
+        return (f + 127) / 128 * 128;
+    }
+    __host__ __device__ static size_t bytes(int nq)
+    {
+        const size_t ring = (size_t)DEC_WARPS * WARP_RING, part = (size_t)2 * DEC_WARPS * nq * (D + 2) * 4;
+        return fixed_bytes(nq) + (ring > part ? ring : part);
     }
 };
 
-template <int BITS, int D, int NGv>
+template <int BITS, int D, int NGv, int CT>
 __global__ void __launch_bounds__(DEC_THREADS, 4)
 decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__restrict__ out, float *__restrict__ lse,
               float *__restrict__ part_ws, int nsplit, int groups_per_split, int qchunks, int seq_len)
 {
     using G_ = Geo<BITS, D>;
-    using Plan = DecodePlan<BITS, D, NGv>;
+    using Plan = DecodePlan<BITS, D, NGv, CT>;
     constexpr int NM = G_::NM, W = G_::W, BST = Plan::BST, TILE_WORDS = 32 * W;
+    constexpr int NSLOT = Plan::NSLOT, SLOT_BYTES = Plan::SLOT_BYTES, KV_BYTES = Plan::KV_BYTES, SZ_BYTES = Plan::SZ_BYTES;
     constexpr int mpg = (D / NGv) / 16;                              // value matrices per channel group
+    constexpr int CPL = D / 32;                                      // channels per lane in per-channel passes
     constexpr float LOG2E = 1.4426950408889634f;
+    constexpr float QMAX = (float)((1 << BITS) - 1);
+    constexpr float R1 = 1.f / G_::ROWF, C1 = 1.f / G_::COLF;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = lane >> 2, t = lane & 3;
     const int split = blockIdx.x, h = blockIdx.y / qchunks, qc = blockIdx.y % qchunks, b = blockIdx.z;
     const int nq = min(8, p.rep - 8 * qc), hq0 = h * p.rep + 8 * qc;
     const int64_t unit = (int64_t)b * p.Hkv + h;
     const int G = p.G, n = seq_len, n_groups = n / G, n_body = n_groups * G;
-    const int TPG = G / KVSINK_TILE, CT = Plan::chunk_tiles(TPG), CPG = TPG / CT;   // tiles per group, tiles per chunk, chunks per group
-    const int NSLOT = Plan::slots(CT), SLOT_BYTES = Plan::slot_bytes(CT);
+    const int TPG = G / KVSINK_TILE, CPG = TPG / CT;                 // tiles and ring chunks per key group
     const uint32_t *bm = c.sink_bitmask + (size_t)b * p.mask_words;
     const float qscale = LOG2E * rsqrtf((float)D);
 
@@ -231,9 +237,8 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
     float *qs = (float *)smem_raw;                                   // [8][D] q * log2e/sqrt(D)
     __half *q16 = (__half *)(qs + 8 * D);                            // [8][D] q as given
     __half *Bs_all = q16 + 8 * D;                                    // [warps][2][nq][BST] key B operand (hi, lo) of the group
-    uint64_t *bars = (uint64_t *)(Bs_all + (size_t)DEC_WARPS * 2 * nq * BST);   // [warps][4] full barriers of the ring slots
-    const size_t fixed = ((size_t)((unsigned char *)(bars + DEC_WARPS * 4) - smem_raw) + 127) / 128 * 128;
-    unsigned char *ring_all = smem_raw + fixed;                      // [warps][NSLOT][SLOT_BYTES]; later reused for the partials
+    uint64_t *bars = (uint64_t *)(Bs_all + (size_t)DEC_WARPS * 2 * nq * BST);   // [warps][8]: 4 chunk slots, 2 parameter slots
+    unsigned char *ring_all = smem_raw + Plan::fixed_bytes(nq);      // [warps][WARP_RING]; later reused for the partials
     float *part = (float *)ring_all;                                 // [2*warps][nq][D+2]
 
     for (int i = tid; i < 8 * D; i += DEC_THREADS) {
@@ -242,19 +247,19 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
         q16[i] = v;
         qs[i] = __half2float(v) * qscale;
     }
-    uint64_t *my_bars = bars + warp * 4;
+    uint64_t *cbar = bars + warp * 8, *pbar = cbar + 4;              // chunk and parameter full-barriers of this warp
     if (lane == 0) {
-        for (int i = 0; i < 4; ++i) mbar_init(&my_bars[i], 1);
+        for (int i = 0; i < 6; ++i) mbar_init(&cbar[i], 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
 
-    const int PS = D + 2;                                            // partial record: o[D], m, l
+    constexpr int PS = D + 2;                                        // partial record: o[D], m, l
 
     // ---------------- packed stream ----------------
-    float m_run[2] = {M_INIT, M_INIT}, l_run[2] = {0.f, 0.f};
+    float m0 = M_INIT, m1 = M_INIT, l0 = 0.f, l1 = 0.f;             // running max / sum of query heads 2t and 2t+1
     float O[NM][4];
-    float bv[NGv][2];                     // sum p*scale*zero per value channel group and head pair
+    float bv[NGv][2];                     // sum p*scale*zero per value channel group and head
     int ev = 60;                          // the value B operand is p * scale * 2^ev; lowered so that it fits fp16
     float evf = pow2i(60);
 #pragma unroll
@@ -269,13 +274,16 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
     const uint8_t *vc_base = c.v_codes + (size_t)unit * p.max_seq * p.row_bytes;
     const float *vs_base = c.v_scale + (size_t)unit * p.max_seq * NGv;
     const float *vz_base = c.v_zero + (size_t)unit * p.max_seq * NGv;
+    const float *ks_base = c.k_scale + (size_t)unit * (p.max_seq / G) * D;
+    const float *kz_base = c.k_zero + (size_t)unit * (p.max_seq / G) * D;
 
-    // Lowers ev so that p * scale * 2^ev stays below 2^13 for a warp-wide maximum scale mx.
+    // Lowers ev so that p * scale * 2^ev stays below 2^13 for the largest |scale| mx among the lanes that share a quad column.
     auto fit_value_scale = [&](float mx) {
-        mx = warp_max(mx);
+#pragma unroll
+        for (int o = 4; o < 32; o <<= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
         int need = 12 - floor_log2(mx);
         need = need > 60 ? 60 : (need < -60 ? -60 : need);
-        if (need < ev) {
+        if (need < ev) {     // warp-uniform: every quad column holds the same tokens
             const float f = pow2i(need - ev);
 #pragma unroll
             for (int m = 0; m < NM; ++m)
@@ -285,86 +293,101 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
             evf = pow2i(ev);
         }
     };
-
-    // Softmax update for NT tiles at once (scores in log2 units, -inf where a token does not take part), then the
-    // value products.  vw / sv / zv: the tiles' value words and the (scale, zero) of tokens g and g+8 of each tile.
-    auto softmax_values = [&](const int NT, float (&s)[2][4], const uint32_t (&vw)[2][W], const float (&sv)[2][2][NGv],
-                              const float (&zv)[2][2][NGv]) {
-        float tm0 = fmaxf(s[0][0], s[0][2]), tm1 = fmaxf(s[0][1], s[0][3]);
-        if (NT == 2) { tm0 = fmaxf(tm0, fmaxf(s[1][0], s[1][2])); tm1 = fmaxf(tm1, fmaxf(s[1][1], s[1][3])); }
+    // New running maxima after a batch of scores with per-lane maxima tm0 / tm1; rescales the accumulators if needed.
+    auto advance_max = [&](float tm0, float tm1) {
 #pragma unroll
         for (int o = 4; o < 32; o <<= 1) {
             tm0 = fmaxf(tm0, __shfl_xor_sync(0xffffffffu, tm0, o));
             tm1 = fmaxf(tm1, __shfl_xor_sync(0xffffffffu, tm1, o));
         }
-        const float mn0 = fmaxf(m_run[0], tm0), mn1 = fmaxf(m_run[1], tm1);
-        if (__any_sync(0xffffffffu, mn0 > m_run[0] || mn1 > m_run[1])) {
-            const float c0 = ex2(m_run[0] - mn0), c1 = ex2(m_run[1] - mn1);
-            l_run[0] *= c0; l_run[1] *= c1;
+        const float mn0 = fmaxf(m0, tm0), mn1 = fmaxf(m1, tm1);
+        if (__any_sync(0xffffffffu, mn0 > m0 || mn1 > m1)) {
+            const float c0 = ex2(m0 - mn0), c1 = ex2(m1 - mn1);
+            l0 *= c0; l1 *= c1;
 #pragma unroll
             for (int j = 0; j < NGv; ++j) { bv[j][0] *= c0; bv[j][1] *= c1; }
 #pragma unroll
             for (int m = 0; m < NM; ++m) { O[m][0] *= c0; O[m][2] *= c0; O[m][1] *= c1; O[m][3] *= c1; }
-            m_run[0] = mn0; m_run[1] = mn1;
+            m0 = mn0; m1 = mn1;
         }
+    };
+    // Value products of one tile: scores s (log2 units, relative maxima already advanced), value words vw, and the
+    // (scale, zero) of tokens g (sv0, zv0) and g+8 (sv1, zv1) per channel group.
+    auto tile_values = [&](const float (&s)[4], const uint32_t (&vw)[W], const float (&sv0)[NGv], const float (&zv0)[NGv],
+                           const float (&sv1)[NGv], const float (&zv1)[NGv]) {
+        const float p0 = ex2(s[0] - m0), p1 = ex2(s[1] - m1), p2 = ex2(s[2] - m0), p3 = ex2(s[3] - m1);
+        l0 += p0 + p2;
+        l1 += p1 + p3;
+        uint32_t va[NM][4];
+        tile_frags<BITS, D>(vw, va);
+        const float evc = evf * C1;
 #pragma unroll
-        for (int k = 0; k < 2; ++k) {
-            if (k >= NT) break;
-            const float p0 = ex2(s[k][0] - mn0), p1 = ex2(s[k][1] - mn1), p2 = ex2(s[k][2] - mn0), p3 = ex2(s[k][3] - mn1);
-            l_run[0] += p0 + p2;
-            l_run[1] += p1 + p3;
-            uint32_t va[NM][4];
-            tile_frags<BITS, D>(vw[k], va);
+        for (int j = 0; j < NGv; ++j) {
+            const float e0 = sv0[j] * evf, e1 = sv1[j] * evc, sz0 = sv0[j] * zv0[j], sz1 = sv1[j] * zv1[j];
+            bv[j][0] = fmaf(p0, sz0, fmaf(p2, sz1, bv[j][0]));
+            bv[j][1] = fmaf(p1, sz0, fmaf(p3, sz1, bv[j][1]));
+            const uint32_t b0 = movm_trans(pack_half2(p0 * e0, p1 * e0));
+            const uint32_t b1 = movm_trans(pack_half2(p2 * e1, p3 * e1));
 #pragma unroll
-            for (int j = 0; j < NGv; ++j) {
-                const float w0 = p0 * sv[k][0][j], w1 = p1 * sv[k][0][j], w2 = p2 * sv[k][1][j], w3 = p3 * sv[k][1][j];
-                bv[j][0] += w0 * zv[k][0][j] + w2 * zv[k][1][j];
-                bv[j][1] += w1 * zv[k][0][j] + w3 * zv[k][1][j];
-                const uint32_t b0 = movm_trans(pack_half2(w0 * evf, w1 * evf));
-                const uint32_t b1 = movm_trans(pack_half2(w2 * (evf / G_::COLF), w3 * (evf / G_::COLF)));
-#pragma unroll
-                for (int mi = 0; mi < mpg; ++mi) mma16816(O[j * mpg + mi], va[j * mpg + mi], b0, b1);
-            }
+            for (int mi = 0; mi < mpg; ++mi) mma16816(O[j * mpg + mi], va[j * mpg + mi], b0, b1);
         }
     };
 
-    // ---- complete key groups of this split: warp w takes groups g_begin + w, + DEC_WARPS, ...; its chunks (CT tiles
-    //      each) arrive through a ring of NSLOT bulk-copy slots, issued NSLOT - 1 chunks ahead by lane 0 ----
+    // ---- complete key groups of this split: warp w takes groups g_begin + w, + DEC_WARPS, ...  Its chunks (CT tiles
+    //      each) arrive through a ring of NSLOT bulk-copy slots filled NSLOT - 1 chunks ahead by lane 0; the key
+    //      parameters of a group arrive one group ahead through two more slots. ----
     const int g_begin = split * groups_per_split, g_end = min(n_groups, g_begin + groups_per_split);
     const int my_groups = g_begin + warp < g_end ? (g_end - g_begin - warp + DEC_WARPS - 1) / DEC_WARPS : 0;
-    const int my_chunks = my_groups * CPG;
-    unsigned char *ring = ring_all + (size_t)warp * NSLOT * SLOT_BYTES;
-    const int KV_BYTES = CT * Plan::TILE_BYTES, SZ_BYTES = CT * 16 * NGv * 4;
-    auto issue_chunk = [&](int ci) {      // lane 0 only
-        const int grp = g_begin + warp + (ci / CPG) * DEC_WARPS;
-        const int T0 = grp * TPG + (ci % CPG) * CT;
-        const int slot = ci % NSLOT;
-        unsigned char *dst = ring + (size_t)slot * SLOT_BYTES;
-        mbar_expect_tx(&my_bars[slot], 2 * KV_BYTES + 2 * SZ_BYTES);
-        bulk_g2s(dst, kc_base + (size_t)T0 * Plan::TILE_BYTES, KV_BYTES, &my_bars[slot]);
-        bulk_g2s(dst + KV_BYTES, vc_base + (size_t)T0 * Plan::TILE_BYTES, KV_BYTES, &my_bars[slot]);
-        bulk_g2s(dst + 2 * KV_BYTES, vs_base + (size_t)T0 * 16 * NGv, SZ_BYTES, &my_bars[slot]);
-        bulk_g2s(dst + 2 * KV_BYTES + SZ_BYTES, vz_base + (size_t)T0 * 16 * NGv, SZ_BYTES, &my_bars[slot]);
+    unsigned char *ring = ring_all + (size_t)warp * Plan::WARP_RING;
+    float *kp_ring = (float *)(ring + NSLOT * SLOT_BYTES);           // [2][scale D | zero D]
+    int iss_g = 0, iss_c = 0;                                        // next chunk to issue: group index, chunk within group
+    auto issue_chunk = [&](int slot) {                               // lane 0 only
+        const int T0 = (g_begin + warp + iss_g * DEC_WARPS) * TPG + iss_c * CT;
+        unsigned char *dst = ring + slot * SLOT_BYTES;
+        mbar_expect_tx(&cbar[slot], SLOT_BYTES);
+        bulk_g2s(dst, kc_base + (size_t)T0 * Plan::TILE_BYTES, KV_BYTES, &cbar[slot]);
+        bulk_g2s(dst + KV_BYTES, vc_base + (size_t)T0 * Plan::TILE_BYTES, KV_BYTES, &cbar[slot]);
+        bulk_g2s(dst + 2 * KV_BYTES, vs_base + (size_t)T0 * 16 * NGv, SZ_BYTES, &cbar[slot]);
+        bulk_g2s(dst + 2 * KV_BYTES + SZ_BYTES, vz_base + (size_t)T0 * 16 * NGv, SZ_BYTES, &cbar[slot]);
+        if (++iss_c == CPG) { iss_c = 0; ++iss_g; }
     };
-    if (lane == 0)
-        for (int ci = 0; ci < NSLOT - 1 && ci < my_chunks; ++ci) issue_chunk(ci);
+    auto issue_params = [&](int gi) {                                // lane 0 only
+        const int grp = g_begin + warp + gi * DEC_WARPS, slot = gi & 1;
+        mbar_expect_tx(&pbar[slot], Plan::KP_BYTES);
+        bulk_g2s(kp_ring + slot * 2 * D, ks_base + (size_t)grp * D, D * 4, &pbar[slot]);
+        bulk_g2s(kp_ring + slot * 2 * D + D, kz_base + (size_t)grp * D, D * 4, &pbar[slot]);
+    };
+    auto wait_bar = [&](uint64_t *bar, unsigned parity) {
+        int polls = 0;
+        bool ok = true;
+        while (!mbar_try_wait(bar, parity)) {
+            if (++polls > DEC_WAIT_LIMIT) { ok = false; break; }
+        }
+        return __all_sync(0xffffffffu, ok);
+    };
+    if (lane == 0 && my_groups > 0) {
+        issue_params(0);
+        for (int i = 0; i < NSLOT - 1 && iss_g < my_groups; ++i) issue_chunk(i);
+    }
+    uint32_t mword_next = my_groups > 0 ? __ldg(bm + (((g_begin + warp) * TPG) >> 1)) : 0u;
     bool stream_ok = true;
+    int ci = 0;                                                      // running chunk index of this warp
 
+#pragma unroll 1
     for (int gi = 0; gi < my_groups && stream_ok; ++gi) {
         const int grp = g_begin + warp + gi * DEC_WARPS;
-        // B operand of the group: fp16(q * scale * 2^sh) per channel and head (sh puts the largest factor of the head
-        // in [2^13, 2^14)), column half pre-divided by COLF; bias = sum_c of the same rounded factors * zero.
-        float bias[2] = {0.f, 0.f}, ksc[2] = {0.f, 0.f};
+        // ---- B operand of the group: fp16(q * scale * 2^sh) per channel and head (sh puts the largest factor of the
+        //      head in [2^13, 2^14)), column half pre-divided by COLF; bias = sum_c of the same rounded factors * zero ----
+        float bias0 = 0.f, bias1 = 0.f, ks0 = 0.f, ks1 = 0.f;
         uint32_t need_lo = 0;     // bit m: matrix m also gets the low half of the split factor (warp-uniform)
         {
-            constexpr int CPL = D / 32;
-            constexpr float QMAX = (float)((1 << BITS) - 1);
-            const float *sc = c.k_scale + ((size_t)unit * (p.max_seq / G) + grp) * D + lane * CPL;
-            const float *ze = c.k_zero + ((size_t)unit * (p.max_seq / G) + grp) * D + lane * CPL;
+            __syncwarp();
+            if (lane == 0 && gi + 1 < my_groups) issue_params(gi + 1);
+            if (!wait_bar(&pbar[gi & 1], (unsigned)(gi >> 1) & 1u)) { stream_ok = false; break; }
+            const float *kp = kp_ring + (gi & 1) * 2 * D;
             float scv[CPL], zev[CPL];
 #pragma unroll
-            for (int e = 0; e < CPL; ++e) { scv[e] = __ldg(sc + e); zev[e] = __ldg(ze + e); }
-            __syncwarp();
+            for (int e = 0; e < CPL; ++e) { scv[e] = kp[lane * CPL + e]; zev[e] = kp[D + lane * CPL + e]; }
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
                 if (i < nq) {
@@ -388,8 +411,8 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
                         big |= fabsf(v[e]) * fmaxf(fabsf(zev[e]), fabsf(QMAX - zev[e])) > 1.6f;
                         bsum += (__half2float(hb) + __half2float(lb)) * zev[e];
                         if ((ch & 8) && G_::COLF != 1.f) {
-                            hb = __hmul(hb, __float2half(1.f / G_::COLF));
-                            lb = __hmul(lb, __float2half(1.f / G_::COLF));
+                            hb = __hmul(hb, __float2half(C1));
+                            lb = __hmul(lb, __float2half(C1));
                         }
                         Bs[i * BST + ch] = hb;
                         Bl[i * BST + ch] = lb;
@@ -400,8 +423,8 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
                     for (int m = 0; m < NM; ++m)
                         if ((bal >> (LPM * m)) & ((1u << LPM) - 1u)) need_lo |= 1u << m;
                     bsum = warp_sum(bsum) * pow2i(-sh);
-                    if (i == 2 * t) { bias[0] = bsum; ksc[0] = pow2i(24 - sh); }
-                    if (i == 2 * t + 1) { bias[1] = bsum; ksc[1] = pow2i(24 - sh); }
+                    if (i == 2 * t) { bias0 = bsum; ks0 = pow2i(24 - sh); }
+                    if (i == 2 * t + 1) { bias1 = bsum; ks1 = pow2i(24 - sh); }
                 }
             }
             __syncwarp();
@@ -412,79 +435,84 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
             bk[m][0] = g < nq ? *(const uint32_t *)(Bs + g * BST + 16 * m + 2 * t) : 0u;
             bk[m][1] = g < nq ? *(const uint32_t *)(Bs + g * BST + 16 * m + 2 * t + 8) : 0u;
         }
-        constexpr float R1 = 1.f / G_::ROWF;
-        const float ks0 = ksc[0], ks1 = ksc[1], ks0r = ksc[0] * R1, ks1r = ksc[1] * R1;
+        const float ks0r = ks0 * R1, ks1r = ks1 * R1;
 
-        for (int cj = 0; cj < CPG; ++cj) {
-            const int ci = gi * CPG + cj, slot = ci % NSLOT;
+#pragma unroll 1
+        for (int cj = 0; cj < CPG; ++cj, ++ci) {
+            const int slot = ci & (NSLOT - 1);
             // refill the slot freed by the previous chunk, then wait for this chunk's bytes
             __syncwarp();
-            if (lane == 0 && ci + NSLOT - 1 < my_chunks) issue_chunk(ci + NSLOT - 1);
-            {
-                const unsigned parity = (unsigned)(ci / NSLOT) & 1u;
-                int polls = 0;
-                while (!mbar_try_wait(&my_bars[slot], parity)) {
-                    if (++polls > DEC_WAIT_LIMIT) { stream_ok = false; break; }
-                }
-                stream_ok = __all_sync(0xffffffffu, stream_ok);
-                if (!stream_ok) {
-                    if (lane == 0) atomicOr(c.status, KVSINK_STATUS_TIMEOUT);
-                    break;
-                }
+            if (lane == 0 && iss_g < my_groups) issue_chunk((ci + NSLOT - 1) & (NSLOT - 1));
+            if (!wait_bar(&cbar[slot], (unsigned)(ci / NSLOT) & 1u)) { stream_ok = false; break; }
+            const uint32_t mword = mword_next;
+            {   // sink bits of the warp's next chunk, fetched one chunk ahead
+                const bool last = cj + 1 == CPG;
+                const int Tn = last ? (grp + DEC_WARPS) * TPG : grp * TPG + (cj + 1) * CT;
+                if (!last || gi + 1 < my_groups) mword_next = __ldg(bm + (Tn >> 1));
             }
-            const unsigned char *sl = ring + (size_t)slot * SLOT_BYTES;
-            const float *ssv = (const float *)(sl + 2 * KV_BYTES), *szv = (const float *)(sl + 2 * KV_BYTES + SZ_BYTES);
-            // largest value scale of the chunk (one float per lane and pass)
-            {
-                float mx = 0.f;
-                for (int i = lane; i < CT * 16 * NGv; i += 32) mx = fmaxf(mx, fabsf(ssv[i]));
-                fit_value_scale(mx);
-            }
+            const uint32_t *kt = (const uint32_t *)(ring + slot * SLOT_BYTES), *vt = kt + KV_BYTES / 4;
+            const float *ssv = (const float *)(vt + KV_BYTES / 4), *szv = ssv + SZ_BYTES / 4;
             const int T0 = grp * TPG + cj * CT;
-            const uint32_t mword = __ldg(bm + (T0 >> 1));
-            float s[2][4];
-            uint32_t vw[2][W];
-            float sv[2][2][NGv], zv[2][2][NGv];
+
+            // scores of the chunk's tiles
+            float s[CT][4];
 #pragma unroll
-            for (int k = 0; k < 2; ++k) {
-                if (k < CT) {
-                    uint32_t kw[W];
-                    load_tile_shared<BITS, D>((const uint32_t *)sl + k * TILE_WORDS, lane, kw);
-                    load_tile_shared<BITS, D>((const uint32_t *)(sl + KV_BYTES) + k * TILE_WORDS, lane, vw[k]);
+            for (int k = 0; k < CT; ++k) {
+                uint32_t kw[W], ka[NM][4];
+                load_tile_shared<BITS, D>(kt + k * TILE_WORDS, lane, kw);
+                tile_frags<BITS, D>(kw, ka);
+                float acc[4] = {0.f, 0.f, 0.f, 0.f};
+                if (need_lo == 0) {
 #pragma unroll
-                    for (int j = 0; j < NGv; ++j) {
-                        sv[k][0][j] = ssv[(k * 16 + g) * NGv + j]; zv[k][0][j] = szv[(k * 16 + g) * NGv + j];
-                        sv[k][1][j] = ssv[(k * 16 + g + 8) * NGv + j]; zv[k][1][j] = szv[(k * 16 + g + 8) * NGv + j];
-                    }
-                    uint32_t ka[NM][4];
-                    tile_frags<BITS, D>(kw, ka);
-                    float acc[4] = {0.f, 0.f, 0.f, 0.f};
-                    if (need_lo == 0) {
+                    for (int m = 0; m < NM; ++m) mma16816(acc, ka[m], bk[m][0], bk[m][1]);
+                } else {
 #pragma unroll
-                        for (int m = 0; m < NM; ++m) mma16816(acc, ka[m], bk[m][0], bk[m][1]);
-                    } else {
-#pragma unroll
-                        for (int m = 0; m < NM; ++m) {
-                            mma16816(acc, ka[m], bk[m][0], bk[m][1]);
-                            if (need_lo & (1u << m)) {
-                                const uint32_t l0 = g < nq ? *(const uint32_t *)(Bl + g * BST + 16 * m + 2 * t) : 0u;
-                                const uint32_t l1 = g < nq ? *(const uint32_t *)(Bl + g * BST + 16 * m + 2 * t + 8) : 0u;
-                                mma16816(acc, ka[m], l0, l1);
-                            }
+                    for (int m = 0; m < NM; ++m) {
+                        mma16816(acc, ka[m], bk[m][0], bk[m][1]);
+                        if (need_lo & (1u << m)) {
+                            const uint32_t h0 = g < nq ? *(const uint32_t *)(Bl + g * BST + 16 * m + 2 * t) : 0u;
+                            const uint32_t h1 = g < nq ? *(const uint32_t *)(Bl + g * BST + 16 * m + 2 * t + 8) : 0u;
+                            mma16816(acc, ka[m], h0, h1);
                         }
                     }
-                    s[k][0] = acc[0] * ks0 - bias[0]; s[k][1] = acc[1] * ks1 - bias[1];
-                    s[k][2] = acc[2] * ks0r - bias[0]; s[k][3] = acc[3] * ks1r - bias[1];
-                    const uint32_t mask16 = (mword >> (16 * ((T0 + k) & 1))) & 0xffffu;
-                    if (mask16) {   // sink tokens are not part of the packed stream (their value parameters are zero)
-                        if ((mask16 >> g) & 1u) s[k][0] = s[k][1] = -INFINITY;
-                        if ((mask16 >> (g + 8)) & 1u) s[k][2] = s[k][3] = -INFINITY;
-                    }
+                }
+                s[k][0] = fmaf(acc[0], ks0, -bias0); s[k][1] = fmaf(acc[1], ks1, -bias1);
+                s[k][2] = fmaf(acc[2], ks0r, -bias0); s[k][3] = fmaf(acc[3], ks1r, -bias1);
+                const uint32_t mask16 = (mword >> (16 * ((T0 + k) & 1))) & 0xffffu;
+                if (mask16) {   // sink tokens are not part of the packed stream (their value parameters are zero)
+                    if ((mask16 >> g) & 1u) s[k][0] = s[k][1] = -INFINITY;
+                    if ((mask16 >> (g + 8)) & 1u) s[k][2] = s[k][3] = -INFINITY;
                 }
             }
-            softmax_values(CT, s, vw, sv, zv);
+            // one softmax step for the whole chunk
+            {
+                float tm0 = fmaxf(s[0][0], s[0][2]), tm1 = fmaxf(s[0][1], s[0][3]);
+                if (CT == 2) { tm0 = fmaxf(tm0, fmaxf(s[CT - 1][0], s[CT - 1][2])); tm1 = fmaxf(tm1, fmaxf(s[CT - 1][1], s[CT - 1][3])); }
+                advance_max(tm0, tm1);
+            }
+            // value scales of this lane's tokens; their maximum bounds the fp16 range needed
+            float sv0[CT][NGv], zv0[CT][NGv], sv1[CT][NGv], zv1[CT][NGv];
+            {
+                float mx = 0.f;
+#pragma unroll
+                for (int k = 0; k < CT; ++k)
+#pragma unroll
+                    for (int j = 0; j < NGv; ++j) {
+                        sv0[k][j] = ssv[(k * 16 + g) * NGv + j]; zv0[k][j] = szv[(k * 16 + g) * NGv + j];
+                        sv1[k][j] = ssv[(k * 16 + g + 8) * NGv + j]; zv1[k][j] = szv[(k * 16 + g + 8) * NGv + j];
+                        mx = fmaxf(mx, fmaxf(fabsf(sv0[k][j]), fabsf(sv1[k][j])));
+                    }
+                fit_value_scale(mx);
+            }
+#pragma unroll
+            for (int k = 0; k < CT; ++k) {
+                uint32_t vw[W];
+                load_tile_shared<BITS, D>(vt + k * TILE_WORDS, lane, vw);
+                tile_values(s[k], vw, sv0[k], zv0[k], sv1[k], zv1[k]);
+            }
         }
     }
+    if (!stream_ok && lane == 0) atomicOr(c.status, KVSINK_STATUS_TIMEOUT);
 
     // ---- tokens of the open group: keys from the fp16 tail (last split only) ----
     if (split == nsplit - 1) {
@@ -507,29 +535,30 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
                 mma16816(acc, a, b0, b1);
             }
             const bool v0 = in0 && !mask_bit(bm, in0 ? tok0 : 0), v1 = in1 && !mask_bit(bm, in1 ? tok1 : 0);
-            float s[2][4];
-            s[0][0] = v0 ? acc[0] * qscale : -INFINITY; s[0][1] = v0 ? acc[1] * qscale : -INFINITY;
-            s[0][2] = v1 ? acc[2] * qscale : -INFINITY; s[0][3] = v1 ? acc[3] * qscale : -INFINITY;
-            uint32_t vw[2][W];
-            load_tile<BITS, D>((const uint32_t *)(vc_base + (size_t)T * p.tile_bytes), lane, vw[0]);
-            float sv[2][2][NGv], zv[2][2][NGv];
+            float s[4];
+            s[0] = v0 ? acc[0] * qscale : -INFINITY; s[1] = v0 ? acc[1] * qscale : -INFINITY;
+            s[2] = v1 ? acc[2] * qscale : -INFINITY; s[3] = v1 ? acc[3] * qscale : -INFINITY;
+            advance_max(fmaxf(s[0], s[2]), fmaxf(s[1], s[3]));
+            uint32_t vw[W];
+            load_tile<BITS, D>((const uint32_t *)(vc_base + (size_t)T * p.tile_bytes), lane, vw);
+            float sv0[NGv], zv0[NGv], sv1[NGv], zv1[NGv];
             float mx = 0.f;
 #pragma unroll
             for (int j = 0; j < NGv; ++j) {   // tokens beyond the sequence have no parameters yet
-                sv[0][0][j] = v0 ? __ldg(vs_base + (size_t)tok0 * NGv + j) : 0.f; zv[0][0][j] = v0 ? __ldg(vz_base + (size_t)tok0 * NGv + j) : 0.f;
-                sv[0][1][j] = v1 ? __ldg(vs_base + (size_t)tok1 * NGv + j) : 0.f; zv[0][1][j] = v1 ? __ldg(vz_base + (size_t)tok1 * NGv + j) : 0.f;
-                mx = fmaxf(mx, fmaxf(fabsf(sv[0][0][j]), fabsf(sv[0][1][j])));
+                sv0[j] = v0 ? __ldg(vs_base + (size_t)tok0 * NGv + j) : 0.f; zv0[j] = v0 ? __ldg(vz_base + (size_t)tok0 * NGv + j) : 0.f;
+                sv1[j] = v1 ? __ldg(vs_base + (size_t)tok1 * NGv + j) : 0.f; zv1[j] = v1 ? __ldg(vz_base + (size_t)tok1 * NGv + j) : 0.f;
+                mx = fmaxf(mx, fmaxf(fabsf(sv0[j]), fabsf(sv1[j])));
             }
             fit_value_scale(mx);
-            softmax_values(1, s, vw, sv, zv);
+            tile_values(s, vw, sv0, zv0, sv1, zv1);
         }
     }
 
     // ---- this warp's packed partial: finish the reductions over the token lanes, convert units ----
 #pragma unroll
     for (int o = 4; o < 32; o <<= 1) {
-        l_run[0] += __shfl_xor_sync(0xffffffffu, l_run[0], o);
-        l_run[1] += __shfl_xor_sync(0xffffffffu, l_run[1], o);
+        l0 += __shfl_xor_sync(0xffffffffu, l0, o);
+        l1 += __shfl_xor_sync(0xffffffffu, l1, o);
 #pragma unroll
         for (int j = 0; j < NGv; ++j) {
             bv[j][0] += __shfl_xor_sync(0xffffffffu, bv[j][0], o);
@@ -538,28 +567,29 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
     }
     __syncthreads();   // every warp has drained its ring: the space now holds the block's partials
     float *my_part = part + (size_t)(2 * warp) * nq * PS;
+    {
+        const float OS0 = pow2i(24 - ev), OS1 = OS0 * R1;
 #pragma unroll
-    for (int m = 0; m < NM; ++m) {
-        const float bj0 = bv[m / mpg][0], bj1 = bv[m / mpg][1];
-        const float OS0 = pow2i(24 - ev), OS1 = OS0 / G_::ROWF;
-        const int ch0 = 16 * m + g, ch1 = ch0 + 8;
-        if (2 * t < nq) {
-            my_part[(2 * t) * PS + ch0] = O[m][0] * OS0 - bj0;
-            my_part[(2 * t) * PS + ch1] = O[m][2] * OS1 - bj0;
+        for (int m = 0; m < NM; ++m) {
+            const float bj0 = bv[m / mpg][0], bj1 = bv[m / mpg][1];
+            const int ch0 = 16 * m + g, ch1 = ch0 + 8;
+            if (2 * t < nq) {
+                my_part[(2 * t) * PS + ch0] = O[m][0] * OS0 - bj0;
+                my_part[(2 * t) * PS + ch1] = O[m][2] * OS1 - bj0;
+            }
+            if (2 * t + 1 < nq) {
+                my_part[(2 * t + 1) * PS + ch0] = O[m][1] * OS0 - bj1;
+                my_part[(2 * t + 1) * PS + ch1] = O[m][3] * OS1 - bj1;
+            }
         }
-        if (2 * t + 1 < nq) {
-            my_part[(2 * t + 1) * PS + ch0] = O[m][1] * OS0 - bj1;
-            my_part[(2 * t + 1) * PS + ch1] = O[m][3] * OS1 - bj1;
+        if (g == 0) {
+            if (2 * t < nq) { my_part[(2 * t) * PS + D] = m0; my_part[(2 * t) * PS + D + 1] = l0; }
+            if (2 * t + 1 < nq) { my_part[(2 * t + 1) * PS + D] = m1; my_part[(2 * t + 1) * PS + D + 1] = l1; }
         }
-    }
-    if (g == 0) {
-        if (2 * t < nq) { my_part[(2 * t) * PS + D] = m_run[0]; my_part[(2 * t) * PS + D + 1] = l_run[0]; }
-        if (2 * t + 1 < nq) { my_part[(2 * t + 1) * PS + D] = m_run[1]; my_part[(2 * t + 1) * PS + D + 1] = l_run[1]; }
     }
 
     // ---------------- sink rows (fp16 side buffer), plain fp32 arithmetic, spread over all warps of all splits ----------------
     {
-        constexpr int CPL = D / 32;
         float ms[8], ls[8], os[8][CPL];
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
@@ -683,16 +713,16 @@ size_t decode_workspace_bytes(const Params &p)
     return (size_t)p.B * p.Hq * max_splits(p) * (p.D + 2) * sizeof(float) + 16;
 }
 
-template <int BITS, int D, int NGV>
-static int launch_decode_n(const Params &p, const kvsink_cache &c, const __half *q, float *out, float *lse, float *ws, cudaStream_t st)
+template <int BITS, int D, int NGV, int CT>
+static int launch_decode_c(const Params &p, const kvsink_cache &c, const __half *q, float *out, float *lse, float *ws, cudaStream_t st)
 {
     const int n_groups = c.seq_len / p.G;
     const int nsplit = choose_splits(p, n_groups);
     const int gps = n_groups > 0 ? (n_groups + nsplit - 1) / nsplit : 0;
     const int qchunks = (p.rep + 7) / 8;
     const int nq_max = p.rep < 8 ? p.rep : 8;
-    const size_t smem = DecodePlan<BITS, D, NGV>::bytes(nq_max, p.G / KVSINK_TILE);
-    auto kern = decode_kernel<BITS, D, NGV>;
+    const size_t smem = DecodePlan<BITS, D, NGV, CT>::bytes(nq_max);
+    auto kern = decode_kernel<BITS, D, NGV, CT>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return KVSINK_ERR_CUDA;
     dim3 grid(nsplit, p.Hkv * qchunks, p.B);
     kern<<<grid, DEC_THREADS, smem, st>>>(p, c, q, out, lse, ws, nsplit, gps, qchunks, c.seq_len);
@@ -702,6 +732,14 @@ static int launch_decode_n(const Params &p, const kvsink_cache &c, const __half 
         if (cudaGetLastError() != cudaSuccess) return KVSINK_ERR_CUDA;
     }
     return KVSINK_OK;
+}
+
+template <int BITS, int D, int NGV>
+static int launch_decode_n(const Params &p, const kvsink_cache &c, const __half *q, float *out, float *lse, float *ws, cudaStream_t st)
+{
+    // ring chunks of two tiles when a key group has an even number of tiles (G a multiple of 32), else of one
+    if ((p.G / KVSINK_TILE) % 2 == 0) return launch_decode_c<BITS, D, NGV, 2>(p, c, q, out, lse, ws, st);
+    return launch_decode_c<BITS, D, NGV, 1>(p, c, q, out, lse, ws, st);
 }
 
 template <int BITS, int D>
