@@ -277,10 +277,12 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
     const float *ks_base = c.k_scale + (size_t)unit * (p.max_seq / G) * D;
     const float *kz_base = c.k_zero + (size_t)unit * (p.max_seq / G) * D;
 
-    // Lowers ev so that p * scale * 2^ev stays below 2^13 for the largest |scale| mx among the lanes that share a quad column.
+    // Lowers ev so that p * scale * 2^ev stays below 2^13 for the largest |scale| mx any lane has seen.
+    // ev_limit = 2^(13 - ev): scales below it need no action, which is the common case and costs one vote.
+    float ev_limit = 0.f;
     auto fit_value_scale = [&](float mx) {
-#pragma unroll
-        for (int o = 4; o < 32; o <<= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+        if (!__any_sync(0xffffffffu, mx >= ev_limit)) return;
+        mx = warp_max(mx);
         int need = 12 - floor_log2(mx);
         need = need > 60 ? 60 : (need < -60 ? -60 : need);
         if (need < ev) {     // warp-uniform: every quad column holds the same tokens
@@ -291,25 +293,26 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
                 for (int i = 0; i < 4; ++i) O[m][i] *= f;
             ev = need;
             evf = pow2i(ev);
+            ev_limit = pow2i(13 - ev);
         }
     };
     // New running maxima after a batch of scores with per-lane maxima tm0 / tm1; rescales the accumulators if needed.
+    // Once the running maxima have settled no lane exceeds them and the step costs one vote.
     auto advance_max = [&](float tm0, float tm1) {
+        if (!__any_sync(0xffffffffu, tm0 > m0 || tm1 > m1)) return;
 #pragma unroll
         for (int o = 4; o < 32; o <<= 1) {
             tm0 = fmaxf(tm0, __shfl_xor_sync(0xffffffffu, tm0, o));
             tm1 = fmaxf(tm1, __shfl_xor_sync(0xffffffffu, tm1, o));
         }
         const float mn0 = fmaxf(m0, tm0), mn1 = fmaxf(m1, tm1);
-        if (__any_sync(0xffffffffu, mn0 > m0 || mn1 > m1)) {
-            const float c0 = ex2(m0 - mn0), c1 = ex2(m1 - mn1);
-            l0 *= c0; l1 *= c1;
+        const float c0 = ex2(m0 - mn0), c1 = ex2(m1 - mn1);
+        l0 *= c0; l1 *= c1;
 #pragma unroll
-            for (int j = 0; j < NGv; ++j) { bv[j][0] *= c0; bv[j][1] *= c1; }
+        for (int j = 0; j < NGv; ++j) { bv[j][0] *= c0; bv[j][1] *= c1; }
 #pragma unroll
-            for (int m = 0; m < NM; ++m) { O[m][0] *= c0; O[m][2] *= c0; O[m][1] *= c1; O[m][3] *= c1; }
-            m0 = mn0; m1 = mn1;
-        }
+        for (int m = 0; m < NM; ++m) { O[m][0] *= c0; O[m][2] *= c0; O[m][1] *= c1; O[m][3] *= c1; }
+        m0 = mn0; m1 = mn1;
     };
     // Value products of one tile: scores s (log2 units, relative maxima already advanced), value words vw, and the
     // (scale, zero) of tokens g (sv0, zv0) and g+8 (sv1, zv1) per channel group.
@@ -478,8 +481,11 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
                 }
                 s[k][0] = fmaf(acc[0], ks0, -bias0); s[k][1] = fmaf(acc[1], ks1, -bias1);
                 s[k][2] = fmaf(acc[2], ks0r, -bias0); s[k][3] = fmaf(acc[3], ks1r, -bias1);
-                const uint32_t mask16 = (mword >> (16 * ((T0 + k) & 1))) & 0xffffu;
-                if (mask16) {   // sink tokens are not part of the packed stream (their value parameters are zero)
+            }
+            if (mword) {   // sink tokens are not part of the packed stream (their value parameters are zero)
+#pragma unroll
+                for (int k = 0; k < CT; ++k) {
+                    const uint32_t mask16 = (mword >> (16 * ((T0 + k) & 1))) & 0xffffu;
                     if ((mask16 >> g) & 1u) s[k][0] = s[k][1] = -INFINITY;
                     if ((mask16 >> (g + 8)) & 1u) s[k][2] = s[k][3] = -INFINITY;
                 }
