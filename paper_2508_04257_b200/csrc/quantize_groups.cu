@@ -104,6 +104,57 @@ __device__ __forceinline__ void pack_matrix(const uint32_t (&pc)[4], int m, uint
     }
 }
 
+// ---- 2-bit coder by thresholds ----
+// code(x) = clamp(rint(x / scale) + zero, 0, 3) is a non-decreasing step function of x, and x is fp16: three fp16
+// thresholds t1 <= t2 <= t3 (the smallest values whose code reaches 1, 2, 3) describe it exactly, and
+// code(x) = [x >= t1] + [x >= t2] + [x >= t3] needs no division, no rounding guard and no conversion.
+// fp16 values in sorted order: sign-magnitude bit pattern -> signed integer (both zeros map to 0).
+__device__ __forceinline__ int h_ord(unsigned b) { return (b & 0x8000u) ? -(int)(b & 0x7fffu) : (int)b; }
+__device__ __forceinline__ unsigned h_unord(int o) { return o >= 0 ? (unsigned)o : (0x8000u | (unsigned)(-o)); }
+__device__ __forceinline__ float h_val(int o) { return __half2float(__ushort_as_half((unsigned short)h_unord(o))); }
+
+// Bit pattern of the smallest finite fp16 value whose code under (scale, zero) is at least `level` (1..qmax), found by
+// evaluating the literal formula around a closed-form estimate; +inf if no finite value reaches it.
+__device__ __noinline__ unsigned code_threshold(float s, float z, int level, float qmax)
+{
+    constexpr int OMAX = 0x7BFF;
+    if (s == 0.f) return 0x7C00u;
+    float est = s * ((float)level - 0.5f - z);
+    est = fminf(fmaxf(est, -65504.f), 65504.f);
+    int o = h_ord(__half_as_ushort(__float2half_ru(est)));
+    bool done = false;
+#pragma unroll 1
+    for (int it = 0; it < 6 && !done; ++it) {
+        if (o > OMAX) return 0x7C00u;
+        if ((int)code_exact(h_val(o), s, z, qmax) >= level) done = true; else ++o;
+    }
+    if (done) {
+        done = false;
+#pragma unroll 1
+        for (int it = 0; it < 6 && !done; ++it) {
+            if (o - 1 < -OMAX || (int)code_exact(h_val(o - 1), s, z, qmax) < level) done = true; else --o;
+        }
+    }
+    if (!done) {   // estimate far off (does not happen for sane parameters): bisection over all finite fp16 values
+        int lo = -OMAX, hi = OMAX + 1;   // invariant: code(lo - 1) < level (vacuous at the bottom), code(hi) >= level or hi beyond the top
+        while (lo < hi) {
+            const int mid = (lo + hi) >> 1;
+            if ((int)code_exact(h_val(mid), s, z, qmax) >= level) hi = mid; else lo = mid + 1;
+        }
+        o = lo;
+        if (o > OMAX) return 0x7C00u;
+    }
+    return h_unord(o);
+}
+
+// Codes of the two elements of a half2 register, positioned: returns acc + w * ([x>=t1] + [x>=t2] + [x>=t3]) per half.
+__device__ __forceinline__ __half2 thermo_accumulate(__half2 acc, uint32_t x2, const __half2 (&t)[3], __half2 w)
+{
+    const __half2 x = *reinterpret_cast<const __half2 *>(&x2);
+    const __half2 cnt = __hadd2(__hadd2(__hge2(x, t[0]), __hge2(x, t[1])), __hge2(x, t[2]));
+    return __hfma2(cnt, w, acc);
+}
+
 // Reduces the lane's pairwise extremes over the eight lanes that hold the other rows (lane bits 2..4).
 __device__ __forceinline__ void reduce_rows(__half2 &mn, __half2 &mx)
 {
@@ -121,6 +172,7 @@ __device__ __forceinline__ void reduce_rows(__half2 &mn, __half2 &mx)
 struct WarpScratch {
     Coder coder[16];
     float2 sz[16];   // (scale, zero) for the exact path
+    __half2 thr[4][2][4];   // 2 bit: thresholds [lane&3][column half][level-1]; the halves are the pair's two keys
 };
 
 template <int BITS, int D, int G>
@@ -220,64 +272,111 @@ quantize_groups_stream(Params p, kvsink_cache c, const __half *__restrict__ k_sr
 #pragma unroll
             for (int T = 0; T < NT; ++T) {
                 const uint32_t m16 = tm[T];
-                const bool r0 = !((m16 >> g) & 1u), r1 = !((m16 >> (g + 8)) & 1u);
                 const __half2 *h = reinterpret_cast<const __half2 *>(a[T]);
-                if (m16 == 0 || r0) { mnA = __hmin2(mnA, h[0]); mxA = __hmax2(mxA, h[0]); mnB = __hmin2(mnB, h[2]); mxB = __hmax2(mxB, h[2]); }
-                if (m16 == 0 || r1) { mnA = __hmin2(mnA, h[1]); mxA = __hmax2(mxA, h[1]); mnB = __hmin2(mnB, h[3]); mxB = __hmax2(mxB, h[3]); }
+                if (m16 == 0) {   // block-uniform, the common case
+                    mnA = __hmin2(mnA, __hmin2(h[0], h[1])); mxA = __hmax2(mxA, __hmax2(h[0], h[1]));
+                    mnB = __hmin2(mnB, __hmin2(h[2], h[3])); mxB = __hmax2(mxB, __hmax2(h[2], h[3]));
+                } else {
+                    if (!((m16 >> g) & 1u)) { mnA = __hmin2(mnA, h[0]); mxA = __hmax2(mxA, h[0]); mnB = __hmin2(mnB, h[2]); mxB = __hmax2(mxB, h[2]); }
+                    if (!((m16 >> (g + 8)) & 1u)) { mnA = __hmin2(mnA, h[1]); mxA = __hmax2(mxA, h[1]); mnB = __hmin2(mnB, h[3]); mxB = __hmax2(mxB, h[3]); }
+                }
             }
             reduce_rows(mnA, mxA);
             reduce_rows(mnB, mxB);
-            // parameters (Eq. 10-11): lanes with g < 4 each take one of the four channels of their column group
-            if (g < 4) {
-                const __half2 mn2 = (g & 2) ? mnB : mnA, mx2 = (g & 2) ? mxB : mxA;
-                const __half lo = (g & 1) ? __high2half(mn2) : __low2half(mn2), hi = (g & 1) ? __high2half(mx2) : __low2half(mx2);
+            // parameters (Eq. 10-11): the lanes of a column group share its four channels (key g & 3)
+            {
+                const int kq = g & 3;
+                const __half2 mn2 = (kq & 2) ? mnB : mnA, mx2 = (kq & 2) ? mxB : mxA;
+                const __half lo = (kq & 1) ? __high2half(mn2) : __low2half(mn2), hi = (kq & 1) ? __high2half(mx2) : __low2half(mx2);
                 const bool any = __half_as_ushort(lo) != 0x7C00;
                 const float mn = __half2float(lo), mx = __half2float(hi);
                 float s, z;
                 group_params(any, mn, mx, qmax, &s, &z);
-                scr.coder[4 * t4 + g] = make_coder(s, z, mn, mx, qmax);
-                scr.sz[4 * t4 + g] = make_float2(s, z);
-                const int ch = 16 * m + 2 * t4 + (g & 1) + 8 * (g >> 1);
-                const size_t o = ((size_t)unit * (p.max_seq / G) + p0 / G) * D + ch;
-                c.k_scale[o] = s;
-                c.k_zero[o] = z;
+                if (g < 4) {
+                    if constexpr (BITS != 2) scr.coder[4 * t4 + kq] = make_coder(s, z, mn, mx, qmax);
+                    scr.sz[4 * t4 + kq] = make_float2(s, z);
+                    const int ch = 16 * m + 2 * t4 + (kq & 1) + 8 * (kq >> 1);
+                    const size_t o = ((size_t)unit * (p.max_seq / G) + p0 / G) * D + ch;
+                    c.k_scale[o] = s;
+                    c.k_zero[o] = z;
+                }
+                if constexpr (BITS == 2) {   // lanes g < 4 find levels 1 and 2 of their key, lanes g >= 4 level 3
+                    __half *th = reinterpret_cast<__half *>(&scr.thr[t4][kq >> 1][0]) + (kq & 1);
+                    if (g < 4) {
+                        th[0] = __ushort_as_half((unsigned short)code_threshold(s, z, 1, qmax));
+                        th[2] = __ushort_as_half((unsigned short)code_threshold(s, z, 2, qmax));
+                    } else {
+                        th[4] = __ushort_as_half((unsigned short)code_threshold(s, z, 3, qmax));
+                    }
+                }
             }
             __syncwarp();
-            Coder kc[4];
-#pragma unroll
-            for (int q = 0; q < 4; ++q) kc[q] = scr.coder[4 * t4 + q];
             const int lo_word = (BITS == 4) ? section_word_offset(NLO, lane, m) : section_word_offset(NLO, lane, m >> 1);
-            const int hi_word = (BITS == 3) ? 32 * NLO + section_word_offset(NHI > 0 ? NHI : 1, lane, m >> 2) : 0;
-            if constexpr (BITS == 3) {   // hi words are OR-ed together by the four warps that share them
-                for (int i = tid; i < 32 * NHI * NT; i += THREADS) xout[(i / (32 * NHI)) * TILE_WORDS + 32 * NLO + i % (32 * NHI)] = 0;
-                __syncthreads();
-            }
+            if constexpr (BITS == 2) {
+                __half2 tA[3], tB[3];
 #pragma unroll
-            for (int T = 0; T < NT; ++T) {
-                uint32_t pc[4], differ = 0;
+                for (int j = 0; j < 3; ++j) { tA[j] = scr.thr[t4][0][j]; tB[j] = scr.thr[t4][1][j]; }
+                const __half2 base = __half2half2(__float2half(1024.f));
+                const __half2 w0 = __half2half2(__float2half(1.f)), w1 = __half2half2(__float2half(4.f));
+                const __half2 w2 = __half2half2(__float2half(16.f)), w3 = __half2half2(__float2half(64.f));
+                const __half2 zero2 = __half2half2(__float2half(0.f));
 #pragma unroll
-                for (int r = 0; r < 4; ++r) pc[r] = code_pair<BITS>(a[T][r], kc[2 * (r >> 1)], kc[2 * (r >> 1) + 1], differ);
-                const uint32_t m16 = tm[T];
-                if (differ | m16) {   // rare: a value too close to a rounding tie, or a tile with sink tokens
-#pragma unroll
-                    for (int r = 0; r < 4; ++r) {
-                        const float2 z0 = scr.sz[4 * t4 + 2 * (r >> 1)], z1 = scr.sz[4 * t4 + 2 * (r >> 1) + 1];
-                        pc[r] = code_pair_exact<BITS>(a[T][r], z0.x, z0.y, z1.x, z1.y);
+                for (int T = 0; T < NT; ++T) {
+                    const uint32_t m16 = tm[T];
+                    __half2 acc = base;
+                    if (m16 == 0) {
+                        acc = thermo_accumulate(acc, a[T][0], tA, w0);
+                        acc = thermo_accumulate(acc, a[T][1], tA, w1);
+                        acc = thermo_accumulate(acc, a[T][2], tB, w2);
+                        acc = thermo_accumulate(acc, a[T][3], tB, w3);
+                    } else {   // sink tokens keep code 0: pair slots 0, 2 are row g, slots 1, 3 row g + 8
+                        const bool s0 = (m16 >> g) & 1u, s1 = (m16 >> (g + 8)) & 1u;
+                        acc = thermo_accumulate(acc, a[T][0], tA, s0 ? zero2 : w0);
+                        acc = thermo_accumulate(acc, a[T][1], tA, s1 ? zero2 : w1);
+                        acc = thermo_accumulate(acc, a[T][2], tB, s0 ? zero2 : w2);
+                        acc = thermo_accumulate(acc, a[T][3], tB, s1 ? zero2 : w3);
                     }
-                    // sink tokens keep code 0 in the packed stream: pair slots 0, 2 are row g, slots 1, 3 row g + 8
-                    if ((m16 >> g) & 1u) pc[0] = pc[2] = 0;
-                    if ((m16 >> (g + 8)) & 1u) pc[1] = pc[3] = 0;
+                    const uint32_t bits = *reinterpret_cast<uint32_t *>(&acc);   // 0x6400 | byte in each half
+                    uint8_t *wb = (uint8_t *)(xout + T * TILE_WORDS + lo_word);
+                    wb[m & 1] = (uint8_t)bits;
+                    wb[2 + (m & 1)] = (uint8_t)(bits >> 16);
                 }
-                uint32_t lo, hi;
-                pack_matrix<BITS>(pc, m, &lo, &hi);
-                uint32_t *tile = xout + T * TILE_WORDS;
-                if constexpr (BITS == 4) {
-                    tile[lo_word] = lo;
-                } else {
-                    uint8_t *wb = (uint8_t *)(tile + lo_word);
-                    wb[m & 1] = (uint8_t)lo;
-                    wb[2 + (m & 1)] = (uint8_t)(lo >> 16);
-                    if constexpr (BITS == 3) atomicOr(&tile[hi_word], hi);
+            } else {
+                Coder kc[4];
+#pragma unroll
+                for (int q = 0; q < 4; ++q) kc[q] = scr.coder[4 * t4 + q];
+                const int hi_word = (BITS == 3) ? 32 * NLO + section_word_offset(NHI > 0 ? NHI : 1, lane, m >> 2) : 0;
+                if constexpr (BITS == 3) {   // hi words are OR-ed together by the four warps that share them
+                    for (int i = tid; i < 32 * NHI * NT; i += THREADS) xout[(i / (32 * NHI)) * TILE_WORDS + 32 * NLO + i % (32 * NHI)] = 0;
+                    __syncthreads();
+                }
+#pragma unroll
+                for (int T = 0; T < NT; ++T) {
+                    uint32_t pc[4], differ = 0;
+#pragma unroll
+                    for (int r = 0; r < 4; ++r) pc[r] = code_pair<BITS>(a[T][r], kc[2 * (r >> 1)], kc[2 * (r >> 1) + 1], differ);
+                    const uint32_t m16 = tm[T];
+                    if (differ | m16) {   // rare: a value too close to a rounding tie, or a tile with sink tokens
+#pragma unroll
+                        for (int r = 0; r < 4; ++r) {
+                            const float2 z0 = scr.sz[4 * t4 + 2 * (r >> 1)], z1 = scr.sz[4 * t4 + 2 * (r >> 1) + 1];
+                            pc[r] = code_pair_exact<BITS>(a[T][r], z0.x, z0.y, z1.x, z1.y);
+                        }
+                        // sink tokens keep code 0 in the packed stream: pair slots 0, 2 are row g, slots 1, 3 row g + 8
+                        if ((m16 >> g) & 1u) pc[0] = pc[2] = 0;
+                        if ((m16 >> (g + 8)) & 1u) pc[1] = pc[3] = 0;
+                    }
+                    uint32_t lo, hi;
+                    pack_matrix<BITS>(pc, m, &lo, &hi);
+                    uint32_t *tile = xout + T * TILE_WORDS;
+                    if constexpr (BITS == 4) {
+                        tile[lo_word] = lo;
+                    } else {
+                        uint8_t *wb = (uint8_t *)(tile + lo_word);
+                        wb[m & 1] = (uint8_t)lo;
+                        wb[2 + (m & 1)] = (uint8_t)(lo >> 16);
+                        if constexpr (BITS == 3) atomicOr(&tile[hi_word], hi);
+                    }
                 }
             }
         } else {
@@ -307,44 +406,76 @@ quantize_groups_stream(Params p, kvsink_cache c, const __half *__restrict__ k_sr
                     }
                     reduce_rows(mnA, mxA);
                     reduce_rows(mnB, mxB);
-                    if (g < 4) {
-                        const __half2 mn2 = (g & 2) ? mnB : mnA, mx2 = (g & 2) ? mxB : mxA;
-                        const __half lo = (g & 1) ? __high2half(mn2) : __low2half(mn2), hi = (g & 1) ? __high2half(mx2) : __low2half(mx2);
-                        const int tk = 2 * t4 + (g & 1) + 8 * (g >> 1);      // token within the tile
+                    {
+                        const int kq = g & 3;
+                        const __half2 mn2 = (kq & 2) ? mnB : mnA, mx2 = (kq & 2) ? mxB : mxA;
+                        const __half lo = (kq & 1) ? __high2half(mn2) : __low2half(mn2), hi = (kq & 1) ? __high2half(mx2) : __low2half(mx2);
+                        const int tk = 2 * t4 + (kq & 1) + 8 * (kq >> 1);      // token within the tile
                         const bool member = !((m16 >> tk) & 1u);
                         const float mn = __half2float(lo), mx = __half2float(hi);
                         float s, z;
                         group_params(member, mn, mx, qmax, &s, &z);
-                        scr.coder[4 * t4 + g] = make_coder(s, z, mn, mx, qmax);
-                        scr.sz[4 * t4 + g] = make_float2(s, z);
-                        const size_t o = ((size_t)unit * p.max_seq + p0 + 16 * T + tk) * NGv + jg;
-                        c.v_scale[o] = s;
-                        c.v_zero[o] = z;
-                    }
-                    __syncwarp();
-                    Coder vc[4];
-#pragma unroll
-                    for (int q = 0; q < 4; ++q) vc[q] = scr.coder[4 * t4 + q];
-#pragma unroll
-                    for (int mi = 0; mi < MPG; ++mi) {
-                        const int m = jg * MPG + mi;
-                        uint32_t pc[4], differ = 0;
-#pragma unroll
-                        for (int r = 0; r < 4; ++r) pc[r] = code_pair<BITS>(a[mi][r], vc[2 * (r >> 1)], vc[2 * (r >> 1) + 1], differ);
-                        if (differ) {   // rare: a value too close to a rounding tie
-#pragma unroll
-                            for (int r = 0; r < 4; ++r) {
-                                const float2 z0 = scr.sz[4 * t4 + 2 * (r >> 1)], z1 = scr.sz[4 * t4 + 2 * (r >> 1) + 1];
-                                pc[r] = code_pair_exact<BITS>(a[mi][r], z0.x, z0.y, z1.x, z1.y);
+                        if (g < 4) {
+                            if constexpr (BITS != 2) scr.coder[4 * t4 + kq] = make_coder(s, z, mn, mx, qmax);
+                            scr.sz[4 * t4 + kq] = make_float2(s, z);
+                            const size_t o = ((size_t)unit * p.max_seq + p0 + 16 * T + tk) * NGv + jg;
+                            c.v_scale[o] = s;
+                            c.v_zero[o] = z;
+                        }
+                        if constexpr (BITS == 2) {
+                            __half *th = reinterpret_cast<__half *>(&scr.thr[t4][kq >> 1][0]) + (kq & 1);
+                            if (g < 4) {
+                                th[0] = __ushort_as_half((unsigned short)code_threshold(s, z, 1, qmax));
+                                th[2] = __ushort_as_half((unsigned short)code_threshold(s, z, 2, qmax));
+                            } else {
+                                th[4] = __ushort_as_half((unsigned short)code_threshold(s, z, 3, qmax));
                             }
                         }
-                        uint32_t lo, hi;
-                        pack_matrix<BITS>(pc, m, &lo, &hi);
-                        if constexpr (BITS == 4) {
-                            wl[m] = lo;
-                        } else {
-                            wl[m >> 1] |= lo << (8 * (m & 1));
-                            if constexpr (BITS == 3) wh[m >> 2] |= hi;
+                    }
+                    __syncwarp();
+                    if constexpr (BITS == 2) {
+                        __half2 tA[3], tB[3];
+#pragma unroll
+                        for (int j = 0; j < 3; ++j) { tA[j] = scr.thr[t4][0][j]; tB[j] = scr.thr[t4][1][j]; }
+                        const __half2 base = __half2half2(__float2half(1024.f));
+                        const __half2 w0 = __half2half2(__float2half(1.f)), w1 = __half2half2(__float2half(4.f));
+                        const __half2 w2 = __half2half2(__float2half(16.f)), w3 = __half2half2(__float2half(64.f));
+#pragma unroll
+                        for (int mi = 0; mi < MPG; ++mi) {
+                            const int m = jg * MPG + mi;
+                            __half2 acc = base;
+                            acc = thermo_accumulate(acc, a[mi][0], tA, w0);
+                            acc = thermo_accumulate(acc, a[mi][1], tA, w1);
+                            acc = thermo_accumulate(acc, a[mi][2], tB, w2);
+                            acc = thermo_accumulate(acc, a[mi][3], tB, w3);
+                            const uint32_t bits = *reinterpret_cast<uint32_t *>(&acc) & 0x00ff00ffu;
+                            wl[m >> 1] |= bits << (8 * (m & 1));
+                        }
+                    } else {
+                        Coder vc[4];
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) vc[q] = scr.coder[4 * t4 + q];
+#pragma unroll
+                        for (int mi = 0; mi < MPG; ++mi) {
+                            const int m = jg * MPG + mi;
+                            uint32_t pc[4], differ = 0;
+#pragma unroll
+                            for (int r = 0; r < 4; ++r) pc[r] = code_pair<BITS>(a[mi][r], vc[2 * (r >> 1)], vc[2 * (r >> 1) + 1], differ);
+                            if (differ) {   // rare: a value too close to a rounding tie
+#pragma unroll
+                                for (int r = 0; r < 4; ++r) {
+                                    const float2 z0 = scr.sz[4 * t4 + 2 * (r >> 1)], z1 = scr.sz[4 * t4 + 2 * (r >> 1) + 1];
+                                    pc[r] = code_pair_exact<BITS>(a[mi][r], z0.x, z0.y, z1.x, z1.y);
+                                }
+                            }
+                            uint32_t lo, hi;
+                            pack_matrix<BITS>(pc, m, &lo, &hi);
+                            if constexpr (BITS == 4) {
+                                wl[m] = lo;
+                            } else {
+                                wl[m >> 1] |= lo << (8 * (m & 1));
+                                if constexpr (BITS == 3) wh[m >> 2] |= hi;
+                            }
                         }
                     }
                     __syncwarp();   // the scratch is rewritten for the next channel group / tile
