@@ -200,8 +200,10 @@ def run_reference(args):
 def run_ours(args):
     import torch.distributed as dist
     import paper_2508_04257_b200 as kv
+    from paper_2508_04257_b200 import dist_util
 
-    rank, world, local = int(os.environ.get("RANK", "0")), int(os.environ.get("WORLD_SIZE", "1")), int(os.environ.get("LOCAL_RANK", "0"))
+    ri = dist_util.rank_info()
+    rank, world, local = ri.rank, ri.world, ri.local_rank
     if not torch.cuda.is_available():
         raise RuntimeError("bench.py needs a CUDA device; there is no CPU fallback")
     torch.cuda.set_device(local)
@@ -209,7 +211,7 @@ def run_ours(args):
     if world > 1:
         dist.init_process_group("nccl", device_id=dev)
 
-    wl = synth.WORKLOADS[args.workload].scaled(seed=synth.WORKLOADS[args.workload].seed + 7919 * rank)
+    wl = synth.WORKLOADS[args.workload].scaled(seed=dist_util.rank_seed(synth.WORKLOADS[args.workload].seed, rank))
     if args.batch > 0:
         wl = wl.scaled(batch=args.batch)
     L = args.instances
@@ -267,15 +269,11 @@ def run_ours(args):
     barrier()
     sampler.region(False)
     clocks = sampler.finish()
-    ms_total = t_a.elapsed_time(t_b)
-    if world > 1:
-        t = torch.tensor([ms_total], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
+    ms_total = dist_util.max_over_ranks(t_a.elapsed_time(t_b), dev)
     ms_step = ms_total / args.steps
     kind_ms = {k: sum(a.elapsed_time(b) for a, b in ev[k]) / max(len(ev[k]), 1) for k in kinds}   # per call
     bytes_step = step_bytes(wl, L)
-    value = world * bytes_step / (ms_step * 1e-3) / 1e9
+    value = dist_util.aggregate_throughput(bytes_step, world, ms_step * 1e-3) / 1e9
     status = kv.read_status(caches[0])
 
     # ---- end to end: pinned host inputs copied in, result copied out, every step
@@ -307,12 +305,8 @@ def run_ours(args):
             e2e_step()
         b.record()
         barrier()
-        ms = a.elapsed_time(b)
-        if world > 1:
-            t = torch.tensor([ms], device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
-        e2e = {"value": world * bytes_step / (ms / args.e2e_steps * 1e-3) / 1e9, "unit": "GB/s", "h2d_bytes_per_step": int(h2d),
+        ms = dist_util.max_over_ranks(a.elapsed_time(b), dev)
+        e2e = {"value": dist_util.aggregate_throughput(bytes_step, world, ms / args.e2e_steps * 1e-3) / 1e9, "unit": "GB/s", "h2d_bytes_per_step": int(h2d),
                "d2h_bytes_per_step": int(d2h), "ms_per_step": ms / args.e2e_steps, "steps": args.e2e_steps}
         del hH, hKV, hnew, hq
 
