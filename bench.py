@@ -81,6 +81,11 @@ def ncu_traffic(kernel_key):
         return None
 
 
+def workload_string(wl):
+    return (f"{wl.name}: B={wl.batch} Hq={wl.n_q_heads} Hkv={wl.n_kv_heads} D={wl.head_dim} S={wl.seq} bits={wl.bits} "
+            f"G={wl.group} k={wl.topk} N={wl.pfn_n}")
+
+
 def measured_peak():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     try:
@@ -190,7 +195,7 @@ def run_reference(args):
     line = {"impl": "reference", "metric": "quantize+decode-attn achieved HBM GB/s", "value": gbs, "unit": "GB/s", "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f32 quantization / f64 attention", "data": "synthetic",
-            "config": {"workload": wl.name, "sample": sample},
+            "config": {"workload": workload_string(wl), "sample": sample},
             "cpu_baseline": {"value": gbs, "unit": "GB/s", "cores": stages["threads"], "kind": "oracle", "sample": sample},
             "e2e": {"value": gbs, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}, "gpu_launches": 0}
     print(json.dumps(line), flush=True)
@@ -341,8 +346,7 @@ def run_ours(args):
     line = {"metric": "quantize+decode-attn achieved HBM GB/s", "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "f32", "data": "synthetic",
-            "config": {"workload": f"{wl.name}: B={wl.batch} Hq={wl.n_q_heads} Hkv={wl.n_kv_heads} D={wl.head_dim} S={wl.seq} bits={wl.bits} "
-                                   f"G={wl.group} k={wl.topk} N={wl.pfn_n}", "instances_per_step": L,
+            "config": {"workload": workload_string(wl), "instances_per_step": L,
                        "l2": f"inputs larger than L2: {L} instances, {bytes_step / 1e6:.0f} MB touched per step; each kernel reads data "
                              "last touched more than 300 MB of traffic earlier",
                        "step": "predict_sinks, then per instance quantize_append(T=S), then per instance quantize_append(T=1) + decode_attention"},
