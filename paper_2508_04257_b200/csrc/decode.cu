@@ -209,7 +209,11 @@ struct DecodePlan {
     }
 };
 
-template <int BITS, int D, int NGv, int CT>
+// PL ("pair layout", for at most four query heads per KV head): query head h owns accumulator columns 2h and 2h+1;
+// column 2h multiplies by the fp16 factor q*scale and column 2h+1 by its fp16 rounding residual, so every score carries
+// the factor to ~22 bits at no extra instruction.  Without PL (five to eight heads) head h owns column h and the
+// residual of channels with large factors goes through a second multiply.
+template <int BITS, int D, int NGv, int CT, bool PL>
 __global__ void __launch_bounds__(DEC_THREADS, 4)
 decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__restrict__ out, float *__restrict__ lse,
               float *__restrict__ part_ws, int nsplit, int groups_per_split, int qchunks, int seq_len)
@@ -299,6 +303,7 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
     // New running maxima after a batch of scores with per-lane maxima tm0 / tm1; rescales the accumulators if needed.
     // Once the running maxima have settled no lane exceeds them and the step costs one vote.
     auto advance_max = [&](float tm0, float tm1) {
+        if (PL) tm1 = M_INIT;
         if (!__any_sync(0xffffffffu, tm0 > m0 || tm1 > m1)) return;
 #pragma unroll
         for (int o = 4; o < 32; o <<= 1) {
@@ -318,7 +323,7 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
     // (scale, zero) of tokens g (sv0, zv0) and g+8 (sv1, zv1) per channel group.
     auto tile_values = [&](const float (&s)[4], const uint32_t (&vw)[W], const float (&sv0)[NGv], const float (&zv0)[NGv],
                            const float (&sv1)[NGv], const float (&zv1)[NGv]) {
-        const float p0 = ex2(s[0] - m0), p1 = ex2(s[1] - m1), p2 = ex2(s[2] - m0), p3 = ex2(s[3] - m1);
+        const float p0 = ex2(s[0] - m0), p1 = PL ? 0.f : ex2(s[1] - m1), p2 = ex2(s[2] - m0), p3 = PL ? 0.f : ex2(s[3] - m1);
         l0 += p0 + p2;
         l1 += p1 + p3;
         uint32_t va[NM][4];
@@ -417,17 +422,28 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
                             hb = __hmul(hb, __float2half(C1));
                             lb = __hmul(lb, __float2half(C1));
                         }
-                        Bs[i * BST + ch] = hb;
-                        Bl[i * BST + ch] = lb;
+                        if (PL) {
+                            Bs[(2 * i) * BST + ch] = hb;
+                            Bs[(2 * i + 1) * BST + ch] = lb;
+                        } else {
+                            Bs[i * BST + ch] = hb;
+                            Bl[i * BST + ch] = lb;
+                        }
                     }
-                    const uint32_t bal = __ballot_sync(0xffffffffu, big);
-                    constexpr int LPM = 16 / CPL;     // lanes per 16-channel matrix
+                    if (!PL) {
+                        const uint32_t bal = __ballot_sync(0xffffffffu, big);
+                        constexpr int LPM = 16 / CPL;     // lanes per 16-channel matrix
 #pragma unroll
-                    for (int m = 0; m < NM; ++m)
-                        if ((bal >> (LPM * m)) & ((1u << LPM) - 1u)) need_lo |= 1u << m;
+                        for (int m = 0; m < NM; ++m)
+                            if ((bal >> (LPM * m)) & ((1u << LPM) - 1u)) need_lo |= 1u << m;
+                    }
                     bsum = warp_sum(bsum) * pow2i(-sh);
-                    if (i == 2 * t) { bias0 = bsum; ks0 = pow2i(24 - sh); }
-                    if (i == 2 * t + 1) { bias1 = bsum; ks1 = pow2i(24 - sh); }
+                    if (PL) {
+                        if (i == t) { bias0 = bsum; ks0 = pow2i(24 - sh); }
+                    } else {
+                        if (i == 2 * t) { bias0 = bsum; ks0 = pow2i(24 - sh); }
+                        if (i == 2 * t + 1) { bias1 = bsum; ks1 = pow2i(24 - sh); }
+                    }
                 }
             }
             __syncwarp();
@@ -435,8 +451,9 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
         uint32_t bk[NM][2];
 #pragma unroll
         for (int m = 0; m < NM; ++m) {
-            bk[m][0] = g < nq ? *(const uint32_t *)(Bs + g * BST + 16 * m + 2 * t) : 0u;
-            bk[m][1] = g < nq ? *(const uint32_t *)(Bs + g * BST + 16 * m + 2 * t + 8) : 0u;
+            const bool col_used = PL ? g < 2 * nq : g < nq;
+            bk[m][0] = col_used ? *(const uint32_t *)(Bs + g * BST + 16 * m + 2 * t) : 0u;
+            bk[m][1] = col_used ? *(const uint32_t *)(Bs + g * BST + 16 * m + 2 * t + 8) : 0u;
         }
         const float ks0r = ks0 * R1, ks1r = ks1 * R1;
 
@@ -465,7 +482,7 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
                 load_tile_shared<BITS, D>(kt + k * TILE_WORDS, lane, kw);
                 tile_frags<BITS, D>(kw, ka);
                 float acc[4] = {0.f, 0.f, 0.f, 0.f};
-                if (need_lo == 0) {
+                if (PL || need_lo == 0) {
 #pragma unroll
                     for (int m = 0; m < NM; ++m) mma16816(acc, ka[m], bk[m][0], bk[m][1]);
                 } else {
@@ -479,8 +496,13 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
                         }
                     }
                 }
-                s[k][0] = fmaf(acc[0], ks0, -bias0); s[k][1] = fmaf(acc[1], ks1, -bias1);
-                s[k][2] = fmaf(acc[2], ks0r, -bias0); s[k][3] = fmaf(acc[3], ks1r, -bias1);
+                if (PL) {   // column 2t: rounded factors, column 2t+1: their residuals
+                    s[k][0] = fmaf(acc[0] + acc[1], ks0, -bias0); s[k][1] = -INFINITY;
+                    s[k][2] = fmaf(acc[2] + acc[3], ks0r, -bias0); s[k][3] = -INFINITY;
+                } else {
+                    s[k][0] = fmaf(acc[0], ks0, -bias0); s[k][1] = fmaf(acc[1], ks1, -bias1);
+                    s[k][2] = fmaf(acc[2], ks0r, -bias0); s[k][3] = fmaf(acc[3], ks1r, -bias1);
+                }
             }
             if (mword) {   // sink tokens are not part of the packed stream (their value parameters are zero)
 #pragma unroll
@@ -536,14 +558,16 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
                 a[1] = in1 ? *(const uint32_t *)(r1 + 16 * m + 2 * t) : 0u;
                 a[2] = in0 ? *(const uint32_t *)(r0 + 16 * m + 2 * t + 8) : 0u;
                 a[3] = in1 ? *(const uint32_t *)(r1 + 16 * m + 2 * t + 8) : 0u;
-                const uint32_t b0 = *(const uint32_t *)(q16 + g * D + 16 * m + 2 * t);
-                const uint32_t b1 = *(const uint32_t *)(q16 + g * D + 16 * m + 2 * t + 8);
+                const int qrow = PL ? (g >> 1) : g;          // query head in accumulator column g
+                const bool qcol = PL ? !(g & 1) : true;
+                const uint32_t b0 = qcol ? *(const uint32_t *)(q16 + qrow * D + 16 * m + 2 * t) : 0u;
+                const uint32_t b1 = qcol ? *(const uint32_t *)(q16 + qrow * D + 16 * m + 2 * t + 8) : 0u;
                 mma16816(acc, a, b0, b1);
             }
             const bool v0 = in0 && !mask_bit(bm, in0 ? tok0 : 0), v1 = in1 && !mask_bit(bm, in1 ? tok1 : 0);
             float s[4];
-            s[0] = v0 ? acc[0] * qscale : -INFINITY; s[1] = v0 ? acc[1] * qscale : -INFINITY;
-            s[2] = v1 ? acc[2] * qscale : -INFINITY; s[3] = v1 ? acc[3] * qscale : -INFINITY;
+            s[0] = v0 ? acc[0] * qscale : -INFINITY; s[1] = (v0 && !PL) ? acc[1] * qscale : -INFINITY;
+            s[2] = v1 ? acc[2] * qscale : -INFINITY; s[3] = (v1 && !PL) ? acc[3] * qscale : -INFINITY;
             advance_max(fmaxf(s[0], s[2]), fmaxf(s[1], s[3]));
             uint32_t vw[W];
             load_tile<BITS, D>((const uint32_t *)(vc_base + (size_t)T * p.tile_bytes), lane, vw);
@@ -579,6 +603,13 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
         for (int m = 0; m < NM; ++m) {
             const float bj0 = bv[m / mpg][0], bj1 = bv[m / mpg][1];
             const int ch0 = 16 * m + g, ch1 = ch0 + 8;
+            if (PL) {
+                if (t < nq) {
+                    my_part[t * PS + ch0] = O[m][0] * OS0 - bj0;
+                    my_part[t * PS + ch1] = O[m][2] * OS1 - bj0;
+                }
+                continue;
+            }
             if (2 * t < nq) {
                 my_part[(2 * t) * PS + ch0] = O[m][0] * OS0 - bj0;
                 my_part[(2 * t) * PS + ch1] = O[m][2] * OS1 - bj0;
@@ -588,7 +619,9 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
                 my_part[(2 * t + 1) * PS + ch1] = O[m][3] * OS1 - bj1;
             }
         }
-        if (g == 0) {
+        if (g == 0 && PL) {
+            if (t < nq) { my_part[t * PS + D] = m0; my_part[t * PS + D + 1] = l0; }
+        } else if (g == 0) {
             if (2 * t < nq) { my_part[(2 * t) * PS + D] = m0; my_part[(2 * t) * PS + D + 1] = l0; }
             if (2 * t + 1 < nq) { my_part[(2 * t + 1) * PS + D] = m1; my_part[(2 * t + 1) * PS + D + 1] = l1; }
         }
@@ -719,8 +752,8 @@ size_t decode_workspace_bytes(const Params &p)
     return (size_t)p.B * p.Hq * max_splits(p) * (p.D + 2) * sizeof(float) + 16;
 }
 
-template <int BITS, int D, int NGV, int CT>
-static int launch_decode_c(const Params &p, const kvsink_cache &c, const __half *q, float *out, float *lse, float *ws, cudaStream_t st)
+template <int BITS, int D, int NGV, int CT, bool PL>
+static int launch_decode_p(const Params &p, const kvsink_cache &c, const __half *q, float *out, float *lse, float *ws, cudaStream_t st)
 {
     const int n_groups = c.seq_len / p.G;
     const int nsplit = choose_splits(p, n_groups);
@@ -728,7 +761,7 @@ static int launch_decode_c(const Params &p, const kvsink_cache &c, const __half 
     const int qchunks = (p.rep + 7) / 8;
     const int nq_max = p.rep < 8 ? p.rep : 8;
     const size_t smem = DecodePlan<BITS, D, NGV, CT>::bytes(nq_max);
-    auto kern = decode_kernel<BITS, D, NGV, CT>;
+    auto kern = decode_kernel<BITS, D, NGV, CT, PL>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return KVSINK_ERR_CUDA;
     dim3 grid(nsplit, p.Hkv * qchunks, p.B);
     kern<<<grid, DEC_THREADS, smem, st>>>(p, c, q, out, lse, ws, nsplit, gps, qchunks, c.seq_len);
@@ -738,6 +771,13 @@ static int launch_decode_c(const Params &p, const kvsink_cache &c, const __half 
         if (cudaGetLastError() != cudaSuccess) return KVSINK_ERR_CUDA;
     }
     return KVSINK_OK;
+}
+
+template <int BITS, int D, int NGV, int CT>
+static int launch_decode_c(const Params &p, const kvsink_cache &c, const __half *q, float *out, float *lse, float *ws, cudaStream_t st)
+{
+    if (p.rep <= 4) return launch_decode_p<BITS, D, NGV, CT, true>(p, c, q, out, lse, ws, st);
+    return launch_decode_p<BITS, D, NGV, CT, false>(p, c, q, out, lse, ws, st);
 }
 
 template <int BITS, int D, int NGV>

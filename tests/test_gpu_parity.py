@@ -23,7 +23,7 @@ def test_tiny_workload_with_appends():
 
 @pytest.mark.parametrize("bits,d,group", [(2, 128, 128), (3, 128, 64), (4, 128, 64), (2, 64, 32), (4, 64, 32), (4, 64, 16),
                                           (2, 128, 32), (3, 128, 128), (4, 128, 256)])
-@pytest.mark.parametrize("hq,hkv", [(4, 4), (8, 2), (6, 2)])
+@pytest.mark.parametrize("hq,hkv", [(4, 4), (8, 2), (6, 2), (16, 2), (12, 1)])
 def test_grid_of_shapes(bits, d, group, hq, hkv):
     # several groups and tiles plus a ragged remainder; sinks at token 0, mid sequence and inside the remainder
     seq = 3 * group + 37
