@@ -223,6 +223,7 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
     constexpr int NM = G_::NM, W = G_::W, BST = Plan::BST, TILE_WORDS = 32 * W;
     constexpr int NSLOT = Plan::NSLOT, SLOT_BYTES = Plan::SLOT_BYTES, KV_BYTES = Plan::KV_BYTES, SZ_BYTES = Plan::SZ_BYTES;
     constexpr int mpg = (D / NGv) / 16;                              // value matrices per channel group
+    constexpr int ST = CT >= 2 ? 2 : 1;                              // tiles per softmax step
     constexpr int CPL = D / 32;                                      // channels per lane in per-channel passes
     constexpr float LOG2E = 1.4426950408889634f;
     constexpr float QMAX = (float)((1 << BITS) - 1);
@@ -377,7 +378,14 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
         issue_params(0);
         for (int i = 0; i < NSLOT - 1 && iss_g < my_groups; ++i) issue_chunk(i);
     }
-    uint32_t mword_next = my_groups > 0 ? __ldg(bm + (((g_begin + warp) * TPG) >> 1)) : 0u;
+    // sink bits of the CT tiles starting at tile T: one 32-bit word covers two tiles
+    auto load_mask_words = [&](int T) {
+        uint2 w;
+        w.x = __ldg(bm + (T >> 1));
+        w.y = CT == 4 ? __ldg(bm + (T >> 1) + 1) : 0u;
+        return w;
+    };
+    uint2 mword_next = my_groups > 0 ? load_mask_words((g_begin + warp) * TPG) : make_uint2(0u, 0u);
     bool stream_ok = true;
     int ci = 0;                                                      // running chunk index of this warp
 
@@ -464,20 +472,25 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
             __syncwarp();
             if (lane == 0 && iss_g < my_groups) issue_chunk((ci + NSLOT - 1) & (NSLOT - 1));
             if (!wait_bar(&cbar[slot], (unsigned)(ci / NSLOT) & 1u)) { stream_ok = false; break; }
-            const uint32_t mword = mword_next;
+            const uint2 mwords = mword_next;
             {   // sink bits of the warp's next chunk, fetched one chunk ahead
                 const bool last = cj + 1 == CPG;
                 const int Tn = last ? (grp + DEC_WARPS) * TPG : grp * TPG + (cj + 1) * CT;
-                if (!last || gi + 1 < my_groups) mword_next = __ldg(bm + (Tn >> 1));
+                if (!last || gi + 1 < my_groups) mword_next = load_mask_words(Tn);
             }
-            const uint32_t *kt = (const uint32_t *)(ring + slot * SLOT_BYTES), *vt = kt + KV_BYTES / 4;
-            const float *ssv = (const float *)(vt + KV_BYTES / 4), *szv = ssv + SZ_BYTES / 4;
-            const int T0 = grp * TPG + cj * CT;
+            const uint32_t *kt0 = (const uint32_t *)(ring + slot * SLOT_BYTES), *vt0 = kt0 + KV_BYTES / 4;
+            const float *ssv0 = (const float *)(vt0 + KV_BYTES / 4), *szv0 = ssv0 + SZ_BYTES / 4;
+#pragma unroll
+            for (int sub = 0; sub < CT / ST; ++sub) {   // softmax steps of ST tiles inside the chunk
+            const uint32_t *kt = kt0 + sub * ST * TILE_WORDS, *vt = vt0 + sub * ST * TILE_WORDS;
+            const float *ssv = ssv0 + sub * ST * 16 * NGv, *szv = szv0 + sub * ST * 16 * NGv;
+            const int T0 = grp * TPG + cj * CT + sub * ST;
+            const uint32_t mword = sub == 0 ? mwords.x : mwords.y;
 
             // scores of the chunk's tiles
-            float s[CT][4];
+            float s[ST][4];
 #pragma unroll
-            for (int k = 0; k < CT; ++k) {
+            for (int k = 0; k < ST; ++k) {
                 uint32_t kw[W], ka[NM][4];
                 load_tile_shared<BITS, D>(kt + k * TILE_WORDS, lane, kw);
                 tile_frags<BITS, D>(kw, ka);
@@ -506,7 +519,7 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
             }
             if (mword) {   // sink tokens are not part of the packed stream (their value parameters are zero)
 #pragma unroll
-                for (int k = 0; k < CT; ++k) {
+                for (int k = 0; k < ST; ++k) {
                     const uint32_t mask16 = (mword >> (16 * ((T0 + k) & 1))) & 0xffffu;
                     if ((mask16 >> g) & 1u) s[k][0] = s[k][1] = -INFINITY;
                     if ((mask16 >> (g + 8)) & 1u) s[k][2] = s[k][3] = -INFINITY;
@@ -515,15 +528,15 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
             // one softmax step for the whole chunk
             {
                 float tm0 = fmaxf(s[0][0], s[0][2]), tm1 = fmaxf(s[0][1], s[0][3]);
-                if (CT == 2) { tm0 = fmaxf(tm0, fmaxf(s[CT - 1][0], s[CT - 1][2])); tm1 = fmaxf(tm1, fmaxf(s[CT - 1][1], s[CT - 1][3])); }
+                if (ST == 2) { tm0 = fmaxf(tm0, fmaxf(s[ST - 1][0], s[ST - 1][2])); tm1 = fmaxf(tm1, fmaxf(s[ST - 1][1], s[ST - 1][3])); }
                 advance_max(tm0, tm1);
             }
             // value scales of this lane's tokens; their maximum bounds the fp16 range needed
-            float sv0[CT][NGv], zv0[CT][NGv], sv1[CT][NGv], zv1[CT][NGv];
+            float sv0[ST][NGv], zv0[ST][NGv], sv1[ST][NGv], zv1[ST][NGv];
             {
                 float mx = 0.f;
 #pragma unroll
-                for (int k = 0; k < CT; ++k)
+                for (int k = 0; k < ST; ++k)
 #pragma unroll
                     for (int j = 0; j < NGv; ++j) {
                         sv0[k][j] = ssv[(k * 16 + g) * NGv + j]; zv0[k][j] = szv[(k * 16 + g) * NGv + j];
@@ -533,10 +546,11 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
                 fit_value_scale(mx);
             }
 #pragma unroll
-            for (int k = 0; k < CT; ++k) {
+            for (int k = 0; k < ST; ++k) {
                 uint32_t vw[W];
                 load_tile_shared<BITS, D>(vt + k * TILE_WORDS, lane, vw);
                 tile_values(s[k], vw, sv0[k], zv0[k], sv1[k], zv1[k]);
+            }
             }
         }
     }
@@ -783,7 +797,10 @@ static int launch_decode_c(const Params &p, const kvsink_cache &c, const __half 
 template <int BITS, int D, int NGV>
 static int launch_decode_n(const Params &p, const kvsink_cache &c, const __half *q, float *out, float *lse, float *ws, cudaStream_t st)
 {
-    // ring chunks of two tiles when a key group has an even number of tiles (G a multiple of 32), else of one
+    // ring chunks of four tiles where a key group divides into them and two slots of that size stay below ~9 KB per
+    // warp, else of two tiles (G a multiple of 32), else of one
+    if constexpr (4 * (2 * 128 * (D * BITS / 64) + 2 * 16 * NGV * 4) <= 4800)
+        if ((p.G / KVSINK_TILE) % 4 == 0) return launch_decode_c<BITS, D, NGV, 4>(p, c, q, out, lse, ws, st);
     if ((p.G / KVSINK_TILE) % 2 == 0) return launch_decode_c<BITS, D, NGV, 2>(p, c, q, out, lse, ws, st);
     return launch_decode_c<BITS, D, NGV, 1>(p, c, q, out, lse, ws, st);
 }
