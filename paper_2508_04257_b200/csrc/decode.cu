@@ -196,7 +196,7 @@ struct DecodePlan {
     static constexpr int SLOT_BYTES = 2 * KV_BYTES + 2 * SZ_BYTES;      // K words, V words, V scales, V zeros of CT tiles
     static constexpr int NSLOT = (9216 / SLOT_BYTES >= 4) ? 4 : 2;      // power of two
     static constexpr int KP_BYTES = 2 * D * 4;                          // key scale + zero of one group
-    static constexpr int WARP_RING = NSLOT * SLOT_BYTES + 2 * KP_BYTES;
+    static constexpr int WARP_RING = NSLOT * SLOT_BYTES + KP_BYTES;
     __host__ __device__ static size_t fixed_bytes(int nq)
     {
         size_t f = 8 * D * 4 + 8 * D * 2 + (size_t)DEC_WARPS * 2 * nq * BST * 2 + DEC_WARPS * 8 * 8;
@@ -348,7 +348,7 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
     const int g_begin = split * groups_per_split, g_end = min(n_groups, g_begin + groups_per_split);
     const int my_groups = g_begin + warp < g_end ? (g_end - g_begin - warp + DEC_WARPS - 1) / DEC_WARPS : 0;
     unsigned char *ring = ring_all + (size_t)warp * Plan::WARP_RING;
-    float *kp_ring = (float *)(ring + NSLOT * SLOT_BYTES);           // [2][scale D | zero D]
+    float *kp_ring = (float *)(ring + NSLOT * SLOT_BYTES);           // [scale D | zero D] of the next group to prepare
     int iss_g = 0, iss_c = 0;                                        // next chunk to issue: group index, chunk within group
     auto issue_chunk = [&](int slot) {                               // lane 0 only
         const int T0 = (g_begin + warp + iss_g * DEC_WARPS) * TPG + iss_c * CT;
@@ -361,10 +361,10 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
         if (++iss_c == CPG) { iss_c = 0; ++iss_g; }
     };
     auto issue_params = [&](int gi) {                                // lane 0 only
-        const int grp = g_begin + warp + gi * DEC_WARPS, slot = gi & 1;
-        mbar_expect_tx(&pbar[slot], Plan::KP_BYTES);
-        bulk_g2s(kp_ring + slot * 2 * D, ks_base + (size_t)grp * D, D * 4, &pbar[slot]);
-        bulk_g2s(kp_ring + slot * 2 * D + D, kz_base + (size_t)grp * D, D * 4, &pbar[slot]);
+        const int grp = g_begin + warp + gi * DEC_WARPS;
+        mbar_expect_tx(&pbar[0], Plan::KP_BYTES);
+        bulk_g2s(kp_ring, ks_base + (size_t)grp * D, D * 4, &pbar[0]);
+        bulk_g2s(kp_ring + D, kz_base + (size_t)grp * D, D * 4, &pbar[0]);
     };
     auto wait_bar = [&](uint64_t *bar, unsigned parity) {
         int polls = 0;
@@ -397,62 +397,74 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
         float bias0 = 0.f, bias1 = 0.f, ks0 = 0.f, ks1 = 0.f;
         uint32_t need_lo = 0;     // bit m: matrix m also gets the low half of the split factor (warp-uniform)
         {
-            __syncwarp();
-            if (lane == 0 && gi + 1 < my_groups) issue_params(gi + 1);
-            if (!wait_bar(&pbar[gi & 1], (unsigned)(gi >> 1) & 1u)) { stream_ok = false; break; }
-            const float *kp = kp_ring + (gi & 1) * 2 * D;
+            if (!wait_bar(&pbar[0], (unsigned)gi & 1u)) { stream_ok = false; break; }
+            const float *kp = kp_ring;
             float scv[CPL], zev[CPL];
 #pragma unroll
             for (int e = 0; e < CPL; ++e) { scv[e] = kp[lane * CPL + e]; zev[e] = kp[D + lane * CPL + e]; }
+            __syncwarp();   // the parameters are in registers: the slot can take the next group's while this one streams
+            if (lane == 0 && gi + 1 < my_groups) issue_params(gi + 1);
+            // one power-of-two scaling for all heads of the group: the largest factor lands in [2^13, 2^14)
+            constexpr int NQL = PL ? 4 : 8;
+            float amax = 0.f;
 #pragma unroll
-            for (int i = 0; i < 8; ++i) {
+            for (int i = 0; i < NQL; ++i)
                 if (i < nq) {
-                    float v[CPL], amax = 0.f;
 #pragma unroll
-                    for (int e = 0; e < CPL; ++e) { v[e] = qs[i * D + lane * CPL + e] * scv[e]; amax = fmaxf(amax, fabsf(v[e])); }
-                    amax = warp_max(amax);
-                    int sh = 13 - floor_log2(amax);
-                    sh = sh > 60 ? 60 : (sh < -60 ? -60 : sh);
-                    const float f = pow2i(sh);
+                    for (int e = 0; e < CPL; ++e) amax = fmaxf(amax, fabsf(qs[i * D + lane * CPL + e] * scv[e]));
+                }
+            amax = warp_max(amax);
+            int sh = 13 - floor_log2(amax);
+            sh = sh > 60 ? 60 : (sh < -60 ? -60 : sh);
+            const float f = pow2i(sh), finv = pow2i(-sh), ksc = pow2i(24 - sh);
+            const bool scaled_col = ((lane * CPL) & 8) && G_::COLF != 1.f;   // this lane's channels sit in the column half
+            const __half2 colf = __half2half2(__float2half(scaled_col ? C1 : 1.f));
+            bool big = false;
+#pragma unroll
+            for (int i = 0; i < NQL; ++i) {
+                if (i < nq) {
                     float bsum = 0.f;
-                    bool big = false;
+                    __half2 hb[CPL / 2], lb[CPL / 2];
 #pragma unroll
-                    for (int e = 0; e < CPL; ++e) {
-                        const int ch = lane * CPL + e;
-                        const float vf = v[e] * f;
-                        __half hb = __float2half_rn(vf);
-                        // fp16 keeps 11 bits of the factor; where that could move a score by more than ~4e-4
-                        // (factor * largest |code - zero| * 2^-12) the rounding residual is kept as a second factor
-                        __half lb = __float2half_rn(vf - __half2float(hb));
-                        big |= fabsf(v[e]) * fmaxf(fabsf(zev[e]), fabsf(QMAX - zev[e])) > 1.6f;
-                        bsum += (__half2float(hb) + __half2float(lb)) * zev[e];
-                        if ((ch & 8) && G_::COLF != 1.f) {
-                            hb = __hmul(hb, __float2half(C1));
-                            lb = __hmul(lb, __float2half(C1));
-                        }
-                        if (PL) {
-                            Bs[(2 * i) * BST + ch] = hb;
-                            Bs[(2 * i + 1) * BST + ch] = lb;
-                        } else {
-                            Bs[i * BST + ch] = hb;
-                            Bl[i * BST + ch] = lb;
-                        }
+                    for (int e = 0; e < CPL; e += 2) {
+                        const float v0 = qs[i * D + lane * CPL + e] * scv[e], v1 = qs[i * D + lane * CPL + e + 1] * scv[e + 1];
+                        const float f0 = v0 * f, f1 = v1 * f;
+                        // fp16 keeps 11 bits of a factor; its rounding residual is kept as a second factor (always with PL,
+                        // else where it could move a score by more than ~4e-4: factor * largest |code - zero| * 2^-12)
+                        const __half2 h = __floats2half2_rn(f0, f1);
+                        const float2 hf = __half22float2(h);
+                        const __half2 l = __floats2half2_rn(f0 - hf.x, f1 - hf.y);
+                        const float2 lf = __half22float2(l);
+                        bsum += (hf.x + lf.x) * zev[e] + (hf.y + lf.y) * zev[e + 1];
+                        if (!PL)
+                            big |= fabsf(v0) * fmaxf(fabsf(zev[e]), fabsf(QMAX - zev[e])) > 1.6f ||
+                                   fabsf(v1) * fmaxf(fabsf(zev[e + 1]), fabsf(QMAX - zev[e + 1])) > 1.6f;
+                        hb[e / 2] = __hmul2(h, colf);
+                        lb[e / 2] = __hmul2(l, colf);
                     }
-                    if (!PL) {
-                        const uint32_t bal = __ballot_sync(0xffffffffu, big);
-                        constexpr int LPM = 16 / CPL;     // lanes per 16-channel matrix
-#pragma unroll
-                        for (int m = 0; m < NM; ++m)
-                            if ((bal >> (LPM * m)) & ((1u << LPM) - 1u)) need_lo |= 1u << m;
-                    }
-                    bsum = warp_sum(bsum) * pow2i(-sh);
-                    if (PL) {
-                        if (i == t) { bias0 = bsum; ks0 = pow2i(24 - sh); }
+                    __half *hrow = PL ? Bs + (2 * i) * BST : Bs + i * BST, *lrow = PL ? Bs + (2 * i + 1) * BST : Bl + i * BST;
+                    if constexpr (CPL == 4) {
+                        *reinterpret_cast<uint2 *>(hrow + lane * CPL) = make_uint2(*reinterpret_cast<uint32_t *>(&hb[0]), *reinterpret_cast<uint32_t *>(&hb[1]));
+                        *reinterpret_cast<uint2 *>(lrow + lane * CPL) = make_uint2(*reinterpret_cast<uint32_t *>(&lb[0]), *reinterpret_cast<uint32_t *>(&lb[1]));
                     } else {
-                        if (i == 2 * t) { bias0 = bsum; ks0 = pow2i(24 - sh); }
-                        if (i == 2 * t + 1) { bias1 = bsum; ks1 = pow2i(24 - sh); }
+                        *reinterpret_cast<__half2 *>(hrow + lane * CPL) = hb[0];
+                        *reinterpret_cast<__half2 *>(lrow + lane * CPL) = lb[0];
+                    }
+                    bsum = warp_sum(bsum) * finv;
+                    if (PL) {
+                        if (i == t) { bias0 = bsum; ks0 = ksc; }
+                    } else {
+                        if (i == 2 * t) { bias0 = bsum; ks0 = ksc; }
+                        if (i == 2 * t + 1) { bias1 = bsum; ks1 = ksc; }
                     }
                 }
+            }
+            if (!PL) {
+                const uint32_t bal = __ballot_sync(0xffffffffu, big);
+                constexpr int LPM = 16 / CPL;     // lanes per 16-channel matrix
+#pragma unroll
+                for (int m = 0; m < NM; ++m)
+                    if ((bal >> (LPM * m)) & ((1u << LPM) - 1u)) need_lo |= 1u << m;
             }
             __syncwarp();
         }
