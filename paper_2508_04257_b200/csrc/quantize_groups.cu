@@ -380,8 +380,11 @@ quantize_groups_stream(Params p, kvsink_cache c, const __half *__restrict__ k_sr
                 }
             }
         } else {
-            // ================= values: a warp owns whole tiles (16 tokens x D channels) =================
-            for (int T = warp; T < NT; T += NW) {
+            // ================= values: a warp owns a tile (16 tokens x D channels), or one channel group of a tile
+            //                    when there are fewer tiles than warps =================
+            constexpr int JG = (NT < NW && !(BITS == 3 && MPG < 4)) ? NGv : 1;   // jobs per tile (3-bit hi words span 4 matrices)
+            for (int job = warp; job < NT * JG; job += NW) {
+                const int T = job / JG, my_jg = job % JG;
                 const uint32_t m16 = tm[T];
                 uint32_t wl[NLO], wh[NHI > 0 ? NHI : 1];
 #pragma unroll
@@ -392,6 +395,7 @@ quantize_groups_stream(Params p, kvsink_cache c, const __half *__restrict__ k_sr
                 const __half *rowp = Xt + (size_t)row * D;
 #pragma unroll
                 for (int jg = 0; jg < NGv; ++jg) {
+                    if (JG > 1 && jg != my_jg) continue;   // warp-uniform
                     uint32_t a[MPG][4];
 #pragma unroll
                     for (int mi = 0; mi < MPG; ++mi)
@@ -482,10 +486,14 @@ quantize_groups_stream(Params p, kvsink_cache c, const __half *__restrict__ k_sr
                 }
                 uint32_t *tile = xout + T * TILE_WORDS;
 #pragma unroll
-                for (int i = 0; i < NLO; ++i) tile[section_word_offset(NLO, lane, i)] = wl[i];
+                for (int i = 0; i < NLO; ++i) {
+                    const int word_jg = ((BITS == 4) ? i : 2 * i) / MPG;   // channel group of the word's matrices
+                    if (JG == 1 || word_jg == my_jg) tile[section_word_offset(NLO, lane, i)] = wl[i];
+                }
                 if constexpr (BITS == 3) {
 #pragma unroll
-                    for (int i = 0; i < NHI; ++i) tile[32 * NLO + section_word_offset(NHI, lane, i)] = wh[i];
+                    for (int i = 0; i < NHI; ++i)
+                        if (JG == 1 || (4 * i) / MPG == my_jg) tile[32 * NLO + section_word_offset(NHI, lane, i)] = wh[i];
                 }
             }
         }
