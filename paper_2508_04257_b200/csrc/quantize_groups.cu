@@ -147,6 +147,42 @@ __device__ __noinline__ unsigned code_threshold(float s, float z, int level, flo
     return h_unord(o);
 }
 
+// The three thresholds of each of a warp's 16 keys with every lane busy.  The lanes g and g + 4 of a column group hold
+// the same key's (s, z): the lower one resolves level 1, the upper one level 2, and they share level 3.
+// Let T = level - zero - 1/2 and o the first fp16 value at or above est = fl(s * T).  Every value below o lies below
+// s * T, so its code stays under the level unless its quotient rounds onto T (checked: `below`).  The value o itself
+// reaches the level unless its quotient is exactly the tie T and rounds to the even neighbour below (common at 2 bit,
+// where scale = range / 3 makes s * T an fp16 value for a third of the groups); its successor is then the threshold,
+// because one fp16 step (>= 2^-12 relative, or 2^-24 absolute next to zero) moves the quotient past T by far more than
+// the 2^-24 relative error of est and the half ulp the rounded quotient can lose.  Estimates outside the finite range,
+// and the rare `below` hit, go to the search above.
+// `th` points at the key's half of thr[t4][column half][0]; consecutive levels are two halves apart.
+__device__ __forceinline__ void warp_thresholds(float s, float z, int g, float qmax, __half *th)
+{
+    constexpr int OMAX = 0x7BFF;
+    const bool upper = g >= 4;
+    // clamp(q, 0, qmax) >= level  <=>  q >= level  for 1 <= level <= qmax
+    auto reaches = [&](int o, float level) { return __fadd_rn(rintf(__fdiv_rn(h_val(o), s)), z) >= level; };
+    const float own = upper ? 2.f : 1.f;
+    const float est_own = s * (own - 0.5f - z), est3 = s * (3.f - 0.5f - z);
+    const int o_own = h_ord(__half_as_ushort(__float2half_ru(fminf(fmaxf(est_own, -65504.f), 65504.f))));
+    const int o3 = h_ord(__half_as_ushort(__float2half_ru(fminf(fmaxf(est3, -65504.f), 65504.f))));
+    const bool own_at = reaches(o_own, own);
+    const bool own_below = o_own > -OMAX && reaches(max(o_own - 1, -OMAX), own);
+    const bool r3 = upper ? (o3 > -OMAX && reaches(max(o3 - 1, -OMAX), 3.f)) : reaches(o3, 3.f);
+    const bool below3 = __shfl_xor_sync(0xffffffffu, (int)r3, 16) != 0;   // meaningful in the lower lane
+    unsigned t_own = h_unord(o_own + (own_at ? 0 : 1));
+    if (s == 0.f) t_own = 0x7C00u;
+    else if (own_below || !(fabsf(est_own) < 65504.f)) t_own = code_threshold(s, z, upper ? 2 : 1, qmax);
+    th[upper ? 2 : 0] = __ushort_as_half((unsigned short)t_own);
+    if (!upper) {
+        unsigned t3 = h_unord(o3 + (r3 ? 0 : 1));
+        if (s == 0.f) t3 = 0x7C00u;
+        else if (below3 || !(fabsf(est3) < 65504.f)) t3 = code_threshold(s, z, 3, qmax);
+        th[4] = __ushort_as_half((unsigned short)t3);
+    }
+}
+
 // Codes of the two elements of a half2 register, positioned: returns acc + w * ([x>=t1] + [x>=t2] + [x>=t3]) per half.
 __device__ __forceinline__ __half2 thermo_accumulate(__half2 acc, uint32_t x2, const __half2 (&t)[3], __half2 w)
 {
@@ -256,6 +292,9 @@ quantize_groups_stream(Params p, kvsink_cache c, const __half *__restrict__ k_sr
         const uint32_t *tm = tmask + buf * NT;
         const int64_t unit = (int64_t)b * p.Hkv + h;
         const int p0 = first_token + grp * G;
+        bool has_sink = false;   // block-uniform; false for almost every item
+#pragma unroll
+        for (int T = 0; T < NT; ++T) has_sink |= tm[T] != 0;
 
         if (kind == 0) {
             // ================= keys: warp m owns channels [16m, 16m+16) of every tile =================
@@ -269,14 +308,18 @@ quantize_groups_stream(Params p, kvsink_cache c, const __half *__restrict__ k_sr
             }
             // extremes per channel over the non-sink tokens: registers 0,1 hold channels (2t, 2t+1), registers 2,3 (2t+8, 2t+9)
             __half2 mnA = H_PINF, mxA = H_NINF, mnB = H_PINF, mxB = H_NINF;
+            if (!has_sink) {
 #pragma unroll
-            for (int T = 0; T < NT; ++T) {
-                const uint32_t m16 = tm[T];
-                const __half2 *h = reinterpret_cast<const __half2 *>(a[T]);
-                if (m16 == 0) {   // block-uniform, the common case
+                for (int T = 0; T < NT; ++T) {
+                    const __half2 *h = reinterpret_cast<const __half2 *>(a[T]);
                     mnA = __hmin2(mnA, __hmin2(h[0], h[1])); mxA = __hmax2(mxA, __hmax2(h[0], h[1]));
                     mnB = __hmin2(mnB, __hmin2(h[2], h[3])); mxB = __hmax2(mxB, __hmax2(h[2], h[3]));
-                } else {
+                }
+            } else {
+#pragma unroll
+                for (int T = 0; T < NT; ++T) {
+                    const uint32_t m16 = tm[T];
+                    const __half2 *h = reinterpret_cast<const __half2 *>(a[T]);
                     if (!((m16 >> g) & 1u)) { mnA = __hmin2(mnA, h[0]); mxA = __hmax2(mxA, h[0]); mnB = __hmin2(mnB, h[2]); mxB = __hmax2(mxB, h[2]); }
                     if (!((m16 >> (g + 8)) & 1u)) { mnA = __hmin2(mnA, h[1]); mxA = __hmax2(mxA, h[1]); mnB = __hmin2(mnB, h[3]); mxB = __hmax2(mxB, h[3]); }
                 }
@@ -300,15 +343,7 @@ quantize_groups_stream(Params p, kvsink_cache c, const __half *__restrict__ k_sr
                     c.k_scale[o] = s;
                     c.k_zero[o] = z;
                 }
-                if constexpr (BITS == 2) {   // lanes g < 4 find levels 1 and 2 of their key, lanes g >= 4 level 3
-                    __half *th = reinterpret_cast<__half *>(&scr.thr[t4][kq >> 1][0]) + (kq & 1);
-                    if (g < 4) {
-                        th[0] = __ushort_as_half((unsigned short)code_threshold(s, z, 1, qmax));
-                        th[2] = __ushort_as_half((unsigned short)code_threshold(s, z, 2, qmax));
-                    } else {
-                        th[4] = __ushort_as_half((unsigned short)code_threshold(s, z, 3, qmax));
-                    }
-                }
+                if constexpr (BITS == 2) warp_thresholds(s, z, g, qmax, reinterpret_cast<__half *>(&scr.thr[t4][kq >> 1][0]) + (kq & 1));
             }
             __syncwarp();
             const int lo_word = (BITS == 4) ? section_word_offset(NLO, lane, m) : section_word_offset(NLO, lane, m >> 1);
@@ -320,26 +355,35 @@ quantize_groups_stream(Params p, kvsink_cache c, const __half *__restrict__ k_sr
                 const __half2 w0 = __half2half2(__float2half(1.f)), w1 = __half2half2(__float2half(4.f));
                 const __half2 w2 = __half2half2(__float2half(16.f)), w3 = __half2half2(__float2half(64.f));
                 const __half2 zero2 = __half2half2(__float2half(0.f));
+                uint8_t *wb0 = (uint8_t *)(xout + lo_word) + (m & 1);
+                if (!has_sink) {
 #pragma unroll
-                for (int T = 0; T < NT; ++T) {
-                    const uint32_t m16 = tm[T];
-                    __half2 acc = base;
-                    if (m16 == 0) {
+                    for (int T = 0; T < NT; ++T) {
+                        __half2 acc = base;
                         acc = thermo_accumulate(acc, a[T][0], tA, w0);
                         acc = thermo_accumulate(acc, a[T][1], tA, w1);
                         acc = thermo_accumulate(acc, a[T][2], tB, w2);
                         acc = thermo_accumulate(acc, a[T][3], tB, w3);
-                    } else {   // sink tokens keep code 0: pair slots 0, 2 are row g, slots 1, 3 row g + 8
+                        const uint32_t bits = *reinterpret_cast<uint32_t *>(&acc);   // 0x6400 | byte in each half
+                        uint8_t *wb = wb0 + T * TILE_WORDS * 4;
+                        wb[0] = (uint8_t)bits;
+                        wb[2] = (uint8_t)(bits >> 16);
+                    }
+                } else {
+#pragma unroll
+                    for (int T = 0; T < NT; ++T) {   // sink tokens keep code 0: pair slots 0, 2 are row g, slots 1, 3 row g + 8
+                        const uint32_t m16 = tm[T];
                         const bool s0 = (m16 >> g) & 1u, s1 = (m16 >> (g + 8)) & 1u;
+                        __half2 acc = base;
                         acc = thermo_accumulate(acc, a[T][0], tA, s0 ? zero2 : w0);
                         acc = thermo_accumulate(acc, a[T][1], tA, s1 ? zero2 : w1);
                         acc = thermo_accumulate(acc, a[T][2], tB, s0 ? zero2 : w2);
                         acc = thermo_accumulate(acc, a[T][3], tB, s1 ? zero2 : w3);
+                        const uint32_t bits = *reinterpret_cast<uint32_t *>(&acc);
+                        uint8_t *wb = wb0 + T * TILE_WORDS * 4;
+                        wb[0] = (uint8_t)bits;
+                        wb[2] = (uint8_t)(bits >> 16);
                     }
-                    const uint32_t bits = *reinterpret_cast<uint32_t *>(&acc);   // 0x6400 | byte in each half
-                    uint8_t *wb = (uint8_t *)(xout + T * TILE_WORDS + lo_word);
-                    wb[m & 1] = (uint8_t)bits;
-                    wb[2 + (m & 1)] = (uint8_t)(bits >> 16);
                 }
             } else {
                 Coder kc[4];
@@ -426,15 +470,8 @@ quantize_groups_stream(Params p, kvsink_cache c, const __half *__restrict__ k_sr
                             c.v_scale[o] = s;
                             c.v_zero[o] = z;
                         }
-                        if constexpr (BITS == 2) {
-                            __half *th = reinterpret_cast<__half *>(&scr.thr[t4][kq >> 1][0]) + (kq & 1);
-                            if (g < 4) {
-                                th[0] = __ushort_as_half((unsigned short)code_threshold(s, z, 1, qmax));
-                                th[2] = __ushort_as_half((unsigned short)code_threshold(s, z, 2, qmax));
-                            } else {
-                                th[4] = __ushort_as_half((unsigned short)code_threshold(s, z, 3, qmax));
-                            }
-                        }
+                        if constexpr (BITS == 2)
+                            warp_thresholds(s, z, g, qmax, reinterpret_cast<__half *>(&scr.thr[t4][kq >> 1][0]) + (kq & 1));
                     }
                     __syncwarp();
                     if constexpr (BITS == 2) {
@@ -500,10 +537,7 @@ quantize_groups_stream(Params p, kvsink_cache c, const __half *__restrict__ k_sr
 
         // ---- sink rows: exact copies into the side buffer at the rank of their position (prefill only) ----
         if (kinds == 2) {
-            bool any = false;
-#pragma unroll
-            for (int T = 0; T < NT; ++T) any |= tm[T] != 0;
-            if (any) {
+            if (has_sink) {
                 const int count = min(c.sink_count[b], p.cap);
                 const int32_t *sp = c.sink_pos + (size_t)b * p.cap;
                 __half *side = (__half *)(kind == 0 ? c.sink_k : c.sink_v);
