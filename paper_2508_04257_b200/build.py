@@ -7,7 +7,7 @@ import subprocess
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libkvsink.so")
-SOURCES = ["api.cu", "predict.cu", "quantize.cu", "quantize_groups.cu", "decode.cu"]
+SOURCES = ["api.cu", "predict.cu", "quantize.cu", "quantize_groups.cu", "quantize_bulk.cu", "decode.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++17", "-lineinfo", "-shared", "-Xcompiler", "-fPIC"]
 
 

@@ -38,7 +38,10 @@ static int derive(const kvsink_config *cfg, Params *p)
 static int quantize_groups(const Params &p, const kvsink_cache &c, const __half *k, const __half *v, int first_token, int n_groups,
                            int64_t sb, int64_t sh, int64_t stt, bool do_v_and_sinks, cudaStream_t st)
 {
-    int rc = launch_quantize_groups_fast(p, c, k, v, first_token, n_groups, sb, sh, stt, do_v_and_sinks, st);
+    int rc = KVSINK_ERR_UNSUPPORTED;
+    if (do_v_and_sinks) rc = launch_quantize_groups_bulk(p, c, k, v, first_token, n_groups, sb, sh, stt, st);
+    if (rc != KVSINK_ERR_UNSUPPORTED) return rc;
+    rc = launch_quantize_groups_fast(p, c, k, v, first_token, n_groups, sb, sh, stt, do_v_and_sinks, st);
     if (rc != KVSINK_ERR_UNSUPPORTED) return rc;
     return launch_quantize_groups(p, c, k, v, first_token, n_groups, sb, sh, stt, do_v_and_sinks, st);
 }

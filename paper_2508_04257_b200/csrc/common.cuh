@@ -95,6 +95,8 @@ int launch_quantize_groups(const Params &p, const kvsink_cache &c, const __half 
                            int n_groups, int64_t sb, int64_t sh, int64_t stt, bool do_v_and_sinks, cudaStream_t st);
 int launch_quantize_groups_fast(const Params &p, const kvsink_cache &c, const __half *k_src, const __half *v_src, int first_token,
                                 int n_groups, int64_t sb, int64_t sh, int64_t stt, bool do_v_and_sinks, cudaStream_t st);
+int launch_quantize_groups_bulk(const Params &p, const kvsink_cache &c, const __half *k_src, const __half *v_src, int first_token,
+                                int n_groups, int64_t sb, int64_t sh, int64_t stt, cudaStream_t st);
 int launch_quantize_tokens(const Params &p, const kvsink_cache &c, const __half *k_src, const __half *v_src, int src_offset,
                            int first_token, int n_tokens, int64_t sb, int64_t sh, int64_t stt, cudaStream_t st);
 int launch_decode(const Params &p, const kvsink_cache &c, const __half *q, float *out, float *lse, void *workspace,

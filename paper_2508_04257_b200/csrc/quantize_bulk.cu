@@ -1,0 +1,560 @@
+// Whole-group quantization (Eq. 8-11 with Algorithm 1's sink exclusion) of a bulk append, fed by tensor-map bulk copies.
+//
+// One persistent block per SM whose warps never synchronise with one another.  Every warp owns one 8 KB stage of
+// shared memory and walks over its own work items: lane 0 issues the item's bulk copies (hardware swizzle, completion
+// on the warp's mbarrier), the warp waits for them, pulls the whole item into registers with ldmatrix, hands the stage
+// to the copies of its next item at once, and then does statistics, parameters, coding and its global stores from
+// registers while that item streams in.  Twenty warps per SM keep 160 KB of copies in flight.
+//
+// An item is 4096 elements of one (sequence, KV head, token group):
+//   keys   : 4096/G channels x G tokens   (per-channel statistics stay inside the warp)
+//   values : 32 tokens x 128 channels     (per-token statistics stay inside the warp)
+// ldmatrix (.trans for values, whose packed tiles are [channel x token]) gives each lane exactly the elements of its
+// pair slots in the packed tile, so the registers that served the min/max pass are coded in place and the lane's
+// packed words come out in the tile's own order.
+//
+// The copies are issued by one elected lane per warp.  (Issuing them from several lanes of one warp inside a
+// divergent loop, and a ring of stages shared by all warps whose parity waits could run two phases ahead, were both
+// tried and both faulted: every mbarrier here belongs to one warp and advances one phase per item.)
+#include <cuda.h>   // CUtensorMap and its enums; the encoder itself is looked up through the runtime
+
+#include <mutex>
+
+#include "common.cuh"
+
+namespace kvsink {
+namespace {
+
+constexpr int QB_D = 128;
+constexpr int QB_STAGE_BYTES = 8192;
+constexpr int QB_WAIT_LIMIT = 1 << 22;   // polls of an mbarrier before a warp gives up (far beyond any real latency)
+constexpr int QB_TILE_BYTES = 512, QB_ROW_BYTES = 32;   // 2-bit tile of 16 tokens x 128 channels
+
+__device__ __forceinline__ void qb_mbar_init(uint64_t *bar, unsigned count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void qb_mbar_expect_tx(uint64_t *bar, unsigned bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool qb_mbar_try_wait(uint64_t *bar, unsigned parity)
+{
+    unsigned ok;
+    asm volatile("{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
+                 : "=r"(ok) : "r"(smem_addr(bar)), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ bool qb_wait(uint64_t *bar, unsigned parity)
+{
+    int polls = 0;
+    while (!qb_mbar_try_wait(bar, parity))
+        if (++polls > QB_WAIT_LIMIT) return false;
+    return true;
+}
+// Tiled bulk copy global -> shared of one box of a rank-4 tensor map; completion is counted on `bar`.
+// The innermost coordinate is a multiple of 8 elements (16 bytes).
+__device__ __forceinline__ void qb_tma_load(void *dst, const CUtensorMap *tm, int c0, int c1, int c2, int c3, uint64_t *bar)
+{
+    asm volatile("cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
+                 ::"r"(smem_addr(dst)), "l"((uint64_t)tm), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(smem_addr(bar)) : "memory");
+}
+__device__ __forceinline__ void qb_ldmatrix_x4(uint32_t (&r)[4], uint32_t addr)
+{
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void qb_ldmatrix_x4_trans(uint32_t (&r)[4], uint32_t addr)
+{
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+
+// fp16 values in sorted order: sign-magnitude bit pattern <-> signed integer (both zeros map to 0).
+constexpr int QB_OMAX = 0x7BFF;
+__device__ __forceinline__ int qb_ord(unsigned b) { return (b & 0x8000u) ? -(int)(b & 0x7fffu) : (int)b; }
+__device__ __forceinline__ unsigned qb_unord(int o) { return o >= 0 ? (unsigned)o : (0x8000u | (unsigned)(-o)); }
+__device__ __forceinline__ float qb_val(int o) { return __half2float(__ushort_as_half((unsigned short)qb_unord(o))); }
+
+// Bit pattern of the smallest finite fp16 value whose code reaches `level`, by bisection over all finite fp16 values
+// with the literal formula; +inf if none does.  Only for the rare keys the closed form below cannot decide.
+__device__ __noinline__ unsigned qb_threshold_search(float s, float z, float level, float qmax)
+{
+    int lo = -QB_OMAX, hi = QB_OMAX + 1;
+    while (lo < hi) {
+        const int mid = (lo + hi) >> 1;
+        if ((float)code_exact(qb_val(mid), s, z, qmax) >= level) hi = mid; else lo = mid + 1;
+    }
+    return lo > QB_OMAX ? 0x7C00u : qb_unord(lo);
+}
+
+// 2-bit coder by thresholds.  code(x) = clamp(rint(x / s) + z, 0, 3) is a non-decreasing step function of the fp16
+// argument, so the smallest fp16 values t1 <= t2 <= t3 whose code reaches 1, 2, 3 describe it exactly and
+// code(x) = [x >= t1] + [x >= t2] + [x >= t3].
+//
+// Threshold of one level, exactly and without a division.  With c = level - z (an integer) the code reaches the
+// level iff rint(fl(x/s)) >= c.  The rounded quotient y = fl(x/s) is a binary32 number, so that holds iff y >= H with
+// H = c - 1/2 when c is even (rint takes the tie to the even integer c) and H = the next binary32 number above
+// c - 1/2 when c is odd.  Round-to-nearest division gives y >= H iff x/s lies above the midpoint M of H and its
+// predecessor, or on it when H has an even mantissa.  M has 25 significant bits and s 24, so s * M is exact in
+// binary64; the threshold is the first fp16 value at or above s * M, or the one after it when x/s == M is a tie
+// that rounds down.
+__device__ __forceinline__ unsigned qb_threshold(float s, double s_half, float z, float level, float qmax)
+{
+    if (s == 0.f) return 0x7C00u;                       // no member: every code is 0
+    if (!(fabsf(z) < 4194304.f)) return qb_threshold_search(s, z, level, qmax);
+    const float c = level - z, h = c - 0.5f, hc = c * 0.5f;     // all exact
+    const unsigned hb = __float_as_uint(h);
+    const float H = hc == rintf(hc) ? h : __uint_as_float(h > 0.f ? hb + 1u : hb - 1u);
+    const unsigned Hb = __float_as_uint(H);
+    const float H_dn = __uint_as_float(H > 0.f ? Hb - 1u : Hb + 1u);        // |H| >= 1/2: never zero
+    const double sm = s_half * ((double)H + (double)H_dn);                  // s * M, exact
+    const __half o = __float2half_ru(__double2float_ru(sm));                // first fp16 value >= s * M (+inf if none)
+    unsigned t = __half_as_ushort(o);
+    if ((double)__half2float(o) == sm && (Hb & 1u)) t = (t & 0x8000u) ? t - 1u : t + 1u;
+    return t;
+}
+
+// acc + w * ([x >= t1] + [x >= t2] + [x >= t3]) on both halves.
+__device__ __forceinline__ __half2 qb_thermo(__half2 acc, uint32_t x2, const __half2 (&t)[3], __half2 w)
+{
+    const __half2 x = *reinterpret_cast<const __half2 *>(&x2);
+    const __half2 cnt = __hadd2(__hadd2(__hge2(x, t[0]), __hge2(x, t[1])), __hge2(x, t[2]));
+    return __hfma2(cnt, w, acc);
+}
+
+__device__ __forceinline__ uint32_t qb_hmin2(uint32_t a, uint32_t b)
+{
+    __half2 r = __hmin2(*reinterpret_cast<__half2 *>(&a), *reinterpret_cast<__half2 *>(&b));
+    return *reinterpret_cast<uint32_t *>(&r);
+}
+__device__ __forceinline__ uint32_t qb_hmax2(uint32_t a, uint32_t b)
+{
+    __half2 r = __hmax2(*reinterpret_cast<__half2 *>(&a), *reinterpret_cast<__half2 *>(&b));
+    return *reinterpret_cast<uint32_t *>(&r);
+}
+
+struct QbShape {
+    int first_token, n_groups;
+    unsigned n_items;
+};
+
+template <int G>
+struct QbGeo {
+    static constexpr int D = QB_D;
+    static constexpr int KC = 4096 / G;           // channels of a key item
+    static constexpr int MT = KC / 16;            // matrices per tile in a key item
+    static constexpr int NT = G / 16;             // tiles per token group
+    static constexpr int NK = D / KC;             // key items per group
+    static constexpr int NV = G / 32;             // value items per group (32 tokens each)
+    static constexpr int IPG = NK + NV;           // items per group
+    static constexpr int Gv = G < D ? G : D, NGv = D / Gv;
+    static constexpr int NS = 2 * D / G;          // statistic sets per item: MT for keys, 2 * NGv for values
+    static constexpr int KPL = NS / 2;            // keys per lane
+    static constexpr int KROWB = 2 * KC;          // bytes per row of a key item in shared memory
+    static constexpr int SCRATCH = 3 * 16 * NS * 2;   // per warp: three thresholds of the item's 16 * NS keys (fp16)
+    static constexpr int WARPS = 20;              // one stage, one mbarrier and the scratch each; 102 registers per thread
+    static_assert(G == 64 || G == 128, "group size");
+    static_assert(MT == NS && 2 * NGv == NS, "statistic sets");
+};
+
+// Position of an item: sequence, KV head, token group and sub-item (keys: channel slab, then values: 32-token slab).
+struct QbPos { int sub, grp, h, b; };
+
+template <int G>
+__device__ __forceinline__ QbPos qb_decode(unsigned id, int n_groups, int Hkv)
+{
+    QbPos q;
+    q.sub = (int)(id % QbGeo<G>::IPG);
+    unsigned ug = id / QbGeo<G>::IPG;
+    q.grp = (int)(ug % (unsigned)n_groups); ug /= (unsigned)n_groups;
+    q.h = (int)(ug % (unsigned)Hkv);
+    q.b = (int)(ug / (unsigned)Hkv);
+    return q;
+}
+// q + step as mixed-radix digits (every digit of step is below its radix).
+template <int G>
+__device__ __forceinline__ QbPos qb_advance(QbPos q, const QbPos &step, int n_groups, int Hkv)
+{
+    q.sub += step.sub; int cy = q.sub >= QbGeo<G>::IPG; q.sub -= cy ? QbGeo<G>::IPG : 0;
+    q.grp += step.grp + cy; cy = q.grp >= n_groups; q.grp -= cy ? n_groups : 0;
+    q.h += step.h + cy; cy = q.h >= Hkv; q.h -= cy ? Hkv : 0;
+    q.b += step.b + cy;
+    return q;
+}
+
+// Sink bits of an item's tokens (up to 128): G/32 words for keys, one word for values; unused words are zero.
+struct QbMask { uint32_t w0, w1, w2, w3; };
+__device__ __forceinline__ uint32_t qb_mask_word(const QbMask &m, int i) { return i == 0 ? m.w0 : (i == 1 ? m.w1 : (i == 2 ? m.w2 : m.w3)); }
+
+template <int G>
+__device__ __forceinline__ void qb_load_mask(const Params &p, const kvsink_cache &c, int q_sub, int q_grp, int q_b, int first_token,
+                                             QbMask &mw)
+{
+    const uint32_t *bm = c.sink_bitmask + (size_t)q_b * p.mask_words;
+    const int p0 = first_token + q_grp * G;
+    mw.w0 = mw.w1 = mw.w2 = mw.w3 = 0u;
+    if (q_sub < QbGeo<G>::NK) {
+        mw.w0 = __ldg(bm + (p0 >> 5));
+        mw.w1 = __ldg(bm + (p0 >> 5) + 1);
+        if (G == 128) { mw.w2 = __ldg(bm + (p0 >> 5) + 2); mw.w3 = __ldg(bm + (p0 >> 5) + 3); }
+    } else {
+        mw.w0 = __ldg(bm + ((p0 + 32 * (q_sub - QbGeo<G>::NK)) >> 5));
+    }
+}
+
+// One stage refill: the bulk copies of item q into `dst`, counted on `bar` (one lane).
+template <int G>
+__device__ __forceinline__ void qb_issue(const CUtensorMap *tm_k, const CUtensorMap *tm_v, const QbPos &q, unsigned char *dst, uint64_t *bar)
+{
+    using Geo = QbGeo<G>;
+    qb_mbar_expect_tx(bar, QB_STAGE_BYTES);
+    if (q.sub < Geo::NK) {
+        qb_tma_load(dst, tm_k, q.sub * Geo::KC, q.grp * G, q.h, q.b, bar);
+    } else {
+        const int tok = q.grp * G + 32 * (q.sub - Geo::NK);
+        qb_tma_load(dst, tm_v, 0, tok, q.h, q.b, bar);
+        qb_tma_load(dst + 4096, tm_v, 64, tok, q.h, q.b, bar);
+    }
+}
+
+template <int BITS, int G>
+__global__ void __launch_bounds__(32 * QbGeo<G>::WARPS, 1)
+quantize_bulk_kernel(Params p, kvsink_cache c, const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v, QbShape sh)
+{
+    using Geo = QbGeo<G>;
+    constexpr int D = QB_D, NS = Geo::NS, KPL = Geo::KPL, MT = Geo::MT, NT = Geo::NT, NGv = Geo::NGv, NW = Geo::WARPS;
+    constexpr int MPS = 16 / NS;                  // matrices per statistic set
+    extern __shared__ __align__(1024) unsigned char smem[];
+    unsigned char *stages = smem;                                               // [warps][8 KB], 1024-byte aligned
+    uint64_t *full = (uint64_t *)(smem + NW * QB_STAGE_BYTES);                  // [warps]
+    __half *thr_all = (__half *)(full + NW);                                    // [warps][3][16 * NS] thresholds
+    const int tid = threadIdx.x, lane = tid & 31;
+    const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);                     // warp-uniform by construction
+    const int g = lane >> 2, t4 = lane & 3, mj = lane >> 3, rr = lane & 7;
+    const float qmax = 3.f;
+
+    if (tid == 0) {
+        for (int i = 0; i < NW; ++i) qb_mbar_init(&full[i], 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();   // the only block-wide barrier
+    if (smem_addr(smem) & 1023u) {   // the swizzle pattern of the stages assumes 1024-byte alignment
+        if (tid == 0) atomicOr(c.status, KVSINK_STATUS_TIMEOUT);
+        return;
+    }
+
+    // ldmatrix row addresses inside a stage: lane constants, the matrix index enters through one XOR and an offset.
+    //   values: two boxes of 64 channels with 128-byte rows (token r at 128 r, 16-byte chunk k at k ^ (r & 7));
+    //           matrix 8T + m = tile T x channels [16m, 16m+16): row 16T + rr + 8 (mj >> 1), chunk 2 (m & 3) + (mj & 1)
+    //   keys:   KROWB-byte rows of KC channels; matrix NT*mi + T: row 16T + rr + 8 (mj & 1), chunk 2 mi + (mj >> 1)
+    const uint32_t lane_v = (uint32_t)((rr + 8 * (mj >> 1)) * 128 + ((((mj & 1) ^ (rr & 1)) | (rr & 6)) << 4));
+    const uint32_t lane_k = Geo::KROWB == 64 ? (uint32_t)((rr + 8 * (mj & 1)) * 64 + ((((mj >> 1) ^ ((rr >> 1) & 1)) | ((rr >> 1) & 2)) << 4))
+                                             : (uint32_t)((rr + 8 * (mj & 1)) * 128 + ((((mj >> 1) ^ (rr & 1)) | (rr & 6)) << 4));
+
+    __half *thr = thr_all + (size_t)warp * (3 * 16 * NS);
+    unsigned char *my_stage = stages + (size_t)warp * QB_STAGE_BYTES;
+    uint64_t *my_full = full + warp;
+
+    // the block's items: in round r the block takes NW consecutive items, one per warp
+    const unsigned id_step = gridDim.x * NW;
+    const QbPos step = qb_decode<G>(id_step, sh.n_groups, p.Hkv);
+    unsigned id = blockIdx.x * NW + warp;
+    QbPos cur = qb_decode<G>(id, sh.n_groups, p.Hkv);
+    QbPos nxt = qb_advance<G>(cur, step, sh.n_groups, p.Hkv);
+    QbMask mw;
+    mw.w0 = mw.w1 = mw.w2 = mw.w3 = 0u;
+    if (id < sh.n_items) {
+        qb_load_mask<G>(p, c, cur.sub, cur.grp, cur.b, sh.first_token, mw);
+        if (lane == 0) qb_issue<G>(&tm_k, &tm_v, cur, my_stage, my_full);
+    }
+    unsigned phase = 0;                           // parity of the stage's current use
+    for (; id < sh.n_items; id += id_step, phase ^= 1u) {
+        // sink bits of the warp's next item, fetched while this one is processed
+        QbMask mw_next;
+        mw_next.w0 = mw_next.w1 = mw_next.w2 = mw_next.w3 = 0u;
+        if (id + id_step < sh.n_items) qb_load_mask<G>(p, c, nxt.sub, nxt.grp, nxt.b, sh.first_token, mw_next);
+        if (!__all_sync(0xffffffffu, qb_wait(my_full, phase))) {
+            if (lane == 0) atomicOr(c.status, KVSINK_STATUS_TIMEOUT);
+            break;
+        }
+        const uint32_t stage = smem_addr(my_stage);
+        const bool is_v = cur.sub >= Geo::NK;     // warp-uniform
+        const int sub = is_v ? cur.sub - Geo::NK : cur.sub;
+        const int64_t unit = (int64_t)cur.b * p.Hkv + cur.h;
+        const int p0 = sh.first_token + cur.grp * G;   // first token of the group (multiple of G)
+
+        // ---- the item's elements, matrix by matrix in the register order of the packed tile; matrices
+        //      [MPS*s, MPS*s + MPS) form statistic set s (keys: one 16-channel matrix column; values: one tile x channel group) ----
+        uint32_t a[16][4];
+        if (is_v) {
+#pragma unroll
+            for (int u = 0; u < 16; ++u) {
+                const int T = u >> 3, m = u & 7;
+                qb_ldmatrix_x4_trans(a[u], ((stage + lane_v) ^ ((m & 3) << 5)) + T * 2048 + (m >> 2) * 4096);
+            }
+        } else {
+#pragma unroll
+            for (int u = 0; u < 16; ++u) {
+                const int mi = u / NT, T = u % NT;
+                qb_ldmatrix_x4(a[u], ((stage + lane_k) ^ (mi << 5)) + T * 16 * Geo::KROWB);
+            }
+        }
+        const bool has_sink = (mw.w0 | mw.w1 | mw.w2 | mw.w3) != 0u;   // the same in every lane; false for almost every item
+
+        // ---- sink rows: exact copies into the side buffer at the rank of their position ----
+        if (has_sink) {
+            const int count = min(c.sink_count[cur.b], p.cap);
+            const int32_t *sp = c.sink_pos + (size_t)cur.b * p.cap;
+            __half *side = (__half *)(is_v ? c.sink_v : c.sink_k);
+            const int tok0 = is_v ? p0 + 32 * sub : p0;
+#pragma unroll
+            for (int wi = 0; wi < 4; ++wi)
+            for (uint32_t rest = qb_mask_word(mw, wi); rest != 0u; rest &= rest - 1u) {   // the set bits only
+                const int r = 32 * wi + __ffs((int)rest) - 1;
+                int lo = 0, hi = count - 1, slot = -1;
+                while (lo <= hi) {
+                    const int mid = (lo + hi) >> 1, v = sp[mid];
+                    if (v == tok0 + r) { slot = mid; break; }
+                    if (v < tok0 + r) lo = mid + 1; else hi = mid - 1;
+                }
+                if (slot < 0) {
+                    if (lane == 0) atomicOr(c.status, KVSINK_STATUS_SINK_MISMATCH);
+                    continue;
+                }
+                __half *dst = side + ((size_t)unit * p.cap + slot) * D;
+                uint32_t src;
+                int n16, off;                     // 16-byte chunks of the row held by this item, first channel
+                if (is_v) {
+                    src = stage + (lane >> 3) * 4096 + r * 128 + (((lane & 7) ^ (r & 7)) << 4);
+                    n16 = 16; off = 0;
+                } else {
+                    const int sw = Geo::KROWB == 64 ? ((r >> 1) & 3) : (r & 7);
+                    src = stage + r * Geo::KROWB + ((lane ^ sw) << 4);
+                    n16 = Geo::KC / 8; off = sub * Geo::KC;
+                }
+                if (lane < n16) {
+                    uint4 v;
+                    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(src));
+                    *(uint4 *)(dst + off + lane * 8) = v;
+                }
+            }
+        }
+
+        // ---- extremes: set s, side 0 covers registers 0,1 (keys: channels 2t,2t+1; values: tokens 2t,2t+1), side 1
+        //      registers 2,3 (the same + 8); keys leave out the rows of sink tokens ----
+        constexpr uint32_t PINF2 = 0x7C007C00u, NINF2 = 0xFC00FC00u;
+        uint32_t mn[NS][2], mx[NS][2];
+#pragma unroll
+        for (int s = 0; s < NS; ++s) { mn[s][0] = mn[s][1] = PINF2; mx[s][0] = mx[s][1] = NINF2; }
+        if (is_v || !has_sink) {
+#pragma unroll
+            for (int u = 0; u < 16; ++u) {
+                const int s = u / MPS;
+                mn[s][0] = qb_hmin2(mn[s][0], qb_hmin2(a[u][0], a[u][1])); mx[s][0] = qb_hmax2(mx[s][0], qb_hmax2(a[u][0], a[u][1]));
+                mn[s][1] = qb_hmin2(mn[s][1], qb_hmin2(a[u][2], a[u][3])); mx[s][1] = qb_hmax2(mx[s][1], qb_hmax2(a[u][2], a[u][3]));
+            }
+        } else {
+#pragma unroll
+            for (int u = 0; u < 16; ++u) {
+                const int s = u / NT, T = u % NT;
+                const uint32_t m16 = (qb_mask_word(mw, T >> 1) >> (16 * (T & 1))) & 0xffffu;
+                if (!((m16 >> g) & 1u)) {
+                    mn[s][0] = qb_hmin2(mn[s][0], a[u][0]); mx[s][0] = qb_hmax2(mx[s][0], a[u][0]);
+                    mn[s][1] = qb_hmin2(mn[s][1], a[u][2]); mx[s][1] = qb_hmax2(mx[s][1], a[u][2]);
+                }
+                if (!((m16 >> (g + 8)) & 1u)) {
+                    mn[s][0] = qb_hmin2(mn[s][0], a[u][1]); mx[s][0] = qb_hmax2(mx[s][0], a[u][1]);
+                    mn[s][1] = qb_hmin2(mn[s][1], a[u][3]); mx[s][1] = qb_hmax2(mx[s][1], a[u][3]);
+                }
+            }
+        }
+        // every lane has consumed its ldmatrix results: the stage can take the warp's next item, which streams in
+        // while this one is coded from registers
+        const QbPos nn = qb_advance<G>(nxt, step, sh.n_groups, p.Hkv);
+        __syncwarp();
+        if (lane == 0 && id + id_step < sh.n_items) qb_issue<G>(&tm_k, &tm_v, nxt, my_stage, my_full);
+
+        // the other rows of a column live in the lanes that differ in bits 2..4
+#pragma unroll
+        for (int o = 4; o < 32; o <<= 1)
+#pragma unroll
+            for (int s = 0; s < NS; ++s)
+#pragma unroll
+                for (int ab = 0; ab < 2; ++ab) {
+                    mn[s][ab] = qb_hmin2(mn[s][ab], __shfl_xor_sync(0xffffffffu, mn[s][ab], o));
+                    mx[s][ab] = qb_hmax2(mx[s][ab], __shfl_xor_sync(0xffffffffu, mx[s][ab], o));
+                }
+
+        // ---- parameters (Eq. 10-11) and thresholds: the eight lanes of a column group share its 4 * NS keys ----
+#pragma unroll
+        for (int j = 0; j < KPL; ++j) {
+            const int kk = g + 8 * j, s_ = kk >> 2, ab_ = (kk >> 1) & 1, e_ = kk & 1;
+            uint32_t smn = 0, smx = 0;
+#pragma unroll
+            for (int s = 0; s < NS; ++s)
+#pragma unroll
+                for (int ab = 0; ab < 2; ++ab)
+                    if (s_ == s && ab_ == ab) { smn = mn[s][ab]; smx = mx[s][ab]; }
+            const unsigned short lo16 = (unsigned short)(e_ ? smn >> 16 : smn & 0xffffu), hi16 = (unsigned short)(e_ ? smx >> 16 : smx & 0xffffu);
+            const float fmn = __half2float(__ushort_as_half(lo16)), fmx = __half2float(__ushort_as_half(hi16));
+            // values: token of the item (set = tile * NGv + channel group); keys: channel of the item (set = matrix)
+            const int idx = 16 * (is_v ? s_ / NGv : s_) + 8 * ab_ + 2 * t4 + e_;
+            const bool member = is_v ? !((mw.w0 >> idx) & 1u) : lo16 != 0x7C00;
+            float s, z;
+            group_params(member, fmn, fmx, qmax, &s, &z);
+            const size_t ov = ((size_t)unit * p.max_seq + p0 + 32 * sub + idx) * NGv + (s_ % NGv);
+            const size_t ok = ((size_t)unit * (p.max_seq / G) + p0 / G) * D + sub * Geo::KC + idx;
+            float *ps = is_v ? c.v_scale + ov : c.k_scale + ok, *pz = is_v ? c.v_zero + ov : c.k_zero + ok;
+            *ps = s;
+            *pz = z;
+            const int pos = 8 * (kk >> 1) + 2 * t4 + e_;
+            const double s_half = 0.5 * (double)s;
+#pragma unroll
+            for (int l = 0; l < 3; ++l) thr[l * (16 * NS) + pos] = __ushort_as_half((unsigned short)qb_threshold(s, s_half, z, (float)(l + 1), qmax));
+        }
+        __syncwarp();
+
+        // ---- coding: every register becomes its byte of packed fields (in both halves) ----
+        const __half2 base = __half2half2(__float2half(1024.f));
+        const __half2 w0 = __half2half2(__float2half(1.f)), w1 = __half2half2(__float2half(4.f));
+        const __half2 w2 = __half2half2(__float2half(16.f)), w3 = __half2half2(__float2half(64.f));
+        uint32_t bits[16];
+#pragma unroll
+        for (int s = 0; s < NS; ++s) {
+            __half2 tq[2][3];
+#pragma unroll
+            for (int ab = 0; ab < 2; ++ab)
+#pragma unroll
+                for (int l = 0; l < 3; ++l) tq[ab][l] = *reinterpret_cast<const __half2 *>(thr + l * (16 * NS) + 8 * (2 * s + ab) + 2 * t4);
+#pragma unroll
+            for (int i = 0; i < MPS; ++i) {
+                const int u = s * MPS + i;
+                __half2 acc = base;
+                acc = qb_thermo(acc, a[u][0], tq[0], w0);
+                acc = qb_thermo(acc, a[u][1], tq[0], w1);
+                acc = qb_thermo(acc, a[u][2], tq[1], w2);
+                acc = qb_thermo(acc, a[u][3], tq[1], w3);
+                bits[u] = *reinterpret_cast<uint32_t *>(&acc);   // 0x6400 | byte in each half
+            }
+        }
+        __syncwarp();   // the scratch is rewritten by the next item
+        if (has_sink && !is_v) {
+            // sink tokens keep code 0: fields 0, 2 of a byte are row g, fields 1, 3 row g + 8 (value items need nothing:
+            // the thresholds of a sink token are +inf)
+#pragma unroll
+            for (int u = 0; u < 16; ++u) {
+                const int T = u % NT;
+                const uint32_t m16 = (qb_mask_word(mw, T >> 1) >> (16 * (T & 1))) & 0xffffu;
+                if ((m16 >> g) & 1u) bits[u] &= 0xffccffccu;
+                if ((m16 >> (g + 8)) & 1u) bits[u] &= 0xff33ff33u;
+            }
+        }
+
+        // ---- packed words: bytes (even matrix lo, odd matrix lo, even matrix hi, odd matrix hi) ----
+        if (is_v) {
+            uint8_t *codes = c.v_codes + ((size_t)unit * p.max_seq) * QB_ROW_BYTES + (size_t)(p0 / KVSINK_TILE + 2 * sub) * QB_TILE_BYTES + lane * 16;
+#pragma unroll
+            for (int T = 0; T < 2; ++T) {
+                uint4 w;
+                w.x = __byte_perm(bits[8 * T + 0], bits[8 * T + 1], 0x6240); w.y = __byte_perm(bits[8 * T + 2], bits[8 * T + 3], 0x6240);
+                w.z = __byte_perm(bits[8 * T + 4], bits[8 * T + 5], 0x6240); w.w = __byte_perm(bits[8 * T + 6], bits[8 * T + 7], 0x6240);
+                *(uint4 *)(codes + T * QB_TILE_BYTES) = w;
+            }
+        } else {
+            uint8_t *codes = c.k_codes + ((size_t)unit * p.max_seq) * QB_ROW_BYTES + (size_t)(p0 / KVSINK_TILE) * QB_TILE_BYTES + lane * 16 +
+                             (sub * MT / 2) * 4;
+#pragma unroll
+            for (int T = 0; T < NT; ++T) {
+                if constexpr (MT == 2) {
+                    *(uint32_t *)(codes + T * QB_TILE_BYTES) = __byte_perm(bits[T], bits[NT + T], 0x6240);
+                } else {
+                    uint2 w;
+                    w.x = __byte_perm(bits[T], bits[NT + T], 0x6240);
+                    w.y = __byte_perm(bits[2 * NT + T], bits[3 * NT + T], 0x6240);
+                    *(uint2 *)(codes + T * QB_TILE_BYTES) = w;
+                }
+            }
+        }
+        cur = nxt;
+        nxt = nn;
+        mw = mw_next;
+    }
+}
+
+// ---- host side ----
+using EncodeTiledFn = CUresult (*)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
+                                   const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn()
+{
+    static std::once_flag once;
+    static EncodeTiledFn fn = nullptr;
+    std::call_once(once, [] {
+        void *ptr = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess && qres == cudaDriverEntryPointSuccess)
+            fn = (EncodeTiledFn)ptr;
+    });
+    return fn;
+}
+
+// fp16 tensor [B][Hkv][T][D] with element strides (sb, sh, stt, 1); box = box_ch channels x box_tok tokens.
+bool make_map(CUtensorMap *tm, const __half *base, const Params &p, int T, int64_t sb, int64_t sh, int64_t stt, int box_ch, int box_tok,
+              CUtensorMapSwizzle swz)
+{
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[4] = {(cuuint64_t)p.D, (cuuint64_t)T, (cuuint64_t)p.Hkv, (cuuint64_t)p.B};
+    // a dimension of extent 1 never advances: any valid stride will do
+    const int64_t s_h = p.Hkv > 1 ? sh : stt * T, s_b = p.B > 1 ? sb : stt * T;
+    if (stt <= 0 || s_h <= 0 || s_b <= 0) return false;
+    const cuuint64_t strides[3] = {(cuuint64_t)stt * 2, (cuuint64_t)s_h * 2, (cuuint64_t)s_b * 2};
+    const cuuint32_t box[4] = {(cuuint32_t)box_ch, (cuuint32_t)box_tok, 1, 1};
+    const cuuint32_t estr[4] = {1, 1, 1, 1};
+    return fn(tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 4, (void *)base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, swz,
+              CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int BITS, int G>
+int launch_bulk(const Params &p, const kvsink_cache &c, const __half *k_src, const __half *v_src, int first_token, int n_groups, int64_t sb,
+                int64_t sh, int64_t stt, cudaStream_t st)
+{
+    using Geo = QbGeo<G>;
+    CUtensorMap tm_k, tm_v;
+    const int T = n_groups * G;
+    if (!make_map(&tm_k, k_src, p, T, sb, sh, stt, Geo::KC, G, Geo::KROWB == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B))
+        return KVSINK_ERR_UNSUPPORTED;
+    if (!make_map(&tm_v, v_src, p, T, sb, sh, stt, 64, 32, CU_TENSOR_MAP_SWIZZLE_128B)) return KVSINK_ERR_UNSUPPORTED;
+    constexpr int NW = Geo::WARPS;
+    constexpr size_t smem = (size_t)NW * (QB_STAGE_BYTES + 8 + Geo::SCRATCH);
+    static_assert(smem <= 227 * 1024, "stages too large");
+    auto kern = quantize_bulk_kernel<BITS, G>;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return KVSINK_ERR_CUDA;
+    QbShape shp;
+    shp.first_token = first_token;
+    shp.n_groups = n_groups;
+    const long n_items = (long)p.B * p.Hkv * n_groups * Geo::IPG;
+    if (n_items >= (1L << 30)) return KVSINK_ERR_UNSUPPORTED;
+    shp.n_items = (unsigned)n_items;
+    long blocks = (n_items + NW - 1) / NW;
+    if (blocks > 148) blocks = 148;
+    kern<<<(unsigned)blocks, 32 * NW, smem, st>>>(p, c, tm_k, tm_v, shp);
+    return cudaGetLastError() == cudaSuccess ? KVSINK_OK : KVSINK_ERR_CUDA;
+}
+
+}  // namespace
+
+// Whole groups of a bulk append (keys, values and sink rows).  Returns KVSINK_ERR_UNSUPPORTED when the shape has no
+// kernel of this kind or the inputs cannot be described by a tensor map; the caller then uses another kernel.
+int launch_quantize_groups_bulk(const Params &p, const kvsink_cache &c, const __half *k_src, const __half *v_src, int first_token,
+                                int n_groups, int64_t sb, int64_t sh, int64_t stt, cudaStream_t st)
+{
+    if (p.D != QB_D || n_groups < 1) return KVSINK_ERR_UNSUPPORTED;
+    if (p.bits == 2 && p.G == 128) return launch_bulk<2, 128>(p, c, k_src, v_src, first_token, n_groups, sb, sh, stt, st);
+    if (p.bits == 2 && p.G == 64) return launch_bulk<2, 64>(p, c, k_src, v_src, first_token, n_groups, sb, sh, stt, st);
+    return KVSINK_ERR_UNSUPPORTED;
+}
+
+}  // namespace kvsink
