@@ -28,7 +28,6 @@ namespace {
 constexpr int QB_D = 128;
 constexpr int QB_STAGE_BYTES = 8192;
 constexpr int QB_WAIT_LIMIT = 1 << 22;   // polls of an mbarrier before a warp gives up (far beyond any real latency)
-constexpr int QB_TILE_BYTES = 512, QB_ROW_BYTES = 32;   // 2-bit tile of 16 tokens x 128 channels
 
 __device__ __forceinline__ void qb_mbar_init(uint64_t *bar, unsigned count)
 {
@@ -134,12 +133,77 @@ __device__ __forceinline__ uint32_t qb_hmax2(uint32_t a, uint32_t b)
     return *reinterpret_cast<uint32_t *>(&r);
 }
 
+// ---- 3- and 4-bit coder: rint(x / scale) + zero without a division per element ----
+// y = fma(x, r, M + zero) with M = 1.5 * 2^23 rounds the product to an integer in the mantissa.  It is evaluated with
+// r = 1/scale nudged down and up by 2^-22: where both agree no rounding of x/scale can fall on the other side of a tie
+// and the agreed integer is the exact answer; where they differ the lane redoes that register with the IEEE division.
+constexpr float QB_MAGIC = 12582912.0f;   // 1.5 * 2^23
+struct __align__(16) QbCoder {
+    float r_lo, r_hi;   // 1/scale nudged down / up; r_lo = +inf forces the exact path
+    float magic;        // M + zero
+    float pad;
+};
+// mn, mx: the group's extremes.  The fast form is used only where it is provably exact: |x/scale| and |zero| far below
+// 2^22 (integer in the mantissa) and the top code cannot exceed qmax (so no clamp is needed).
+__device__ __forceinline__ QbCoder qb_make_coder(float scale, float zero, float mn, float mx, float qmax)
+{
+    QbCoder c;
+    c.pad = 0.f;
+    if (scale == 0.f) {   // no member, or sink token: code 0
+        c.r_lo = c.r_hi = 0.f;
+        c.magic = QB_MAGIC;
+        return c;
+    }
+    const float r = __frcp_rn(scale);
+    const float absmax = fmaxf(fabsf(mn), fabsf(mx));
+    const bool top_fits = __fadd_rn(rintf(__fdiv_rn(mx, scale)), zero) <= qmax;
+    const bool ok = absmax * r < 2097152.f && fabsf(zero) < 2097152.f && r < 3.0e38f && top_fits;
+    c.r_lo = ok ? __fmul_rn(r, 1.f - 2.384185791015625e-07f) : __int_as_float(0x7f800000);
+    c.r_hi = ok ? __fmul_rn(r, 1.f + 2.384185791015625e-07f) : r;
+    c.magic = QB_MAGIC + (ok ? zero : 0.f);
+    return c;
+}
+// Codes of the two elements of a half2 register -> (code_lo | code_hi << 16); `differ` collects disagreement bits.
+__device__ __forceinline__ uint32_t qb_code_pair(uint32_t h2, const QbCoder &c0, const QbCoder &c1, uint32_t &differ)
+{
+    const float2 x = __half22float2(*reinterpret_cast<const __half2 *>(&h2));
+    const float a0 = fmaf(x.x, c0.r_lo, c0.magic), b0 = fmaf(x.x, c0.r_hi, c0.magic);
+    const float a1 = fmaf(x.y, c1.r_lo, c1.magic), b1 = fmaf(x.y, c1.r_hi, c1.magic);
+    differ |= (__float_as_uint(a0) ^ __float_as_uint(b0)) | (__float_as_uint(a1) ^ __float_as_uint(b1));
+    // low halves of the two results (the bit pattern of 1.5 * 2^23 has a zero low half)
+    return __byte_perm(__float_as_uint(a0), __float_as_uint(a1), 0x5410);
+}
+__device__ __noinline__ uint32_t qb_code_pair_exact(uint32_t h2, float s0, float z0, float s1, float z1, float qmax)
+{
+    const float2 x = __half22float2(*reinterpret_cast<const __half2 *>(&h2));
+    const uint32_t c0 = s0 == 0.f ? 0u : code_exact(x.x, s0, z0, qmax);
+    const uint32_t c1 = s1 == 0.f ? 0u : code_exact(x.y, s1, z1, qmax);
+    return c0 | (c1 << 16);
+}
+// Bits contributed by matrix m of a tile to a lane's words, from its four code pairs pc[r] (pair slots 4m + r).
+//   4 bit: the whole word m in `lo`.
+//   3 bit: the low two bits of the codes as a byte in each half of `lo` (byte m & 1 of each half of word m >> 1);
+//          `hi` holds this matrix's bits of word m >> 2 of the second section, already in place.
+template <int BITS>
+__device__ __forceinline__ void qb_pack_matrix(const uint32_t (&pc)[4], int m, uint32_t *lo, uint32_t *hi)
+{
+    if constexpr (BITS == 4) {
+        *lo = pc[0] | (pc[1] << 4) | (pc[2] << 8) | (pc[3] << 12);
+        *hi = 0;
+    } else {
+        *lo = (pc[0] & 0x00030003u) | ((pc[1] & 0x00030003u) << 2) | ((pc[2] & 0x00030003u) << 4) | ((pc[3] & 0x00030003u) << 6);
+        const uint32_t h = ((pc[0] >> 2) & 0x00010001u) | (((pc[1] >> 2) & 0x00010001u) << 1) | (((pc[2] >> 2) & 0x00010001u) << 4) |
+                           (((pc[3] >> 2) & 0x00010001u) << 5);
+        *hi = h << (8 * (m & 1) + 2 * (1 - ((m >> 1) & 1)));
+    }
+}
+
 struct QbShape {
     int first_token, n_groups;
     unsigned n_items;
 };
 
-template <int G>
+template <int G, int BITS = 2>
 struct QbGeo {
     static constexpr int D = QB_D;
     static constexpr int KC = 4096 / G;           // channels of a key item
@@ -152,9 +216,12 @@ struct QbGeo {
     static constexpr int NS = 2 * D / G;          // statistic sets per item: MT for keys, 2 * NGv for values
     static constexpr int KPL = NS / 2;            // keys per lane
     static constexpr int KROWB = 2 * KC;          // bytes per row of a key item in shared memory
-    static constexpr int SCRATCH = 3 * 16 * NS * 2;   // per warp: three thresholds of the item's 16 * NS keys (fp16)
+    // per warp and for each of the item's 16 * NS keys: three fp16 thresholds (2 bit), or a coder and (scale, zero)
+    static constexpr int SCRATCH = BITS == 2 ? 3 * 16 * NS * 2 : 16 * NS * (int)(sizeof(QbCoder) + sizeof(float2));
+    static constexpr int TILE_BYTES = 256 * BITS, ROW_BYTES = 16 * BITS;   // packed tile of 16 tokens x 128 channels
     static constexpr int WARPS = 20;              // one stage, one mbarrier and the scratch each; 102 registers per thread
     static_assert(G == 64 || G == 128, "group size");
+    static_assert(BITS != 3 || G == 64, "a 3-bit key item must cover whole words of the high-bit section (64 channels)");
     static_assert(MT == NS && 2 * NGv == NS, "statistic sets");
 };
 
@@ -219,20 +286,20 @@ __device__ __forceinline__ void qb_issue(const CUtensorMap *tm_k, const CUtensor
 }
 
 template <int BITS, int G>
-__global__ void __launch_bounds__(32 * QbGeo<G>::WARPS, 1)
+__global__ void __launch_bounds__(32 * QbGeo<G, BITS>::WARPS, 1)
 quantize_bulk_kernel(Params p, kvsink_cache c, const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v, QbShape sh)
 {
-    using Geo = QbGeo<G>;
+    using Geo = QbGeo<G, BITS>;
     constexpr int D = QB_D, NS = Geo::NS, KPL = Geo::KPL, MT = Geo::MT, NT = Geo::NT, NGv = Geo::NGv, NW = Geo::WARPS;
     constexpr int MPS = 16 / NS;                  // matrices per statistic set
     extern __shared__ __align__(1024) unsigned char smem[];
     unsigned char *stages = smem;                                               // [warps][8 KB], 1024-byte aligned
     uint64_t *full = (uint64_t *)(smem + NW * QB_STAGE_BYTES);                  // [warps]
-    __half *thr_all = (__half *)(full + NW);                                    // [warps][3][16 * NS] thresholds
+    unsigned char *scratch = (unsigned char *)(full + NW);                      // [warps][SCRATCH], 16-byte aligned
     const int tid = threadIdx.x, lane = tid & 31;
     const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);                     // warp-uniform by construction
     const int g = lane >> 2, t4 = lane & 3, mj = lane >> 3, rr = lane & 7;
-    const float qmax = 3.f;
+    const float qmax = (float)((1 << BITS) - 1);
 
     if (tid == 0) {
         for (int i = 0; i < NW; ++i) qb_mbar_init(&full[i], 1);
@@ -252,7 +319,9 @@ quantize_bulk_kernel(Params p, kvsink_cache c, const __grid_constant__ CUtensorM
     const uint32_t lane_k = Geo::KROWB == 64 ? (uint32_t)((rr + 8 * (mj & 1)) * 64 + ((((mj >> 1) ^ ((rr >> 1) & 1)) | ((rr >> 1) & 2)) << 4))
                                              : (uint32_t)((rr + 8 * (mj & 1)) * 128 + ((((mj >> 1) ^ (rr & 1)) | (rr & 6)) << 4));
 
-    __half *thr = thr_all + (size_t)warp * (3 * 16 * NS);
+    __half *thr = (__half *)(scratch + (size_t)warp * Geo::SCRATCH);            // 2 bit: [3][16 * NS] thresholds
+    QbCoder *coder = (QbCoder *)(scratch + (size_t)warp * Geo::SCRATCH);        // 3, 4 bit: [16 * NS] coders ...
+    float2 *sz = (float2 *)(coder + 16 * NS);                                   // ... and [16 * NS] (scale, zero)
     unsigned char *my_stage = stages + (size_t)warp * QB_STAGE_BYTES;
     uint64_t *my_full = full + warp;
 
@@ -409,70 +478,146 @@ quantize_bulk_kernel(Params p, kvsink_cache c, const __grid_constant__ CUtensorM
             *ps = s;
             *pz = z;
             const int pos = 8 * (kk >> 1) + 2 * t4 + e_;
-            const double s_half = 0.5 * (double)s;
+            if constexpr (BITS == 2) {
+                const double s_half = 0.5 * (double)s;
 #pragma unroll
-            for (int l = 0; l < 3; ++l) thr[l * (16 * NS) + pos] = __ushort_as_half((unsigned short)qb_threshold(s, s_half, z, (float)(l + 1), qmax));
+                for (int l = 0; l < 3; ++l)
+                    thr[l * (16 * NS) + pos] = __ushort_as_half((unsigned short)qb_threshold(s, s_half, z, (float)(l + 1), qmax));
+            } else {
+                coder[pos] = qb_make_coder(s, z, fmn, fmx, qmax);
+                sz[pos] = make_float2(s, z);
+            }
         }
         __syncwarp();
 
-        // ---- coding: every register becomes its byte of packed fields (in both halves) ----
-        const __half2 base = __half2half2(__float2half(1024.f));
-        const __half2 w0 = __half2half2(__float2half(1.f)), w1 = __half2half2(__float2half(4.f));
-        const __half2 w2 = __half2half2(__float2half(16.f)), w3 = __half2half2(__float2half(64.f));
-        uint32_t bits[16];
+        const size_t tile0 = (size_t)unit * (p.max_seq / KVSINK_TILE) + p0 / KVSINK_TILE + (is_v ? 2 * sub : 0);
+        uint8_t *codes = (is_v ? c.v_codes : c.k_codes) + tile0 * Geo::TILE_BYTES;
+        if constexpr (BITS == 2) {
+            // ---- coding: every register becomes its byte of packed fields (in both halves) ----
+            const __half2 base = __half2half2(__float2half(1024.f));
+            const __half2 w0 = __half2half2(__float2half(1.f)), w1 = __half2half2(__float2half(4.f));
+            const __half2 w2 = __half2half2(__float2half(16.f)), w3 = __half2half2(__float2half(64.f));
+            uint32_t bits[16];
 #pragma unroll
-        for (int s = 0; s < NS; ++s) {
-            __half2 tq[2][3];
+            for (int s = 0; s < NS; ++s) {
+                __half2 tq[2][3];
 #pragma unroll
-            for (int ab = 0; ab < 2; ++ab)
+                for (int ab = 0; ab < 2; ++ab)
 #pragma unroll
-                for (int l = 0; l < 3; ++l) tq[ab][l] = *reinterpret_cast<const __half2 *>(thr + l * (16 * NS) + 8 * (2 * s + ab) + 2 * t4);
+                    for (int l = 0; l < 3; ++l) tq[ab][l] = *reinterpret_cast<const __half2 *>(thr + l * (16 * NS) + 8 * (2 * s + ab) + 2 * t4);
 #pragma unroll
-            for (int i = 0; i < MPS; ++i) {
-                const int u = s * MPS + i;
-                __half2 acc = base;
-                acc = qb_thermo(acc, a[u][0], tq[0], w0);
-                acc = qb_thermo(acc, a[u][1], tq[0], w1);
-                acc = qb_thermo(acc, a[u][2], tq[1], w2);
-                acc = qb_thermo(acc, a[u][3], tq[1], w3);
-                bits[u] = *reinterpret_cast<uint32_t *>(&acc);   // 0x6400 | byte in each half
+                for (int i = 0; i < MPS; ++i) {
+                    const int u = s * MPS + i;
+                    __half2 acc = base;
+                    acc = qb_thermo(acc, a[u][0], tq[0], w0);
+                    acc = qb_thermo(acc, a[u][1], tq[0], w1);
+                    acc = qb_thermo(acc, a[u][2], tq[1], w2);
+                    acc = qb_thermo(acc, a[u][3], tq[1], w3);
+                    bits[u] = *reinterpret_cast<uint32_t *>(&acc);   // 0x6400 | byte in each half
+                }
             }
-        }
-        __syncwarp();   // the scratch is rewritten by the next item
-        if (has_sink && !is_v) {
-            // sink tokens keep code 0: fields 0, 2 of a byte are row g, fields 1, 3 row g + 8 (value items need nothing:
-            // the thresholds of a sink token are +inf)
+            __syncwarp();   // the scratch is rewritten by the next item
+            if (has_sink && !is_v) {
+                // sink tokens keep code 0: fields 0, 2 of a byte are row g, fields 1, 3 row g + 8 (value items need
+                // nothing: the thresholds of a sink token are +inf)
 #pragma unroll
-            for (int u = 0; u < 16; ++u) {
-                const int T = u % NT;
-                const uint32_t m16 = (qb_mask_word(mw, T >> 1) >> (16 * (T & 1))) & 0xffffu;
-                if ((m16 >> g) & 1u) bits[u] &= 0xffccffccu;
-                if ((m16 >> (g + 8)) & 1u) bits[u] &= 0xff33ff33u;
+                for (int u = 0; u < 16; ++u) {
+                    const int T = u % NT;
+                    const uint32_t m16 = (qb_mask_word(mw, T >> 1) >> (16 * (T & 1))) & 0xffffu;
+                    if ((m16 >> g) & 1u) bits[u] &= 0xffccffccu;
+                    if ((m16 >> (g + 8)) & 1u) bits[u] &= 0xff33ff33u;
+                }
             }
-        }
-
-        // ---- packed words: bytes (even matrix lo, odd matrix lo, even matrix hi, odd matrix hi) ----
-        if (is_v) {
-            uint8_t *codes = c.v_codes + ((size_t)unit * p.max_seq) * QB_ROW_BYTES + (size_t)(p0 / KVSINK_TILE + 2 * sub) * QB_TILE_BYTES + lane * 16;
+            // ---- packed words: bytes (even matrix lo, odd matrix lo, even matrix hi, odd matrix hi) ----
+            if (is_v) {
 #pragma unroll
-            for (int T = 0; T < 2; ++T) {
-                uint4 w;
-                w.x = __byte_perm(bits[8 * T + 0], bits[8 * T + 1], 0x6240); w.y = __byte_perm(bits[8 * T + 2], bits[8 * T + 3], 0x6240);
-                w.z = __byte_perm(bits[8 * T + 4], bits[8 * T + 5], 0x6240); w.w = __byte_perm(bits[8 * T + 6], bits[8 * T + 7], 0x6240);
-                *(uint4 *)(codes + T * QB_TILE_BYTES) = w;
+                for (int T = 0; T < 2; ++T) {
+                    uint4 w;
+                    w.x = __byte_perm(bits[8 * T + 0], bits[8 * T + 1], 0x6240); w.y = __byte_perm(bits[8 * T + 2], bits[8 * T + 3], 0x6240);
+                    w.z = __byte_perm(bits[8 * T + 4], bits[8 * T + 5], 0x6240); w.w = __byte_perm(bits[8 * T + 6], bits[8 * T + 7], 0x6240);
+                    *(uint4 *)(codes + T * Geo::TILE_BYTES + lane * 16) = w;
+                }
+            } else {
+#pragma unroll
+                for (int T = 0; T < NT; ++T) {
+                    uint8_t *dst = codes + T * Geo::TILE_BYTES + lane * 16 + (sub * MT / 2) * 4;
+                    if constexpr (MT == 2) {
+                        *(uint32_t *)dst = __byte_perm(bits[T], bits[NT + T], 0x6240);
+                    } else {
+                        uint2 w;
+                        w.x = __byte_perm(bits[T], bits[NT + T], 0x6240);
+                        w.y = __byte_perm(bits[2 * NT + T], bits[3 * NT + T], 0x6240);
+                        *(uint2 *)dst = w;
+                    }
+                }
             }
         } else {
-            uint8_t *codes = c.k_codes + ((size_t)unit * p.max_seq) * QB_ROW_BYTES + (size_t)(p0 / KVSINK_TILE) * QB_TILE_BYTES + lane * 16 +
-                             (sub * MT / 2) * 4;
+            // ---- coding, 3 and 4 bit: set by set (its four keys' coders from the scratch), matrix by matrix ----
+            uint32_t lo[16], hi[16];
 #pragma unroll
-            for (int T = 0; T < NT; ++T) {
-                if constexpr (MT == 2) {
-                    *(uint32_t *)(codes + T * QB_TILE_BYTES) = __byte_perm(bits[T], bits[NT + T], 0x6240);
-                } else {
-                    uint2 w;
-                    w.x = __byte_perm(bits[T], bits[NT + T], 0x6240);
-                    w.y = __byte_perm(bits[2 * NT + T], bits[3 * NT + T], 0x6240);
-                    *(uint2 *)(codes + T * QB_TILE_BYTES) = w;
+            for (int s = 0; s < NS; ++s) {
+                QbCoder kc[4];   // keys (side 0: e 0, 1; side 1: e 0, 1) of this lane's columns
+#pragma unroll
+                for (int q = 0; q < 4; ++q) kc[q] = coder[8 * (2 * s + (q >> 1)) + 2 * t4 + (q & 1)];
+#pragma unroll
+                for (int i = 0; i < MPS; ++i) {
+                    const int u = s * MPS + i;
+                    const int m = is_v ? (u & 7) : sub * MT + u / NT;   // matrix of the tile
+                    uint32_t pc[4];
+#pragma unroll
+                    for (int r = 0; r < 4; ++r) {
+                        uint32_t differ = 0;
+                        pc[r] = qb_code_pair(a[u][r], kc[2 * (r >> 1)], kc[2 * (r >> 1) + 1], differ);
+                        if (differ) {   // a value too close to a rounding tie (fp16 inputs land on exact ties often)
+                            const float2 z0 = sz[8 * (2 * s + (r >> 1)) + 2 * t4], z1 = sz[8 * (2 * s + (r >> 1)) + 2 * t4 + 1];
+                            pc[r] = qb_code_pair_exact(a[u][r], z0.x, z0.y, z1.x, z1.y, qmax);
+                        }
+                    }
+                    if (has_sink && !is_v) {   // sink tokens keep code 0: pair slots 0, 2 are row g, slots 1, 3 row g + 8
+                        const int T = u % NT;
+                        const uint32_t m16 = (qb_mask_word(mw, T >> 1) >> (16 * (T & 1))) & 0xffffu;
+                        if ((m16 >> g) & 1u) pc[0] = pc[2] = 0;
+                        if ((m16 >> (g + 8)) & 1u) pc[1] = pc[3] = 0;
+                    }
+                    qb_pack_matrix<BITS>(pc, m, &lo[u], &hi[u]);
+                }
+            }
+            __syncwarp();   // the scratch is rewritten by the next item
+            // ---- packed words.  4 bit: word m of a lane is matrix m, planes of four words.  3 bit: low section as for
+            //      2 bit (word m >> 1, byte m & 1 of each half), high section at 512 bytes (word m >> 2, two per lane) ----
+            if (is_v) {
+#pragma unroll
+                for (int T = 0; T < 2; ++T) {
+                    uint8_t *dst = codes + T * Geo::TILE_BYTES;
+                    if constexpr (BITS == 4) {
+                        *(uint4 *)(dst + lane * 16) = make_uint4(lo[8 * T], lo[8 * T + 1], lo[8 * T + 2], lo[8 * T + 3]);
+                        *(uint4 *)(dst + 512 + lane * 16) = make_uint4(lo[8 * T + 4], lo[8 * T + 5], lo[8 * T + 6], lo[8 * T + 7]);
+                    } else {
+                        uint4 w;
+                        w.x = lo[8 * T + 0] | (lo[8 * T + 1] << 8); w.y = lo[8 * T + 2] | (lo[8 * T + 3] << 8);
+                        w.z = lo[8 * T + 4] | (lo[8 * T + 5] << 8); w.w = lo[8 * T + 6] | (lo[8 * T + 7] << 8);
+                        *(uint4 *)(dst + lane * 16) = w;
+                        uint2 h;
+                        h.x = hi[8 * T + 0] | hi[8 * T + 1] | hi[8 * T + 2] | hi[8 * T + 3];
+                        h.y = hi[8 * T + 4] | hi[8 * T + 5] | hi[8 * T + 6] | hi[8 * T + 7];
+                        *(uint2 *)(dst + 512 + lane * 8) = h;
+                    }
+                }
+            } else {
+#pragma unroll
+                for (int T = 0; T < NT; ++T) {
+                    uint8_t *dst = codes + T * Geo::TILE_BYTES;
+                    if constexpr (BITS == 4 && MT == 4) {          // matrices 4 sub .. 4 sub + 3: plane `sub`
+                        *(uint4 *)(dst + sub * 512 + lane * 16) = make_uint4(lo[T], lo[NT + T], lo[2 * NT + T], lo[3 * NT + T]);
+                    } else if constexpr (BITS == 4) {              // matrices 2 sub, 2 sub + 1: half of a lane's plane entry
+                        *(uint2 *)(dst + (sub >> 1) * 512 + lane * 16 + (sub & 1) * 8) = make_uint2(lo[T], lo[NT + T]);
+                    } else {                                       // 3 bit, 64 channels: two low words and one whole high word
+                        uint2 w;
+                        w.x = lo[T] | (lo[NT + T] << 8);
+                        w.y = lo[2 * NT + T] | (lo[3 * NT + T] << 8);
+                        *(uint2 *)(dst + lane * 16 + sub * 8) = w;
+                        *(uint32_t *)(dst + 512 + lane * 8 + sub * 4) = hi[T] | hi[NT + T] | hi[2 * NT + T] | hi[3 * NT + T];
+                    }
                 }
             }
         }
@@ -521,7 +666,7 @@ template <int BITS, int G>
 int launch_bulk(const Params &p, const kvsink_cache &c, const __half *k_src, const __half *v_src, int first_token, int n_groups, int64_t sb,
                 int64_t sh, int64_t stt, cudaStream_t st)
 {
-    using Geo = QbGeo<G>;
+    using Geo = QbGeo<G, BITS>;
     CUtensorMap tm_k, tm_v;
     const int T = n_groups * G;
     if (!make_map(&tm_k, k_src, p, T, sb, sh, stt, Geo::KC, G, Geo::KROWB == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B))
@@ -554,6 +699,9 @@ int launch_quantize_groups_bulk(const Params &p, const kvsink_cache &c, const __
     if (p.D != QB_D || n_groups < 1) return KVSINK_ERR_UNSUPPORTED;
     if (p.bits == 2 && p.G == 128) return launch_bulk<2, 128>(p, c, k_src, v_src, first_token, n_groups, sb, sh, stt, st);
     if (p.bits == 2 && p.G == 64) return launch_bulk<2, 64>(p, c, k_src, v_src, first_token, n_groups, sb, sh, stt, st);
+    if (p.bits == 3 && p.G == 64) return launch_bulk<3, 64>(p, c, k_src, v_src, first_token, n_groups, sb, sh, stt, st);
+    if (p.bits == 4 && p.G == 128) return launch_bulk<4, 128>(p, c, k_src, v_src, first_token, n_groups, sb, sh, stt, st);
+    if (p.bits == 4 && p.G == 64) return launch_bulk<4, 64>(p, c, k_src, v_src, first_token, n_groups, sb, sh, stt, st);
     return KVSINK_ERR_UNSUPPORTED;
 }
 
