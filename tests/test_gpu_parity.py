@@ -117,3 +117,22 @@ def test_strided_inputs():
     kt = K.permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3)
     vt = V.permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3)
     run_both(wl, K=kt, V=vt)
+
+
+@pytest.mark.parametrize("bits,group", [(2, 128), (2, 64), (3, 64), (4, 64), (4, 128)])
+def test_bulk_append_kernel_strided_and_sink_dense(bits, group):
+    # head_dim 128 with whole groups takes the tensor-map kernel: padded rows, [B, S, H, D] storage, and a prompt in
+    # which a third of the tokens are sinks (runs that straddle tile and group boundaries, one group of sinks only)
+    wl = TINY.scaled(bits=bits, head_dim=128, group=group, n_q_heads=6, n_kv_heads=3, batch=2, seq=5 * group + 9, topk=5,
+                     pfn_n=2, seed=4000 + bits * 10 + group)
+    K, V = synth.make_kv(wl, 0, "cuda")
+    big_k = torch.zeros((wl.batch, wl.n_kv_heads, wl.seq + 8, wl.head_dim + 64), dtype=torch.float16, device="cuda")
+    big_v = torch.zeros_like(big_k)
+    big_k[:, :, :wl.seq, :wl.head_dim] = K
+    big_v[:, :, :wl.seq, :wl.head_dim] = V
+    run_both(wl, K=big_k[:, :, :wl.seq, :wl.head_dim], V=big_v[:, :, :wl.seq, :wl.head_dim], appends=1)
+    kt = K.permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3)
+    vt = V.permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3)
+    run_both(wl, K=kt, V=vt)
+    dense = wl.scaled(topk=wl.seq // 3, pfn_n=group + 3, seed=wl.seed + 1)    # first-N covers the whole first group
+    run_both(dense, appends=1)
