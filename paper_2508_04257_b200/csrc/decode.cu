@@ -229,7 +229,7 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
     constexpr float QMAX = (float)((1 << BITS) - 1);
     constexpr float R1 = 1.f / G_::ROWF, C1 = 1.f / G_::COLF;
 
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = lane >> 2, t = lane & 3;
+    const int tid = threadIdx.x, lane = tid & 31, warp = __shfl_sync(0xffffffffu, tid >> 5, 0), g = lane >> 2, t = lane & 3;
     const int split = blockIdx.x, h = blockIdx.y / qchunks, qc = blockIdx.y % qchunks, b = blockIdx.z;
     const int nq = min(8, p.rep - 8 * qc), hq0 = h * p.rep + 8 * qc;
     const int64_t unit = (int64_t)b * p.Hkv + h;
