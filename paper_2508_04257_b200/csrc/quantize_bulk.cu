@@ -371,27 +371,34 @@ quantize_bulk_kernel(Params p, kvsink_cache c, const __grid_constant__ CUtensorM
         }
         const bool has_sink = (mw.w0 | mw.w1 | mw.w2 | mw.w3) != 0u;   // the same in every lane; false for almost every item
 
-        // ---- sink rows: exact copies into the side buffer at the rank of their position ----
+        // ---- sink rows: exact copies into the side buffer at the rank of their position.  One binary search finds
+        //      the rank of the item's first sink token; the list is ascending and holds every masked token, so the
+        //      item's other sink tokens follow it one by one ----
         if (has_sink) {
             const int count = min(c.sink_count[cur.b], p.cap);
             const int32_t *sp = c.sink_pos + (size_t)cur.b * p.cap;
             __half *side = (__half *)(is_v ? c.sink_v : c.sink_k);
             const int tok0 = is_v ? p0 + 32 * sub : p0;
+            int slot = -1;                        // rank of the next sink token of the item
 #pragma unroll
             for (int wi = 0; wi < 4; ++wi)
             for (uint32_t rest = qb_mask_word(mw, wi); rest != 0u; rest &= rest - 1u) {   // the set bits only
                 const int r = 32 * wi + __ffs((int)rest) - 1;
-                int lo = 0, hi = count - 1, slot = -1;
-                while (lo <= hi) {
-                    const int mid = (lo + hi) >> 1, v = sp[mid];
-                    if (v == tok0 + r) { slot = mid; break; }
-                    if (v < tok0 + r) lo = mid + 1; else hi = mid - 1;
-                }
                 if (slot < 0) {
+                    int lo = 0, hi = count - 1;
+                    while (lo <= hi) {
+                        const int mid = (lo + hi) >> 1, v = sp[mid];
+                        if (v == tok0 + r) { slot = mid; break; }
+                        if (v < tok0 + r) lo = mid + 1; else hi = mid - 1;
+                    }
+                    if (slot < 0) slot = count;   // not in the list: reported below
+                }
+                const int my = slot++;
+                if (my >= count || sp[my] != tok0 + r) {
                     if (lane == 0) atomicOr(c.status, KVSINK_STATUS_SINK_MISMATCH);
                     continue;
                 }
-                __half *dst = side + ((size_t)unit * p.cap + slot) * D;
+                __half *dst = side + ((size_t)unit * p.cap + my) * D;
                 uint32_t src;
                 int n16, off;                     // 16-byte chunks of the row held by this item, first channel
                 if (is_v) {
