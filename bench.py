@@ -334,16 +334,26 @@ def run_ours(args):
 
     cpu = None
     if world == 1 and args.cpu_heads > 0:
+        # the oracle as it stands on the host cores: whole steps (predict once, then every instance) over the sample,
+        # repeated until about ten seconds of CPU work have been timed
         heads = min(wl.n_kv_heads, args.cpu_heads)
         sub, hH2, hK, hV, hk1, hv1, hq2 = oracle_sample(synth.WORKLOADS[args.workload], heads)
-        st = oracle_pass(sub, hH2, hK, hV, hk1, hv1, hq2)
-        for _ in range(L - 1):          # the step has L instances: time the oracle on as many passes
-            more = oracle_pass(sub, hH2, hK, hV, hk1, hv1, hq2)
-            for k in ("quantize", "append", "decode"):
-                st[k] += more[k]
+        st, steps_done, t_cpu0 = None, 0, time.perf_counter()
+        while steps_done == 0 or (time.perf_counter() - t_cpu0 < args.cpu_seconds and steps_done < 64):
+            one = oracle_pass(sub, hH2, hK, hV, hk1, hv1, hq2)
+            for _ in range(L - 1):          # the step has L instances: time the oracle on as many passes
+                more = oracle_pass(sub, hH2, hK, hV, hk1, hv1, hq2)
+                for k in ("quantize", "append", "decode"):
+                    one[k] += more[k]
+            if st is None:
+                st = one
+            else:
+                for k in kinds:
+                    st[k] += one[k]
+            steps_done += 1
         secs = st["predict"] + st["quantize"] + st["append"] + st["decode"]
-        cpu = {"value": step_bytes(sub, L) / secs / 1e9, "unit": "GB/s", "cores": st["threads"], "kind": "oracle",
-               "sample": f"{L} instances, all {wl.batch} sequences x first {heads} of {wl.n_kv_heads} KV heads of {wl.name}",
+        cpu = {"value": steps_done * step_bytes(sub, L) / secs / 1e9, "unit": "GB/s", "cores": st["threads"], "kind": "oracle",
+               "sample": f"{steps_done} steps of {L} instances, all {wl.batch} sequences x first {heads} of {wl.n_kv_heads} KV heads of {wl.name}",
                "seconds": secs, "stage_seconds": {k: st[k] for k in kinds}}
 
     launches_per_step = 2 + L * (1 + 1 + 2)
@@ -374,6 +384,7 @@ def main():
     ap.add_argument("--batch", type=int, default=0, help="override the workload's batch (profiling a smaller case)")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--cpu-heads", type=int, default=32, help="KV heads in the CPU-oracle sample (0 = skip)")
+    ap.add_argument("--cpu-seconds", type=float, default=10.0, help="CPU work to time for the oracle baseline")
     ap.add_argument("--ref-heads", type=int, default=4, help="KV heads per step of --impl reference")
     args = ap.parse_args()
     if args.impl == "reference":
