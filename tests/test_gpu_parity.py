@@ -136,3 +136,11 @@ def test_bulk_append_kernel_strided_and_sink_dense(bits, group):
     run_both(wl, K=kt, V=vt)
     dense = wl.scaled(topk=wl.seq // 3, pfn_n=group + 3, seed=wl.seed + 1)    # first-N covers the whole first group
     run_both(dense, appends=1)
+
+
+@pytest.mark.parametrize("bits,group,n_groups", [(2, 128, 1), (2, 64, 2), (3, 64, 1), (4, 128, 2)])
+def test_bulk_append_kernel_smallest_launches(bits, group, n_groups):
+    # one sequence, one KV head: fewer work items than one block has warps, extents of 1 in the tensor map
+    wl = TINY.scaled(bits=bits, head_dim=128, group=group, n_q_heads=1, n_kv_heads=1, batch=1, seq=n_groups * group, topk=3,
+                     pfn_n=1, seed=5000 + bits * 10 + group)
+    run_both(wl, appends=1)
