@@ -246,6 +246,9 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
     unsigned char *ring_all = smem_raw + Plan::fixed_bytes(nq);      // [warps][WARP_RING]; later reused for the partials
     float *part = (float *)ring_all;                                 // [2*warps][nq][D+2]
 
+    // launched with programmatic stream serialization: everything above overlaps the tail of the kernel before this
+    // one in the stream; nothing it may have written (the query, the cache) is read before this point
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     for (int i = tid; i < 8 * D; i += DEC_THREADS) {
         const int qh = i / D, ch = i % D;
         __half v = qh < nq ? q[((size_t)b * p.Hq + hq0 + qh) * D + ch] : __float2half(0.f);
@@ -260,6 +263,26 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
     __syncthreads();
 
     constexpr int PS = D + 2;                                        // partial record: o[D], m, l
+
+    // Sink rows of the side buffer are shared out over all warps of all splits and handled after the stream; the
+    // first row of this warp is fetched now, so that its latency hides behind the stream.
+    const int sink_n = min(c.sink_count[b], p.cap);
+    const int sink_worker = split * DEC_WARPS + warp, sink_workers = nsplit * DEC_WARPS;
+    int sink_pos_next = -1;
+    uint32_t sink_k_next[CPL / 2], sink_v_next[CPL / 2];
+    auto fetch_sink = [&](int j) {
+        sink_pos_next = -1;
+#pragma unroll
+        for (int e = 0; e < CPL / 2; ++e) sink_k_next[e] = sink_v_next[e] = 0u;
+        if (j < sink_n) {
+            sink_pos_next = c.sink_pos[(size_t)b * p.cap + j];
+            const uint32_t *kr = (const uint32_t *)((const __half *)c.sink_k + ((size_t)unit * p.cap + j) * D + lane * CPL);
+            const uint32_t *vr = (const uint32_t *)((const __half *)c.sink_v + ((size_t)unit * p.cap + j) * D + lane * CPL);
+#pragma unroll
+            for (int e = 0; e < CPL / 2; ++e) { sink_k_next[e] = kr[e]; sink_v_next[e] = vr[e]; }
+        }
+    };
+    fetch_sink(sink_worker);
 
     // ---------------- packed stream ----------------
     float m0 = M_INIT, m1 = M_INIT, l0 = 0.f, l1 = 0.f;             // running max / sum of query heads 2t and 2t+1
@@ -350,21 +373,27 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
     unsigned char *ring = ring_all + (size_t)warp * Plan::WARP_RING;
     float *kp_ring = (float *)(ring + NSLOT * SLOT_BYTES);           // [scale D | zero D] of the next group to prepare
     int iss_g = 0, iss_c = 0;                                        // next chunk to issue: group index, chunk within group
-    auto issue_chunk = [&](int slot) {                               // lane 0 only
+    // Every lane keeps the issue bookkeeping (so that addresses and counters stay warp-uniform values); lane 0 alone
+    // issues the copies.
+    auto issue_chunk = [&](int slot) {
         const int T0 = (g_begin + warp + iss_g * DEC_WARPS) * TPG + iss_c * CT;
         unsigned char *dst = ring + slot * SLOT_BYTES;
-        mbar_expect_tx(&cbar[slot], SLOT_BYTES);
-        bulk_g2s(dst, kc_base + (size_t)T0 * Plan::TILE_BYTES, KV_BYTES, &cbar[slot]);
-        bulk_g2s(dst + KV_BYTES, vc_base + (size_t)T0 * Plan::TILE_BYTES, KV_BYTES, &cbar[slot]);
-        bulk_g2s(dst + 2 * KV_BYTES, vs_base + (size_t)T0 * 16 * NGv, SZ_BYTES, &cbar[slot]);
-        bulk_g2s(dst + 2 * KV_BYTES + SZ_BYTES, vz_base + (size_t)T0 * 16 * NGv, SZ_BYTES, &cbar[slot]);
+        if (lane == 0) {
+            mbar_expect_tx(&cbar[slot], SLOT_BYTES);
+            bulk_g2s(dst, kc_base + (size_t)T0 * Plan::TILE_BYTES, KV_BYTES, &cbar[slot]);
+            bulk_g2s(dst + KV_BYTES, vc_base + (size_t)T0 * Plan::TILE_BYTES, KV_BYTES, &cbar[slot]);
+            bulk_g2s(dst + 2 * KV_BYTES, vs_base + (size_t)T0 * 16 * NGv, SZ_BYTES, &cbar[slot]);
+            bulk_g2s(dst + 2 * KV_BYTES + SZ_BYTES, vz_base + (size_t)T0 * 16 * NGv, SZ_BYTES, &cbar[slot]);
+        }
         if (++iss_c == CPG) { iss_c = 0; ++iss_g; }
     };
-    auto issue_params = [&](int gi) {                                // lane 0 only
+    auto issue_params = [&](int gi) {
         const int grp = g_begin + warp + gi * DEC_WARPS;
-        mbar_expect_tx(&pbar[0], Plan::KP_BYTES);
-        bulk_g2s(kp_ring, ks_base + (size_t)grp * D, D * 4, &pbar[0]);
-        bulk_g2s(kp_ring + D, kz_base + (size_t)grp * D, D * 4, &pbar[0]);
+        if (lane == 0) {
+            mbar_expect_tx(&pbar[0], Plan::KP_BYTES);
+            bulk_g2s(kp_ring, ks_base + (size_t)grp * D, D * 4, &pbar[0]);
+            bulk_g2s(kp_ring + D, kz_base + (size_t)grp * D, D * 4, &pbar[0]);
+        }
     };
     auto wait_bar = [&](uint64_t *bar, unsigned parity) {
         int polls = 0;
@@ -374,7 +403,7 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
         }
         return __all_sync(0xffffffffu, ok);
     };
-    if (lane == 0 && my_groups > 0) {
+    if (my_groups > 0) {
         issue_params(0);
         for (int i = 0; i < NSLOT - 1 && iss_g < my_groups; ++i) issue_chunk(i);
     }
@@ -403,7 +432,7 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
 #pragma unroll
             for (int e = 0; e < CPL; ++e) { scv[e] = kp[lane * CPL + e]; zev[e] = kp[D + lane * CPL + e]; }
             __syncwarp();   // the parameters are in registers: the slot can take the next group's while this one streams
-            if (lane == 0 && gi + 1 < my_groups) issue_params(gi + 1);
+            if (gi + 1 < my_groups) issue_params(gi + 1);
             // one power-of-two scaling for all heads of the group: the largest factor lands in [2^13, 2^14)
             constexpr int NQL = PL ? 4 : 8;
             float amax = 0.f;
@@ -482,7 +511,7 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
             const int slot = ci & (NSLOT - 1);
             // refill the slot freed by the previous chunk, then wait for this chunk's bytes
             __syncwarp();
-            if (lane == 0 && iss_g < my_groups) issue_chunk((ci + NSLOT - 1) & (NSLOT - 1));
+            if (iss_g < my_groups) issue_chunk((ci + NSLOT - 1) & (NSLOT - 1));
             if (!wait_bar(&cbar[slot], (unsigned)(ci / NSLOT) & 1u)) { stream_ok = false; break; }
             const uint2 mwords = mword_next;
             {   // sink bits of the warp's next chunk, fetched one chunk ahead
@@ -567,6 +596,7 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
         }
     }
     if (!stream_ok && lane == 0) atomicOr(c.status, KVSINK_STATUS_TIMEOUT);
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the merge kernel may be scheduled; it waits for this grid's end
 
     // ---- tokens of the open group: keys from the fp16 tail (last split only) ----
     if (split == nsplit - 1) {
@@ -653,7 +683,7 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
         }
     }
 
-    // ---------------- sink rows (fp16 side buffer), plain fp32 arithmetic, spread over all warps of all splits ----------------
+    // ---------------- sink rows (fp16 side buffer), plain fp32 arithmetic ----------------
     {
         float ms[8], ls[8], os[8][CPL];
 #pragma unroll
@@ -662,16 +692,17 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
 #pragma unroll
             for (int e = 0; e < CPL; ++e) os[i][e] = 0.f;
         }
-        const int count = min(c.sink_count[b], p.cap);
-        const int worker = split * DEC_WARPS + warp, nworkers = nsplit * DEC_WARPS;
-        for (int j = worker; j < count; j += nworkers) {
-            const int pos = c.sink_pos[(size_t)b * p.cap + j];
-            if (pos < 0 || pos >= n) continue;
-            const __half *kr = (const __half *)c.sink_k + ((size_t)unit * p.cap + j) * D + lane * CPL;
-            const __half *vr = (const __half *)c.sink_v + ((size_t)unit * p.cap + j) * D + lane * CPL;
+        for (int j = sink_worker; j < sink_n; j += sink_workers) {
+            const int pos = sink_pos_next;
             float kf[CPL], vf[CPL];
 #pragma unroll
-            for (int e = 0; e < CPL; ++e) { kf[e] = __half2float(kr[e]); vf[e] = __half2float(vr[e]); }
+            for (int e = 0; e < CPL / 2; ++e) {
+                const float2 k2 = __half22float2(*reinterpret_cast<const __half2 *>(&sink_k_next[e]));
+                const float2 v2 = __half22float2(*reinterpret_cast<const __half2 *>(&sink_v_next[e]));
+                kf[2 * e] = k2.x; kf[2 * e + 1] = k2.y; vf[2 * e] = v2.x; vf[2 * e + 1] = v2.y;
+            }
+            fetch_sink(j + sink_workers);   // the next row streams in while this one is used
+            if (pos < 0 || pos >= n) continue;
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
                 if (i < nq) {
@@ -731,6 +762,9 @@ __global__ void decode_merge_kernel(const float *__restrict__ part_ws, int nspli
     const size_t oq = blockIdx.x;
     const int ch = threadIdx.x;
     const float *base = part_ws + oq * nsplit * PS;
+    // launched with programmatic stream serialization: the blocks may start while the split kernel drains, and wait
+    // here until all of it has completed and its records are visible
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     float M = M_INIT;
     for (int s = 0; s < nsplit; ++s) M = fmaxf(M, base[(size_t)s * PS + D]);
     float acc = 0.f, L = 0.f;
@@ -789,12 +823,27 @@ static int launch_decode_p(const Params &p, const kvsink_cache &c, const __half 
     const size_t smem = DecodePlan<BITS, D, NGV, CT>::bytes(nq_max);
     auto kern = decode_kernel<BITS, D, NGV, CT, PL>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return KVSINK_ERR_CUDA;
-    dim3 grid(nsplit, p.Hkv * qchunks, p.B);
-    kern<<<grid, DEC_THREADS, smem, st>>>(p, c, q, out, lse, ws, nsplit, gps, qchunks, c.seq_len);
-    if (cudaGetLastError() != cudaSuccess) return KVSINK_ERR_CUDA;
+    cudaLaunchAttribute pdl[1];
+    pdl[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    pdl[0].val.programmaticStreamSerializationAllowed = 1;
+    {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(nsplit, p.Hkv * qchunks, p.B);
+        cfg.blockDim = dim3(DEC_THREADS);
+        cfg.dynamicSmemBytes = smem;
+        cfg.stream = st;
+        cfg.attrs = pdl;
+        cfg.numAttrs = 1;
+        if (cudaLaunchKernelEx(&cfg, kern, p, c, q, out, lse, ws, nsplit, gps, qchunks, (int)c.seq_len) != cudaSuccess) return KVSINK_ERR_CUDA;
+    }
     if (nsplit > 1) {
-        decode_merge_kernel<<<p.B * p.Hq, D, 0, st>>>(ws, nsplit, D, out, lse);
-        if (cudaGetLastError() != cudaSuccess) return KVSINK_ERR_CUDA;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(p.B * p.Hq);
+        cfg.blockDim = dim3(D);
+        cfg.stream = st;
+        cfg.attrs = pdl;
+        cfg.numAttrs = 1;
+        if (cudaLaunchKernelEx(&cfg, decode_merge_kernel, (const float *)ws, nsplit, (int)D, out, lse) != cudaSuccess) return KVSINK_ERR_CUDA;
     }
     return KVSINK_OK;
 }
