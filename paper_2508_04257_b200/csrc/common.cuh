@@ -86,6 +86,28 @@ __device__ __forceinline__ uint32_t code_exact(float x, float scale, float zero,
     return (uint32_t)(int)q;
 }
 
+// Programmatic stream serialization (dependent launch).  A kernel launched with launch_pdl may be scheduled while its
+// predecessor in the stream is still draining; it must call pdl_wait() before it reads or writes anything a predecessor
+// may have touched.  pdl_wait() returns once every prerequisite grid has completed and its writes are visible (at once
+// when the kernel was launched the ordinary way).
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args)
+{
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kern, KArgs(args)...);
+}
+
 __device__ __forceinline__ bool mask_bit(const uint32_t *__restrict__ bm, int pos) { return (bm[pos >> 5] >> (pos & 31)) & 1u; }
 
 // Launchers implemented in the kernel translation units; all return a KVSINK_* code.

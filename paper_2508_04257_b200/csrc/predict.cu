@@ -15,6 +15,7 @@ __global__ void sink_score_listed(const uint16_t *__restrict__ H, int S, int64_t
 {
     int i = blockIdx.x * blockDim.x + threadIdx.x;
     int b = blockIdx.y;
+    pdl_wait();
     if (i >= S) return;
     const uint16_t *row = H + b * sb + i * ss;
     unsigned best = 0;
@@ -32,6 +33,7 @@ __global__ void sink_score_all(const uint16_t *__restrict__ H, int S, int d, int
 {
     int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
     int b = blockIdx.y;
+    pdl_wait();
     if (warp >= S) return;
     const uint16_t *row = H + b * sb + warp * ss;
     unsigned best = 0;
@@ -82,6 +84,7 @@ sink_select(const uint16_t *__restrict__ score, int score_stride, int S, int k, 
     const int b = blockIdx.x, tid = threadIdx.x;
     const uint16_t *sc = score + (size_t)b * score_stride;
     const int kk = k < S ? k : S;
+    pdl_wait();
     int vstar = 0x10000, r = 0;   // no score exceeds 0x10000: no top-k selection when kk == 0
     if (kk > 0) {
         if (tid < 256) hist[tid] = 0;
@@ -158,14 +161,16 @@ int launch_predict_sinks(const Params &p, const __half *hidden, int S, int64_t s
             cl.n = p.n_channels;
             for (int i = 0; i < 8; ++i) cl.c[i] = p.channels[i];
             dim3 grid((S + 255) / 256, p.B);
-            sink_score_listed<<<grid, 256, 0, st>>>((const uint16_t *)hidden, S, sb, ss, cl, score, stride);
+            if (launch_pdl(sink_score_listed, grid, dim3(256), 0, st, (const uint16_t *)hidden, S, sb, ss, cl, score, stride) != cudaSuccess)
+                return KVSINK_ERR_CUDA;
         } else {
             dim3 grid((S + 7) / 8, p.B);
-            sink_score_all<<<grid, 256, 0, st>>>((const uint16_t *)hidden, S, p.hidden, sb, ss, score, stride);
+            if (launch_pdl(sink_score_all, grid, dim3(256), 0, st, (const uint16_t *)hidden, S, p.hidden, sb, ss, score, stride) != cudaSuccess)
+                return KVSINK_ERR_CUDA;
         }
     }
-    sink_select<<<p.B, SEL_THREADS, 0, st>>>(score, stride, S, p.topk, p.pfn_n, p.mask_words, p.cap, bitmask, sink_pos, sink_count);
-    return cudaGetLastError() == cudaSuccess ? KVSINK_OK : KVSINK_ERR_CUDA;
+    return launch_pdl(sink_select, dim3(p.B), dim3(SEL_THREADS), 0, st, (const uint16_t *)score, stride, S, p.topk, p.pfn_n, p.mask_words,
+                      p.cap, bitmask, sink_pos, sink_count) == cudaSuccess ? KVSINK_OK : KVSINK_ERR_CUDA;
 }
 
 }  // namespace kvsink

@@ -240,6 +240,7 @@ quantize_tokens_kernel(Params p, kvsink_cache c, const __half *__restrict__ k_sr
     const float qmax = (float)((1 << p.bits) - 1);
     const uint32_t *bm = c.sink_bitmask + (size_t)b * p.mask_words;
     if (tid < KVSINK_TILE) present[tid] = (tile * KVSINK_TILE + tid >= t_lo && tile * KVSINK_TILE + tid < t_hi) ? 1 : 0;
+    pdl_wait();
 
     const int cpl = D / 32;   // channels per lane (2 or 4)
     for (int pos = t_lo + warp; pos < t_hi; pos += QT_THREADS / 32) {
@@ -309,8 +310,8 @@ int launch_quantize_tokens(const Params &p, const kvsink_cache &c, const __half 
     if (n_tokens <= 0) return KVSINK_OK;
     int tiles = (first_token + n_tokens - 1) / KVSINK_TILE - first_token / KVSINK_TILE + 1;
     dim3 grid(tiles, p.Hkv, p.B);
-    quantize_tokens_kernel<<<grid, QT_THREADS, 0, st>>>(p, c, k_src, v_src, src_offset, first_token, n_tokens, sb, sh, stt);
-    return cudaGetLastError() == cudaSuccess ? KVSINK_OK : KVSINK_ERR_CUDA;
+    return launch_pdl(quantize_tokens_kernel, grid, dim3(QT_THREADS), 0, st, p, c, k_src, v_src, src_offset, first_token, n_tokens, sb, sh,
+                      stt) == cudaSuccess ? KVSINK_OK : KVSINK_ERR_CUDA;
 }
 
 }  // namespace kvsink

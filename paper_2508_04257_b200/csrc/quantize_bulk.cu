@@ -306,6 +306,7 @@ quantize_bulk_kernel(Params p, kvsink_cache c, const __grid_constant__ CUtensorM
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();   // the only block-wide barrier
+    pdl_wait();        // nothing before this line touches global memory
     if (smem_addr(smem) & 1023u) {   // the swizzle pattern of the stages assumes 1024-byte alignment
         if (tid == 0) atomicOr(c.status, KVSINK_STATUS_TIMEOUT);
         return;
@@ -692,8 +693,7 @@ int launch_bulk(const Params &p, const kvsink_cache &c, const __half *k_src, con
     shp.n_items = (unsigned)n_items;
     long blocks = (n_items + NW - 1) / NW;
     if (blocks > 148) blocks = 148;
-    kern<<<(unsigned)blocks, 32 * NW, smem, st>>>(p, c, tm_k, tm_v, shp);
-    return cudaGetLastError() == cudaSuccess ? KVSINK_OK : KVSINK_ERR_CUDA;
+    return launch_pdl(kern, dim3((unsigned)blocks), dim3(32 * NW), smem, st, p, c, tm_k, tm_v, shp) == cudaSuccess ? KVSINK_OK : KVSINK_ERR_CUDA;
 }
 
 }  // namespace
