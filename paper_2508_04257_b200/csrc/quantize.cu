@@ -65,6 +65,51 @@ __device__ __forceinline__ uint32_t assemble_word(int bits, int D, int word, Get
     return out;
 }
 
+// The same walk over a word's fields, for the insert path: get(m,row,col) returns the code, or a value >= 0x100 for an
+// element that is not being written; *fieldmask receives the bits of the fields that are.
+template <typename Get>
+__device__ __forceinline__ uint32_t assemble_word_masked(int bits, int D, int word, Get get, uint32_t *fieldmask)
+{
+    uint32_t out = 0, msk = 0;
+    int lane, i, m, row, col;
+    auto put = [&](uint32_t v, uint32_t width_mask, int shift) {
+        const bool on = v < 0x100u;
+        out |= on ? (v & width_mask) << shift : 0u;
+        msk |= on ? width_mask << shift : 0u;
+    };
+    if (bits == 2 || bits == 4) {
+        const int n = D * bits / 64, fields = 16 / bits;
+        section_word_owner(n, word, &lane, &i);
+        for (int k = 0; k < fields; ++k)
+            for (int e = 0; e < 2; ++e) {
+                slot_to_elem(lane, fields * i + k, e, &m, &row, &col);
+                put(get(m, row, col), (1u << bits) - 1u, 16 * e + bits * k);
+            }
+    } else {
+        const int nlo = D / 32, nhi = D / 64;
+        if (word < 32 * nlo) {
+            section_word_owner(nlo, word, &lane, &i);
+            for (int k = 0; k < 8; ++k)
+                for (int e = 0; e < 2; ++e) {
+                    slot_to_elem(lane, 8 * i + k, e, &m, &row, &col);
+                    put(get(m, row, col), 3u, 16 * e + 2 * k);
+                }
+        } else {
+            int j;
+            section_word_owner(nhi, word - 32 * nlo, &lane, &j);
+            for (int w = 0; w < 2; ++w)
+                for (int k = 0; k < 8; ++k)
+                    for (int e = 0; e < 2; ++e) {
+                        slot_to_elem(lane, 8 * (2 * j + w) + k, e, &m, &row, &col);
+                        const uint32_t v = get(m, row, col);
+                        put(v < 0x100u ? v >> 2 : v, 1u, 16 * e + 4 * (k >> 1) + 2 * (1 - w) + (k & 1));
+                    }
+        }
+    }
+    *fieldmask = msk;
+    return out;
+}
+
 // ---------------------------------------------------------------------------------------------------------
 // Whole groups: one block per (token group, KV head, sequence).  Keys per channel over the group's non-sink
 // tokens, values per token, sink rows to the side buffer.
@@ -297,10 +342,10 @@ quantize_tokens_kernel(Params p, kvsink_cache c, const __half *__restrict__ k_sr
     const bool fresh = (t_lo % KVSINK_TILE) == 0;   // no earlier token lives in this tile
     for (int word = tid; word < tile_words; word += QT_THREADS) {
         uint32_t keep = fresh ? 0u : vout[word];
-        uint32_t newbits = assemble_word(p.bits, D, word, [&](int m, int row, int col) {
-            return present[col] ? (uint32_t)vcode[col * D + 16 * m + row] : 0u; });
-        uint32_t fieldmask = assemble_word(p.bits, D, word, [&](int m, int row, int col) { return present[col] ? 0xffu : 0u; });
-        vout[word] = (keep & ~fieldmask) | newbits;
+        uint32_t fieldmask;
+        const uint32_t newbits = assemble_word_masked(p.bits, D, word, [&](int m, int row, int col) {
+            return present[col] ? (uint32_t)vcode[col * D + 16 * m + row] : 0x100u; }, &fieldmask);
+        if (fieldmask || fresh) vout[word] = (keep & ~fieldmask) | newbits;   // a fresh tile is written whole
     }
 }
 
