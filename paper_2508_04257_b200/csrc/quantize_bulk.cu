@@ -4,7 +4,7 @@
 // shared memory and walks over its own work items: lane 0 issues the item's bulk copies (hardware swizzle, completion
 // on the warp's mbarrier), the warp waits for them, pulls the whole item into registers with ldmatrix, hands the stage
 // to the copies of its next item at once, and then does statistics, parameters, coding and its global stores from
-// registers while that item streams in.  Twenty warps per SM keep 160 KB of copies in flight.
+// registers while that item streams in.  Sixteen to twenty warps per SM keep 128-160 KB of copies in flight.
 //
 // An item is 4096 elements of one (sequence, KV head, token group):
 //   keys   : 4096/G channels x G tokens   (per-channel statistics stay inside the warp)
@@ -219,7 +219,9 @@ struct QbGeo {
     // per warp and for each of the item's 16 * NS keys: three fp16 thresholds (2 bit), or a coder and (scale, zero)
     static constexpr int SCRATCH = BITS == 2 ? 3 * 16 * NS * 2 : 16 * NS * (int)(sizeof(QbCoder) + sizeof(float2));
     static constexpr int TILE_BYTES = 256 * BITS, ROW_BYTES = 16 * BITS;   // packed tile of 16 tokens x 128 channels
-    static constexpr int WARPS = 20;              // one stage, one mbarrier and the scratch each; 102 registers per thread
+    // warps per block, each with one stage, one mbarrier and its scratch: 20 (96 registers per thread) for the 2-bit
+    // coder; 16 (128 registers) for the 3- and 4-bit coder, which spills at 96 and measures 9 % faster this way
+    static constexpr int WARPS = BITS == 2 ? 20 : 16;
     static_assert(G == 64 || G == 128, "group size");
     static_assert(BITS != 3 || G == 64, "a 3-bit key item must cover whole words of the high-bit section (64 channels)");
     static_assert(MT == NS && 2 * NGv == NS, "statistic sets");
