@@ -72,6 +72,38 @@ __device__ __forceinline__ int block_excl_count(bool flag, int *total, unsigned 
     return before + within;
 }
 
+// Largest bin index whose suffix count (keys in bins >= it) reaches `need`, and how many of that bin's keys are still
+// needed, from a 256-bin histogram; one warp, eight bins per lane.  need >= 1; if the histogram holds fewer than
+// `need` keys the answer is bin 0.
+__device__ __forceinline__ void find_bin(const unsigned *hist, int need, int *bin_out, int *rest_out)
+{
+    const int lane = threadIdx.x & 31;
+    // lane l owns bins 255 - 8l ... 248 - 8l (descending), so that a prefix over lanes is a suffix over bins
+    unsigned h[8], mine = 0;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) { h[j] = hist[255 - 8 * lane - j]; mine += h[j]; }
+    unsigned incl = mine;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const unsigned x = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += x;
+    }
+    const unsigned before = incl - mine;                         // keys in the bins above this lane's
+    const unsigned hit = __ballot_sync(0xffffffffu, (int)incl >= need);
+    const int owner = hit ? __ffs((int)hit) - 1 : 31;            // first lane whose bins reach the count
+    if (lane == owner) {
+        int cum = (int)before, bin = 255 - 8 * lane;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            bin = 255 - 8 * lane - j;
+            if (cum + (int)h[j] >= need || bin == 0) break;
+            cum += (int)h[j];
+        }
+        *bin_out = bin;
+        *rest_out = need - cum;
+    }
+}
+
 // One block per sequence: 2-pass radix select of the k-th largest 16-bit score, then an ordered pass that
 // breaks ties by index, ORs the first N tokens in and emits mask words and ascending positions.
 __global__ void __launch_bounds__(SEL_THREADS)
@@ -80,7 +112,7 @@ sink_select(const uint16_t *__restrict__ score, int score_stride, int S, int k, 
 {
     __shared__ unsigned hist[256];
     __shared__ unsigned warp_tot[32];
-    __shared__ int s_hi, s_need, s_vstar, s_r;
+    __shared__ int s_hi, s_need, s_lo, s_r;
     const int b = blockIdx.x, tid = threadIdx.x;
     const uint16_t *sc = score + (size_t)b * score_stride;
     const int kk = k < S ? k : S;
@@ -91,15 +123,7 @@ sink_select(const uint16_t *__restrict__ score, int score_stride, int S, int k, 
         __syncthreads();
         for (int i = tid; i < S; i += SEL_THREADS) atomicAdd(&hist[sc[i] >> 8], 1u);
         __syncthreads();
-        if (tid == 0) {
-            int cum = 0, bin = 255;
-            for (; bin > 0; --bin) {
-                if (cum + (int)hist[bin] >= kk) break;
-                cum += (int)hist[bin];
-            }
-            s_hi = bin;
-            s_need = kk - cum;
-        }
+        if (tid < 32) find_bin(hist, kk, &s_hi, &s_need);
         __syncthreads();
         const int hi = s_hi;
         if (tid < 256) hist[tid] = 0;
@@ -109,17 +133,9 @@ sink_select(const uint16_t *__restrict__ score, int score_stride, int S, int k, 
             if ((int)(v >> 8) == hi) atomicAdd(&hist[v & 0xffu], 1u);
         }
         __syncthreads();
-        if (tid == 0) {
-            int cum = 0, bin = 255, need = s_need;
-            for (; bin > 0; --bin) {
-                if (cum + (int)hist[bin] >= need) break;
-                cum += (int)hist[bin];
-            }
-            s_vstar = (hi << 8) | bin;
-            s_r = need - cum;
-        }
+        if (tid < 32) find_bin(hist, s_need, &s_lo, &s_r);
         __syncthreads();
-        vstar = s_vstar;
+        vstar = (hi << 8) | s_lo;
         r = s_r;
     }
     int run_eq = 0, run_sel = 0;
