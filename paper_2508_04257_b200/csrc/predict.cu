@@ -51,25 +51,29 @@ __global__ void sink_score_all(const uint16_t *__restrict__ H, int S, int d, int
 
 constexpr int SEL_THREADS = 1024;
 
-// Exclusive prefix count of `flag` over the block in thread order; *total = number of set flags.
-__device__ __forceinline__ int block_excl_count(bool flag, int *total, unsigned *warp_tot)
+// Exclusive prefix sum of `v` over the block in thread order; *total = the sum over the block.
+__device__ __forceinline__ int block_excl_sum(int v, int *total, unsigned *warp_tot)
 {
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
-    unsigned bal = __ballot_sync(0xffffffffu, flag);
-    int within = __popc(bal & ((1u << lane) - 1u));
-    if (lane == 0) warp_tot[w] = __popc(bal);
-    __syncthreads();
-    unsigned v = warp_tot[lane];
-    unsigned incl = v;
+    int incl = v;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
-        unsigned x = __shfl_up_sync(0xffffffffu, incl, o);
+        const int x = __shfl_up_sync(0xffffffffu, incl, o);
         if (lane >= o) incl += x;
     }
-    int before = (int)__shfl_sync(0xffffffffu, incl - v, w);
-    *total = (int)__shfl_sync(0xffffffffu, incl, 31);
+    if (lane == 31) warp_tot[w] = (unsigned)incl;
     __syncthreads();
-    return before + within;
+    const unsigned t = warp_tot[lane];           // SEL_THREADS / 32 == 32 warps
+    unsigned tincl = t;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const unsigned x = __shfl_up_sync(0xffffffffu, tincl, o);
+        if (lane >= o) tincl += x;
+    }
+    const int before = (int)__shfl_sync(0xffffffffu, tincl - t, w);
+    *total = (int)__shfl_sync(0xffffffffu, tincl, 31);
+    __syncthreads();
+    return before + incl - v;
 }
 
 // Largest bin index whose suffix count (keys in bins >= it) reaches `need`, and how many of that bin's keys are still
@@ -138,20 +142,49 @@ sink_select(const uint16_t *__restrict__ score, int score_stride, int S, int k, 
         vstar = (hi << 8) | s_lo;
         r = s_r;
     }
+    // Ordered pass, TPT consecutive tokens per thread and step: two block scans per TPT * 1024 tokens.
+    constexpr int TPT = 4;
     int run_eq = 0, run_sel = 0;
-    const int S_round = (S + SEL_THREADS - 1) / SEL_THREADS * SEL_THREADS;
-    for (int base = 0; base < S_round; base += SEL_THREADS) {
-        const int i = base + tid;
-        const int key = i < S ? (int)sc[i] : -1;
-        const bool gt = key > vstar, eq = key == vstar;
+    const int lane = tid & 31;
+    const int step = SEL_THREADS * TPT;
+    const int S_round = (S + step - 1) / step * step;
+    for (int base = 0; base < S_round; base += step) {
+        const int i0 = base + TPT * tid;
+        int key[TPT];
+        if (i0 + TPT <= S) {   // the score rows are 16-byte aligned and i0 is a multiple of 4
+            const uint2 v = *reinterpret_cast<const uint2 *>(sc + i0);
+            key[0] = (int)(v.x & 0xffffu); key[1] = (int)(v.x >> 16); key[2] = (int)(v.y & 0xffffu); key[3] = (int)(v.y >> 16);
+        } else {
+#pragma unroll
+            for (int j = 0; j < TPT; ++j) key[j] = i0 + j < S ? (int)sc[i0 + j] : -1;
+        }
+        int n_eq = 0;
+#pragma unroll
+        for (int j = 0; j < TPT; ++j) n_eq += key[j] == vstar;
         int tot_eq;
-        const int eq_rank = run_eq + block_excl_count(eq, &tot_eq, warp_tot);
-        const bool sel = i < S && (i < N || gt || (eq && eq_rank < r));
-        const unsigned word = __ballot_sync(0xffffffffu, sel);
-        if ((tid & 31) == 0 && (i >> 5) < mask_words) bitmask[(size_t)b * mask_words + (i >> 5)] = word;
+        int eq_rank = run_eq + block_excl_sum(n_eq, &tot_eq, warp_tot);
+        unsigned nib = 0;
+#pragma unroll
+        for (int j = 0; j < TPT; ++j) {
+            const bool eq = key[j] == vstar;
+            const bool sel = i0 + j < S && (i0 + j < N || key[j] > vstar || (eq && eq_rank < r));
+            eq_rank += eq;
+            nib |= (unsigned)sel << j;
+        }
+        // eight threads share a mask word
+        unsigned word = nib << (4 * (lane & 7));
+        word |= __shfl_xor_sync(0xffffffffu, word, 1);
+        word |= __shfl_xor_sync(0xffffffffu, word, 2);
+        word |= __shfl_xor_sync(0xffffffffu, word, 4);
+        if ((lane & 7) == 0 && (i0 >> 5) < mask_words) bitmask[(size_t)b * mask_words + (i0 >> 5)] = word;
         int tot_sel;
-        const int rank = run_sel + block_excl_count(sel, &tot_sel, warp_tot);
-        if (sel && rank < cap) sink_pos[(size_t)b * cap + rank] = i;
+        int rank = run_sel + block_excl_sum(__popc(nib), &tot_sel, warp_tot);
+#pragma unroll
+        for (int j = 0; j < TPT; ++j)
+            if ((nib >> j) & 1u) {
+                if (rank < cap) sink_pos[(size_t)b * cap + rank] = i0 + j;
+                ++rank;
+            }
         run_eq += tot_eq;
         run_sel += tot_sel;
     }
