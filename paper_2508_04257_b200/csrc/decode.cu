@@ -223,7 +223,7 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
     constexpr int NM = G_::NM, W = G_::W, BST = Plan::BST, TILE_WORDS = 32 * W;
     constexpr int NSLOT = Plan::NSLOT, SLOT_BYTES = Plan::SLOT_BYTES, KV_BYTES = Plan::KV_BYTES, SZ_BYTES = Plan::SZ_BYTES;
     constexpr int mpg = (D / NGv) / 16;                              // value matrices per channel group
-    constexpr int ST = CT >= 2 ? 2 : 1;                              // tiles per softmax step
+    constexpr int ST = CT >= 4 ? 4 : (CT >= 2 ? 2 : 1);                              // tiles per softmax step
     constexpr int CPL = D / 32;                                      // channels per lane in per-channel passes
     constexpr float LOG2E = 1.4426950408889634f;
     constexpr float QMAX = (float)((1 << BITS) - 1);
@@ -526,7 +526,7 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
             const uint32_t *kt = kt0 + sub * ST * TILE_WORDS, *vt = vt0 + sub * ST * TILE_WORDS;
             const float *ssv = ssv0 + sub * ST * 16 * NGv, *szv = szv0 + sub * ST * 16 * NGv;
             const int T0 = grp * TPG + cj * CT + sub * ST;
-            const uint32_t mword = sub == 0 ? mwords.x : mwords.y;
+            const uint32_t mword = ST == 4 ? (mwords.x | mwords.y) : (sub == 0 ? mwords.x : mwords.y);
 
             // scores of the chunk's tiles
             float s[ST][4];
@@ -561,7 +561,7 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
             if (mword) {   // sink tokens are not part of the packed stream (their value parameters are zero)
 #pragma unroll
                 for (int k = 0; k < ST; ++k) {
-                    const uint32_t mask16 = (mword >> (16 * ((T0 + k) & 1))) & 0xffffu;
+                    const uint32_t mask16 = ((ST == 4 ? (k < 2 ? mwords.x : mwords.y) : mword) >> (16 * ((T0 + k) & 1))) & 0xffffu;
                     if ((mask16 >> g) & 1u) s[k][0] = s[k][1] = -INFINITY;
                     if ((mask16 >> (g + 8)) & 1u) s[k][2] = s[k][3] = -INFINITY;
                 }
@@ -569,7 +569,8 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
             // one softmax step for the whole chunk
             {
                 float tm0 = fmaxf(s[0][0], s[0][2]), tm1 = fmaxf(s[0][1], s[0][3]);
-                if (ST == 2) { tm0 = fmaxf(tm0, fmaxf(s[ST - 1][0], s[ST - 1][2])); tm1 = fmaxf(tm1, fmaxf(s[ST - 1][1], s[ST - 1][3])); }
+#pragma unroll
+                for (int k = 1; k < ST; ++k) { tm0 = fmaxf(tm0, fmaxf(s[k][0], s[k][2])); tm1 = fmaxf(tm1, fmaxf(s[k][1], s[k][3])); }
                 advance_max(tm0, tm1);
             }
             // value scales of this lane's tokens; their maximum bounds the fp16 range needed
