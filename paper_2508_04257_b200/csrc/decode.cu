@@ -10,6 +10,8 @@
 // Each warp streams whole key groups of one (sequence, KV head) unit; sequence splits are merged by a second
 // kernel.  Sink tokens are masked out of the packed stream and added from the fp16 side buffer under the same
 // softmax; keys of the open group come from the fp16 tail.
+#include <cooperative_groups.h>
+
 #include <mutex>
 
 #include "common.cuh"
@@ -216,7 +218,7 @@ struct DecodePlan {
 template <int BITS, int D, int NGv, int CT, bool PL>
 __global__ void __launch_bounds__(DEC_THREADS, 4)
 decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__restrict__ out, float *__restrict__ lse,
-              float *__restrict__ part_ws, int nsplit, int groups_per_split, int qchunks, int seq_len)
+              float *__restrict__ part_ws, int nsplit, int groups_per_split, int qchunks, int seq_len, int cluster_merge)
 {
     using G_ = Geo<BITS, D>;
     using Plan = DecodePlan<BITS, D, NGv, CT>;
@@ -749,10 +751,37 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
             out[oq * D + ch] = L > 0.f ? acc / L : 0.f;
             if (lse && ch == 0) lse[oq] = L > 0.f ? (M + log2f(L)) * 0.6931471805599453f : -INFINITY;
         } else {
-            float *wsr = part_ws + (oq * nsplit + split) * PS;
+            // the split's record: to the workspace for the merge kernel, or, when the splits of a unit form a thread-block
+            // cluster, to this block's shared memory (the query tables are no longer needed) for the cluster's first block
+            float *wsr = cluster_merge ? qs + (size_t)qh * PS : part_ws + (oq * nsplit + split) * PS;
             wsr[ch] = acc;
             if (ch == 0) { wsr[D] = M; wsr[D + 1] = L; }
         }
+    }
+    if (cluster_merge) {
+        // the splits of a unit are the blocks of one cluster: its first block reads the records of the others through
+        // distributed shared memory and merges them in split order (the same arithmetic as the merge kernel)
+        namespace cg = cooperative_groups;
+        cg::cluster_group cluster = cg::this_cluster();
+        cluster.sync();
+        if (split == 0) {
+            for (int idx = tid; idx < nq * D; idx += DEC_THREADS) {
+                const int qh = idx / D, ch = idx % D;
+                float M = M_INIT;
+                for (int sp = 0; sp < nsplit; ++sp) M = fmaxf(M, cluster.map_shared_rank(qs, sp)[(size_t)qh * PS + D]);
+                float acc = 0.f, L = 0.f;
+                for (int sp = 0; sp < nsplit; ++sp) {
+                    const float *pr = cluster.map_shared_rank(qs, sp) + (size_t)qh * PS;
+                    const float f = ex2(pr[D] - M);
+                    acc += pr[ch] * f;
+                    L += pr[D + 1] * f;
+                }
+                const size_t oq = (size_t)b * p.Hq + hq0 + qh;
+                out[oq * D + ch] = L > 0.f ? acc / L : 0.f;
+                if (lse && ch == 0) lse[oq] = L > 0.f ? (M + log2f(L)) * 0.6931471805599453f : -INFINITY;
+            }
+        }
+        cluster.sync();   // nobody's shared memory goes away while the first block reads it
     }
 }
 
@@ -824,9 +853,12 @@ static int launch_decode_p(const Params &p, const kvsink_cache &c, const __half 
     const size_t smem = DecodePlan<BITS, D, NGV, CT>::bytes(nq_max);
     auto kern = decode_kernel<BITS, D, NGV, CT, PL>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return KVSINK_ERR_CUDA;
-    cudaLaunchAttribute pdl[1];
+    cudaLaunchAttribute pdl[2];
     pdl[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     pdl[0].val.programmaticStreamSerializationAllowed = 1;
+    // up to eight splits (the portable cluster size): the splits of a unit are launched as one thread-block cluster and
+    // merged inside the kernel through distributed shared memory; more splits go through the workspace and the merge kernel
+    const bool cluster_merge = nsplit > 1 && nsplit <= 8;
     {
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3(nsplit, p.Hkv * qchunks, p.B);
@@ -835,9 +867,17 @@ static int launch_decode_p(const Params &p, const kvsink_cache &c, const __half 
         cfg.stream = st;
         cfg.attrs = pdl;
         cfg.numAttrs = 1;
-        if (cudaLaunchKernelEx(&cfg, kern, p, c, q, out, lse, ws, nsplit, gps, qchunks, (int)c.seq_len) != cudaSuccess) return KVSINK_ERR_CUDA;
+        if (cluster_merge) {
+            pdl[1].id = cudaLaunchAttributeClusterDimension;
+            pdl[1].val.clusterDim.x = nsplit;
+            pdl[1].val.clusterDim.y = 1;
+            pdl[1].val.clusterDim.z = 1;
+            cfg.numAttrs = 2;
+        }
+        if (cudaLaunchKernelEx(&cfg, kern, p, c, q, out, lse, ws, nsplit, gps, qchunks, (int)c.seq_len, (int)cluster_merge) != cudaSuccess)
+            return KVSINK_ERR_CUDA;
     }
-    if (nsplit > 1) {
+    if (nsplit > 1 && !cluster_merge) {
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3(p.B * p.Hq);
         cfg.blockDim = dim3(D);
