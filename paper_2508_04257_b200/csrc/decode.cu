@@ -858,8 +858,8 @@ static int launch_decode_p(const Params &p, const kvsink_cache &c, const __half 
     pdl[0].val.programmaticStreamSerializationAllowed = 1;
     // up to eight splits (the portable cluster size): the splits of a unit are launched as one thread-block cluster and
     // merged inside the kernel through distributed shared memory; more splits go through the workspace and the merge kernel
-    const bool cluster_merge = nsplit > 1 && nsplit <= 8;
-    {
+    bool cluster_merge = nsplit > 1 && nsplit <= 8;
+    for (;;) {
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3(nsplit, p.Hkv * qchunks, p.B);
         cfg.blockDim = dim3(DEC_THREADS);
@@ -874,8 +874,10 @@ static int launch_decode_p(const Params &p, const kvsink_cache &c, const __half 
             pdl[1].val.clusterDim.z = 1;
             cfg.numAttrs = 2;
         }
-        if (cudaLaunchKernelEx(&cfg, kern, p, c, q, out, lse, ws, nsplit, gps, qchunks, (int)c.seq_len, (int)cluster_merge) != cudaSuccess)
-            return KVSINK_ERR_CUDA;
+        if (cudaLaunchKernelEx(&cfg, kern, p, c, q, out, lse, ws, nsplit, gps, qchunks, (int)c.seq_len, (int)cluster_merge) == cudaSuccess) break;
+        (void)cudaGetLastError();
+        if (!cluster_merge) return KVSINK_ERR_CUDA;
+        cluster_merge = false;   // a cluster that cannot be placed: the same launch without one, merged by the second kernel
     }
     if (nsplit > 1 && !cluster_merge) {
         cudaLaunchConfig_t cfg = {};
