@@ -2,9 +2,10 @@
  * libkvsink -- KVSink quantized-KV-cache hot path for NVIDIA B200 (sm_100a).
  *
  * C ABI.  Every pointer documented "device" must point to CUDA device memory owned by the caller;
- * "host" pointers are ordinary host memory.  The library allocates no device memory, keeps no global
- * state, launches all work asynchronously on the caller's stream and never synchronises, except in
- * kvsink_read_status.  Every entry point returns 0 (KVSINK_OK) or a negative KVSINK_ERR_* code; argument
+ * "host" pointers are ordinary host memory.  The library allocates no device memory, keeps no state
+ * between calls (it caches two lookups: the driver's tensor-map encoder and, for kvsink_decode_attention_static,
+ * the device address of its built-in scratch), launches all work asynchronously on the caller's stream and never
+ * synchronises, except in kvsink_read_status.  Every entry point returns 0 (KVSINK_OK) or a negative KVSINK_ERR_* code; argument
  * errors are detected on the host before anything is launched.  Nothing traps or spins on the device.
  *
  * Citations are to arXiv 2508.04257 ("KVSink"): Eq. 3 / Eq. 7 (attention, split into sink and non-sink
