@@ -349,10 +349,118 @@ quantize_tokens_kernel(Params p, kvsink_cache c, const __half *__restrict__ k_sr
     }
 }
 
+// ---------------------------------------------------------------------------------------------------------
+// One token per sequence (the decode-time append): one warp per (sequence, KV head).  The value row is coded and its
+// fields go straight into the tile's words: every channel's field has its own place (lane, word, bit) in the tile, so
+// the lanes clear and set their fields with word atomics and nothing but the token's own fields is touched.
+// ---------------------------------------------------------------------------------------------------------
+constexpr int QA_WARPS = 4;
+
+// Word (index among the tile's 32-bit words) and bit position of the field of matrix element (m, row, col); for 3 bit
+// the low two bits, and through *hi_word / *hi_shift the high bit.
+__device__ __forceinline__ void field_place(int bits, int D, int m, int row, int col, int *word, int *shift, int *hi_word, int *hi_shift)
+{
+    const int lane = 4 * (row & 7) + ((col & 7) >> 1), e = col & 1;
+    const int s = 4 * m + (row >> 3) + 2 * (col >> 3);
+    if (bits == 3) {
+        const int nlo = D / 32, nhi = D / 64, i = s >> 3, k = s & 7;
+        *word = section_word_offset(nlo, lane, i);
+        *shift = 16 * e + 2 * k;
+        *hi_word = 32 * nlo + section_word_offset(nhi, lane, i >> 1);
+        *hi_shift = 16 * e + 4 * (k >> 1) + 2 * (1 - (i & 1)) + (k & 1);
+    } else {
+        const int n = D * bits / 64, fields = 16 / bits;
+        *word = section_word_offset(n, lane, s / fields);
+        *shift = 16 * e + bits * (s % fields);
+        *hi_word = *hi_shift = 0;
+    }
+}
+
+__global__ void __launch_bounds__(32 * QA_WARPS)
+append_one_kernel(Params p, kvsink_cache c, const __half *__restrict__ k_src, const __half *__restrict__ v_src, int src_token, int pos,
+                  int64_t sb, int64_t sh, int64_t stt)
+{
+    const int D = p.D, G = p.G;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int64_t unit = (int64_t)blockIdx.x * QA_WARPS + warp;
+    pdl_wait();
+    if (unit >= (int64_t)p.B * p.Hkv) return;
+    const int b = (int)(unit / p.Hkv), h = (int)(unit % p.Hkv);
+    const float qmax = (float)((1 << p.bits) - 1);
+    const int cpl = D / 32;   // channels per lane (2 or 4)
+    const int64_t src = b * sb + h * sh + (int64_t)src_token * stt;
+    const bool sink = mask_bit(c.sink_bitmask + (size_t)b * p.mask_words, pos);
+    float x[4];
+    __half kx[4], vx[4];
+    for (int e = 0; e < cpl; ++e) {
+        vx[e] = v_src[src + lane * cpl + e];
+        x[e] = __half2float(vx[e]);
+        kx[e] = k_src[src + lane * cpl + e];
+    }
+    // key row -> tail
+    __half *tail = (__half *)c.k_tail + ((size_t)unit * G + pos % G) * D;
+    for (int e = 0; e < cpl; ++e) tail[lane * cpl + e] = kx[e];
+    if (sink) {
+        const int count = min(c.sink_count[b], p.cap);
+        const int slot = find_slot(c.sink_pos + (size_t)b * p.cap, count, pos);
+        if (slot < 0) {
+            if (lane == 0) atomicOr(c.status, KVSINK_STATUS_SINK_MISMATCH);
+        } else {
+            __half *dk = (__half *)c.sink_k + ((size_t)unit * p.cap + slot) * D;
+            __half *dv = (__half *)c.sink_v + ((size_t)unit * p.cap + slot) * D;
+            for (int e = 0; e < cpl; ++e) {
+                dk[lane * cpl + e] = kx[e];
+                dv[lane * cpl + e] = vx[e];
+            }
+        }
+    }
+    // value row: min / max over the lanes of each channel group, parameters, codes
+    float mn = x[0], mx = x[0];
+    for (int e = 1; e < cpl; ++e) { mn = fminf(mn, x[e]); mx = fmaxf(mx, x[e]); }
+    const int lanes_per_group = p.Gv / cpl;
+    for (int o = 1; o < lanes_per_group; o <<= 1) {
+        mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, o));
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    }
+    float s, z;
+    group_params(!sink, mn, mx, qmax, &s, &z);
+    if (lane % lanes_per_group == 0) {
+        const size_t o = ((size_t)unit * p.max_seq + pos) * p.NGv + lane / lanes_per_group;
+        c.v_scale[o] = s;
+        c.v_zero[o] = z;
+    }
+    // the token's fields in its tile; a tile whose first token this is is written whole (zeros elsewhere)
+    const int tile = pos / KVSINK_TILE, col = pos % KVSINK_TILE;
+    uint32_t *vout = (uint32_t *)(c.v_codes + (size_t)unit * p.max_seq * p.row_bytes + (size_t)tile * p.tile_bytes);
+    const bool fresh = col == 0;
+    if (fresh) {
+        for (int w = lane; w < p.tile_bytes / 4; w += 32) vout[w] = 0u;
+        __syncwarp();
+    }
+    for (int e = 0; e < cpl; ++e) {
+        const int ch = lane * cpl + e;
+        const uint32_t code = sink ? 0u : code_exact(x[e], s, z, qmax);
+        int word, shift, hi_word, hi_shift;
+        field_place(p.bits, D, ch >> 4, ch & 15, col, &word, &shift, &hi_word, &hi_shift);
+        const uint32_t lo_mask = p.bits == 3 ? 3u : (1u << p.bits) - 1u;
+        if (!fresh) atomicAnd(&vout[word], ~(lo_mask << shift));
+        if (code & lo_mask) atomicOr(&vout[word], (code & lo_mask) << shift);
+        if (p.bits == 3) {
+            if (!fresh) atomicAnd(&vout[hi_word], ~(1u << hi_shift));
+            if (code >> 2) atomicOr(&vout[hi_word], 1u << hi_shift);
+        }
+    }
+}
+
 int launch_quantize_tokens(const Params &p, const kvsink_cache &c, const __half *k_src, const __half *v_src, int src_offset,
                            int first_token, int n_tokens, int64_t sb, int64_t sh, int64_t stt, cudaStream_t st)
 {
     if (n_tokens <= 0) return KVSINK_OK;
+    if (n_tokens == 1) {
+        const long units = (long)p.B * p.Hkv;
+        return launch_pdl(append_one_kernel, dim3((unsigned)((units + QA_WARPS - 1) / QA_WARPS)), dim3(32 * QA_WARPS), 0, st, p, c, k_src, v_src,
+                          src_offset, first_token, sb, sh, stt) == cudaSuccess ? KVSINK_OK : KVSINK_ERR_CUDA;
+    }
     int tiles = (first_token + n_tokens - 1) / KVSINK_TILE - first_token / KVSINK_TILE + 1;
     dim3 grid(tiles, p.Hkv, p.B);
     return launch_pdl(quantize_tokens_kernel, grid, dim3(QT_THREADS), 0, st, p, c, k_src, v_src, src_offset, first_token, n_tokens, sb, sh,
