@@ -785,26 +785,44 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
     }
 }
 
-// Merge of the sequence splits: one block per (sequence, query head), one thread per channel.
+// Merge of the sequence splits (more than eight per unit): one block per (sequence, query head); thread (ch, sl) folds the
+// records sl, sl + MERGE_SLICES, ... of channel ch, and the slices are combined in a fixed order (bit-reproducible).
+constexpr int MERGE_SLICES = 4;
+
 __global__ void decode_merge_kernel(const float *__restrict__ part_ws, int nsplit, int D, float *__restrict__ out, float *__restrict__ lse)
 {
+    __shared__ float sh_acc[MERGE_SLICES][128], sh_m[MERGE_SLICES], sh_l[MERGE_SLICES];
     const int PS = D + 2;
     const size_t oq = blockIdx.x;
-    const int ch = threadIdx.x;
+    const int ch = threadIdx.x, sl = threadIdx.y;
     const float *base = part_ws + oq * nsplit * PS;
     // launched with programmatic stream serialization: the blocks may start while the split kernel drains, and wait
     // here until all of it has completed and its records are visible
     asm volatile("griddepcontrol.wait;" ::: "memory");
     float M = M_INIT;
-    for (int s = 0; s < nsplit; ++s) M = fmaxf(M, base[(size_t)s * PS + D]);
+    for (int s = sl; s < nsplit; s += MERGE_SLICES) M = fmaxf(M, base[(size_t)s * PS + D]);
     float acc = 0.f, L = 0.f;
-    for (int s = 0; s < nsplit; ++s) {
+    for (int s = sl; s < nsplit; s += MERGE_SLICES) {
         const float f = ex2(base[(size_t)s * PS + D] - M);
         acc += base[(size_t)s * PS + ch] * f;
         L += base[(size_t)s * PS + D + 1] * f;
     }
-    out[oq * D + ch] = L > 0.f ? acc / L : 0.f;
-    if (lse && ch == 0) lse[oq] = L > 0.f ? (M + log2f(L)) * 0.6931471805599453f : -INFINITY;
+    sh_acc[sl][ch] = acc;
+    if (ch == 0) { sh_m[sl] = M; sh_l[sl] = L; }
+    __syncthreads();
+    if (sl != 0) return;
+    float Mt = M_INIT;
+#pragma unroll
+    for (int i = 0; i < MERGE_SLICES; ++i) Mt = fmaxf(Mt, sh_m[i]);
+    float at = 0.f, Lt = 0.f;
+#pragma unroll
+    for (int i = 0; i < MERGE_SLICES; ++i) {
+        const float f = ex2(sh_m[i] - Mt);
+        at += sh_acc[i][ch] * f;
+        Lt += sh_l[i] * f;
+    }
+    out[oq * D + ch] = Lt > 0.f ? at / Lt : 0.f;
+    if (lse && ch == 0) lse[oq] = Lt > 0.f ? (Mt + log2f(Lt)) * 0.6931471805599453f : -INFINITY;
 }
 
 // ---- host side ----
@@ -882,7 +900,7 @@ static int launch_decode_p(const Params &p, const kvsink_cache &c, const __half 
     if (nsplit > 1 && !cluster_merge) {
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3(p.B * p.Hq);
-        cfg.blockDim = dim3(D);
+        cfg.blockDim = dim3(D, MERGE_SLICES);
         cfg.stream = st;
         cfg.attrs = pdl;
         cfg.numAttrs = 1;
