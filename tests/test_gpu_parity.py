@@ -144,3 +144,14 @@ def test_bulk_append_kernel_smallest_launches(bits, group, n_groups):
     wl = TINY.scaled(bits=bits, head_dim=128, group=group, n_q_heads=1, n_kv_heads=1, batch=1, seq=n_groups * group, topk=3,
                      pfn_n=1, seed=5000 + bits * 10 + group)
     run_both(wl, appends=1)
+
+
+@pytest.mark.parametrize("hq,hkv,batch,groups", [(16, 16, 8, 24), (8, 4, 12, 40), (4, 4, 3, 33)])
+def test_decode_split_counts_that_merge_inside_a_cluster(hq, hkv, batch, groups):
+    # enough (sequence, KV head) units that a unit gets two to eight sequence splits: those run as one thread-block
+    # cluster and merge through distributed shared memory instead of the merge kernel
+    wl = TINY.scaled(bits=2, head_dim=128, group=32, n_q_heads=hq, n_kv_heads=hkv, batch=batch, seq=32 * groups + 11, topk=6,
+                     pfn_n=1, seed=6000 + hq + batch)
+    r = run_both(wl, appends=1)
+    out2, _ = kv.decode_attention(configs(wl)[1], r["gpu_cache"], r["q"])
+    assert bits_equal(out2.cpu().numpy(), r["out"].cpu().numpy())      # the merge order is fixed
