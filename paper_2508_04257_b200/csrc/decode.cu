@@ -215,7 +215,12 @@ struct DecodePlan {
 // column 2h multiplies by the fp16 factor q*scale and column 2h+1 by its fp16 rounding residual, so every score carries
 // the factor to ~22 bits at no extra instruction.  Without PL (five to eight heads) head h owns column h and the
 // residual of channels with large factors goes through a second multiply.
-template <int BITS, int D, int NGv, int CT, bool PL>
+// I8 (2 bit, one query head per KV head): the key side runs on the integer tensor path.  The four bytes of a stored
+// word are four channels of one token row, so the word masked with 0x03.., 0x0c.., 0x30.., 0xc0.. is the u8 A fragment
+// of one m16n8k32 (fields in place: x1, x4 for the rows g + 8, x16 for the upper contraction slots, x64 for both); the B
+// operand holds the factor q * scale * 2^sh of each channel as three signed 7-bit limbs in three accumulator columns
+// (divided by 16 beforehand for the upper slots), sums are exact in int32.
+template <int BITS, int D, int NGv, int CT, bool PL, bool I8 = false>
 __global__ void __launch_bounds__(DEC_THREADS, 4)
 decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__restrict__ out, float *__restrict__ lse,
               float *__restrict__ part_ws, int nsplit, int groups_per_split, int qchunks, int seq_len, int cluster_merge)
@@ -435,6 +440,34 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
             for (int e = 0; e < CPL; ++e) { scv[e] = kp[lane * CPL + e]; zev[e] = kp[D + lane * CPL + e]; }
             __syncwarp();   // the parameters are in registers: the slot can take the next group's while this one streams
             if (gi + 1 < my_groups) issue_params(gi + 1);
+            if constexpr (I8) {
+                // limbs of the one head's factors: f = q * scale * 2^sh with the largest |f| in [2^19, 2^20)
+                float v[CPL], amax = 0.f;
+#pragma unroll
+                for (int e = 0; e < CPL; ++e) { v[e] = qs[lane * CPL + e] * scv[e]; amax = fmaxf(amax, fabsf(v[e])); }
+                amax = warp_max(amax);
+                int sh = 19 - floor_log2(amax);
+                sh = sh > 60 ? 60 : (sh < -60 ? -60 : sh);
+                const bool upper = ((lane * CPL) & 8) != 0;           // channels in the upper contraction slots
+                const float pre = upper ? pow2i(sh - 4) : pow2i(sh);
+                const int mtx = (lane * CPL) >> 4, colbase = (lane * CPL) & 15;
+                signed char *tab = reinterpret_cast<signed char *>(Bs) + ((mtx >> 1) * 2 + (colbase >> 3)) * 48;   // [word][half][limb][t][byte]
+                float bsum = 0.f;
+#pragma unroll
+                for (int e = 0; e < CPL; ++e) {
+                    const float fp = v[e] * pre;
+                    const float l0 = rintf(fp * (1.f / 16384.f)), r = fmaf(-l0, 16384.f, fp);
+                    const float l1 = rintf(r * (1.f / 128.f)), l2 = rintf(fmaf(-l1, 128.f, r));
+                    const float F = fmaf(l0, 16384.f, fmaf(l1, 128.f, l2)) * (upper ? 16.f : 1.f);   // the factor the MMAs apply
+                    bsum = fmaf(F, zev[e], bsum);
+                    const int col = colbase + e, at = ((col & 7) >> 1) * 4 + (mtx & 1) + 2 * (col & 1);
+                    tab[at] = (signed char)(int)l0;
+                    tab[16 + at] = (signed char)(int)l1;
+                    tab[32 + at] = (signed char)(int)l2;
+                }
+                bsum = warp_sum(bsum) * pow2i(-sh);
+                if (t == 0) { bias0 = bsum; ks0 = pow2i(-sh); }
+            } else {
             // one power-of-two scaling for all heads of the group: the largest factor lands in [2^13, 2^14)
             constexpr int NQL = PL ? 4 : 8;
             float amax = 0.f;
@@ -497,14 +530,26 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
                 for (int m = 0; m < NM; ++m)
                     if ((bal >> (LPM * m)) & ((1u << LPM) - 1u)) need_lo |= 1u << m;
             }
+            }
             __syncwarp();
         }
         uint32_t bk[NM][2];
+        if constexpr (I8) {
+            // B fragments of the four words: column g = limb g, contraction slots 4t .. 4t + 3 (lower, upper)
+#pragma unroll
+            for (int m = 0; m < NM; ++m) bk[m][0] = bk[m][1] = 0u;
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int c2 = 0; c2 < 2; ++c2)
+                    bk[i][c2] = g < 3 ? *reinterpret_cast<const uint32_t *>(reinterpret_cast<const signed char *>(Bs) + (i * 2 + c2) * 48 + g * 16 + 4 * t) : 0u;
+        } else {
 #pragma unroll
         for (int m = 0; m < NM; ++m) {
             const bool col_used = PL ? g < 2 * nq : g < nq;
             bk[m][0] = col_used ? *(const uint32_t *)(Bs + g * BST + 16 * m + 2 * t) : 0u;
             bk[m][1] = col_used ? *(const uint32_t *)(Bs + g * BST + 16 * m + 2 * t + 8) : 0u;
+        }
         }
         const float ks0r = ks0 * R1, ks1r = ks1 * R1;
 
@@ -534,6 +579,25 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
             float s[ST][4];
 #pragma unroll
             for (int k = 0; k < ST; ++k) {
+                if constexpr (I8) {
+                    uint32_t kw[W];
+                    load_tile_shared<BITS, D>(kt + k * TILE_WORDS, lane, kw);
+                    int ia[4] = {0, 0, 0, 0};
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const uint32_t x = kw[i];
+                        asm volatile("mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                                     : "+r"(ia[0]), "+r"(ia[1]), "+r"(ia[2]), "+r"(ia[3])
+                                     : "r"(x & 0x03030303u), "r"(x & 0x0c0c0c0cu), "r"(x & 0x30303030u), "r"(x & 0xc0c0c0c0u), "r"(bk[i][0]), "r"(bk[i][1]));
+                    }
+                    // lane t = 0 holds limbs 0, 1 (columns 0, 1), its neighbour limb 2 (column 2)
+                    const int v0 = __shfl_down_sync(0xffffffffu, ia[0], 1), v1 = __shfl_down_sync(0xffffffffu, ia[2], 1);
+                    const float tg = fmaf((float)ia[0], 16384.f, fmaf((float)ia[1], 128.f, (float)v0));
+                    const float th = fmaf((float)ia[2], 16384.f, fmaf((float)ia[3], 128.f, (float)v1));
+                    s[k][0] = t == 0 ? fmaf(tg, ks0, -bias0) : -INFINITY; s[k][1] = -INFINITY;
+                    s[k][2] = t == 0 ? fmaf(th, ks0r, -bias0) : -INFINITY; s[k][3] = -INFINITY;
+                    continue;
+                }
                 uint32_t kw[W], ka[NM][4];
                 load_tile_shared<BITS, D>(kt + k * TILE_WORDS, lane, kw);
                 tile_frags<BITS, D>(kw, ka);
@@ -860,7 +924,7 @@ size_t decode_workspace_bytes(const Params &p)
     return (size_t)p.B * p.Hq * max_splits(p) * (p.D + 2) * sizeof(float) + 16;
 }
 
-template <int BITS, int D, int NGV, int CT, bool PL>
+template <int BITS, int D, int NGV, int CT, bool PL, bool I8 = false>
 static int launch_decode_p(const Params &p, const kvsink_cache &c, const __half *q, float *out, float *lse, float *ws, cudaStream_t st)
 {
     const int n_groups = c.seq_len / p.G;
@@ -869,7 +933,7 @@ static int launch_decode_p(const Params &p, const kvsink_cache &c, const __half 
     const int qchunks = (p.rep + 7) / 8;
     const int nq_max = p.rep < 8 ? p.rep : 8;
     const size_t smem = DecodePlan<BITS, D, NGV, CT>::bytes(nq_max);
-    auto kern = decode_kernel<BITS, D, NGV, CT, PL>;
+    auto kern = decode_kernel<BITS, D, NGV, CT, PL, I8>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return KVSINK_ERR_CUDA;
     cudaLaunchAttribute pdl[2];
     pdl[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
@@ -912,6 +976,8 @@ static int launch_decode_p(const Params &p, const kvsink_cache &c, const __half 
 template <int BITS, int D, int NGV, int CT>
 static int launch_decode_c(const Params &p, const kvsink_cache &c, const __half *q, float *out, float *lse, float *ws, cudaStream_t st)
 {
+    if constexpr (BITS == 2 && D == 128)
+        if (p.rep == 1) return launch_decode_p<BITS, D, NGV, CT, true, true>(p, c, q, out, lse, ws, st);
     if (p.rep <= 4) return launch_decode_p<BITS, D, NGV, CT, true>(p, c, q, out, lse, ws, st);
     return launch_decode_p<BITS, D, NGV, CT, false>(p, c, q, out, lse, ws, st);
 }
