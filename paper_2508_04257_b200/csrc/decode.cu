@@ -215,11 +215,12 @@ struct DecodePlan {
 // column 2h multiplies by the fp16 factor q*scale and column 2h+1 by its fp16 rounding residual, so every score carries
 // the factor to ~22 bits at no extra instruction.  Without PL (five to eight heads) head h owns column h and the
 // residual of channels with large factors goes through a second multiply.
-// I8 (2 bit, one query head per KV head): the key side runs on the integer tensor path.  The four bytes of a stored
-// word are four channels of one token row, so the word masked with 0x03.., 0x0c.., 0x30.., 0xc0.. is the u8 A fragment
-// of one m16n8k32 (fields in place: x1, x4 for the rows g + 8, x16 for the upper contraction slots, x64 for both); the B
-// operand holds the factor q * scale * 2^sh of each channel as three signed 7-bit limbs in three accumulator columns
-// (divided by 16 beforehand for the upper slots), sums are exact in int32.
+// I8 (2 or 4 bit, one query head per KV head): the key side runs on the integer tensor path.  The four bytes of a stored
+// word are four channels of one token row.  2 bit: the word masked with 0x03.., 0x0c.., 0x30.., 0xc0.. is the u8 A
+// fragment of one m16n8k32 (fields in place: x1, x4 for the rows g + 8, x16 for the upper contraction slots, x64 for
+// both).  4 bit: a word masked with 0x0f.. and 0xf0.. gives the registers of rows g and g + 8 (x16), two words (two
+// matrices) make one fragment.  The B operand holds the factor q * scale * 2^sh of each channel as three signed 7-bit
+// limbs in three accumulator columns (2 bit: divided by 16 beforehand for the upper slots); sums are exact in int32.
 template <int BITS, int D, int NGv, int CT, bool PL, bool I8 = false>
 __global__ void __launch_bounds__(DEC_THREADS, 4)
 decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__restrict__ out, float *__restrict__ lse,
@@ -448,10 +449,12 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
                 amax = warp_max(amax);
                 int sh = 19 - floor_log2(amax);
                 sh = sh > 60 ? 60 : (sh < -60 ? -60 : sh);
-                const bool upper = ((lane * CPL) & 8) != 0;           // channels in the upper contraction slots
+                const bool upper = BITS == 2 && ((lane * CPL) & 8) != 0;   // 2 bit: channels in the upper contraction slots (x16 in place)
                 const float pre = upper ? pow2i(sh - 4) : pow2i(sh);
                 const int mtx = (lane * CPL) >> 4, colbase = (lane * CPL) & 15;
-                signed char *tab = reinterpret_cast<signed char *>(Bs) + ((mtx >> 1) * 2 + (colbase >> 3)) * 48;   // [word][half][limb][t][byte]
+                // table [MMA][lower / upper slots][limb][t][byte]; 2 bit: MMA = word = matrix pair, upper = column half;
+                // 4 bit: MMA = matrix pair, upper = odd matrix
+                signed char *tab = reinterpret_cast<signed char *>(Bs) + ((mtx >> 1) * 2 + (BITS == 2 ? (colbase >> 3) : (mtx & 1))) * 48;
                 float bsum = 0.f;
 #pragma unroll
                 for (int e = 0; e < CPL; ++e) {
@@ -460,7 +463,8 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
                     const float l1 = rintf(r * (1.f / 128.f)), l2 = rintf(fmaf(-l1, 128.f, r));
                     const float F = fmaf(l0, 16384.f, fmaf(l1, 128.f, l2)) * (upper ? 16.f : 1.f);   // the factor the MMAs apply
                     bsum = fmaf(F, zev[e], bsum);
-                    const int col = colbase + e, at = ((col & 7) >> 1) * 4 + (mtx & 1) + 2 * (col & 1);
+                    const int col = colbase + e;
+                    const int at = ((col & 7) >> 1) * 4 + (BITS == 2 ? (mtx & 1) + 2 * (col & 1) : 2 * (col & 1) + (col >> 3));
                     tab[at] = (signed char)(int)l0;
                     tab[16 + at] = (signed char)(int)l1;
                     tab[32 + at] = (signed char)(int)l2;
@@ -585,10 +589,17 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
                     int ia[4] = {0, 0, 0, 0};
 #pragma unroll
                     for (int i = 0; i < 4; ++i) {
-                        const uint32_t x = kw[i];
+                        uint32_t a0, a1, a2, a3;
+                        if constexpr (BITS == 2) {
+                            const uint32_t x = kw[i];
+                            a0 = x & 0x03030303u; a1 = x & 0x0c0c0c0cu; a2 = x & 0x30303030u; a3 = x & 0xc0c0c0c0u;
+                        } else {
+                            const uint32_t x = kw[2 * i], y = kw[2 * i + 1];
+                            a0 = x & 0x0f0f0f0fu; a1 = x & 0xf0f0f0f0u; a2 = y & 0x0f0f0f0fu; a3 = y & 0xf0f0f0f0u;
+                        }
                         asm volatile("mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
                                      : "+r"(ia[0]), "+r"(ia[1]), "+r"(ia[2]), "+r"(ia[3])
-                                     : "r"(x & 0x03030303u), "r"(x & 0x0c0c0c0cu), "r"(x & 0x30303030u), "r"(x & 0xc0c0c0c0u), "r"(bk[i][0]), "r"(bk[i][1]));
+                                     : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(bk[i][0]), "r"(bk[i][1]));
                     }
                     // lane t = 0 holds limbs 0, 1 (columns 0, 1), its neighbour limb 2 (column 2)
                     const int v0 = __shfl_down_sync(0xffffffffu, ia[0], 1), v1 = __shfl_down_sync(0xffffffffu, ia[2], 1);
@@ -976,7 +987,7 @@ static int launch_decode_p(const Params &p, const kvsink_cache &c, const __half 
 template <int BITS, int D, int NGV, int CT>
 static int launch_decode_c(const Params &p, const kvsink_cache &c, const __half *q, float *out, float *lse, float *ws, cudaStream_t st)
 {
-    if constexpr (BITS == 2 && D == 128)
+    if constexpr ((BITS == 2 || BITS == 4) && D == 128)
         if (p.rep == 1) return launch_decode_p<BITS, D, NGV, CT, true, true>(p, c, q, out, lse, ws, st);
     if (p.rep <= 4) return launch_decode_p<BITS, D, NGV, CT, true>(p, c, q, out, lse, ws, st);
     return launch_decode_p<BITS, D, NGV, CT, false>(p, c, q, out, lse, ws, st);
