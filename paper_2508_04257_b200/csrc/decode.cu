@@ -215,12 +215,14 @@ struct DecodePlan {
 // column 2h multiplies by the fp16 factor q*scale and column 2h+1 by its fp16 rounding residual, so every score carries
 // the factor to ~22 bits at no extra instruction.  Without PL (five to eight heads) head h owns column h and the
 // residual of channels with large factors goes through a second multiply.
-// I8 (2 or 4 bit, one query head per KV head): the key side runs on the integer tensor path.  The four bytes of a stored
+// I8 (one query head per KV head): the key side runs on the integer tensor path.  The four bytes of a stored
 // word are four channels of one token row.  2 bit: the word masked with 0x03.., 0x0c.., 0x30.., 0xc0.. is the u8 A
 // fragment of one m16n8k32 (fields in place: x1, x4 for the rows g + 8, x16 for the upper contraction slots, x64 for
 // both).  4 bit: a word masked with 0x0f.. and 0xf0.. gives the registers of rows g and g + 8 (x16), two words (two
 // matrices) make one fragment.  The B operand holds the factor q * scale * 2^sh of each channel as three signed 7-bit
-// limbs in three accumulator columns (2 bit: divided by 16 beforehand for the upper slots); sums are exact in int32.
+// limbs in three accumulator columns (2, 3 bit: divided by 16 beforehand for the upper slots); sums are exact in int32.
+// 3 bit: the low two bits as for 2 bit, the high bits of the second section (same byte structure) through four more
+// MMAs with the same B operands into accumulators of their own.
 template <int BITS, int D, int NGv, int CT, bool PL, bool I8 = false>
 __global__ void __launch_bounds__(DEC_THREADS, 4)
 decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__restrict__ out, float *__restrict__ lse,
@@ -449,12 +451,12 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
                 amax = warp_max(amax);
                 int sh = 19 - floor_log2(amax);
                 sh = sh > 60 ? 60 : (sh < -60 ? -60 : sh);
-                const bool upper = BITS == 2 && ((lane * CPL) & 8) != 0;   // 2 bit: channels in the upper contraction slots (x16 in place)
+                const bool upper = BITS != 4 && ((lane * CPL) & 8) != 0;   // 2, 3 bit: channels in the upper contraction slots (x16 in place)
                 const float pre = upper ? pow2i(sh - 4) : pow2i(sh);
                 const int mtx = (lane * CPL) >> 4, colbase = (lane * CPL) & 15;
                 // table [MMA][lower / upper slots][limb][t][byte]; 2 bit: MMA = word = matrix pair, upper = column half;
                 // 4 bit: MMA = matrix pair, upper = odd matrix
-                signed char *tab = reinterpret_cast<signed char *>(Bs) + ((mtx >> 1) * 2 + (BITS == 2 ? (colbase >> 3) : (mtx & 1))) * 48;
+                signed char *tab = reinterpret_cast<signed char *>(Bs) + ((mtx >> 1) * 2 + (BITS != 4 ? (colbase >> 3) : (mtx & 1))) * 48;
                 float bsum = 0.f;
 #pragma unroll
                 for (int e = 0; e < CPL; ++e) {
@@ -464,7 +466,7 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
                     const float F = fmaf(l0, 16384.f, fmaf(l1, 128.f, l2)) * (upper ? 16.f : 1.f);   // the factor the MMAs apply
                     bsum = fmaf(F, zev[e], bsum);
                     const int col = colbase + e;
-                    const int at = ((col & 7) >> 1) * 4 + (BITS == 2 ? (mtx & 1) + 2 * (col & 1) : 2 * (col & 1) + (col >> 3));
+                    const int at = ((col & 7) >> 1) * 4 + (BITS != 4 ? (mtx & 1) + 2 * (col & 1) : 2 * (col & 1) + (col >> 3));
                     tab[at] = (signed char)(int)l0;
                     tab[16 + at] = (signed char)(int)l1;
                     tab[32 + at] = (signed char)(int)l2;
@@ -587,10 +589,25 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
                     uint32_t kw[W];
                     load_tile_shared<BITS, D>(kt + k * TILE_WORDS, lane, kw);
                     int ia[4] = {0, 0, 0, 0};
+                    int ih0[4] = {0, 0, 0, 0}, ih1[4] = {0, 0, 0, 0};   // 3 bit: the high bits of the even / odd words
 #pragma unroll
                     for (int i = 0; i < 4; ++i) {
                         uint32_t a0, a1, a2, a3;
-                        if constexpr (BITS == 2) {
+                        if constexpr (BITS == 3) {
+                            // the second section has the byte structure of the first: the high bits of word i sit at bits
+                            // 2, 3, 6, 7 (even i) or 0, 1, 4, 5 (odd i) of the bytes of word 4 + i / 2
+                            const uint32_t hw = kw[4 + (i >> 1)];
+                            if ((i & 1) == 0) {
+                                asm volatile("mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                                             : "+r"(ih0[0]), "+r"(ih0[1]), "+r"(ih0[2]), "+r"(ih0[3])
+                                             : "r"(hw & 0x04040404u), "r"(hw & 0x08080808u), "r"(hw & 0x40404040u), "r"(hw & 0x80808080u), "r"(bk[i][0]), "r"(bk[i][1]));
+                            } else {
+                                asm volatile("mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                                             : "+r"(ih1[0]), "+r"(ih1[1]), "+r"(ih1[2]), "+r"(ih1[3])
+                                             : "r"(hw & 0x01010101u), "r"(hw & 0x02020202u), "r"(hw & 0x10101010u), "r"(hw & 0x20202020u), "r"(bk[i][0]), "r"(bk[i][1]));
+                            }
+                        }
+                        if constexpr (BITS != 4) {
                             const uint32_t x = kw[i];
                             a0 = x & 0x03030303u; a1 = x & 0x0c0c0c0cu; a2 = x & 0x30303030u; a3 = x & 0xc0c0c0c0u;
                         } else {
@@ -601,12 +618,18 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
                                      : "+r"(ia[0]), "+r"(ia[1]), "+r"(ia[2]), "+r"(ia[3])
                                      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(bk[i][0]), "r"(bk[i][1]));
                     }
+                    if constexpr (BITS == 3) {
+                        // code = low + 4 * high; in place the high bits weigh 4, 8 (rows g, g + 8) in even words and 1, 2 in
+                        // odd ones, the low fields 1, 4: rows g in units of 1, rows g + 8 in units of 4
+                        ia[0] += ih0[0] + 4 * ih1[0]; ia[1] += ih0[1] + 4 * ih1[1];
+                        ia[2] += 2 * ih0[2] + 8 * ih1[2]; ia[3] += 2 * ih0[3] + 8 * ih1[3];
+                    }
                     // lane t = 0 holds limbs 0, 1 (columns 0, 1), its neighbour limb 2 (column 2)
                     const int v0 = __shfl_down_sync(0xffffffffu, ia[0], 1), v1 = __shfl_down_sync(0xffffffffu, ia[2], 1);
                     const float tg = fmaf((float)ia[0], 16384.f, fmaf((float)ia[1], 128.f, (float)v0));
                     const float th = fmaf((float)ia[2], 16384.f, fmaf((float)ia[3], 128.f, (float)v1));
                     s[k][0] = t == 0 ? fmaf(tg, ks0, -bias0) : -INFINITY; s[k][1] = -INFINITY;
-                    s[k][2] = t == 0 ? fmaf(th, ks0r, -bias0) : -INFINITY; s[k][3] = -INFINITY;
+                    s[k][2] = t == 0 ? fmaf(th, ks0 * (BITS == 4 ? 0.0625f : 0.25f), -bias0) : -INFINITY; s[k][3] = -INFINITY;
                     continue;
                 }
                 uint32_t kw[W], ka[NM][4];
@@ -987,7 +1010,7 @@ static int launch_decode_p(const Params &p, const kvsink_cache &c, const __half 
 template <int BITS, int D, int NGV, int CT>
 static int launch_decode_c(const Params &p, const kvsink_cache &c, const __half *q, float *out, float *lse, float *ws, cudaStream_t st)
 {
-    if constexpr ((BITS == 2 || BITS == 4) && D == 128)
+    if constexpr (D == 128)
         if (p.rep == 1) return launch_decode_p<BITS, D, NGV, CT, true, true>(p, c, q, out, lse, ws, st);
     if (p.rep <= 4) return launch_decode_p<BITS, D, NGV, CT, true>(p, c, q, out, lse, ws, st);
     return launch_decode_p<BITS, D, NGV, CT, false>(p, c, q, out, lse, ws, st);
