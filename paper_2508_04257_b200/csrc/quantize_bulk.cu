@@ -137,6 +137,8 @@ __device__ __forceinline__ uint32_t qb_hmax2(uint32_t a, uint32_t b)
 // y = fma(x, r, M + zero) with M = 1.5 * 2^23 rounds the product to an integer in the mantissa.  It is evaluated with
 // r = 1/scale nudged down and up by 2^-22: where both agree no rounding of x/scale can fall on the other side of a tie
 // and the agreed integer is the exact answer; where they differ the lane redoes that register with the IEEE division.
+// The two elements of a register share one packed FMA per reciprocal; a matrix (four registers) is tested with one
+// branch, and inside it only the registers that disagreed are redone.
 constexpr float QB_MAGIC = 12582912.0f;   // 1.5 * 2^23
 struct __align__(16) QbCoder {
     float r_lo, r_hi;   // 1/scale nudged down / up; r_lo = +inf forces the exact path
@@ -163,15 +165,34 @@ __device__ __forceinline__ QbCoder qb_make_coder(float scale, float zero, float 
     c.magic = QB_MAGIC + (ok ? zero : 0.f);
     return c;
 }
+// The coders of two adjacent keys (the two elements of a half2 register), field by field, so that each field is the
+// operand pair of one packed fp32 FMA.
+struct __align__(16) QbCoder2 {
+    float r_lo[2], r_hi[2];
+    float magic[2], pad[2];
+};
+__device__ __forceinline__ unsigned long long qb_pair(float lo, float hi)
+{
+    unsigned long long r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
 // Codes of the two elements of a half2 register -> (code_lo | code_hi << 16); `differ` collects disagreement bits.
-__device__ __forceinline__ uint32_t qb_code_pair(uint32_t h2, const QbCoder &c0, const QbCoder &c1, uint32_t &differ)
+// Both elements go through one packed FMA per nudged reciprocal (fma.rn.f32x2: two IEEE FMAs, one instruction).
+__device__ __forceinline__ uint32_t qb_code_pair(uint32_t h2, unsigned long long r_lo, unsigned long long r_hi, unsigned long long magic,
+                                                 uint32_t &differ)
 {
     const float2 x = __half22float2(*reinterpret_cast<const __half2 *>(&h2));
-    const float a0 = fmaf(x.x, c0.r_lo, c0.magic), b0 = fmaf(x.x, c0.r_hi, c0.magic);
-    const float a1 = fmaf(x.y, c1.r_lo, c1.magic), b1 = fmaf(x.y, c1.r_hi, c1.magic);
-    differ |= (__float_as_uint(a0) ^ __float_as_uint(b0)) | (__float_as_uint(a1) ^ __float_as_uint(b1));
+    const unsigned long long xx = qb_pair(x.x, x.y);
+    unsigned long long a, b;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(a) : "l"(xx), "l"(r_lo), "l"(magic));
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(b) : "l"(xx), "l"(r_hi), "l"(magic));
+    uint32_t a0, a1, b0, b1;
+    asm("mov.b64 {%0, %1}, %2;" : "=r"(a0), "=r"(a1) : "l"(a));
+    asm("mov.b64 {%0, %1}, %2;" : "=r"(b0), "=r"(b1) : "l"(b));
+    differ |= (a0 ^ b0) | (a1 ^ b1);
     // low halves of the two results (the bit pattern of 1.5 * 2^23 has a zero low half)
-    return __byte_perm(__float_as_uint(a0), __float_as_uint(a1), 0x5410);
+    return __byte_perm(a0, a1, 0x5410);
 }
 __device__ __noinline__ uint32_t qb_code_pair_exact(uint32_t h2, float s0, float z0, float s1, float z1, float qmax)
 {
@@ -216,8 +237,9 @@ struct QbGeo {
     static constexpr int NS = 2 * D / G;          // statistic sets per item: MT for keys, 2 * NGv for values
     static constexpr int KPL = NS / 2;            // keys per lane
     static constexpr int KROWB = 2 * KC;          // bytes per row of a key item in shared memory
-    // per warp and for each of the item's 16 * NS keys: three fp16 thresholds (2 bit), or a coder and (scale, zero)
-    static constexpr int SCRATCH = BITS == 2 ? 3 * 16 * NS * 2 : 16 * NS * (int)(sizeof(QbCoder) + sizeof(float2));
+    // per warp and for each of the item's 16 * NS keys: three fp16 thresholds (2 bit), or a coder (stored by key pair)
+    // and (scale, zero)
+    static constexpr int SCRATCH = BITS == 2 ? 3 * 16 * NS * 2 : 8 * NS * (int)sizeof(QbCoder2) + 16 * NS * (int)sizeof(float2);
     static constexpr int TILE_BYTES = 256 * BITS, ROW_BYTES = 16 * BITS;   // packed tile of 16 tokens x 128 channels
     // warps per block, each with one stage, one mbarrier and its scratch: 20 (96 registers per thread) for the 2-bit
     // coder; 16 (128 registers) for the 3- and 4-bit coder, which spills at 96 and measures 9 % faster this way
@@ -323,8 +345,8 @@ quantize_bulk_kernel(Params p, kvsink_cache c, const __grid_constant__ CUtensorM
                                              : (uint32_t)((rr + 8 * (mj & 1)) * 128 + ((((mj >> 1) ^ (rr & 1)) | (rr & 6)) << 4));
 
     __half *thr = (__half *)(scratch + (size_t)warp * Geo::SCRATCH);            // 2 bit: [3][16 * NS] thresholds
-    QbCoder *coder = (QbCoder *)(scratch + (size_t)warp * Geo::SCRATCH);        // 3, 4 bit: [16 * NS] coders ...
-    float2 *sz = (float2 *)(coder + 16 * NS);                                   // ... and [16 * NS] (scale, zero)
+    QbCoder2 *coder = (QbCoder2 *)(scratch + (size_t)warp * Geo::SCRATCH);      // 3, 4 bit: [8 * NS] coders of key pairs ...
+    float2 *sz = (float2 *)(coder + 8 * NS);                                   // ... and [16 * NS] (scale, zero)
     unsigned char *my_stage = stages + (size_t)warp * QB_STAGE_BYTES;
     uint64_t *my_full = full + warp;
 
@@ -494,7 +516,11 @@ quantize_bulk_kernel(Params p, kvsink_cache c, const __grid_constant__ CUtensorM
                 for (int l = 0; l < 3; ++l)
                     thr[l * (16 * NS) + pos] = __ushort_as_half((unsigned short)qb_threshold(s, s_half, z, (float)(l + 1), qmax));
             } else {
-                coder[pos] = qb_make_coder(s, z, fmn, fmx, qmax);
+                const QbCoder cc = qb_make_coder(s, z, fmn, fmx, qmax);
+                QbCoder2 *c2 = coder + (pos >> 1);
+                c2->r_lo[e_] = cc.r_lo;
+                c2->r_hi[e_] = cc.r_hi;
+                c2->magic[e_] = cc.magic;
                 sz[pos] = make_float2(s, z);
             }
         }
@@ -566,22 +592,33 @@ quantize_bulk_kernel(Params p, kvsink_cache c, const __grid_constant__ CUtensorM
             uint32_t lo[16], hi[16];
 #pragma unroll
             for (int s = 0; s < NS; ++s) {
-                QbCoder kc[4];   // keys (side 0: e 0, 1; side 1: e 0, 1) of this lane's columns
+                unsigned long long k_lo[2], k_hi[2], k_magic[2];   // key pairs of this lane's columns (side 0, side 1)
 #pragma unroll
-                for (int q = 0; q < 4; ++q) kc[q] = coder[8 * (2 * s + (q >> 1)) + 2 * t4 + (q & 1)];
+                for (int q = 0; q < 2; ++q) {
+                    const QbCoder2 *c2 = coder + 4 * (2 * s + q) + t4;
+                    const float4 rr = *reinterpret_cast<const float4 *>(c2->r_lo);
+                    const float2 mm = *reinterpret_cast<const float2 *>(c2->magic);
+                    k_lo[q] = qb_pair(rr.x, rr.y);
+                    k_hi[q] = qb_pair(rr.z, rr.w);
+                    k_magic[q] = qb_pair(mm.x, mm.y);
+                }
 #pragma unroll
                 for (int i = 0; i < MPS; ++i) {
                     const int u = s * MPS + i;
                     const int m = is_v ? (u & 7) : sub * MT + u / NT;   // matrix of the tile
                     uint32_t pc[4];
 #pragma unroll
-                    for (int r = 0; r < 4; ++r) {
-                        uint32_t differ = 0;
-                        pc[r] = qb_code_pair(a[u][r], kc[2 * (r >> 1)], kc[2 * (r >> 1) + 1], differ);
-                        if (differ) {   // a value too close to a rounding tie (fp16 inputs land on exact ties often)
-                            const float2 z0 = sz[8 * (2 * s + (r >> 1)) + 2 * t4], z1 = sz[8 * (2 * s + (r >> 1)) + 2 * t4 + 1];
-                            pc[r] = qb_code_pair_exact(a[u][r], z0.x, z0.y, z1.x, z1.y, qmax);
-                        }
+                    uint32_t differ[4] = {0u, 0u, 0u, 0u};
+#pragma unroll
+                    for (int r = 0; r < 4; ++r) pc[r] = qb_code_pair(a[u][r], k_lo[r >> 1], k_hi[r >> 1], k_magic[r >> 1], differ[r]);
+                    if (differ[0] | differ[1] | differ[2] | differ[3]) {
+                        // a value too close to a rounding tie (fp16 inputs land on exact ties often): redo those registers
+#pragma unroll
+                        for (int r = 0; r < 4; ++r)
+                            if (differ[r]) {
+                                const float2 z0 = sz[8 * (2 * s + (r >> 1)) + 2 * t4], z1 = sz[8 * (2 * s + (r >> 1)) + 2 * t4 + 1];
+                                pc[r] = qb_code_pair_exact(a[u][r], z0.x, z0.y, z1.x, z1.y, qmax);
+                            }
                     }
                     if (has_sink && !is_v) {   // sink tokens keep code 0: pair slots 0, 2 are row g, slots 1, 3 row g + 8
                         const int T = u % NT;
