@@ -359,7 +359,7 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
                            const float (&sv1)[NGv], const float (&zv1)[NGv]) {
         const float p0 = ex2(s[0] - m0), p1 = PL ? 0.f : ex2(s[1] - m1), p2 = ex2(s[2] - m0), p3 = PL ? 0.f : ex2(s[3] - m1);
         l0 += p0 + p2;
-        l1 += p1 + p3;
+        if (!PL) l1 += p1 + p3;
         uint32_t va[NM][4];
         tile_frags<BITS, D>(vw, va);
         const float evc = evf * C1;
@@ -367,9 +367,10 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
         for (int j = 0; j < NGv; ++j) {
             const float e0 = sv0[j] * evf, e1 = sv1[j] * evc, sz0 = sv0[j] * zv0[j], sz1 = sv1[j] * zv1[j];
             bv[j][0] = fmaf(p0, sz0, fmaf(p2, sz1, bv[j][0]));
-            bv[j][1] = fmaf(p1, sz0, fmaf(p3, sz1, bv[j][1]));
-            const uint32_t b0 = movm_trans(pack_half2(p0 * e0, p1 * e0));
-            const uint32_t b1 = movm_trans(pack_half2(p2 * e1, p3 * e1));
+            if (!PL) bv[j][1] = fmaf(p1, sz0, fmaf(p3, sz1, bv[j][1]));
+            // with PL the odd columns carry no probability: a literal zero (0 * e is not foldable under IEEE rules)
+            const uint32_t b0 = movm_trans(pack_half2(p0 * e0, PL ? 0.f : p1 * e0));
+            const uint32_t b1 = movm_trans(pack_half2(p2 * e1, PL ? 0.f : p3 * e1));
 #pragma unroll
             for (int mi = 0; mi < mpg; ++mi) mma16816(O[j * mpg + mi], va[j * mpg + mi], b0, b1);
         }
