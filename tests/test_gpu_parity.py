@@ -94,6 +94,21 @@ def test_constant_groups_negative_zero_and_extremes():
     run_both(wl, K=K, V=V)
 
 
+@pytest.mark.parametrize("bits", [2, 3, 4])
+def test_wide_factor_range_with_one_query_head_per_kv_head(bits):
+    # head_dim 128 with as many query as KV heads: channels whose q * scale differ by several orders of magnitude, large
+    # zero-points, constant and zero channels
+    wl = TINY.scaled(seq=160, group=32, bits=bits, head_dim=128, batch=2, n_q_heads=2, n_kv_heads=2, seed=80 + bits)
+    K, V = synth.make_kv(wl, 0, "cuda")
+    K[:, :, :, 3] = 2.5
+    K[:, :, :, 4] = 0.0
+    K[:, :, :, 6] *= 300.0                                                         # one loud channel
+    K[:, :, :, 70] *= 1e-3                                                         # one quiet channel
+    K[:, :, :, 8] = 300.0 + torch.arange(160, device="cuda").half() * 0.25        # far from zero: large |zero|
+    K[:, :, :, 100] = -40.0 + torch.randn(160, device="cuda").half() * 0.01
+    run_both(wl, K=K, V=V)
+
+
 def test_bit_identical_across_runs_and_split_counts():
     wl = TINY.scaled(seq=32 * 40 + 5, group=32, bits=2, head_dim=128, n_q_heads=4, n_kv_heads=1, batch=1, topk=20, seed=12)
     r1 = run_both(wl)
