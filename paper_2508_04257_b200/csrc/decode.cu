@@ -464,8 +464,9 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
                     const float fp = v[e] * pre;
                     const float l0 = rintf(fp * (1.f / 16384.f)), r = fmaf(-l0, 16384.f, fp);
                     const float l1 = rintf(r * (1.f / 128.f)), l2 = rintf(fmaf(-l1, 128.f, r));
-                    const float F = fmaf(l0, 16384.f, fmaf(l1, 128.f, l2)) * (upper ? 16.f : 1.f);   // the factor the MMAs apply
-                    bsum = fmaf(F, zev[e], bsum);
+                    // the zero-point term takes the unrounded factor: the limbs' rounding then meets the codes (at most
+                    // qmax) only, not code - zero, which is large for a channel far from zero with a narrow range
+                    bsum = fmaf(upper ? fp * 16.f : fp, zev[e], bsum);
                     const int col = colbase + e;
                     const int at = ((col & 7) >> 1) * 4 + (BITS != 4 ? (mtx & 1) + 2 * (col & 1) : 2 * (col & 1) + (col >> 3));
                     tab[at] = (signed char)(int)l0;
