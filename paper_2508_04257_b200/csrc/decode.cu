@@ -628,8 +628,9 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
                     }
                     // lane t = 0 holds limbs 0, 1 (columns 0, 1), its neighbour limb 2 (column 2)
                     const int v0 = __shfl_down_sync(0xffffffffu, ia[0], 1), v1 = __shfl_down_sync(0xffffffffu, ia[2], 1);
-                    const float tg = fmaf((float)ia[0], 16384.f, fmaf((float)ia[1], 128.f, (float)v0));
-                    const float th = fmaf((float)ia[2], 16384.f, fmaf((float)ia[3], 128.f, (float)v1));
+                    // the two lower limbs combine in int32 (below 2^29 for every code width), then one conversion each
+                    const float tg = fmaf((float)ia[0], 16384.f, (float)(ia[1] * 128 + v0));
+                    const float th = fmaf((float)ia[2], 16384.f, (float)(ia[3] * 128 + v1));
                     s[k][0] = t == 0 ? fmaf(tg, ks0, -bias0) : -INFINITY; s[k][1] = -INFINITY;
                     s[k][2] = t == 0 ? fmaf(th, ks0 * (BITS == 4 ? 0.0625f : 0.25f), -bias0) : -INFINITY; s[k][3] = -INFINITY;
                     continue;
