@@ -220,7 +220,7 @@ struct DecodePlan {
 // fragment of one m16n8k32 (fields in place: x1, x4 for the rows g + 8, x16 for the upper contraction slots, x64 for
 // both).  4 bit: a word masked with 0x0f.. and 0xf0.. gives the registers of rows g and g + 8 (x16), two words (two
 // matrices) make one fragment.  The B operand holds the factor q * scale * 2^sh of each channel as three signed 7-bit
-// limbs in three accumulator columns (2, 3 bit: divided by 16 beforehand for the upper slots); sums are exact in int32.
+// limbs in four accumulator columns (2, 3 bit: divided by 16 beforehand for the upper slots); sums are exact in int32.
 // 3 bit: the low two bits as for 2 bit, the high bits of the second section (same byte structure) through four more
 // MMAs with the same B operands into accumulators of their own.
 template <int BITS, int D, int NGv, int CT, bool PL, bool I8 = false>
@@ -350,7 +350,7 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
 #pragma unroll
         for (int j = 0; j < NGv; ++j) { bv[j][0] *= c0; bv[j][1] *= c1; }
 #pragma unroll
-        for (int m = 0; m < NM; ++m) { O[m][0] *= c0; O[m][2] *= c0; O[m][1] *= c1; O[m][3] *= c1; }
+        for (int m = 0; m < NM; ++m) { O[m][0] *= c0; O[m][2] *= c0; O[m][1] *= PL ? c0 : c1; O[m][3] *= PL ? c0 : c1; }
         m0 = mn0; m1 = mn1;
     };
     // Value products of one tile: scores s (log2 units, relative maxima already advanced), value words vw, and the
@@ -368,9 +368,18 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
             const float e0 = sv0[j] * evf, e1 = sv1[j] * evc, sz0 = sv0[j] * zv0[j], sz1 = sv1[j] * zv1[j];
             bv[j][0] = fmaf(p0, sz0, fmaf(p2, sz1, bv[j][0]));
             if (!PL) bv[j][1] = fmaf(p1, sz0, fmaf(p3, sz1, bv[j][1]));
-            // with PL the odd columns carry no probability: a literal zero (0 * e is not foldable under IEEE rules)
-            const uint32_t b0 = movm_trans(pack_half2(p0 * e0, PL ? 0.f : p1 * e0));
-            const uint32_t b1 = movm_trans(pack_half2(p2 * e1, PL ? 0.f : p3 * e1));
+            uint32_t b0, b1;
+            if constexpr (PL) {
+                // the odd columns carry the fp16 rounding residual of the weight p * scale: the outputs keep the weight
+                // to ~22 bits (columns 2h and 2h+1 are added at the end)
+                const float x0 = p0 * e0, x1 = p2 * e1;
+                const float r0 = x0 - __half2float(__float2half_rn(x0)), r1 = x1 - __half2float(__float2half_rn(x1));
+                b0 = movm_trans(pack_half2(x0, r0));
+                b1 = movm_trans(pack_half2(x1, r1));
+            } else {
+                b0 = movm_trans(pack_half2(p0 * e0, p1 * e0));
+                b1 = movm_trans(pack_half2(p2 * e1, p3 * e1));
+            }
 #pragma unroll
             for (int mi = 0; mi < mpg; ++mi) mma16816(O[j * mpg + mi], va[j * mpg + mi], b0, b1);
         }
@@ -445,25 +454,28 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
             __syncwarp();   // the parameters are in registers: the slot can take the next group's while this one streams
             if (gi + 1 < my_groups) issue_params(gi + 1);
             if constexpr (I8) {
-                // limbs of the one head's factors: f = q * scale * 2^sh with the largest |f| in [2^19, 2^20)
+                // limbs of the one head's factors: f = q * scale * 2^sh with the largest |f| in [2^26, 2^27), four signed
+                // 7-bit limbs each: every factor is kept to 2^-27 of the group's largest one (2^-23 where the factor is
+                // pre-divided for the upper contraction slots), finer than binary32 keeps the factor itself
                 float v[CPL], amax = 0.f;
 #pragma unroll
                 for (int e = 0; e < CPL; ++e) { v[e] = qs[lane * CPL + e] * scv[e]; amax = fmaxf(amax, fabsf(v[e])); }
                 amax = warp_max(amax);
-                int sh = 19 - floor_log2(amax);
+                int sh = 26 - floor_log2(amax);
                 sh = sh > 60 ? 60 : (sh < -60 ? -60 : sh);
                 const bool upper = BITS != 4 && ((lane * CPL) & 8) != 0;   // 2, 3 bit: channels in the upper contraction slots (x16 in place)
                 const float pre = upper ? pow2i(sh - 4) : pow2i(sh);
                 const int mtx = (lane * CPL) >> 4, colbase = (lane * CPL) & 15;
                 // table [MMA][lower / upper slots][limb][t][byte]; 2 bit: MMA = word = matrix pair, upper = column half;
                 // 4 bit: MMA = matrix pair, upper = odd matrix
-                signed char *tab = reinterpret_cast<signed char *>(Bs) + ((mtx >> 1) * 2 + (BITS != 4 ? (colbase >> 3) : (mtx & 1))) * 48;
+                signed char *tab = reinterpret_cast<signed char *>(Bs) + ((mtx >> 1) * 2 + (BITS != 4 ? (colbase >> 3) : (mtx & 1))) * 64;
                 float bsum = 0.f;
 #pragma unroll
                 for (int e = 0; e < CPL; ++e) {
                     const float fp = v[e] * pre;
-                    const float l0 = rintf(fp * (1.f / 16384.f)), r = fmaf(-l0, 16384.f, fp);
-                    const float l1 = rintf(r * (1.f / 128.f)), l2 = rintf(fmaf(-l1, 128.f, r));
+                    const float l0 = rintf(fp * (1.f / 2097152.f)), r1 = fmaf(-l0, 2097152.f, fp);
+                    const float l1 = rintf(r1 * (1.f / 16384.f)), r2 = fmaf(-l1, 16384.f, r1);
+                    const float l2 = rintf(r2 * (1.f / 128.f)), l3 = rintf(fmaf(-l2, 128.f, r2));
                     // the zero-point term takes the unrounded factor: the limbs' rounding then meets the codes (at most
                     // qmax) only, not code - zero, which is large for a channel far from zero with a narrow range
                     bsum = fmaf(upper ? fp * 16.f : fp, zev[e], bsum);
@@ -472,6 +484,7 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
                     tab[at] = (signed char)(int)l0;
                     tab[16 + at] = (signed char)(int)l1;
                     tab[32 + at] = (signed char)(int)l2;
+                    tab[48 + at] = (signed char)(int)l3;
                 }
                 bsum = warp_sum(bsum) * pow2i(-sh);
                 if (t == 0) { bias0 = bsum; ks0 = pow2i(-sh); }
@@ -550,7 +563,7 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
             for (int i = 0; i < 4; ++i)
 #pragma unroll
                 for (int c2 = 0; c2 < 2; ++c2)
-                    bk[i][c2] = g < 3 ? *reinterpret_cast<const uint32_t *>(reinterpret_cast<const signed char *>(Bs) + (i * 2 + c2) * 48 + g * 16 + 4 * t) : 0u;
+                    bk[i][c2] = g < 4 ? *reinterpret_cast<const uint32_t *>(reinterpret_cast<const signed char *>(Bs) + (i * 2 + c2) * 64 + g * 16 + 4 * t) : 0u;
         } else {
 #pragma unroll
         for (int m = 0; m < NM; ++m) {
@@ -626,11 +639,12 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
                         ia[0] += ih0[0] + 4 * ih1[0]; ia[1] += ih0[1] + 4 * ih1[1];
                         ia[2] += 2 * ih0[2] + 8 * ih1[2]; ia[3] += 2 * ih0[3] + 8 * ih1[3];
                     }
-                    // lane t = 0 holds limbs 0, 1 (columns 0, 1), its neighbour limb 2 (column 2)
-                    const int v0 = __shfl_down_sync(0xffffffffu, ia[0], 1), v1 = __shfl_down_sync(0xffffffffu, ia[2], 1);
-                    // the two lower limbs combine in int32 (below 2^29 for every code width), then one conversion each
-                    const float tg = fmaf((float)ia[0], 16384.f, (float)(ia[1] * 128 + v0));
-                    const float th = fmaf((float)ia[2], 16384.f, (float)(ia[3] * 128 + v1));
+                    // lane t = 0 holds limbs 0, 1 (columns 0, 1), its neighbour limbs 2, 3 (columns 2, 3): each lane combines
+                    // its pair in int32 (below 2^31 for every code width), then one conversion per pair
+                    const int xg = ia[0] * 128 + ia[1], xh = ia[2] * 128 + ia[3];
+                    const int yg = __shfl_down_sync(0xffffffffu, xg, 1), yh = __shfl_down_sync(0xffffffffu, xh, 1);
+                    const float tg = fmaf((float)xg, 16384.f, (float)yg);
+                    const float th = fmaf((float)xh, 16384.f, (float)yh);
                     s[k][0] = t == 0 ? fmaf(tg, ks0, -bias0) : -INFINITY; s[k][1] = -INFINITY;
                     s[k][2] = t == 0 ? fmaf(th, ks0 * (BITS == 4 ? 0.0625f : 0.25f), -bias0) : -INFINITY; s[k][3] = -INFINITY;
                     continue;
@@ -765,8 +779,8 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
             const int ch0 = 16 * m + g, ch1 = ch0 + 8;
             if (PL) {
                 if (t < nq) {
-                    my_part[t * PS + ch0] = O[m][0] * OS0 - bj0;
-                    my_part[t * PS + ch1] = O[m][2] * OS1 - bj0;
+                    my_part[t * PS + ch0] = (O[m][0] + O[m][1]) * OS0 - bj0;
+                    my_part[t * PS + ch1] = (O[m][2] + O[m][3]) * OS1 - bj0;
                 }
                 continue;
             }

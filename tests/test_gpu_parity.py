@@ -94,18 +94,22 @@ def test_constant_groups_negative_zero_and_extremes():
     run_both(wl, K=K, V=V)
 
 
+@pytest.mark.parametrize("seed", range(6))
+@pytest.mark.parametrize("hq,hkv", [(2, 2), (8, 2)])
 @pytest.mark.parametrize("bits", [2, 3, 4])
-def test_wide_factor_range_with_one_query_head_per_kv_head(bits):
-    # head_dim 128 with as many query as KV heads: channels whose q * scale differ by several orders of magnitude, large
-    # zero-points, constant and zero channels
-    wl = TINY.scaled(seq=160, group=32, bits=bits, head_dim=128, batch=2, n_q_heads=2, n_kv_heads=2, seed=80 + bits)
+def test_wide_factor_range(bits, hq, hkv, seed):
+    # head_dim 128, one and four query heads per KV head: channels whose q * scale differ by several orders of magnitude
+    # (one 300 times louder, one 1000 times quieter than the rest), large zero-points (a ramp far from zero, and seeded
+    # noise of 0.01 around -40, |zero| ~ 1e4), constant and zero channels
+    wl = TINY.scaled(seq=160, group=32, bits=bits, head_dim=128, batch=2, n_q_heads=hq, n_kv_heads=hkv, seed=500 + seed)
     K, V = synth.make_kv(wl, 0, "cuda")
+    g = torch.Generator("cuda").manual_seed(seed)
     K[:, :, :, 3] = 2.5
     K[:, :, :, 4] = 0.0
-    K[:, :, :, 6] *= 300.0                                                         # one loud channel
-    K[:, :, :, 70] *= 1e-3                                                         # one quiet channel
-    K[:, :, :, 8] = 300.0 + torch.arange(160, device="cuda").half() * 0.25        # far from zero: large |zero|
-    K[:, :, :, 100] = -40.0 + (torch.arange(160, device="cuda") % 7).half() * 0.004   # narrow range far from zero: |zero| ~ 1e4
+    K[:, :, :, 6] *= 300.0
+    K[:, :, :, 70] *= 1e-3
+    K[:, :, :, 8] = 300.0 + torch.arange(160, device="cuda").half() * 0.25
+    K[:, :, :, 100] = -40.0 + torch.randn(160, device="cuda", generator=g).half() * 0.01
     run_both(wl, K=K, V=V)
 
 
