@@ -4,7 +4,7 @@
  * C ABI.  Every pointer documented "device" must point to CUDA device memory owned by the caller;
  * "host" pointers are ordinary host memory.  The library allocates no device memory, keeps no state
  * between calls (it caches two lookups: the driver's tensor-map encoder and, for kvsink_decode_attention_static,
- * the device address of its built-in scratch), launches all work asynchronously on the caller's stream and never
+ * the device address of its built-in scratch; and it counts its kernel launches, see kvsink_launch_count), launches all work asynchronously on the caller's stream and never
  * synchronises, except in kvsink_read_status.  Every entry point returns 0 (KVSINK_OK) or a negative KVSINK_ERR_* code; argument
  * errors are detected on the host before anything is launched.  Nothing traps or spins on the device.
  *
@@ -171,7 +171,9 @@ int kvsink_decode_attention(const kvsink_config *cfg, const kvsink_cache *cache,
  *     KVSINK_STATIC_SCRATCH_BYTES, otherwise KVSINK_ERR_STATIC_SCRATCH is returned and nothing is launched
  *     (use kvsink_decode_attention with your own workspace then).
  *   - The first call on each device looks up the array's device address (a CUDA runtime query, made with that
- *     device current, no allocation).  Make that first call outside of any stream capture.
+ *     device current, no allocation).  Make that first call outside of any stream capture.  The address is kept for
+ *     the life of the device's primary context: after cudaDeviceReset (or anything else that destroys that context)
+ *     the cached address is stale and this entry point must not be used again in the process.
  *   - All calls on a device share the one array, which keeps whatever the previous call left in it.  Nothing in
  *     it has to start at zero -- each call overwrites every record it later reads -- but two calls whose kernels
  *     overlap on the GPU (different streams, no ordering between them) race on it and corrupt each other's
@@ -182,6 +184,10 @@ int kvsink_decode_attention_static(const kvsink_config *cfg, const kvsink_cache 
 
 /* Copies the device status word to *host_status and waits for the stream (the only call that synchronises). */
 int kvsink_read_status(const kvsink_cache *cache, int32_t *host_status, void *cuda_stream);
+
+/* Kernel launches the library has made in this process since it was loaded (host counter; every entry point adds the
+ * kernels it launched).  For accounting in benchmarks and tests; not a step of the paper's method. */
+unsigned long long kvsink_launch_count(void);
 
 /* Static text for a status code. */
 const char *kvsink_strerror(int code);

@@ -16,7 +16,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _LIB_PATH = os.path.join(_HERE, "libkvsink.so")
 
 EXPORTS = ("kvsink_cache_sizes", "kvsink_predict_sinks", "kvsink_quantize_append", "kvsink_decode_attention",
-           "kvsink_decode_attention_static", "kvsink_read_status", "kvsink_strerror")
+           "kvsink_decode_attention_static", "kvsink_read_status", "kvsink_launch_count", "kvsink_strerror")
 STATIC_SCRATCH_BYTES = 4 * 1024 * 1024
 
 
@@ -56,6 +56,7 @@ def lib():
             raise ImportError(f"{_LIB_PATH} is missing: build it with `python -m paper_2508_04257_b200.build`")
         _lib = C.CDLL(_LIB_PATH)
         _lib.kvsink_strerror.restype = C.c_char_p
+        _lib.kvsink_launch_count.restype = C.c_ulonglong
         for name in EXPORTS:
             getattr(_lib, name)
     return _lib
@@ -192,6 +193,11 @@ def decode_attention_static(cfg: Config, cache: KVCache, q: torch.Tensor, out: t
     if rc:
         raise KvsinkError(rc, "kvsink_decode_attention_static")
     return out, lse
+
+
+def launch_count() -> int:
+    """kvsink_launch_count: kernel launches the library has made in this process."""
+    return int(lib().kvsink_launch_count())
 
 
 def read_status(cache: KVCache) -> int:

@@ -3,6 +3,8 @@
 
 using namespace kvsink;
 
+std::atomic<unsigned long long> kvsink::g_launches{0};
+
 static int derive(const kvsink_config *cfg, Params *p)
 {
     if (!cfg) return KVSINK_ERR_BAD_ARG;
@@ -169,6 +171,8 @@ extern "C" int kvsink_read_status(const kvsink_cache *cache, int32_t *host_statu
     if (cudaStreamSynchronize(st) != cudaSuccess) return KVSINK_ERR_CUDA;
     return KVSINK_OK;
 }
+
+extern "C" unsigned long long kvsink_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
 extern "C" const char *kvsink_strerror(int code)
 {

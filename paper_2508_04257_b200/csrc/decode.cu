@@ -1007,7 +1007,10 @@ static int launch_decode_p(const Params &p, const kvsink_cache &c, const __half 
             pdl[1].val.clusterDim.z = 1;
             cfg.numAttrs = 2;
         }
-        if (cudaLaunchKernelEx(&cfg, kern, p, c, q, out, lse, ws, nsplit, gps, qchunks, (int)c.seq_len, (int)cluster_merge) == cudaSuccess) break;
+        if (cudaLaunchKernelEx(&cfg, kern, p, c, q, out, lse, ws, nsplit, gps, qchunks, (int)c.seq_len, (int)cluster_merge) == cudaSuccess) {
+            note_launch();
+            break;
+        }
         (void)cudaGetLastError();
         if (!cluster_merge) return KVSINK_ERR_CUDA;
         cluster_merge = false;   // a cluster that cannot be placed: the same launch without one, merged by the second kernel
@@ -1020,6 +1023,7 @@ static int launch_decode_p(const Params &p, const kvsink_cache &c, const __half 
         cfg.attrs = pdl;
         cfg.numAttrs = 1;
         if (cudaLaunchKernelEx(&cfg, decode_merge_kernel, (const float *)ws, nsplit, (int)D, out, lse) != cudaSuccess) return KVSINK_ERR_CUDA;
+        note_launch();
     }
     return KVSINK_OK;
 }

@@ -9,6 +9,15 @@ struct ChannelList {
     int c[8];
 };
 
+// Magnitude key of an fp16 value: its 15-bit pattern, which orders finite values and infinity as |x| does.  A NaN
+// (pattern above 0x7c00) compares false against everything in the reference comparison `|x| > best`, so it never raises
+// a score: its key is 0.
+__device__ __forceinline__ unsigned magnitude_key(uint16_t h)
+{
+    const unsigned a = h & 0x7fffu;
+    return a > 0x7c00u ? 0u : a;
+}
+
 // score = max over listed channels of |H| as the 15-bit magnitude pattern of the fp16 value (order-preserving).
 __global__ void sink_score_listed(const uint16_t *__restrict__ H, int S, int64_t sb, int64_t ss, ChannelList cl,
                                   uint16_t *__restrict__ score, int score_stride)
@@ -21,7 +30,7 @@ __global__ void sink_score_listed(const uint16_t *__restrict__ H, int S, int64_t
     unsigned best = 0;
 #pragma unroll 1
     for (int j = 0; j < cl.n; ++j) {
-        unsigned a = __ldg(row + cl.c[j]) & 0x7fffu;
+        unsigned a = magnitude_key(__ldg(row + cl.c[j]));
         best = a > best ? a : best;
     }
     score[(size_t)b * score_stride + i] = (uint16_t)best;
@@ -38,7 +47,7 @@ __global__ void sink_score_all(const uint16_t *__restrict__ H, int S, int d, int
     const uint16_t *row = H + b * sb + warp * ss;
     unsigned best = 0;
     for (int c = lane; c < d; c += 32) {
-        unsigned a = __ldg(row + c) & 0x7fffu;
+        unsigned a = magnitude_key(__ldg(row + c));
         best = a > best ? a : best;
     }
 #pragma unroll

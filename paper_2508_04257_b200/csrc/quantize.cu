@@ -259,6 +259,7 @@ int launch_quantize_groups(const Params &p, const kvsink_cache &c, const __half 
     if (cudaFuncSetAttribute(quantize_groups_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
         return KVSINK_ERR_CUDA;
     dim3 grid(n_groups, p.Hkv, p.B);
+    note_launch();
     quantize_groups_kernel<<<grid, QG_THREADS, smem, st>>>(p, c, k_src, v_src, first_token, sb, sh, stt, do_v_and_sinks ? 1 : 0);
     return cudaGetLastError() == cudaSuccess ? KVSINK_OK : KVSINK_ERR_CUDA;
 }

@@ -587,6 +587,7 @@ static int launch_stream(const Params &p, const kvsink_cache &c, const __half *k
     if (per_sm > cap) per_sm = cap;
     long blocks = 148L * per_sm;
     if (blocks > n_items) blocks = n_items;
+    note_launch();
     kern<<<(unsigned)blocks, 32 * NW, smem, st>>>(p, c, k_src, v_src, first_token, n_groups, sb, sh, stt, kinds);
     return cudaGetLastError() == cudaSuccess ? KVSINK_OK : KVSINK_ERR_CUDA;
 }

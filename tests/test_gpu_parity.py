@@ -78,6 +78,22 @@ def test_ties_in_the_score_go_to_the_lower_index():
     run_both(wl0, H=H)
 
 
+def test_nan_and_infinity_in_the_hidden_state():
+    # an infinite value outranks every finite one; a NaN never raises a token's score (the comparison |x| > best is false)
+    wl = TINY.scaled(seq=200, topk=4, pfn_n=1, batch=2, seed=21)
+    H = synth.make_hidden(wl, "cuda")
+    c0, c1 = wl.channels[0], wl.channels[1]
+    H[0, 50, c0] = float("nan")
+    H[0, 60, c1] = float("inf")
+    H[1, 70, c0] = float("-inf")
+    H[1, 71, c0] = float("nan")
+    H[1, 71, c1] = 3.0
+    r = run_both(wl, H=H)
+    pos = r["oracle_cache"].sink_pos.reshape(wl.batch, -1)
+    assert 60 in pos[0] and 50 not in pos[0] and 70 in pos[1]
+    run_both(wl.scaled(channels=()), H=H)
+
+
 def test_constant_groups_negative_zero_and_extremes():
     wl = TINY.scaled(seq=128, group=32, bits=4, batch=1, n_q_heads=2, n_kv_heads=2, seed=8)
     K, V = synth.make_kv(wl, 0, "cuda")

@@ -1,8 +1,10 @@
 """GPU parity at the full sizes of the five workloads, in the launch configuration the benchmark times.
 
-The oracle cannot redo a whole workload in seconds, so it is run one (sequence, KV head) unit at a time on
-sampled units: sink prediction for the unit's whole sequence, the unit's packed codes / parameters / side buffer
-bit for bit, then one appended token and the unit's attention outputs within tolerance."""
+The single-layer workloads are compared in full: every (sequence, KV head) unit's packed codes, parameters, side
+buffer and tail bit for bit, and every attention output within tolerance.  The 32-layer workload holds 2048 units of
+8192 tokens per layer; there the oracle is run one unit at a time on 64 units spread over the whole index range, on
+two of the layers: sink prediction for the unit's whole sequence, the unit's arrays bit for bit, then one appended
+token and the unit's attention outputs within tolerance."""
 import numpy as np
 import pytest
 import torch
@@ -11,7 +13,7 @@ import oracle
 import paper_2508_04257_b200 as kv
 from paper_2508_04257_b200 import synth
 
-from parity_util import assert_close, bits_equal, np16
+from parity_util import assert_close, bits_equal, np16, run_both
 
 pytestmark = pytest.mark.gpu
 
@@ -31,7 +33,7 @@ def _unit_slice(t, wl, b, h, per_unit):
     return t[u * per_unit:(u + 1) * per_unit].cpu().numpy()
 
 
-def check_units(wl, H, layers, units, n_seq_checked=2):
+def check_units(wl, H, layers, units, n_seq_checked=2, layer0=0):
     """layers: list of (K, V) device tensors; units: list of (b, h)."""
     gcfg, ucfg = _gpu_cfg(wl), _unit_cfg(wl)
     rep = wl.n_q_heads // wl.n_kv_heads
@@ -54,7 +56,7 @@ def check_units(wl, H, layers, units, n_seq_checked=2):
         assert bits_equal(g_bm[b:b + 1], bm) and bits_equal(g_pos[b:b + 1], pos) and g_cnt[b] == cnt[0]
         seq_masks[b] = (bm, pos, cnt)
     worst = 0.0
-    for li, (K, V) in enumerate(layers):
+    for li, (K, V) in enumerate(layers, start=layer0):
         cache = kv.KVCache(gcfg, sinks)
         kv.quantize_append(gcfg, cache, K, V)
         k1, v1 = synth.make_new_token(wl, li, 0, "cuda")
@@ -87,33 +89,49 @@ def check_units(wl, H, layers, units, n_seq_checked=2):
     return worst
 
 
-def test_llama2_7b_layer_full_size():
-    wl = synth.WORKLOADS["llama2_7b_layer"]
+def check_whole_workload(wl):
+    """Every unit of a single-layer workload: prediction, prefill, one appended token, attention."""
     H = synth.make_hidden(wl, "cuda")
-    worst = check_units(wl, H, [synth.make_kv(wl, 0, "cuda")], [(0, 0), (3, 17), (7, 31), (5, 8)])
-    print("config 2 worst attention error", worst)
+    K, V = synth.make_kv(wl, 0, "cuda")
+    r = run_both(wl, appends=1, H=H, K=K, V=V)
+    planted = synth.sink_positions(wl)
+    oc = r["oracle_cache"]
+    cap = wl.topk + wl.pfn_n
+    for b in range(wl.batch):                      # every sequence: the planted outliers (and the first N) are found
+        want = sorted(set(planted[b].tolist()) | set(range(wl.pfn_n)))
+        assert oc.sink_pos.reshape(wl.batch, cap)[b, :oc.sink_count[b]].tolist() == want
+    return r["err"]
+
+
+def test_llama2_7b_layer_full_size():
+    print("config 2 worst attention error", check_whole_workload(synth.WORKLOADS["llama2_7b_layer"]))
 
 
 def test_llama3_8b_gqa_full_size():
-    wl = synth.WORKLOADS["llama3_8b_gqa"]
-    H = synth.make_hidden(wl, "cuda")
-    check_units(wl, H, [synth.make_kv(wl, 0, "cuda")], [(0, 0), (3, 7), (2, 4)])
+    print("config 3 worst attention error", check_whole_workload(synth.WORKLOADS["llama3_8b_gqa"]))
 
 
 def test_long_context_gqa_full_size():
-    wl = synth.WORKLOADS["long_gqa"]
-    H = synth.make_hidden(wl, "cuda")
-    check_units(wl, H, [synth.make_kv(wl, 0, "cuda")], [(0, 0), (0, 5)])
+    print("config 5 worst attention error", check_whole_workload(synth.WORKLOADS["long_gqa"]))
+
+
+def _spread_units(wl, n, shift):
+    """n (sequence, KV head) units spread evenly over the unit index range, every KV head and many sequences among them."""
+    nu = wl.batch * wl.n_kv_heads
+    step = nu // n
+    units = [(i * step + (i * 13 + shift) % step) for i in range(n)]
+    return [(u // wl.n_kv_heads, u % wl.n_kv_heads) for u in units]
 
 
 @pytest.mark.parametrize("name", ["decode32_3bit", "decode32_4bit"])
 def test_decode32_full_batch_two_layers(name):
-    """Full batch and sequence of the 32-layer decode workload; two of the 32 layers (each 8.6 GB of fp16 input)."""
+    """Full batch and sequence of the 32-layer decode workload; two of the 32 layers (each 8.6 GB of fp16 input), 64 units
+    of each, the first and the last unit among them."""
     wl = synth.WORKLOADS[name]
     H = synth.make_hidden(wl, "cuda")
-    layers = [synth.make_kv(wl, 0, "cuda")]
-    check_units(wl, H, layers, [(0, 0), (63, 31), (17, 5)])
-    del layers
-    torch.cuda.empty_cache()
-    layers = [synth.make_kv(wl, 1, "cuda")]
-    check_units(wl, H, layers, [(40, 12)])
+    for layer, shift in ((0, 0), (1, 5)):
+        units = _spread_units(wl, 62, shift) + [(0, 0), (wl.batch - 1, wl.n_kv_heads - 1)]
+        layers = [synth.make_kv(wl, layer, "cuda")]
+        check_units(wl, H, layers, sorted(set(units)), layer0=layer)
+        del layers
+        torch.cuda.empty_cache()

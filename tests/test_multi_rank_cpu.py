@@ -1,8 +1,11 @@
 """The multi-GPU path of the benchmark on CPU: two gloo ranks.  The hot path shards by sequence with no data-path
 collective, so what needs testing is the plumbing: per-rank seeds give disjoint batches, the slowest rank's time
 is what every rank sees, and the aggregate counts the units of all ranks."""
+import json
 import os
 import socket
+import subprocess
+import sys
 
 import numpy as np
 import torch
@@ -57,3 +60,15 @@ def test_two_gloo_ranks_shard_by_sequence_and_take_the_slowest_time():
 def test_single_process_is_the_identity():
     assert dist_util.max_over_ranks(3.5, "cpu") == 3.5
     assert dist_util.aggregate_throughput(10.0, 1, 2.0) == 5.0
+
+
+def test_bench_starts_its_own_ranks():
+    """`bench.py --gpus 2` without a launcher starts two ranks itself; here only the plumbing runs (gloo, no kernels)."""
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    r = subprocess.run([sys.executable, os.path.join(root, "bench.py"), "--gpus", "2", "--plumbing-only"], capture_output=True, text=True,
+                       env=env, timeout=300)
+    assert r.returncode == 0, r.stderr[-2000:]
+    lines = [json.loads(l) for l in r.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1                                   # rank 0 alone prints
+    assert lines[0]["n_gpus"] == 2 and lines[0]["ms_per_step"] == 2.0 and lines[0]["scaling"] == "weak"

@@ -36,8 +36,13 @@ def test_static_scratch_matches_the_workspace_entry_point_twice_in_a_row():
         ref, ref_lse = kv.decode_attention(cfg, cache, q)
         out = torch.full(shape, float("nan"), dtype=torch.float32, device="cuda")
         lse = torch.full(shape[:2], float("nan"), dtype=torch.float32, device="cuda")
+        torch.cuda.synchronize()
+        if call == 1:       # the first call has made the one-time address lookup; from now on device memory must not move
+            free_before, allocated_before = torch.cuda.mem_get_info()[0], torch.cuda.memory_allocated()
         kv.decode_attention_static(cfg, cache, q, out, lse)
         torch.cuda.synchronize()
+        if call == 1:
+            assert torch.cuda.mem_get_info()[0] == free_before and torch.cuda.memory_allocated() == allocated_before
         o, r = out.cpu().numpy(), ref.cpu().numpy()
         assert np.all(np.isfinite(o))
         assert np.all(np.abs(o - r) <= ATOL + RTOL * np.abs(r)), f"call {call}: max diff {np.abs(o - r).max():.3e}"
