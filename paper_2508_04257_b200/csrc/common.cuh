@@ -115,6 +115,16 @@ inline cudaError_t launch_pdl(void (*kern)(KArgs...), dim3 grid, dim3 block, siz
     return cudaLaunchKernelEx(&cfg, kern, KArgs(args)...);
 }
 
+// Decode attention: warps per block, the "no score yet" value of a running maximum, and 2^x.
+constexpr int DEC_WARPS = 4;
+constexpr float M_INIT = -1.0e30f;
+__device__ __forceinline__ float ex2(float x)
+{
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
 __device__ __forceinline__ bool mask_bit(const uint32_t *__restrict__ bm, int pos) { return (bm[pos >> 5] >> (pos & 31)) & 1u; }
 
 // Launchers implemented in the kernel translation units; all return a KVSINK_* code.
@@ -131,6 +141,12 @@ int launch_quantize_tokens(const Params &p, const kvsink_cache &c, const __half 
 int launch_decode(const Params &p, const kvsink_cache &c, const __half *q, float *out, float *lse, void *workspace,
                   size_t workspace_bytes, cudaStream_t st);
 int launch_decode_static(const Params &p, const kvsink_cache &c, const __half *q, float *out, float *lse, cudaStream_t st);
+int launch_decode_b2(const Params &p, const kvsink_cache &c, const __half *q, float *out, float *lse, float *ws, cudaStream_t st);
+int launch_decode_b3(const Params &p, const kvsink_cache &c, const __half *q, float *out, float *lse, float *ws, cudaStream_t st);
+int launch_decode_b4(const Params &p, const kvsink_cache &c, const __half *q, float *out, float *lse, float *ws, cudaStream_t st);
+int launch_decode_merge(const float *ws, int nsplit, int D, int n_rows, float *out, float *lse, cudaStream_t st);
+int max_splits(const Params &p);
+int choose_splits(const Params &p, int n_groups);
 size_t decode_workspace_bytes(const Params &p);
 size_t predict_workspace_bytes(const Params &p);
 

@@ -1,904 +1,10 @@
-// Single-token decode attention over the packed cache (Eq. 3 with Eq. 7's split into sink and non-sink sums).
-//
-// A packed tile is the register image of the m16n8k16 A operand, so a lane's 128-bit load IS its fragment.
-// Codes are never converted: a b-bit field masked in place is an fp16 subnormal (code * 2^k * 2^-24), which the
-// tensor core multiplies exactly; the power-of-two position factors are folded into the B operand (column half)
-// and into the fp32 epilogue (row half).
-//   scores   S[token, head] = sum_c code[token, c] * (q[head, c] * scale[c]) - sum_c q*scale*zero      (keys)
-//   outputs  O[c, head]     = sum_t code[c, t] * (p[t, head] * scale[t])  - sum_t p*scale*zero         (values)
-// with M = 16 tokens (keys) or 16 channels (values), N = 8 query heads of one KV head, fp32 accumulation.
-// Each warp streams whole key groups of one (sequence, KV head) unit; sequence splits are merged by a second
-// kernel.  Sink tokens are masked out of the packed stream and added from the fp16 side buffer under the same
-// softmax; keys of the open group come from the fp16 tail.
-#include <cooperative_groups.h>
-
+// Decode attention, host side: split heuristic, merge of the sequence splits, dispatch over the code width, and the
+// entry point that keeps its scratch inside the library image.  The split kernel itself is in decode_kernel.cuh.
 #include <mutex>
 
 #include "common.cuh"
 
 namespace kvsink {
-
-constexpr int DEC_WARPS = 4;
-constexpr int DEC_THREADS = DEC_WARPS * 32;
-constexpr float M_INIT = -1.0e30f;
-
-__device__ __forceinline__ float ex2(float x)
-{
-    float y;
-    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-    return y;
-}
-
-__device__ __forceinline__ void mma16816(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1)
-{
-    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
-}
-
-__device__ __forceinline__ uint32_t movm_trans(uint32_t v)
-{
-    uint32_t o;
-    asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(o) : "r"(v));
-    return o;
-}
-
-__device__ __forceinline__ uint32_t pack_half2(float lo, float hi)
-{
-    __half2 h = __floats2half2_rn(lo, hi);
-    return *reinterpret_cast<uint32_t *>(&h);
-}
-
-// floor(log2(x)) of a positive normal float; -127 for zero and subnormals.
-__device__ __forceinline__ int floor_log2(float x) { return (int)((__float_as_uint(x) >> 23) & 0xffu) - 127; }
-// 2^e for -126 <= e <= 127.
-__device__ __forceinline__ float pow2i(int e) { return __uint_as_float((uint32_t)(e + 127) << 23); }
-
-__device__ __forceinline__ float warp_max(float v)
-{
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
-    return v;
-}
-
-template <int BITS, int D>
-struct Geo {
-    static constexpr int W = D * BITS / 64;                  // 32-bit words per lane per tile
-    static constexpr int NLO = (BITS == 3) ? D / 32 : W;     // words per lane in the first section
-    static constexpr int NHI = (BITS == 3) ? D / 64 : 0;
-    static constexpr int NM = D / 16;                        // 16x16 matrices per tile
-    // value of a masked field = code * ROWF^(row half) * COLF^(col half) * 2^-24
-    static constexpr float ROWF = (BITS == 2) ? 4.f : (BITS == 3 ? 1.f : 16.f);
-    static constexpr float COLF = (BITS == 4) ? 1.f : 16.f;
-};
-
-// A lane's words of one tile: section planes of up to four words per lane.
-template <int N>
-__device__ __forceinline__ void load_section(const uint32_t *__restrict__ sec, int lane, uint32_t *w)
-{
-#pragma unroll
-    for (int p = 0; p * 4 < N; ++p) {
-        const int u = (N - 4 * p) > 4 ? 4 : (N - 4 * p);
-        const uint32_t *src = sec + u * lane;
-        if (u == 4) {
-            uint4 v = __ldg((const uint4 *)src);
-            w[4 * p] = v.x; w[4 * p + 1] = v.y; w[4 * p + 2] = v.z; w[4 * p + 3] = v.w;
-        } else if (u == 2) {
-            uint2 v = __ldg((const uint2 *)src);
-            w[4 * p] = v.x; w[4 * p + 1] = v.y;
-        } else {
-#pragma unroll
-            for (int i = 0; i < u; ++i) w[4 * p + i] = __ldg(src + i);
-        }
-        sec += 32 * u;
-    }
-}
-
-// The same from a tile image in shared memory.
-template <int N>
-__device__ __forceinline__ void load_section_shared(const uint32_t *sec, int lane, uint32_t *w)
-{
-#pragma unroll
-    for (int p = 0; p * 4 < N; ++p) {
-        const int u = (N - 4 * p) > 4 ? 4 : (N - 4 * p);
-        const uint32_t *src = sec + u * lane;
-        if (u == 4) {
-            uint4 v = *(const uint4 *)src;
-            w[4 * p] = v.x; w[4 * p + 1] = v.y; w[4 * p + 2] = v.z; w[4 * p + 3] = v.w;
-        } else if (u == 2) {
-            uint2 v = *(const uint2 *)src;
-            w[4 * p] = v.x; w[4 * p + 1] = v.y;
-        } else {
-#pragma unroll
-            for (int i = 0; i < u; ++i) w[4 * p + i] = src[i];
-        }
-        sec += 32 * u;
-    }
-}
-
-template <int BITS, int D>
-__device__ __forceinline__ void load_tile_shared(const uint32_t *tile, int lane, uint32_t (&w)[Geo<BITS, D>::W])
-{
-    using G_ = Geo<BITS, D>;
-    load_section_shared<G_::NLO>(tile, lane, w);
-    if constexpr (BITS == 3) load_section_shared<G_::NHI>(tile + 32 * G_::NLO, lane, w + G_::NLO);
-}
-
-template <int BITS, int D>
-__device__ __forceinline__ void load_tile(const uint32_t *__restrict__ tile, int lane, uint32_t (&w)[Geo<BITS, D>::W])
-{
-    using G_ = Geo<BITS, D>;
-    load_section<G_::NLO>(tile, lane, w);
-    if constexpr (BITS == 3) load_section<G_::NHI>(tile + 32 * G_::NLO, lane, w + G_::NLO);
-}
-
-// Masked fields of a lane's words as the A registers of the tile's NM matrices.
-template <int BITS, int D>
-__device__ __forceinline__ void tile_frags(const uint32_t (&w)[Geo<BITS, D>::W], uint32_t (&a)[Geo<BITS, D>::NM][4])
-{
-    using G_ = Geo<BITS, D>;
-    if constexpr (BITS == 2) {
-#pragma unroll
-        for (int i = 0; i < G_::W; ++i) {
-            const uint32_t x = w[i], y = x >> 8;
-            a[2 * i][0] = x & 0x00030003u; a[2 * i][1] = x & 0x000c000cu; a[2 * i][2] = x & 0x00300030u; a[2 * i][3] = x & 0x00c000c0u;
-            a[2 * i + 1][0] = y & 0x00030003u; a[2 * i + 1][1] = y & 0x000c000cu; a[2 * i + 1][2] = y & 0x00300030u; a[2 * i + 1][3] = y & 0x00c000c0u;
-        }
-    } else if constexpr (BITS == 4) {
-#pragma unroll
-        for (int i = 0; i < G_::W; ++i) {
-            const uint32_t x = w[i], y = x >> 8;
-            a[i][0] = x & 0x000f000fu; a[i][1] = x & 0x00f000f0u; a[i][2] = y & 0x000f000fu; a[i][3] = y & 0x00f000f0u;
-        }
-    } else {
-#pragma unroll
-        for (int i = 0; i < G_::NLO; ++i) {
-            const uint32_t x = w[i];
-            const uint32_t hh = (i & 1) ? (w[G_::NLO + i / 2] << 2) : w[G_::NLO + i / 2];
-            const uint32_t me = (x & 0x33333333u) | (hh & 0xccccccccu);                 // even fields, 3 bits at 4j
-            const uint32_t mo = ((x >> 2) & 0x33333333u) | ((hh >> 1) & 0xccccccccu);   // odd fields
-            const uint32_t me8 = me >> 8, mo8 = mo >> 8;
-            a[2 * i][0] = me & 0x00070007u; a[2 * i][1] = mo & 0x00070007u; a[2 * i][2] = me & 0x00700070u; a[2 * i][3] = mo & 0x00700070u;
-            a[2 * i + 1][0] = me8 & 0x00070007u; a[2 * i + 1][1] = mo8 & 0x00070007u; a[2 * i + 1][2] = me8 & 0x00700070u; a[2 * i + 1][3] = mo8 & 0x00700070u;
-        }
-    }
-}
-
-// ---- per-warp bulk-copy ring (TMA, cp.async.bulk) ----
-__device__ __forceinline__ void mbar_init(uint64_t *bar, unsigned count)
-{
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(bar)), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint64_t *bar, unsigned bytes)
-{
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, unsigned parity)
-{
-    unsigned ok;
-    asm volatile("{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
-                 : "=r"(ok) : "r"(smem_addr(bar)), "r"(parity) : "memory");
-    return ok != 0;
-}
-// Global -> shared bulk copy; addresses and size are multiples of 16 bytes; completion is counted on `bar`.
-__device__ __forceinline__ void bulk_g2s(void *dst, const void *src, unsigned bytes, uint64_t *bar)
-{
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                 ::"r"(smem_addr(dst)), "l"(src), "r"(bytes), "r"(smem_addr(bar)) : "memory");
-}
-
-constexpr int DEC_WAIT_LIMIT = 1 << 22;   // polls of a full-barrier before a warp gives up (far beyond any real latency)
-
-// Shared-memory plan of a decode block, shared by the kernel and the launcher.  CT = tiles per ring chunk.
-template <int BITS, int D, int NGv, int CT>
-struct DecodePlan {
-    static constexpr int W = D * BITS / 64, TILE_BYTES = 128 * W;
-    static constexpr int BST = D + 8;                                   // padded row stride of the key B tables (bank spread)
-    static constexpr int KV_BYTES = CT * TILE_BYTES, SZ_BYTES = CT * 16 * NGv * 4;
-    static constexpr int SLOT_BYTES = 2 * KV_BYTES + 2 * SZ_BYTES;      // K words, V words, V scales, V zeros of CT tiles
-    static constexpr int NSLOT = (9216 / SLOT_BYTES >= 4) ? 4 : 2;      // power of two
-    static constexpr int KP_BYTES = 2 * D * 4;                          // key scale + zero of one group
-    static constexpr int WARP_RING = NSLOT * SLOT_BYTES + KP_BYTES;
-    __host__ __device__ static size_t fixed_bytes(int nq)
-    {
-        size_t f = 8 * D * 4 + 8 * D * 2 + (size_t)DEC_WARPS * 2 * nq * BST * 2 + DEC_WARPS * 8 * 8;
-        return (f + 127) / 128 * 128;
-    }
-    __host__ __device__ static size_t bytes(int nq)
-    {
-        const size_t ring = (size_t)DEC_WARPS * WARP_RING, part = (size_t)2 * DEC_WARPS * nq * (D + 2) * 4;
-        return fixed_bytes(nq) + (ring > part ? ring : part);
-    }
-};
-
-// PL ("pair layout", for at most four query heads per KV head): query head h owns accumulator columns 2h and 2h+1;
-// column 2h multiplies by the fp16 factor q*scale and column 2h+1 by its fp16 rounding residual, so every score carries
-// the factor to ~22 bits at no extra instruction.  Without PL (five to eight heads) head h owns column h and the
-// residual of channels with large factors goes through a second multiply.
-// I8 (one query head per KV head): the key side runs on the integer tensor path.  The four bytes of a stored
-// word are four channels of one token row.  2 bit: the word masked with 0x03.., 0x0c.., 0x30.., 0xc0.. is the u8 A
-// fragment of one m16n8k32 (fields in place: x1, x4 for the rows g + 8, x16 for the upper contraction slots, x64 for
-// both).  4 bit: a word masked with 0x0f.. and 0xf0.. gives the registers of rows g and g + 8 (x16), two words (two
-// matrices) make one fragment.  The B operand holds the factor q * scale * 2^sh of each channel as three signed 7-bit
-// limbs in four accumulator columns (2, 3 bit: divided by 16 beforehand for the upper slots); sums are exact in int32.
-// 3 bit: the low two bits as for 2 bit, the high bits of the second section (same byte structure) through four more
-// MMAs with the same B operands into accumulators of their own.
-template <int BITS, int D, int NGv, int CT, bool PL, bool I8 = false>
-__global__ void __launch_bounds__(DEC_THREADS, 4)
-decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__restrict__ out, float *__restrict__ lse,
-              float *__restrict__ part_ws, int nsplit, int groups_per_split, int qchunks, int seq_len, int cluster_merge)
-{
-    using G_ = Geo<BITS, D>;
-    using Plan = DecodePlan<BITS, D, NGv, CT>;
-    constexpr int NM = G_::NM, W = G_::W, BST = Plan::BST, TILE_WORDS = 32 * W;
-    constexpr int NSLOT = Plan::NSLOT, SLOT_BYTES = Plan::SLOT_BYTES, KV_BYTES = Plan::KV_BYTES, SZ_BYTES = Plan::SZ_BYTES;
-    constexpr int mpg = (D / NGv) / 16;                              // value matrices per channel group
-    constexpr int ST = CT >= 4 ? 4 : (CT >= 2 ? 2 : 1);                              // tiles per softmax step
-    constexpr int CPL = D / 32;                                      // channels per lane in per-channel passes
-    constexpr float LOG2E = 1.4426950408889634f;
-    constexpr float QMAX = (float)((1 << BITS) - 1);
-    constexpr float R1 = 1.f / G_::ROWF, C1 = 1.f / G_::COLF;
-
-    const int tid = threadIdx.x, lane = tid & 31, warp = __shfl_sync(0xffffffffu, tid >> 5, 0), g = lane >> 2, t = lane & 3;
-    const int split = blockIdx.x, h = blockIdx.y / qchunks, qc = blockIdx.y % qchunks, b = blockIdx.z;
-    const int nq = min(8, p.rep - 8 * qc), hq0 = h * p.rep + 8 * qc;
-    const int64_t unit = (int64_t)b * p.Hkv + h;
-    const int G = p.G, n = seq_len, n_groups = n / G, n_body = n_groups * G;
-    const int TPG = G / KVSINK_TILE, CPG = TPG / CT;                 // tiles and ring chunks per key group
-    const uint32_t *bm = c.sink_bitmask + (size_t)b * p.mask_words;
-    const float qscale = LOG2E * rsqrtf((float)D);
-
-    extern __shared__ __align__(128) unsigned char smem_raw[];
-    float *qs = (float *)smem_raw;                                   // [8][D] q * log2e/sqrt(D)
-    __half *q16 = (__half *)(qs + 8 * D);                            // [8][D] q as given
-    __half *Bs_all = q16 + 8 * D;                                    // [warps][2][nq][BST] key B operand (hi, lo) of the group
-    uint64_t *bars = (uint64_t *)(Bs_all + (size_t)DEC_WARPS * 2 * nq * BST);   // [warps][8]: 4 chunk slots, 2 parameter slots
-    unsigned char *ring_all = smem_raw + Plan::fixed_bytes(nq);      // [warps][WARP_RING]; later reused for the partials
-    float *part = (float *)ring_all;                                 // [2*warps][nq][D+2]
-
-    // launched with programmatic stream serialization: everything above overlaps the tail of the kernel before this
-    // one in the stream; nothing it may have written (the query, the cache) is read before this point
-    asm volatile("griddepcontrol.wait;" ::: "memory");
-    for (int i = tid; i < 8 * D; i += DEC_THREADS) {
-        const int qh = i / D, ch = i % D;
-        __half v = qh < nq ? q[((size_t)b * p.Hq + hq0 + qh) * D + ch] : __float2half(0.f);
-        q16[i] = v;
-        qs[i] = __half2float(v) * qscale;
-    }
-    uint64_t *cbar = bars + warp * 8, *pbar = cbar + 4;              // chunk and parameter full-barriers of this warp
-    if (lane == 0) {
-        for (int i = 0; i < 6; ++i) mbar_init(&cbar[i], 1);
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    }
-    __syncthreads();
-
-    constexpr int PS = D + 2;                                        // partial record: o[D], m, l
-
-    // Sink rows of the side buffer are shared out over all warps of all splits and handled after the stream; the
-    // first row of this warp is fetched now, so that its latency hides behind the stream.
-    const int sink_n = min(c.sink_count[b], p.cap);
-    const int sink_worker = split * DEC_WARPS + warp, sink_workers = nsplit * DEC_WARPS;
-    int sink_pos_next = -1;
-    uint32_t sink_k_next[CPL / 2], sink_v_next[CPL / 2];
-    auto fetch_sink = [&](int j) {
-        sink_pos_next = -1;
-#pragma unroll
-        for (int e = 0; e < CPL / 2; ++e) sink_k_next[e] = sink_v_next[e] = 0u;
-        if (j < sink_n) {
-            sink_pos_next = c.sink_pos[(size_t)b * p.cap + j];
-            const uint32_t *kr = (const uint32_t *)((const __half *)c.sink_k + ((size_t)unit * p.cap + j) * D + lane * CPL);
-            const uint32_t *vr = (const uint32_t *)((const __half *)c.sink_v + ((size_t)unit * p.cap + j) * D + lane * CPL);
-#pragma unroll
-            for (int e = 0; e < CPL / 2; ++e) { sink_k_next[e] = kr[e]; sink_v_next[e] = vr[e]; }
-        }
-    };
-    fetch_sink(sink_worker);
-
-    // ---------------- packed stream ----------------
-    float m0 = M_INIT, m1 = M_INIT, l0 = 0.f, l1 = 0.f;             // running max / sum of query heads 2t and 2t+1
-    float O[NM][4];
-    float bv[NGv][2];                     // sum p*scale*zero per value channel group and head
-    int ev = 60;                          // the value B operand is p * scale * 2^ev; lowered so that it fits fp16
-    float evf = pow2i(60);
-#pragma unroll
-    for (int m = 0; m < NM; ++m)
-#pragma unroll
-        for (int i = 0; i < 4; ++i) O[m][i] = 0.f;
-#pragma unroll
-    for (int j = 0; j < NGv; ++j) bv[j][0] = bv[j][1] = 0.f;
-
-    __half *Bs = Bs_all + (size_t)warp * 2 * nq * BST, *Bl = Bs + (size_t)nq * BST;
-    const uint8_t *kc_base = c.k_codes + (size_t)unit * p.max_seq * p.row_bytes;
-    const uint8_t *vc_base = c.v_codes + (size_t)unit * p.max_seq * p.row_bytes;
-    const float *vs_base = c.v_scale + (size_t)unit * p.max_seq * NGv;
-    const float *vz_base = c.v_zero + (size_t)unit * p.max_seq * NGv;
-    const float *ks_base = c.k_scale + (size_t)unit * (p.max_seq / G) * D;
-    const float *kz_base = c.k_zero + (size_t)unit * (p.max_seq / G) * D;
-
-    // Lowers ev so that p * scale * 2^ev stays below 2^13 for the largest |scale| mx any lane has seen.
-    // ev_limit = 2^(13 - ev): scales below it need no action, which is the common case and costs one vote.
-    float ev_limit = 0.f;
-    auto fit_value_scale = [&](float mx) {
-        if (!__any_sync(0xffffffffu, mx >= ev_limit)) return;
-        mx = warp_max(mx);
-        int need = 12 - floor_log2(mx);
-        need = need > 60 ? 60 : (need < -60 ? -60 : need);
-        if (need < ev) {     // warp-uniform: every quad column holds the same tokens
-            const float f = pow2i(need - ev);
-#pragma unroll
-            for (int m = 0; m < NM; ++m)
-#pragma unroll
-                for (int i = 0; i < 4; ++i) O[m][i] *= f;
-            ev = need;
-            evf = pow2i(ev);
-            ev_limit = pow2i(13 - ev);
-        }
-    };
-    // New running maxima after a batch of scores with per-lane maxima tm0 / tm1; rescales the accumulators if needed.
-    // Once the running maxima have settled no lane exceeds them and the step costs one vote.
-    auto advance_max = [&](float tm0, float tm1) {
-        if (PL) tm1 = M_INIT;
-        if (!__any_sync(0xffffffffu, tm0 > m0 || tm1 > m1)) return;
-#pragma unroll
-        for (int o = 4; o < 32; o <<= 1) {
-            tm0 = fmaxf(tm0, __shfl_xor_sync(0xffffffffu, tm0, o));
-            tm1 = fmaxf(tm1, __shfl_xor_sync(0xffffffffu, tm1, o));
-        }
-        const float mn0 = fmaxf(m0, tm0), mn1 = fmaxf(m1, tm1);
-        const float c0 = ex2(m0 - mn0), c1 = ex2(m1 - mn1);
-        l0 *= c0; l1 *= c1;
-#pragma unroll
-        for (int j = 0; j < NGv; ++j) { bv[j][0] *= c0; bv[j][1] *= c1; }
-#pragma unroll
-        for (int m = 0; m < NM; ++m) { O[m][0] *= c0; O[m][2] *= c0; O[m][1] *= PL ? c0 : c1; O[m][3] *= PL ? c0 : c1; }
-        m0 = mn0; m1 = mn1;
-    };
-    // Value products of one tile: scores s (log2 units, relative maxima already advanced), value words vw, and the
-    // (scale, zero) of tokens g (sv0, zv0) and g+8 (sv1, zv1) per channel group.
-    auto tile_values = [&](const float (&s)[4], const uint32_t (&vw)[W], const float (&sv0)[NGv], const float (&zv0)[NGv],
-                           const float (&sv1)[NGv], const float (&zv1)[NGv]) {
-        const float p0 = ex2(s[0] - m0), p1 = PL ? 0.f : ex2(s[1] - m1), p2 = ex2(s[2] - m0), p3 = PL ? 0.f : ex2(s[3] - m1);
-        l0 += p0 + p2;
-        if (!PL) l1 += p1 + p3;
-        uint32_t va[NM][4];
-        tile_frags<BITS, D>(vw, va);
-        const float evc = evf * C1;
-#pragma unroll
-        for (int j = 0; j < NGv; ++j) {
-            const float e0 = sv0[j] * evf, e1 = sv1[j] * evc, sz0 = sv0[j] * zv0[j], sz1 = sv1[j] * zv1[j];
-            bv[j][0] = fmaf(p0, sz0, fmaf(p2, sz1, bv[j][0]));
-            if (!PL) bv[j][1] = fmaf(p1, sz0, fmaf(p3, sz1, bv[j][1]));
-            uint32_t b0, b1;
-            if constexpr (PL) {
-                // the odd columns carry the fp16 rounding residual of the weight p * scale: the outputs keep the weight
-                // to ~22 bits (columns 2h and 2h+1 are added at the end)
-                const float x0 = p0 * e0, x1 = p2 * e1;
-                const float r0 = x0 - __half2float(__float2half_rn(x0)), r1 = x1 - __half2float(__float2half_rn(x1));
-                b0 = movm_trans(pack_half2(x0, r0));
-                b1 = movm_trans(pack_half2(x1, r1));
-            } else {
-                b0 = movm_trans(pack_half2(p0 * e0, p1 * e0));
-                b1 = movm_trans(pack_half2(p2 * e1, p3 * e1));
-            }
-#pragma unroll
-            for (int mi = 0; mi < mpg; ++mi) mma16816(O[j * mpg + mi], va[j * mpg + mi], b0, b1);
-        }
-    };
-
-    // ---- complete key groups of this split: warp w takes groups g_begin + w, + DEC_WARPS, ...  Its chunks (CT tiles
-    //      each) arrive through a ring of NSLOT bulk-copy slots filled NSLOT - 1 chunks ahead by lane 0; the key
-    //      parameters of a group arrive one group ahead through two more slots. ----
-    const int g_begin = split * groups_per_split, g_end = min(n_groups, g_begin + groups_per_split);
-    const int my_groups = g_begin + warp < g_end ? (g_end - g_begin - warp + DEC_WARPS - 1) / DEC_WARPS : 0;
-    unsigned char *ring = ring_all + (size_t)warp * Plan::WARP_RING;
-    float *kp_ring = (float *)(ring + NSLOT * SLOT_BYTES);           // [scale D | zero D] of the next group to prepare
-    int iss_g = 0, iss_c = 0;                                        // next chunk to issue: group index, chunk within group
-    // Every lane keeps the issue bookkeeping (so that addresses and counters stay warp-uniform values); lane 0 alone
-    // issues the copies.
-    auto issue_chunk = [&](int slot) {
-        const int T0 = (g_begin + warp + iss_g * DEC_WARPS) * TPG + iss_c * CT;
-        unsigned char *dst = ring + slot * SLOT_BYTES;
-        if (lane == 0) {
-            mbar_expect_tx(&cbar[slot], SLOT_BYTES);
-            bulk_g2s(dst, kc_base + (size_t)T0 * Plan::TILE_BYTES, KV_BYTES, &cbar[slot]);
-            bulk_g2s(dst + KV_BYTES, vc_base + (size_t)T0 * Plan::TILE_BYTES, KV_BYTES, &cbar[slot]);
-            bulk_g2s(dst + 2 * KV_BYTES, vs_base + (size_t)T0 * 16 * NGv, SZ_BYTES, &cbar[slot]);
-            bulk_g2s(dst + 2 * KV_BYTES + SZ_BYTES, vz_base + (size_t)T0 * 16 * NGv, SZ_BYTES, &cbar[slot]);
-        }
-        if (++iss_c == CPG) { iss_c = 0; ++iss_g; }
-    };
-    auto issue_params = [&](int gi) {
-        const int grp = g_begin + warp + gi * DEC_WARPS;
-        if (lane == 0) {
-            mbar_expect_tx(&pbar[0], Plan::KP_BYTES);
-            bulk_g2s(kp_ring, ks_base + (size_t)grp * D, D * 4, &pbar[0]);
-            bulk_g2s(kp_ring + D, kz_base + (size_t)grp * D, D * 4, &pbar[0]);
-        }
-    };
-    auto wait_bar = [&](uint64_t *bar, unsigned parity) {
-        int polls = 0;
-        bool ok = true;
-        while (!mbar_try_wait(bar, parity)) {
-            if (++polls > DEC_WAIT_LIMIT) { ok = false; break; }
-        }
-        return __all_sync(0xffffffffu, ok);
-    };
-    if (my_groups > 0) {
-        issue_params(0);
-        for (int i = 0; i < NSLOT - 1 && iss_g < my_groups; ++i) issue_chunk(i);
-    }
-    // sink bits of the CT tiles starting at tile T: one 32-bit word covers two tiles
-    auto load_mask_words = [&](int T) {
-        uint2 w;
-        w.x = __ldg(bm + (T >> 1));
-        w.y = CT == 4 ? __ldg(bm + (T >> 1) + 1) : 0u;
-        return w;
-    };
-    uint2 mword_next = my_groups > 0 ? load_mask_words((g_begin + warp) * TPG) : make_uint2(0u, 0u);
-    bool stream_ok = true;
-    int ci = 0;                                                      // running chunk index of this warp
-
-#pragma unroll 1
-    for (int gi = 0; gi < my_groups && stream_ok; ++gi) {
-        const int grp = g_begin + warp + gi * DEC_WARPS;
-        // ---- B operand of the group: fp16(q * scale * 2^sh) per channel and head (sh puts the largest factor of the
-        //      head in [2^13, 2^14)), column half pre-divided by COLF; bias = sum_c of the same rounded factors * zero ----
-        float bias0 = 0.f, bias1 = 0.f, ks0 = 0.f, ks1 = 0.f;
-        uint32_t need_lo = 0;     // bit m: matrix m also gets the low half of the split factor (warp-uniform)
-        {
-            if (!wait_bar(&pbar[0], (unsigned)gi & 1u)) { stream_ok = false; break; }
-            const float *kp = kp_ring;
-            float scv[CPL], zev[CPL];
-#pragma unroll
-            for (int e = 0; e < CPL; ++e) { scv[e] = kp[lane * CPL + e]; zev[e] = kp[D + lane * CPL + e]; }
-            __syncwarp();   // the parameters are in registers: the slot can take the next group's while this one streams
-            if (gi + 1 < my_groups) issue_params(gi + 1);
-            if constexpr (I8) {
-                // limbs of the one head's factors: f = q * scale * 2^sh with the largest |f| in [2^26, 2^27), four signed
-                // 7-bit limbs each: every factor is kept to 2^-27 of the group's largest one (2^-23 where the factor is
-                // pre-divided for the upper contraction slots), finer than binary32 keeps the factor itself
-                float v[CPL], amax = 0.f;
-#pragma unroll
-                for (int e = 0; e < CPL; ++e) { v[e] = qs[lane * CPL + e] * scv[e]; amax = fmaxf(amax, fabsf(v[e])); }
-                amax = warp_max(amax);
-                int sh = 26 - floor_log2(amax);
-                sh = sh > 60 ? 60 : (sh < -60 ? -60 : sh);
-                const bool upper = BITS != 4 && ((lane * CPL) & 8) != 0;   // 2, 3 bit: channels in the upper contraction slots (x16 in place)
-                const float pre = upper ? pow2i(sh - 4) : pow2i(sh);
-                const int mtx = (lane * CPL) >> 4, colbase = (lane * CPL) & 15;
-                // table [MMA][lower / upper slots][limb][t][byte]; 2 bit: MMA = word = matrix pair, upper = column half;
-                // 4 bit: MMA = matrix pair, upper = odd matrix
-                signed char *tab = reinterpret_cast<signed char *>(Bs) + ((mtx >> 1) * 2 + (BITS != 4 ? (colbase >> 3) : (mtx & 1))) * 64;
-                float bsum = 0.f;
-#pragma unroll
-                for (int e = 0; e < CPL; ++e) {
-                    const float fp = v[e] * pre;
-                    const float l0 = rintf(fp * (1.f / 2097152.f)), r1 = fmaf(-l0, 2097152.f, fp);
-                    const float l1 = rintf(r1 * (1.f / 16384.f)), r2 = fmaf(-l1, 16384.f, r1);
-                    const float l2 = rintf(r2 * (1.f / 128.f)), l3 = rintf(fmaf(-l2, 128.f, r2));
-                    // the zero-point term takes the unrounded factor: the limbs' rounding then meets the codes (at most
-                    // qmax) only, not code - zero, which is large for a channel far from zero with a narrow range
-                    bsum = fmaf(upper ? fp * 16.f : fp, zev[e], bsum);
-                    const int col = colbase + e;
-                    const int at = ((col & 7) >> 1) * 4 + (BITS != 4 ? (mtx & 1) + 2 * (col & 1) : 2 * (col & 1) + (col >> 3));
-                    tab[at] = (signed char)(int)l0;
-                    tab[16 + at] = (signed char)(int)l1;
-                    tab[32 + at] = (signed char)(int)l2;
-                    tab[48 + at] = (signed char)(int)l3;
-                }
-                bsum = warp_sum(bsum) * pow2i(-sh);
-                if (t == 0) { bias0 = bsum; ks0 = pow2i(-sh); }
-            } else {
-            // one power-of-two scaling for all heads of the group: the largest factor lands in [2^13, 2^14)
-            constexpr int NQL = PL ? 4 : 8;
-            float amax = 0.f;
-#pragma unroll
-            for (int i = 0; i < NQL; ++i)
-                if (i < nq) {
-#pragma unroll
-                    for (int e = 0; e < CPL; ++e) amax = fmaxf(amax, fabsf(qs[i * D + lane * CPL + e] * scv[e]));
-                }
-            amax = warp_max(amax);
-            int sh = 13 - floor_log2(amax);
-            sh = sh > 60 ? 60 : (sh < -60 ? -60 : sh);
-            const float f = pow2i(sh), finv = pow2i(-sh), ksc = pow2i(24 - sh);
-            const bool scaled_col = ((lane * CPL) & 8) && G_::COLF != 1.f;   // this lane's channels sit in the column half
-            const __half2 colf = __half2half2(__float2half(scaled_col ? C1 : 1.f));
-            bool big = false;
-#pragma unroll
-            for (int i = 0; i < NQL; ++i) {
-                if (i < nq) {
-                    float bsum = 0.f;
-                    __half2 hb[CPL / 2], lb[CPL / 2];
-#pragma unroll
-                    for (int e = 0; e < CPL; e += 2) {
-                        const float v0 = qs[i * D + lane * CPL + e] * scv[e], v1 = qs[i * D + lane * CPL + e + 1] * scv[e + 1];
-                        const float f0 = v0 * f, f1 = v1 * f;
-                        // fp16 keeps 11 bits of a factor; its rounding residual is kept as a second factor (always with PL,
-                        // else where it could move a score by more than ~4e-4: factor * largest |code - zero| * 2^-12)
-                        const __half2 h = __floats2half2_rn(f0, f1);
-                        const float2 hf = __half22float2(h);
-                        const __half2 l = __floats2half2_rn(f0 - hf.x, f1 - hf.y);
-                        const float2 lf = __half22float2(l);
-                        bsum += (hf.x + lf.x) * zev[e] + (hf.y + lf.y) * zev[e + 1];
-                        if (!PL)
-                            big |= fabsf(v0) * fmaxf(fabsf(zev[e]), fabsf(QMAX - zev[e])) > 1.6f ||
-                                   fabsf(v1) * fmaxf(fabsf(zev[e + 1]), fabsf(QMAX - zev[e + 1])) > 1.6f;
-                        hb[e / 2] = __hmul2(h, colf);
-                        lb[e / 2] = __hmul2(l, colf);
-                    }
-                    __half *hrow = PL ? Bs + (2 * i) * BST : Bs + i * BST, *lrow = PL ? Bs + (2 * i + 1) * BST : Bl + i * BST;
-                    if constexpr (CPL == 4) {
-                        *reinterpret_cast<uint2 *>(hrow + lane * CPL) = make_uint2(*reinterpret_cast<uint32_t *>(&hb[0]), *reinterpret_cast<uint32_t *>(&hb[1]));
-                        *reinterpret_cast<uint2 *>(lrow + lane * CPL) = make_uint2(*reinterpret_cast<uint32_t *>(&lb[0]), *reinterpret_cast<uint32_t *>(&lb[1]));
-                    } else {
-                        *reinterpret_cast<__half2 *>(hrow + lane * CPL) = hb[0];
-                        *reinterpret_cast<__half2 *>(lrow + lane * CPL) = lb[0];
-                    }
-                    bsum = warp_sum(bsum) * finv;
-                    if (PL) {
-                        if (i == t) { bias0 = bsum; ks0 = ksc; }
-                    } else {
-                        if (i == 2 * t) { bias0 = bsum; ks0 = ksc; }
-                        if (i == 2 * t + 1) { bias1 = bsum; ks1 = ksc; }
-                    }
-                }
-            }
-            if (!PL) {
-                const uint32_t bal = __ballot_sync(0xffffffffu, big);
-                constexpr int LPM = 16 / CPL;     // lanes per 16-channel matrix
-#pragma unroll
-                for (int m = 0; m < NM; ++m)
-                    if ((bal >> (LPM * m)) & ((1u << LPM) - 1u)) need_lo |= 1u << m;
-            }
-            }
-            __syncwarp();
-        }
-        uint32_t bk[NM][2];
-        if constexpr (I8) {
-            // B fragments of the four words: column g = limb g, contraction slots 4t .. 4t + 3 (lower, upper)
-#pragma unroll
-            for (int m = 0; m < NM; ++m) bk[m][0] = bk[m][1] = 0u;
-#pragma unroll
-            for (int i = 0; i < 4; ++i)
-#pragma unroll
-                for (int c2 = 0; c2 < 2; ++c2)
-                    bk[i][c2] = g < 4 ? *reinterpret_cast<const uint32_t *>(reinterpret_cast<const signed char *>(Bs) + (i * 2 + c2) * 64 + g * 16 + 4 * t) : 0u;
-        } else {
-#pragma unroll
-        for (int m = 0; m < NM; ++m) {
-            const bool col_used = PL ? g < 2 * nq : g < nq;
-            bk[m][0] = col_used ? *(const uint32_t *)(Bs + g * BST + 16 * m + 2 * t) : 0u;
-            bk[m][1] = col_used ? *(const uint32_t *)(Bs + g * BST + 16 * m + 2 * t + 8) : 0u;
-        }
-        }
-        const float ks0r = ks0 * R1, ks1r = ks1 * R1;
-
-#pragma unroll 1
-        for (int cj = 0; cj < CPG; ++cj, ++ci) {
-            const int slot = ci & (NSLOT - 1);
-            // refill the slot freed by the previous chunk, then wait for this chunk's bytes
-            __syncwarp();
-            if (iss_g < my_groups) issue_chunk((ci + NSLOT - 1) & (NSLOT - 1));
-            if (!wait_bar(&cbar[slot], (unsigned)(ci / NSLOT) & 1u)) { stream_ok = false; break; }
-            const uint2 mwords = mword_next;
-            {   // sink bits of the warp's next chunk, fetched one chunk ahead
-                const bool last = cj + 1 == CPG;
-                const int Tn = last ? (grp + DEC_WARPS) * TPG : grp * TPG + (cj + 1) * CT;
-                if (!last || gi + 1 < my_groups) mword_next = load_mask_words(Tn);
-            }
-            const uint32_t *kt0 = (const uint32_t *)(ring + slot * SLOT_BYTES), *vt0 = kt0 + KV_BYTES / 4;
-            const float *ssv0 = (const float *)(vt0 + KV_BYTES / 4), *szv0 = ssv0 + SZ_BYTES / 4;
-#pragma unroll
-            for (int sub = 0; sub < CT / ST; ++sub) {   // softmax steps of ST tiles inside the chunk
-            const uint32_t *kt = kt0 + sub * ST * TILE_WORDS, *vt = vt0 + sub * ST * TILE_WORDS;
-            const float *ssv = ssv0 + sub * ST * 16 * NGv, *szv = szv0 + sub * ST * 16 * NGv;
-            const int T0 = grp * TPG + cj * CT + sub * ST;
-            const uint32_t mword = ST == 4 ? (mwords.x | mwords.y) : (sub == 0 ? mwords.x : mwords.y);
-
-            // scores of the chunk's tiles
-            float s[ST][4];
-#pragma unroll
-            for (int k = 0; k < ST; ++k) {
-                if constexpr (I8) {
-                    uint32_t kw[W];
-                    load_tile_shared<BITS, D>(kt + k * TILE_WORDS, lane, kw);
-                    int ia[4] = {0, 0, 0, 0};
-                    int ih0[4] = {0, 0, 0, 0}, ih1[4] = {0, 0, 0, 0};   // 3 bit: the high bits of the even / odd words
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        uint32_t a0, a1, a2, a3;
-                        if constexpr (BITS == 3) {
-                            // the second section has the byte structure of the first: the high bits of word i sit at bits
-                            // 2, 3, 6, 7 (even i) or 0, 1, 4, 5 (odd i) of the bytes of word 4 + i / 2
-                            const uint32_t hw = kw[4 + (i >> 1)];
-                            if ((i & 1) == 0) {
-                                asm volatile("mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-                                             : "+r"(ih0[0]), "+r"(ih0[1]), "+r"(ih0[2]), "+r"(ih0[3])
-                                             : "r"(hw & 0x04040404u), "r"(hw & 0x08080808u), "r"(hw & 0x40404040u), "r"(hw & 0x80808080u), "r"(bk[i][0]), "r"(bk[i][1]));
-                            } else {
-                                asm volatile("mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-                                             : "+r"(ih1[0]), "+r"(ih1[1]), "+r"(ih1[2]), "+r"(ih1[3])
-                                             : "r"(hw & 0x01010101u), "r"(hw & 0x02020202u), "r"(hw & 0x10101010u), "r"(hw & 0x20202020u), "r"(bk[i][0]), "r"(bk[i][1]));
-                            }
-                        }
-                        if constexpr (BITS != 4) {
-                            const uint32_t x = kw[i];
-                            a0 = x & 0x03030303u; a1 = x & 0x0c0c0c0cu; a2 = x & 0x30303030u; a3 = x & 0xc0c0c0c0u;
-                        } else {
-                            const uint32_t x = kw[2 * i], y = kw[2 * i + 1];
-                            a0 = x & 0x0f0f0f0fu; a1 = x & 0xf0f0f0f0u; a2 = y & 0x0f0f0f0fu; a3 = y & 0xf0f0f0f0u;
-                        }
-                        asm volatile("mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-                                     : "+r"(ia[0]), "+r"(ia[1]), "+r"(ia[2]), "+r"(ia[3])
-                                     : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(bk[i][0]), "r"(bk[i][1]));
-                    }
-                    if constexpr (BITS == 3) {
-                        // code = low + 4 * high; in place the high bits weigh 4, 8 (rows g, g + 8) in even words and 1, 2 in
-                        // odd ones, the low fields 1, 4: rows g in units of 1, rows g + 8 in units of 4
-                        ia[0] += ih0[0] + 4 * ih1[0]; ia[1] += ih0[1] + 4 * ih1[1];
-                        ia[2] += 2 * ih0[2] + 8 * ih1[2]; ia[3] += 2 * ih0[3] + 8 * ih1[3];
-                    }
-                    // lane t = 0 holds limbs 0, 1 (columns 0, 1), its neighbour limbs 2, 3 (columns 2, 3): each lane combines
-                    // its pair in int32 (below 2^31 for every code width), then one conversion per pair
-                    const int xg = ia[0] * 128 + ia[1], xh = ia[2] * 128 + ia[3];
-                    const int yg = __shfl_down_sync(0xffffffffu, xg, 1), yh = __shfl_down_sync(0xffffffffu, xh, 1);
-                    const float tg = fmaf((float)xg, 16384.f, (float)yg);
-                    const float th = fmaf((float)xh, 16384.f, (float)yh);
-                    s[k][0] = t == 0 ? fmaf(tg, ks0, -bias0) : -INFINITY; s[k][1] = -INFINITY;
-                    s[k][2] = t == 0 ? fmaf(th, ks0 * (BITS == 4 ? 0.0625f : 0.25f), -bias0) : -INFINITY; s[k][3] = -INFINITY;
-                    continue;
-                }
-                uint32_t kw[W], ka[NM][4];
-                load_tile_shared<BITS, D>(kt + k * TILE_WORDS, lane, kw);
-                tile_frags<BITS, D>(kw, ka);
-                float acc[4] = {0.f, 0.f, 0.f, 0.f};
-                if (PL || need_lo == 0) {
-#pragma unroll
-                    for (int m = 0; m < NM; ++m) mma16816(acc, ka[m], bk[m][0], bk[m][1]);
-                } else {
-#pragma unroll
-                    for (int m = 0; m < NM; ++m) {
-                        mma16816(acc, ka[m], bk[m][0], bk[m][1]);
-                        if (need_lo & (1u << m)) {
-                            const uint32_t h0 = g < nq ? *(const uint32_t *)(Bl + g * BST + 16 * m + 2 * t) : 0u;
-                            const uint32_t h1 = g < nq ? *(const uint32_t *)(Bl + g * BST + 16 * m + 2 * t + 8) : 0u;
-                            mma16816(acc, ka[m], h0, h1);
-                        }
-                    }
-                }
-                if (PL) {   // column 2t: rounded factors, column 2t+1: their residuals
-                    s[k][0] = fmaf(acc[0] + acc[1], ks0, -bias0); s[k][1] = -INFINITY;
-                    s[k][2] = fmaf(acc[2] + acc[3], ks0r, -bias0); s[k][3] = -INFINITY;
-                } else {
-                    s[k][0] = fmaf(acc[0], ks0, -bias0); s[k][1] = fmaf(acc[1], ks1, -bias1);
-                    s[k][2] = fmaf(acc[2], ks0r, -bias0); s[k][3] = fmaf(acc[3], ks1r, -bias1);
-                }
-            }
-            if (mword) {   // sink tokens are not part of the packed stream (their value parameters are zero)
-#pragma unroll
-                for (int k = 0; k < ST; ++k) {
-                    const uint32_t mask16 = ((ST == 4 ? (k < 2 ? mwords.x : mwords.y) : mword) >> (16 * ((T0 + k) & 1))) & 0xffffu;
-                    if ((mask16 >> g) & 1u) s[k][0] = s[k][1] = -INFINITY;
-                    if ((mask16 >> (g + 8)) & 1u) s[k][2] = s[k][3] = -INFINITY;
-                }
-            }
-            // one softmax step for the whole chunk
-            {
-                float tm0 = fmaxf(s[0][0], s[0][2]), tm1 = fmaxf(s[0][1], s[0][3]);
-#pragma unroll
-                for (int k = 1; k < ST; ++k) { tm0 = fmaxf(tm0, fmaxf(s[k][0], s[k][2])); tm1 = fmaxf(tm1, fmaxf(s[k][1], s[k][3])); }
-                advance_max(tm0, tm1);
-            }
-            // value scales of this lane's tokens; their maximum bounds the fp16 range needed
-            float sv0[ST][NGv], zv0[ST][NGv], sv1[ST][NGv], zv1[ST][NGv];
-            {
-                float mx = 0.f;
-#pragma unroll
-                for (int k = 0; k < ST; ++k)
-#pragma unroll
-                    for (int j = 0; j < NGv; ++j) {
-                        sv0[k][j] = ssv[(k * 16 + g) * NGv + j]; zv0[k][j] = szv[(k * 16 + g) * NGv + j];
-                        sv1[k][j] = ssv[(k * 16 + g + 8) * NGv + j]; zv1[k][j] = szv[(k * 16 + g + 8) * NGv + j];
-                        mx = fmaxf(mx, fmaxf(fabsf(sv0[k][j]), fabsf(sv1[k][j])));
-                    }
-                fit_value_scale(mx);
-            }
-#pragma unroll
-            for (int k = 0; k < ST; ++k) {
-                uint32_t vw[W];
-                load_tile_shared<BITS, D>(vt + k * TILE_WORDS, lane, vw);
-                tile_values(s[k], vw, sv0[k], zv0[k], sv1[k], zv1[k]);
-            }
-            }
-        }
-    }
-    if (!stream_ok && lane == 0) atomicOr(c.status, KVSINK_STATUS_TIMEOUT);
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the merge kernel may be scheduled; it waits for this grid's end
-
-    // ---- tokens of the open group: keys from the fp16 tail (last split only) ----
-    if (split == nsplit - 1) {
-        const __half *tail = (const __half *)c.k_tail + (size_t)unit * G * D;
-        const int T_begin = n_body / KVSINK_TILE, T_end = (n + KVSINK_TILE - 1) / KVSINK_TILE;
-        for (int T = T_begin + warp; T < T_end; T += DEC_WARPS) {
-            const int tok0 = T * KVSINK_TILE + g, tok1 = tok0 + 8;
-            const bool in0 = tok0 < n, in1 = tok1 < n;
-            const __half *r0 = tail + (size_t)(tok0 % G) * D, *r1 = tail + (size_t)(tok1 % G) * D;
-            float acc[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-            for (int m = 0; m < NM; ++m) {
-                uint32_t a[4];
-                a[0] = in0 ? *(const uint32_t *)(r0 + 16 * m + 2 * t) : 0u;
-                a[1] = in1 ? *(const uint32_t *)(r1 + 16 * m + 2 * t) : 0u;
-                a[2] = in0 ? *(const uint32_t *)(r0 + 16 * m + 2 * t + 8) : 0u;
-                a[3] = in1 ? *(const uint32_t *)(r1 + 16 * m + 2 * t + 8) : 0u;
-                const int qrow = PL ? (g >> 1) : g;          // query head in accumulator column g
-                const bool qcol = PL ? !(g & 1) : true;
-                const uint32_t b0 = qcol ? *(const uint32_t *)(q16 + qrow * D + 16 * m + 2 * t) : 0u;
-                const uint32_t b1 = qcol ? *(const uint32_t *)(q16 + qrow * D + 16 * m + 2 * t + 8) : 0u;
-                mma16816(acc, a, b0, b1);
-            }
-            const bool v0 = in0 && !mask_bit(bm, in0 ? tok0 : 0), v1 = in1 && !mask_bit(bm, in1 ? tok1 : 0);
-            float s[4];
-            s[0] = v0 ? acc[0] * qscale : -INFINITY; s[1] = (v0 && !PL) ? acc[1] * qscale : -INFINITY;
-            s[2] = v1 ? acc[2] * qscale : -INFINITY; s[3] = (v1 && !PL) ? acc[3] * qscale : -INFINITY;
-            advance_max(fmaxf(s[0], s[2]), fmaxf(s[1], s[3]));
-            uint32_t vw[W];
-            load_tile<BITS, D>((const uint32_t *)(vc_base + (size_t)T * p.tile_bytes), lane, vw);
-            float sv0[NGv], zv0[NGv], sv1[NGv], zv1[NGv];
-            float mx = 0.f;
-#pragma unroll
-            for (int j = 0; j < NGv; ++j) {   // tokens beyond the sequence have no parameters yet
-                sv0[j] = v0 ? __ldg(vs_base + (size_t)tok0 * NGv + j) : 0.f; zv0[j] = v0 ? __ldg(vz_base + (size_t)tok0 * NGv + j) : 0.f;
-                sv1[j] = v1 ? __ldg(vs_base + (size_t)tok1 * NGv + j) : 0.f; zv1[j] = v1 ? __ldg(vz_base + (size_t)tok1 * NGv + j) : 0.f;
-                mx = fmaxf(mx, fmaxf(fabsf(sv0[j]), fabsf(sv1[j])));
-            }
-            fit_value_scale(mx);
-            tile_values(s, vw, sv0, zv0, sv1, zv1);
-        }
-    }
-
-    // ---- this warp's packed partial: finish the reductions over the token lanes, convert units ----
-#pragma unroll
-    for (int o = 4; o < 32; o <<= 1) {
-        l0 += __shfl_xor_sync(0xffffffffu, l0, o);
-        l1 += __shfl_xor_sync(0xffffffffu, l1, o);
-#pragma unroll
-        for (int j = 0; j < NGv; ++j) {
-            bv[j][0] += __shfl_xor_sync(0xffffffffu, bv[j][0], o);
-            bv[j][1] += __shfl_xor_sync(0xffffffffu, bv[j][1], o);
-        }
-    }
-    __syncthreads();   // every warp has drained its ring: the space now holds the block's partials
-    float *my_part = part + (size_t)(2 * warp) * nq * PS;
-    {
-        const float OS0 = pow2i(24 - ev), OS1 = OS0 * R1;
-#pragma unroll
-        for (int m = 0; m < NM; ++m) {
-            const float bj0 = bv[m / mpg][0], bj1 = bv[m / mpg][1];
-            const int ch0 = 16 * m + g, ch1 = ch0 + 8;
-            if (PL) {
-                if (t < nq) {
-                    my_part[t * PS + ch0] = (O[m][0] + O[m][1]) * OS0 - bj0;
-                    my_part[t * PS + ch1] = (O[m][2] + O[m][3]) * OS1 - bj0;
-                }
-                continue;
-            }
-            if (2 * t < nq) {
-                my_part[(2 * t) * PS + ch0] = O[m][0] * OS0 - bj0;
-                my_part[(2 * t) * PS + ch1] = O[m][2] * OS1 - bj0;
-            }
-            if (2 * t + 1 < nq) {
-                my_part[(2 * t + 1) * PS + ch0] = O[m][1] * OS0 - bj1;
-                my_part[(2 * t + 1) * PS + ch1] = O[m][3] * OS1 - bj1;
-            }
-        }
-        if (g == 0 && PL) {
-            if (t < nq) { my_part[t * PS + D] = m0; my_part[t * PS + D + 1] = l0; }
-        } else if (g == 0) {
-            if (2 * t < nq) { my_part[(2 * t) * PS + D] = m0; my_part[(2 * t) * PS + D + 1] = l0; }
-            if (2 * t + 1 < nq) { my_part[(2 * t + 1) * PS + D] = m1; my_part[(2 * t + 1) * PS + D + 1] = l1; }
-        }
-    }
-
-    // ---------------- sink rows (fp16 side buffer), plain fp32 arithmetic ----------------
-    {
-        float ms[8], ls[8], os[8][CPL];
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            ms[i] = M_INIT; ls[i] = 0.f;
-#pragma unroll
-            for (int e = 0; e < CPL; ++e) os[i][e] = 0.f;
-        }
-        for (int j = sink_worker; j < sink_n; j += sink_workers) {
-            const int pos = sink_pos_next;
-            float kf[CPL], vf[CPL];
-#pragma unroll
-            for (int e = 0; e < CPL / 2; ++e) {
-                const float2 k2 = __half22float2(*reinterpret_cast<const __half2 *>(&sink_k_next[e]));
-                const float2 v2 = __half22float2(*reinterpret_cast<const __half2 *>(&sink_v_next[e]));
-                kf[2 * e] = k2.x; kf[2 * e + 1] = k2.y; vf[2 * e] = v2.x; vf[2 * e + 1] = v2.y;
-            }
-            fetch_sink(j + sink_workers);   // the next row streams in while this one is used
-            if (pos < 0 || pos >= n) continue;
-#pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                if (i < nq) {
-                    float d = 0.f;
-#pragma unroll
-                    for (int e = 0; e < CPL; ++e) d += qs[i * D + lane * CPL + e] * kf[e];
-                    const float sc = warp_sum(d);
-                    const float mnew = fmaxf(ms[i], sc);
-                    const float corr = ex2(ms[i] - mnew), pp = ex2(sc - mnew);
-                    ls[i] = ls[i] * corr + pp;
-#pragma unroll
-                    for (int e = 0; e < CPL; ++e) os[i][e] = os[i][e] * corr + pp * vf[e];
-                    ms[i] = mnew;
-                }
-            }
-        }
-        float *sp = my_part + (size_t)nq * PS;
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            if (i < nq) {
-#pragma unroll
-                for (int e = 0; e < CPL; ++e) sp[i * PS + lane * CPL + e] = os[i][e];
-                if (lane == 0) { sp[i * PS + D] = ms[i]; sp[i * PS + D + 1] = ls[i]; }
-            }
-        }
-    }
-    __syncthreads();
-
-    // ---- merge the block's partials; write the result or this split's partial ----
-    for (int idx = tid; idx < nq * D; idx += DEC_THREADS) {
-        const int qh = idx / D, ch = idx % D;
-        float M = M_INIT;
-        for (int w = 0; w < 2 * DEC_WARPS; ++w) M = fmaxf(M, part[((size_t)w * nq + qh) * PS + D]);
-        float acc = 0.f, L = 0.f;
-        for (int w = 0; w < 2 * DEC_WARPS; ++w) {
-            const float *pr = part + ((size_t)w * nq + qh) * PS;
-            const float f = ex2(pr[D] - M);
-            acc += pr[ch] * f;
-            L += pr[D + 1] * f;
-        }
-        const size_t oq = (size_t)b * p.Hq + hq0 + qh;
-        if (nsplit == 1) {
-            out[oq * D + ch] = L > 0.f ? acc / L : 0.f;
-            if (lse && ch == 0) lse[oq] = L > 0.f ? (M + log2f(L)) * 0.6931471805599453f : -INFINITY;
-        } else {
-            // the split's record: to the workspace for the merge kernel, or, when the splits of a unit form a thread-block
-            // cluster, to this block's shared memory (the query tables are no longer needed) for the cluster's first block
-            float *wsr = cluster_merge ? qs + (size_t)qh * PS : part_ws + (oq * nsplit + split) * PS;
-            wsr[ch] = acc;
-            if (ch == 0) { wsr[D] = M; wsr[D + 1] = L; }
-        }
-    }
-    if (cluster_merge) {
-        // the splits of a unit are the blocks of one cluster: its first block reads the records of the others through
-        // distributed shared memory and merges them in split order (the same arithmetic as the merge kernel)
-        namespace cg = cooperative_groups;
-        cg::cluster_group cluster = cg::this_cluster();
-        cluster.sync();
-        if (split == 0) {
-            for (int idx = tid; idx < nq * D; idx += DEC_THREADS) {
-                const int qh = idx / D, ch = idx % D;
-                float M = M_INIT;
-                for (int sp = 0; sp < nsplit; ++sp) M = fmaxf(M, cluster.map_shared_rank(qs, sp)[(size_t)qh * PS + D]);
-                float acc = 0.f, L = 0.f;
-                for (int sp = 0; sp < nsplit; ++sp) {
-                    const float *pr = cluster.map_shared_rank(qs, sp) + (size_t)qh * PS;
-                    const float f = ex2(pr[D] - M);
-                    acc += pr[ch] * f;
-                    L += pr[D + 1] * f;
-                }
-                const size_t oq = (size_t)b * p.Hq + hq0 + qh;
-                out[oq * D + ch] = L > 0.f ? acc / L : 0.f;
-                if (lse && ch == 0) lse[oq] = L > 0.f ? (M + log2f(L)) * 0.6931471805599453f : -INFINITY;
-            }
-        }
-        cluster.sync();   // nobody's shared memory goes away while the first block reads it
-    }
-}
 
 // Merge of the sequence splits (more than eight per unit): one block per (sequence, query head); thread (ch, sl) folds the
 // records sl, sl + MERGE_SLICES, ... of channel ch, and the slices are combined in a fixed order (bit-reproducible).
@@ -940,10 +46,26 @@ __global__ void decode_merge_kernel(const float *__restrict__ part_ws, int nspli
     if (lse && ch == 0) lse[oq] = Lt > 0.f ? (Mt + log2f(Lt)) * 0.6931471805599453f : -INFINITY;
 }
 
+int launch_decode_merge(const float *ws, int nsplit, int D, int n_rows, float *out, float *lse, cudaStream_t st)
+{
+    cudaLaunchAttribute pdl[1];
+    pdl[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    pdl[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(n_rows);
+    cfg.blockDim = dim3(D, MERGE_SLICES);
+    cfg.stream = st;
+    cfg.attrs = pdl;
+    cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, decode_merge_kernel, ws, nsplit, D, out, lse) != cudaSuccess) return KVSINK_ERR_CUDA;
+    note_launch();
+    return KVSINK_OK;
+}
+
 // ---- host side ----
 constexpr int DEC_SLOTS = 148 * 4;   // resident blocks the split heuristic plans for
 
-static int max_splits(const Params &p)
+int max_splits(const Params &p)
 {
     const int qchunks = (p.rep + 7) / 8;
     const long units = (long)p.B * p.Hkv * qchunks;
@@ -953,7 +75,7 @@ static int max_splits(const Params &p)
     return (int)(ns < 1 ? 1 : ns);
 }
 
-static int choose_splits(const Params &p, int n_groups)
+int choose_splits(const Params &p, int n_groups)
 {
     const int qchunks = (p.rep + 7) / 8;
     const long units = (long)p.B * p.Hkv * qchunks;
@@ -975,101 +97,14 @@ size_t decode_workspace_bytes(const Params &p)
     return (size_t)p.B * p.Hq * max_splits(p) * (p.D + 2) * sizeof(float) + 16;
 }
 
-template <int BITS, int D, int NGV, int CT, bool PL, bool I8 = false>
-static int launch_decode_p(const Params &p, const kvsink_cache &c, const __half *q, float *out, float *lse, float *ws, cudaStream_t st)
-{
-    const int n_groups = c.seq_len / p.G;
-    const int nsplit = choose_splits(p, n_groups);
-    const int gps = n_groups > 0 ? (n_groups + nsplit - 1) / nsplit : 0;
-    const int qchunks = (p.rep + 7) / 8;
-    const int nq_max = p.rep < 8 ? p.rep : 8;
-    const size_t smem = DecodePlan<BITS, D, NGV, CT>::bytes(nq_max);
-    auto kern = decode_kernel<BITS, D, NGV, CT, PL, I8>;
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return KVSINK_ERR_CUDA;
-    cudaLaunchAttribute pdl[2];
-    pdl[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    pdl[0].val.programmaticStreamSerializationAllowed = 1;
-    // up to eight splits (the portable cluster size): the splits of a unit are launched as one thread-block cluster and
-    // merged inside the kernel through distributed shared memory; more splits go through the workspace and the merge kernel
-    bool cluster_merge = nsplit > 1 && nsplit <= 8;
-    for (;;) {
-        cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3(nsplit, p.Hkv * qchunks, p.B);
-        cfg.blockDim = dim3(DEC_THREADS);
-        cfg.dynamicSmemBytes = smem;
-        cfg.stream = st;
-        cfg.attrs = pdl;
-        cfg.numAttrs = 1;
-        if (cluster_merge) {
-            pdl[1].id = cudaLaunchAttributeClusterDimension;
-            pdl[1].val.clusterDim.x = nsplit;
-            pdl[1].val.clusterDim.y = 1;
-            pdl[1].val.clusterDim.z = 1;
-            cfg.numAttrs = 2;
-        }
-        if (cudaLaunchKernelEx(&cfg, kern, p, c, q, out, lse, ws, nsplit, gps, qchunks, (int)c.seq_len, (int)cluster_merge) == cudaSuccess) {
-            note_launch();
-            break;
-        }
-        (void)cudaGetLastError();
-        if (!cluster_merge) return KVSINK_ERR_CUDA;
-        cluster_merge = false;   // a cluster that cannot be placed: the same launch without one, merged by the second kernel
-    }
-    if (nsplit > 1 && !cluster_merge) {
-        cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3(p.B * p.Hq);
-        cfg.blockDim = dim3(D, MERGE_SLICES);
-        cfg.stream = st;
-        cfg.attrs = pdl;
-        cfg.numAttrs = 1;
-        if (cudaLaunchKernelEx(&cfg, decode_merge_kernel, (const float *)ws, nsplit, (int)D, out, lse) != cudaSuccess) return KVSINK_ERR_CUDA;
-        note_launch();
-    }
-    return KVSINK_OK;
-}
-
-template <int BITS, int D, int NGV, int CT>
-static int launch_decode_c(const Params &p, const kvsink_cache &c, const __half *q, float *out, float *lse, float *ws, cudaStream_t st)
-{
-    if constexpr (D == 128)
-        if (p.rep == 1) return launch_decode_p<BITS, D, NGV, CT, true, true>(p, c, q, out, lse, ws, st);
-    if (p.rep <= 4) return launch_decode_p<BITS, D, NGV, CT, true>(p, c, q, out, lse, ws, st);
-    return launch_decode_p<BITS, D, NGV, CT, false>(p, c, q, out, lse, ws, st);
-}
-
-template <int BITS, int D, int NGV>
-static int launch_decode_n(const Params &p, const kvsink_cache &c, const __half *q, float *out, float *lse, float *ws, cudaStream_t st)
-{
-    // ring chunks of four tiles where a key group divides into them and two slots of that size stay below ~9 KB per
-    // warp, else of two tiles (G a multiple of 32), else of one
-    if constexpr (4 * (2 * 128 * (D * BITS / 64) + 2 * 16 * NGV * 4) <= 4800)
-        if ((p.G / KVSINK_TILE) % 4 == 0) return launch_decode_c<BITS, D, NGV, 4>(p, c, q, out, lse, ws, st);
-    if ((p.G / KVSINK_TILE) % 2 == 0) return launch_decode_c<BITS, D, NGV, 2>(p, c, q, out, lse, ws, st);
-    return launch_decode_c<BITS, D, NGV, 1>(p, c, q, out, lse, ws, st);
-}
-
-template <int BITS, int D>
-static int launch_decode_t(const Params &p, const kvsink_cache &c, const __half *q, float *out, float *lse, float *ws, cudaStream_t st)
-{
-    if (p.NGv == 1) return launch_decode_n<BITS, D, 1>(p, c, q, out, lse, ws, st);
-    if (p.NGv == 2) return launch_decode_n<BITS, D, 2>(p, c, q, out, lse, ws, st);
-    if (p.NGv == 4) return launch_decode_n<BITS, D, 4>(p, c, q, out, lse, ws, st);
-    return KVSINK_ERR_UNSUPPORTED;
-}
-
 int launch_decode(const Params &p, const kvsink_cache &c, const __half *q, float *out, float *lse, void *workspace,
                   size_t workspace_bytes, cudaStream_t st)
 {
     if (workspace_bytes < decode_workspace_bytes(p)) return KVSINK_ERR_WORKSPACE;
     float *ws = (float *)workspace;
-    if (p.D == 128) {
-        if (p.bits == 2) return launch_decode_t<2, 128>(p, c, q, out, lse, ws, st);
-        if (p.bits == 3) return launch_decode_t<3, 128>(p, c, q, out, lse, ws, st);
-        if (p.bits == 4) return launch_decode_t<4, 128>(p, c, q, out, lse, ws, st);
-    } else if (p.D == 64) {
-        if (p.bits == 2) return launch_decode_t<2, 64>(p, c, q, out, lse, ws, st);
-        if (p.bits == 4) return launch_decode_t<4, 64>(p, c, q, out, lse, ws, st);
-    }
+    if (p.bits == 2) return launch_decode_b2(p, c, q, out, lse, ws, st);
+    if (p.bits == 3) return launch_decode_b3(p, c, q, out, lse, ws, st);
+    if (p.bits == 4) return launch_decode_b4(p, c, q, out, lse, ws, st);
     return KVSINK_ERR_UNSUPPORTED;
 }
 
