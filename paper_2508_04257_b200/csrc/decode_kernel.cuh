@@ -262,6 +262,20 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
 
     constexpr int PS = D + 2;                                        // partial record: o[D], m, l
 
+    // Integer key side: lane l prepares the B operand bytes of one group of four contraction slots, (MMA l/8, lower or
+    // upper slots (l/4)%2, slots 4(l%4) ... +3); these are its four channels and their query values.
+    int i8_ch[4] = {0, 0, 0, 0};
+    float i8_q[4] = {0.f, 0.f, 0.f, 0.f};
+    if constexpr (I8) {
+        const int mi = lane >> 3, c2 = (lane >> 2) & 1, tq = lane & 3;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            i8_ch[e] = BITS != 4 ? 16 * (2 * mi + (e & 1)) + 8 * c2 + 2 * tq + (e >> 1)
+                                 : 16 * (2 * mi + c2) + 8 * (e & 1) + 2 * tq + (e >> 1);
+            i8_q[e] = qs[i8_ch[e]];
+        }
+    }
+
     // Sink rows of the side buffer are shared out over all warps of all splits and handled after the stream; the
     // first row of this warp is fetched now, so that its latency hides behind the stream.
     const int sink_n = min(c.sink_count[b], p.cap);
@@ -444,43 +458,44 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
             const float *kp = kp_ring;
             float scv[CPL], zev[CPL];
 #pragma unroll
-            for (int e = 0; e < CPL; ++e) { scv[e] = kp[lane * CPL + e]; zev[e] = kp[D + lane * CPL + e]; }
+            for (int e = 0; e < CPL; ++e) {
+                const int ch = I8 ? i8_ch[e] : lane * CPL + e;
+                scv[e] = kp[ch]; zev[e] = kp[D + ch];
+            }
             __syncwarp();   // the parameters are in registers: the slot can take the next group's while this one streams
             if (gi + 1 < my_groups) issue_params(gi + 1);
             if constexpr (I8) {
-                // limbs of the one head's factors: f = q * scale * 2^sh with the largest |f| in [2^26, 2^27), four signed
-                // 7-bit limbs each: every factor is kept to 2^-27 of the group's largest one (2^-23 where the factor is
-                // pre-divided for the upper contraction slots), finer than binary32 keeps the factor itself
-                float v[CPL], amax = 0.f;
+                // limbs of the one head's factors: F = rint(q * scale * 2^sh) with the largest |F| in [2^29, 2^30), cut into
+                // four signed bytes (radix 256): every factor is kept to 2^-30 of the group's largest one (2^-26 where the
+                // factor is pre-divided for the upper contraction slots), finer than binary32 keeps the factor itself.
+                // Adding 0x808080 propagates the carries of the signed digits and the exclusive-or removes the offset again.
+                float v[4], amax = 0.f, bsum = 0.f;
 #pragma unroll
-                for (int e = 0; e < CPL; ++e) { v[e] = qs[lane * CPL + e] * scv[e]; amax = fmaxf(amax, fabsf(v[e])); }
-                amax = warp_max(amax);
-                int sh = 26 - floor_log2(amax);
-                sh = sh > 60 ? 60 : (sh < -60 ? -60 : sh);
-                const bool upper = BITS != 4 && ((lane * CPL) & 8) != 0;   // 2, 3 bit: channels in the upper contraction slots (x16 in place)
-                const float pre = upper ? pow2i(sh - 4) : pow2i(sh);
-                const int mtx = (lane * CPL) >> 4, colbase = (lane * CPL) & 15;
-                // table [MMA][lower / upper slots][limb][t][byte]; 2 bit: MMA = word = matrix pair, upper = column half;
-                // 4 bit: MMA = matrix pair, upper = odd matrix
-                signed char *tab = reinterpret_cast<signed char *>(Bs) + ((mtx >> 1) * 2 + (BITS != 4 ? (colbase >> 3) : (mtx & 1))) * 64;
-                float bsum = 0.f;
-#pragma unroll
-                for (int e = 0; e < CPL; ++e) {
-                    const float fp = v[e] * pre;
-                    const float l0 = rintf(fp * (1.f / 2097152.f)), r1 = fmaf(-l0, 2097152.f, fp);
-                    const float l1 = rintf(r1 * (1.f / 16384.f)), r2 = fmaf(-l1, 16384.f, r1);
-                    const float l2 = rintf(r2 * (1.f / 128.f)), l3 = rintf(fmaf(-l2, 128.f, r2));
+                for (int e = 0; e < 4; ++e) {
+                    v[e] = i8_q[e] * scv[e];
+                    amax = fmaxf(amax, fabsf(v[e]));
                     // the zero-point term takes the unrounded factor: the limbs' rounding then meets the codes (at most
                     // qmax) only, not code - zero, which is large for a channel far from zero with a narrow range
-                    bsum = fmaf(upper ? fp * 16.f : fp, zev[e], bsum);
-                    const int col = colbase + e;
-                    const int at = ((col & 7) >> 1) * 4 + (BITS != 4 ? (mtx & 1) + 2 * (col & 1) : 2 * (col & 1) + (col >> 3));
-                    tab[at] = (signed char)(int)l0;
-                    tab[16 + at] = (signed char)(int)l1;
-                    tab[32 + at] = (signed char)(int)l2;
-                    tab[48 + at] = (signed char)(int)l3;
+                    bsum = fmaf(v[e], zev[e], bsum);
                 }
-                bsum = warp_sum(bsum) * pow2i(-sh);
+                amax = __uint_as_float(__reduce_max_sync(0xffffffffu, __float_as_uint(amax)));   // non-negative floats order as integers
+                int sh = 29 - floor_log2(amax);
+                sh = sh > 60 ? 60 : (sh < -60 ? -60 : sh);
+                const bool upper = BITS != 4 && (lane & 4) != 0;   // 2, 3 bit: this lane's channels sit in the upper contraction slots (x16 in place)
+                const float pre = upper ? pow2i(sh - 4) : pow2i(sh);
+                uint32_t d[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) d[e] = ((uint32_t)__float2int_rn(v[e] * pre) + 0x00808080u) ^ 0x00808080u;
+                // byte transpose: word j = byte j of the four channels, in contraction-slot order
+                const uint32_t t0 = __byte_perm(d[0], d[1], 0x5140), t1 = __byte_perm(d[0], d[1], 0x7362);
+                const uint32_t t2 = __byte_perm(d[2], d[3], 0x5140), t3 = __byte_perm(d[2], d[3], 0x7362);
+                // table [MMA][lower / upper slots][limb, most significant first][t][byte]: this lane owns one 4-byte slot group
+                uint32_t *tab = reinterpret_cast<uint32_t *>(Bs) + (lane >> 2) * 16 + (lane & 3);
+                tab[0] = __byte_perm(t1, t3, 0x7632);
+                tab[4] = __byte_perm(t1, t3, 0x5410);
+                tab[8] = __byte_perm(t0, t2, 0x7632);
+                tab[12] = __byte_perm(t0, t2, 0x5410);
+                bsum = warp_sum(bsum);
                 if (t == 0) { bias0 = bsum; ks0 = pow2i(-sh); }
             } else {
             // one power-of-two scaling for all heads of the group: the largest factor lands in [2^13, 2^14)
@@ -632,11 +647,11 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
                         ia[2] += 2 * ih0[2] + 8 * ih1[2]; ia[3] += 2 * ih0[3] + 8 * ih1[3];
                     }
                     // lane t = 0 holds limbs 0, 1 (columns 0, 1), its neighbour limbs 2, 3 (columns 2, 3): each lane combines
-                    // its pair in int32 (below 2^31 for every code width), then one conversion per pair
-                    const int xg = ia[0] * 128 + ia[1], xh = ia[2] * 128 + ia[3];
-                    const int yg = __shfl_down_sync(0xffffffffu, xg, 1), yh = __shfl_down_sync(0xffffffffu, xh, 1);
-                    const float tg = fmaf((float)xg, 16384.f, (float)yg);
-                    const float th = fmaf((float)xh, 16384.f, (float)yh);
+                    // its pair (every column sum is below 2^24, exact in binary32), then the pairs combine
+                    const float xg = fmaf((float)ia[0], 256.f, (float)ia[1]), xh = fmaf((float)ia[2], 256.f, (float)ia[3]);
+                    const float yg = __shfl_down_sync(0xffffffffu, xg, 1), yh = __shfl_down_sync(0xffffffffu, xh, 1);
+                    const float tg = fmaf(xg, 65536.f, yg);
+                    const float th = fmaf(xh, 65536.f, yh);
                     s[k][0] = t == 0 ? fmaf(tg, ks0, -bias0) : -INFINITY; s[k][1] = -INFINITY;
                     s[k][2] = t == 0 ? fmaf(th, ks0 * (BITS == 4 ? 0.0625f : 0.25f), -bias0) : -INFINITY; s[k][3] = -INFINITY;
                     continue;
