@@ -210,13 +210,15 @@ struct DecodePlan {
 // limbs in four accumulator columns (2, 3 bit: divided by 16 beforehand for the upper slots); sums are exact in int32.
 // 3 bit: the low two bits as for 2 bit, the high bits of the second section (same byte structure) through four more
 // MMAs with the same B operands into accumulators of their own.
-template <int BITS, int D, int NGv, int CT, bool PL, bool I8 = false>
+// I8 = 2 (two to four query heads per KV head, 2 and 4 bit): the same with two B operands per word, which hold the upper
+// and the lower byte pair of every head's factors in the pair layout's columns.
+template <int BITS, int D, int NGv, int CT, bool PL, int I8 = 0>
 __global__ void __launch_bounds__(DEC_THREADS, 4)
 decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__restrict__ out, float *__restrict__ lse,
               float *__restrict__ part_ws, int nsplit, int groups_per_split, int qchunks, int seq_len, int cluster_merge)
 {
     using G_ = Geo<BITS, D>;
-    constexpr int NQMAX = I8 ? 1 : (PL ? 4 : 8);
+    constexpr int NQMAX = I8 == 1 ? 1 : (PL ? 4 : 8);
     using Plan = DecodePlan<BITS, D, NGv, CT, NQMAX>;
     constexpr int NM = G_::NM, W = G_::W, BST = Plan::BST, TILE_WORDS = 32 * W;
     constexpr int NSLOT = Plan::NSLOT, SLOT_BYTES = Plan::SLOT_BYTES, KV_BYTES = Plan::KV_BYTES, SZ_BYTES = Plan::SZ_BYTES;
@@ -229,7 +231,7 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
 
     const int tid = threadIdx.x, lane = tid & 31, warp = __shfl_sync(0xffffffffu, tid >> 5, 0), g = lane >> 2, t = lane & 3;
     const int split = blockIdx.x, h = blockIdx.y / qchunks, qc = blockIdx.y % qchunks, b = blockIdx.z;
-    const int nq = I8 ? 1 : min(NQMAX, p.rep - 8 * qc), hq0 = h * p.rep + 8 * qc;
+    const int nq = I8 == 1 ? 1 : min(NQMAX, p.rep - 8 * qc), hq0 = h * p.rep + 8 * qc;
     const int64_t unit = (int64_t)b * p.Hkv + h;
     const int G = p.G, n = seq_len, n_groups = n / G, n_body = n_groups * G;
     const int TPG = G / KVSINK_TILE, CPG = TPG / CT;                 // tiles and ring chunks per key group
@@ -272,7 +274,7 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
         for (int e = 0; e < 4; ++e) {
             i8_ch[e] = BITS != 4 ? 16 * (2 * mi + (e & 1)) + 8 * c2 + 2 * tq + (e >> 1)
                                  : 16 * (2 * mi + c2) + 8 * (e & 1) + 2 * tq + (e >> 1);
-            i8_q[e] = qs[i8_ch[e]];
+            if (I8 == 1) i8_q[e] = qs[i8_ch[e]];
         }
     }
 
@@ -464,7 +466,7 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
             }
             __syncwarp();   // the parameters are in registers: the slot can take the next group's while this one streams
             if (gi + 1 < my_groups) issue_params(gi + 1);
-            if constexpr (I8) {
+            if constexpr (I8 == 1) {
                 // limbs of the one head's factors: F = rint(q * scale * 2^sh) with the largest |F| in [2^29, 2^30), cut into
                 // four signed bytes (radix 256): every factor is kept to 2^-30 of the group's largest one (2^-26 where the
                 // factor is pre-divided for the upper contraction slots), finer than binary32 keeps the factor itself.
@@ -497,6 +499,43 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
                 tab[12] = __byte_perm(t0, t2, 0x5410);
                 bsum = warp_sum(bsum);
                 if (t == 0) { bias0 = bsum; ks0 = pow2i(-sh); }
+            } else if constexpr (I8 == 2) {
+                // up to four heads: the same four signed bytes per factor and head, each head with its own power of two.
+                // The two most significant bytes of every head fill the eight columns of one B operand (head h in columns
+                // 2h, 2h+1), the two less significant ones those of a second: lane t then finds both halves of head t's sum
+                // in its own accumulators.  Table [MMA][lower / upper slots][operand][column][t] in 32-bit words.
+                const bool upper = BITS != 4 && (lane & 4) != 0;
+                uint32_t *tab = reinterpret_cast<uint32_t *>(Bs) + (lane >> 2) * 64 + (lane & 3);
+#pragma unroll
+                for (int hh = 0; hh < 4; ++hh) {
+                    uint32_t w3 = 0u, w2 = 0u, w1 = 0u, w0 = 0u;
+                    if (hh < nq) {
+                        float v[4], amax = 0.f, bsum = 0.f;
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            v[e] = qs[hh * D + i8_ch[e]] * scv[e];
+                            amax = fmaxf(amax, fabsf(v[e]));
+                            bsum = fmaf(v[e], zev[e], bsum);
+                        }
+                        amax = __uint_as_float(__reduce_max_sync(0xffffffffu, __float_as_uint(amax)));
+                        int sh = 29 - floor_log2(amax);
+                        sh = sh > 60 ? 60 : (sh < -60 ? -60 : sh);
+                        const float pre = upper ? pow2i(sh - 4) : pow2i(sh);
+                        uint32_t d[4];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) d[e] = ((uint32_t)__float2int_rn(v[e] * pre) + 0x00808080u) ^ 0x00808080u;
+                        const uint32_t t0 = __byte_perm(d[0], d[1], 0x5140), t1 = __byte_perm(d[0], d[1], 0x7362);
+                        const uint32_t t2 = __byte_perm(d[2], d[3], 0x5140), t3 = __byte_perm(d[2], d[3], 0x7362);
+                        w3 = __byte_perm(t1, t3, 0x7632); w2 = __byte_perm(t1, t3, 0x5410);
+                        w1 = __byte_perm(t0, t2, 0x7632); w0 = __byte_perm(t0, t2, 0x5410);
+                        bsum = warp_sum(bsum);
+                        if (t == hh) { bias0 = bsum; ks0 = pow2i(-sh); }
+                    }
+                    tab[(2 * hh) * 4] = w3;
+                    tab[(2 * hh + 1) * 4] = w2;
+                    tab[(8 + 2 * hh) * 4] = w1;
+                    tab[(8 + 2 * hh + 1) * 4] = w0;
+                }
             } else {
             // one power-of-two scaling for all heads of the group: the largest factor lands in [2^13, 2^14)
             constexpr int NQL = PL ? 4 : 8;
@@ -564,7 +603,17 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
             __syncwarp();
         }
         uint32_t bk[NM][2];
-        if constexpr (I8) {
+        if constexpr (I8 == 2) {
+            // B fragments of the four words, first operand (bk[0..3]) and second (bk[4..7]): column g, slots 4t .. 4t + 3
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int c2 = 0; c2 < 2; ++c2) {
+                    const uint32_t *e = reinterpret_cast<const uint32_t *>(Bs) + (i * 2 + c2) * 64 + g * 4 + t;
+                    bk[i][c2] = e[0];
+                    bk[4 + i][c2] = e[32];
+                }
+        } else if constexpr (I8 == 1) {
             // B fragments of the four words: column g = limb g, contraction slots 4t .. 4t + 3 (lower, upper)
 #pragma unroll
             for (int m = 0; m < NM; ++m) bk[m][0] = bk[m][1] = 0u;
@@ -607,7 +656,35 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
             float s[ST][4];
 #pragma unroll
             for (int k = 0; k < ST; ++k) {
-                if constexpr (I8) {
+                if constexpr (I8 == 2) {
+                    uint32_t kw[W];
+                    load_tile_shared<BITS, D>(kt + k * TILE_WORDS, lane, kw);
+                    int ia[4] = {0, 0, 0, 0}, ib[4] = {0, 0, 0, 0};   // upper / lower byte pair of the heads' sums
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        uint32_t a0, a1, a2, a3;
+                        if constexpr (BITS != 4) {
+                            const uint32_t x = kw[i];
+                            a0 = x & 0x03030303u; a1 = x & 0x0c0c0c0cu; a2 = x & 0x30303030u; a3 = x & 0xc0c0c0c0u;
+                        } else {
+                            const uint32_t x = kw[2 * i], y = kw[2 * i + 1];
+                            a0 = x & 0x0f0f0f0fu; a1 = x & 0xf0f0f0f0u; a2 = y & 0x0f0f0f0fu; a3 = y & 0xf0f0f0f0u;
+                        }
+                        asm volatile("mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                                     : "+r"(ia[0]), "+r"(ia[1]), "+r"(ia[2]), "+r"(ia[3])
+                                     : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(bk[i][0]), "r"(bk[i][1]));
+                        asm volatile("mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                                     : "+r"(ib[0]), "+r"(ib[1]), "+r"(ib[2]), "+r"(ib[3])
+                                     : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(bk[4 + i][0]), "r"(bk[4 + i][1]));
+                    }
+                    // lane t holds head t: bytes 3, 2 of its sum in the first accumulators, bytes 1, 0 in the second
+                    const float tg = fmaf(fmaf((float)ia[0], 256.f, (float)ia[1]), 65536.f, fmaf((float)ib[0], 256.f, (float)ib[1]));
+                    const float th = fmaf(fmaf((float)ia[2], 256.f, (float)ia[3]), 65536.f, fmaf((float)ib[2], 256.f, (float)ib[3]));
+                    s[k][0] = fmaf(tg, ks0, -bias0); s[k][1] = -INFINITY;
+                    s[k][2] = fmaf(th, ks0 * (BITS == 4 ? 0.0625f : 0.25f), -bias0); s[k][3] = -INFINITY;
+                    continue;
+                }
+                if constexpr (I8 == 1) {
                     uint32_t kw[W];
                     load_tile_shared<BITS, D>(kt + k * TILE_WORDS, lane, kw);
                     int ia[4] = {0, 0, 0, 0};
@@ -908,14 +985,14 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
 }
 
 // ---- launch: one instantiation per (bits, head size, value groups per row, chunk size, key-side variant) ----
-template <int BITS, int D, int NGV, int CT, bool PL, bool I8 = false>
+template <int BITS, int D, int NGV, int CT, bool PL, int I8 = 0>
 static int launch_decode_p(const Params &p, const kvsink_cache &c, const __half *q, float *out, float *lse, float *ws, cudaStream_t st)
 {
     const int n_groups = c.seq_len / p.G;
     const int nsplit = choose_splits(p, n_groups);
     const int gps = n_groups > 0 ? (n_groups + nsplit - 1) / nsplit : 0;
     const int qchunks = (p.rep + 7) / 8;
-    const size_t smem = DecodePlan<BITS, D, NGV, CT, I8 ? 1 : (PL ? 4 : 8)>::BYTES;
+    const size_t smem = DecodePlan<BITS, D, NGV, CT, I8 == 1 ? 1 : (PL ? 4 : 8)>::BYTES;
     auto kern = decode_kernel<BITS, D, NGV, CT, PL, I8>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return KVSINK_ERR_CUDA;
     cudaLaunchAttribute pdl[2];
@@ -955,7 +1032,9 @@ template <int BITS, int D, int NGV, int CT>
 static int launch_decode_c(const Params &p, const kvsink_cache &c, const __half *q, float *out, float *lse, float *ws, cudaStream_t st)
 {
     if constexpr (D == 128)
-        if (p.rep == 1) return launch_decode_p<BITS, D, NGV, CT, true, true>(p, c, q, out, lse, ws, st);
+        if (p.rep == 1) return launch_decode_p<BITS, D, NGV, CT, true, 1>(p, c, q, out, lse, ws, st);
+    if constexpr (D == 128 && BITS != 3)
+        if (p.rep <= 4) return launch_decode_p<BITS, D, NGV, CT, true, 2>(p, c, q, out, lse, ws, st);
     if (p.rep <= 4) return launch_decode_p<BITS, D, NGV, CT, true>(p, c, q, out, lse, ws, st);
     return launch_decode_p<BITS, D, NGV, CT, false>(p, c, q, out, lse, ws, st);
 }
