@@ -154,26 +154,27 @@ __device__ __forceinline__ void tile_frags(const uint32_t (&w)[Geo<BITS, D>::W],
 }
 
 // ---- per-warp bulk-copy ring (TMA, cp.async.bulk) ----
-__device__ __forceinline__ void mbar_init(uint64_t *bar, unsigned count)
+// Barriers and copy destinations are passed as 32-bit shared-window addresses, converted once per warp.
+__device__ __forceinline__ void mbar_init(uint32_t bar, unsigned count)
 {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(bar)), "r"(count) : "memory");
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
 }
-__device__ __forceinline__ void mbar_expect_tx(uint64_t *bar, unsigned bytes)
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, unsigned bytes)
 {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)), "r"(bytes) : "memory");
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
-__device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, unsigned parity)
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, unsigned parity)
 {
     unsigned ok;
     asm volatile("{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
-                 : "=r"(ok) : "r"(smem_addr(bar)), "r"(parity) : "memory");
+                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
 }
 // Global -> shared bulk copy; addresses and size are multiples of 16 bytes; completion is counted on `bar`.
-__device__ __forceinline__ void bulk_g2s(void *dst, const void *src, unsigned bytes, uint64_t *bar)
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void *src, unsigned bytes, uint32_t bar)
 {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                 ::"r"(smem_addr(dst)), "l"(src), "r"(bytes), "r"(smem_addr(bar)) : "memory");
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
 }
 
 constexpr int DEC_WAIT_LIMIT = 1 << 22;   // polls of a full-barrier before a warp gives up (far beyond any real latency)
@@ -246,9 +247,10 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
     unsigned char *ring_all = smem_raw + Plan::FIXED;                // [warps][WARP_RING]; later reused for the partials
     float *part = (float *)ring_all;                                 // [2*warps][nq][D+2]
 
-    uint64_t *cbar = bars + warp * 8, *pbar = cbar + 4;              // chunk and parameter full-barriers of this warp
+    // chunk full-barriers (one per ring slot) and the parameter full-barrier of this warp, as shared-window addresses
+    const uint32_t cbar = smem_addr(bars + warp * 8), pbar = cbar + 4 * 8;
     if (lane == 0) {
-        for (int i = 0; i < 6; ++i) mbar_init(&cbar[i], 1);
+        for (int i = 0; i < 5; ++i) mbar_init(cbar + 8 * i, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     // launched with programmatic stream serialization: everything above overlaps the tail of the kernel before this
@@ -404,15 +406,16 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
     int iss = 0;                                                     // chunks issued so far
     uint32_t iss_kv = (uint32_t)w_begin * TPG * Plan::TILE_BYTES;    // byte offset of the next chunk in the code arrays
     uint32_t iss_sz = (uint32_t)w_begin * TPG * 16 * NGv * 4;        // and in the value parameter arrays
+    const uint32_t ring_s = smem_addr(ring), kp_s = smem_addr(kp_ring);
     auto issue_chunk = [&]() {
         const int slot = iss & (NSLOT - 1);
-        unsigned char *dst = ring + slot * SLOT_BYTES;
+        const uint32_t dst = ring_s + slot * SLOT_BYTES, bar = cbar + 8 * slot;
         if (lane == 0) {
-            mbar_expect_tx(&cbar[slot], SLOT_BYTES);
-            bulk_g2s(dst, kc_base + iss_kv, KV_BYTES, &cbar[slot]);
-            bulk_g2s(dst + KV_BYTES, vc_base + iss_kv, KV_BYTES, &cbar[slot]);
-            bulk_g2s(dst + 2 * KV_BYTES, (const unsigned char *)vs_base + iss_sz, SZ_BYTES, &cbar[slot]);
-            bulk_g2s(dst + 2 * KV_BYTES + SZ_BYTES, (const unsigned char *)vz_base + iss_sz, SZ_BYTES, &cbar[slot]);
+            mbar_expect_tx(bar, SLOT_BYTES);
+            bulk_g2s(dst, kc_base + iss_kv, KV_BYTES, bar);
+            bulk_g2s(dst + KV_BYTES, vc_base + iss_kv, KV_BYTES, bar);
+            bulk_g2s(dst + 2 * KV_BYTES, (const unsigned char *)vs_base + iss_sz, SZ_BYTES, bar);
+            bulk_g2s(dst + 2 * KV_BYTES + SZ_BYTES, (const unsigned char *)vz_base + iss_sz, SZ_BYTES, bar);
         }
         ++iss;
         iss_kv += KV_BYTES;
@@ -420,12 +423,12 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
     };
     auto issue_params = [&](int gi) {
         if (lane == 0) {
-            mbar_expect_tx(&pbar[0], Plan::KP_BYTES);
-            bulk_g2s(kp_ring, ks_base + (size_t)(w_begin + gi) * D, D * 4, &pbar[0]);
-            bulk_g2s(kp_ring + D, kz_base + (size_t)(w_begin + gi) * D, D * 4, &pbar[0]);
+            mbar_expect_tx(pbar, Plan::KP_BYTES);
+            bulk_g2s(kp_s, ks_base + (size_t)(w_begin + gi) * D, D * 4, pbar);
+            bulk_g2s(kp_s + D * 4, kz_base + (size_t)(w_begin + gi) * D, D * 4, pbar);
         }
     };
-    auto wait_bar = [&](uint64_t *bar, unsigned parity) {
+    auto wait_bar = [&](uint32_t bar, unsigned parity) {
         int polls = 0;
         bool ok = true;
         while (!mbar_try_wait(bar, parity)) {
@@ -456,7 +459,7 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
         float bias0 = 0.f, bias1 = 0.f, ks0 = 0.f, ks1 = 0.f;
         uint32_t need_lo = 0;     // bit m: matrix m also gets the low half of the split factor (warp-uniform)
         {
-            if (!wait_bar(&pbar[0], (unsigned)gi & 1u)) { stream_ok = false; break; }
+            if (!wait_bar(pbar, (unsigned)gi & 1u)) { stream_ok = false; break; }
             const float *kp = kp_ring;
             float scv[CPL], zev[CPL];
 #pragma unroll
@@ -638,7 +641,7 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
             // refill the slot freed by the previous chunk, then wait for this chunk's bytes
             __syncwarp();
             if (iss < n_chunks) issue_chunk();
-            if (!wait_bar(&cbar[slot], (unsigned)(ci / NSLOT) & 1u)) { stream_ok = false; break; }
+            if (!wait_bar(cbar + 8 * slot, (unsigned)(ci / NSLOT) & 1u)) { stream_ok = false; break; }
             const uint2 mwords = mword_next;
             {   // sink bits of the warp's next chunk, fetched one chunk ahead
                 if (ci + 1 < n_chunks) mword_next = load_mask_words(grp * TPG + (cj + 1) * CT);   // the warp's chunks are consecutive
@@ -762,7 +765,9 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
             if (mword) {   // sink tokens are not part of the packed stream (their value parameters are zero)
 #pragma unroll
                 for (int k = 0; k < ST; ++k) {
-                    const uint32_t mask16 = ((ST == 4 ? (k < 2 ? mwords.x : mwords.y) : mword) >> (16 * ((T0 + k) & 1))) & 0xffffu;
+                    // a chunk of an even number of tiles starts on an even tile: the half of the word is known at compile time
+                    const int half = (CT % 2 == 0) ? (k & 1) : ((T0 + k) & 1);
+                    const uint32_t mask16 = ((ST == 4 ? (k < 2 ? mwords.x : mwords.y) : mword) >> (16 * half)) & 0xffffu;
                     if ((mask16 >> g) & 1u) s[k][0] = s[k][1] = -INFINITY;
                     if ((mask16 >> (g + 8)) & 1u) s[k][2] = s[k][3] = -INFINITY;
                 }
