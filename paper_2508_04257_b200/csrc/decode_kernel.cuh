@@ -256,6 +256,9 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
     // launched with programmatic stream serialization: everything above overlaps the tail of the kernel before this
     // one in the stream; nothing it may have written (the query, the cache) is read before this point
     asm volatile("griddepcontrol.wait;" ::: "memory");
+    // the next kernel in the stream may be scheduled from now on: its blocks take whatever room this grid leaves, set
+    // themselves up, and wait at the same point until this grid has completed
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     for (int i = tid; i < NQMAX * D; i += DEC_THREADS) {
         const int qh = i / D, ch = i % D;
         __half v = qh < nq ? q[((size_t)b * p.Hq + hq0 + qh) * D + ch] : __float2half(0.f);
@@ -803,7 +806,6 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
         }
     }
     if (!stream_ok && lane == 0) atomicOr(c.status, KVSINK_STATUS_TIMEOUT);
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the merge kernel may be scheduled; it waits for this grid's end
 
     // ---- tokens of the open group: keys from the fp16 tail (last split only) ----
     if (split == nsplit - 1) {
