@@ -136,7 +136,8 @@ int kvsink_predict_sinks(const kvsink_config *cfg, const void *hidden, int32_t S
  * scale = zero = 0).  Values are coded on arrival; a key waits in k_tail until its G-token group is complete.
  *   k_new, v_new  device, fp16, element (b, h, t, c) at base + b*stride_b + h*stride_h + t*stride_t + c;
  *                 strides in elements, multiples of 8; both tensors share the strides.
- *   T             T == 1 at any time; T > 1 only while seq_len is a multiple of G (for instance the prefill).
+ *   T             any T >= 0 at any time (prefill, chunked prefill, one decode token): a chunk may start and end inside
+ *                 a key group; the result is the same as appending its tokens one by one.
  * On success cache->seq_len (host) is advanced by T.
  */
 int kvsink_quantize_append(const kvsink_config *cfg, kvsink_cache *cache, const void *k_new, const void *v_new, int32_t T,

@@ -205,3 +205,81 @@ def quantize_group(x: np.ndarray, member: np.ndarray, bits: int):
     lib().kvo_quantize_group(x.ctypes.data_as(C.c_void_p), m.ctypes.data_as(C.c_void_p), C.c_int(x.shape[0]),
                              C.c_int(bits), C.byref(sc), C.byref(ze), codes.ctypes.data_as(C.c_void_p))
     return np.float32(sc.value), np.float32(ze.value), codes
+
+
+# ---- analysis routines (Section 3.1 / Appendix D; Section 4.1, Table 1) ----
+def channel_absmax(hidden: np.ndarray) -> np.ndarray:
+    """hidden: float16 [B, S, d] (last axis contiguous). Returns float32 [d]: the largest |H| of every channel."""
+    h = _u16(hidden)
+    assert h.ndim == 3 and h.strides[2] == 2
+    B, S, d = h.shape
+    out = np.zeros(d, np.float32)
+    _check(lib().kvo_channel_absmax(h.ctypes.data_as(C.c_void_p), C.c_int32(B), C.c_int32(S), C.c_int32(d), C.c_int64(h.strides[0] // 2),
+                                    C.c_int64(h.strides[1] // 2), out.ctypes.data_as(C.c_void_p)), "channel_absmax")
+    return out
+
+
+def quant_error(cfg: Config, x: np.ndarray, bitmask: np.ndarray, per_channel: bool, exclude_sinks: bool) -> np.ndarray:
+    """x: float16 [B, Hkv, T, D]. Returns float64 [4]: (sum sq err, elements) over groups without / with a sink token."""
+    a = _u16(x)
+    assert a.ndim == 4 and a.strides[3] == 2
+    bm = np.ascontiguousarray(bitmask, np.uint32)
+    out = np.zeros(4, np.float64)
+    _check(lib().kvo_quant_error(C.byref(cfg.c()), a.ctypes.data_as(C.c_void_p), C.c_int32(a.shape[2]), C.c_int64(a.strides[0] // 2),
+                                 C.c_int64(a.strides[1] // 2), C.c_int64(a.strides[2] // 2), C.c_int(int(per_channel)),
+                                 C.c_int(int(exclude_sinks)), bm.ctypes.data_as(C.c_void_p), out.ctypes.data_as(C.c_void_p)), "quant_error")
+    return out
+
+
+# ---- static (calibrated) parameters (Section 5.1 scheme; Appendix C; Algorithm 1's remark on calibration) ----
+class _Static(C.Structure):
+    _fields_ = [("k_scale", C.c_void_p), ("k_zero", C.c_void_p), ("v_scale", C.c_void_p), ("v_zero", C.c_void_p)]
+
+
+class StaticParams:
+    """Calibrated (scale, zero): keys float32 [Hkv, D] per channel, values float32 [Hkv, D / v_group] per channel group."""
+
+    def __init__(self, cfg: Config):
+        ngv = cfg.head_dim // min(cfg.group, cfg.head_dim)
+        self.k_scale = np.zeros((cfg.n_kv_heads, cfg.head_dim), np.float32)
+        self.k_zero = np.zeros_like(self.k_scale)
+        self.v_scale = np.zeros((cfg.n_kv_heads, ngv), np.float32)
+        self.v_zero = np.zeros_like(self.v_scale)
+
+    def c(self) -> _Static:
+        p = lambda a: a.ctypes.data_as(C.c_void_p)
+        return _Static(p(self.k_scale), p(self.k_zero), p(self.v_scale), p(self.v_zero))
+
+
+def calibrate(cfg: Config, k_cal: np.ndarray, v_cal: np.ndarray, bitmask: np.ndarray) -> StaticParams:
+    """Global min-max calibration over k_cal, v_cal float16 [B, Hkv, T, D] with the masked (sink) tokens left out."""
+    k, v = _u16(k_cal), _u16(v_cal)
+    assert k.shape == v.shape and k.strides == v.strides and k.strides[3] == 2
+    bm = np.ascontiguousarray(bitmask, np.uint32)
+    sp = StaticParams(cfg)
+    cs = sp.c()
+    _check(lib().kvo_calibrate(C.byref(cfg.c()), k.ctypes.data_as(C.c_void_p), v.ctypes.data_as(C.c_void_p), C.c_int32(k.shape[2]),
+                               C.c_int64(k.strides[0] // 2), C.c_int64(k.strides[1] // 2), C.c_int64(k.strides[2] // 2),
+                               bm.ctypes.data_as(C.c_void_p), C.byref(cs)), "calibrate")
+    return sp
+
+
+def quantize_append_calibrated(cfg: Config, cache: Cache, sp: StaticParams, k_new: np.ndarray, v_new: np.ndarray) -> None:
+    k, v = _u16(k_new), _u16(v_new)
+    assert k.shape == v.shape and k.strides == v.strides and k.strides[3] == 2
+    cc, cs = cache.c(), sp.c()
+    rc = lib().kvo_quantize_append_calibrated(C.byref(cfg.c()), C.byref(cc), C.byref(cs), k.ctypes.data_as(C.c_void_p),
+                                              v.ctypes.data_as(C.c_void_p), C.c_int32(k.shape[2]), C.c_int64(k.strides[0] // 2),
+                                              C.c_int64(k.strides[1] // 2), C.c_int64(k.strides[2] // 2))
+    _check(rc, "quantize_append_calibrated")
+    cache.seq_len = cc.seq_len
+
+
+def decode_attention_calibrated(cfg: Config, cache: Cache, sp: StaticParams, q: np.ndarray):
+    qq = np.ascontiguousarray(_u16(q))
+    out = np.zeros((cfg.batch, cfg.n_q_heads, cfg.head_dim), np.float64)
+    lse = np.zeros((cfg.batch, cfg.n_q_heads), np.float64)
+    cc, cs = cache.c(), sp.c()
+    _check(lib().kvo_decode_attention_calibrated(C.byref(cfg.c()), C.byref(cc), C.byref(cs), qq.ctypes.data_as(C.c_void_p),
+                                                 out.ctypes.data_as(C.c_void_p), lse.ctypes.data_as(C.c_void_p)), "decode_attention_calibrated")
+    return out, lse

@@ -557,3 +557,251 @@ int kvo_decode_attention(const kvo_config *c, const kvo_cache *cache, const uint
     }
     return KVO_OK;
 }
+
+/* =====================================================================================================
+ * Analysis routines (Section 3.1 / Appendix D: where the extreme activations sit; Section 4.1, Table 1: what
+ * sink tokens do to the quantization error).
+ * ===================================================================================================== */
+
+/*
+ * Largest magnitude of every hidden channel over all tokens of all sequences: out[c] = max_{b,i} |H[b,i,c]|.
+ * This is the scan from which the few "outlier channels" of a model (Appendix D, the table of emergence layers and
+ * outlier channels) are read off: they are the channels whose maximum is orders of magnitude above the rest, and the
+ * emergence layer is the first layer whose scan shows them.  A NaN never raises a maximum (|x| > best is false).
+ */
+int kvo_channel_absmax(const uint16_t *hidden, int32_t B, int32_t S, int32_t d, int64_t stride_b, int64_t stride_s, float *out)
+{
+    if (!hidden || !out || B < 0 || S < 0 || d < 1) return KVO_ERR_BAD_ARG;
+    for (int c = 0; c < d; ++c) out[c] = 0.0f;
+    for (int b = 0; b < B; ++b)
+        for (int i = 0; i < S; ++i) {
+            const uint16_t *row = hidden + b * stride_b + i * stride_s;
+            for (int c = 0; c < d; ++c) {
+                float a = fabsf(half_to_float(row[c]));
+                if (a > out[c]) out[c] = a;
+            }
+        }
+    return KVO_OK;
+}
+
+/*
+ * Quantization error in the shape of Table 1 (Section 4.1): round-to-nearest asymmetric quantization (Eq. 8-11) of a
+ * tensor x [B,Hkv,T,D], squared error (x - x')^2 with x' = scale * (Q - zero) (Eq. 9), summed separately over the
+ * quantization groups that contain no sink token and over those that contain at least one.
+ *   per_channel != 0 : groups of `group` consecutive tokens of one channel (keys, per channel); a last, shorter group
+ *                      takes the remaining tokens
+ *   per_channel == 0 : groups of min(group, D) consecutive channels of one token (per token)
+ *   exclude_sinks == 0: plain RTN, every token takes part in its group's min / max (the table's dynamic rows)
+ *   exclude_sinks != 0: KVSink: sink tokens take no part in the statistics and are not quantized (no error counted)
+ * out[0], out[1]: sum of squared errors and number of elements over groups without a sink token;
+ * out[2], out[3]: the same over groups with one.  MSE = out[0] / out[1] and out[2] / out[3].
+ */
+int kvo_quant_error(const kvo_config *c, const uint16_t *x, int32_t T, int64_t stride_b, int64_t stride_h, int64_t stride_t,
+                    int per_channel, int exclude_sinks, const uint32_t *bitmask, double *out)
+{
+    int rc = check_config(c);
+    if (rc) return rc;
+    if (!x || !bitmask || !out || T < 0 || T > c->max_seq) return KVO_ERR_BAD_ARG;
+    const int D = c->head_dim, G = c->group, gv = v_group_of(c);
+    const int buf = G > D ? G : D;
+    float *xs = (float *)malloc(sizeof(float) * (size_t)buf);
+    uint8_t *mem = (uint8_t *)malloc((size_t)buf);
+    int32_t *codes = (int32_t *)malloc(sizeof(int32_t) * (size_t)buf);
+    out[0] = out[1] = out[2] = out[3] = 0.0;
+    for (int b = 0; b < c->batch; ++b)
+        for (int h = 0; h < c->n_kv_heads; ++h) {
+            const uint16_t *base = x + b * stride_b + h * stride_h;
+            if (per_channel) {
+                for (int t0 = 0; t0 < T; t0 += G) {
+                    int n = T - t0 < G ? T - t0 : G, has_sink = 0;
+                    for (int t = 0; t < n; ++t) has_sink |= mask_bit(bitmask, c, b, t0 + t);
+                    for (int ch = 0; ch < D; ++ch) {
+                        float sc = 0.0f, ze = 0.0f;
+                        for (int t = 0; t < n; ++t) {
+                            xs[t] = half_to_float(base[(int64_t)(t0 + t) * stride_t + ch]);
+                            mem[t] = (uint8_t)(exclude_sinks ? !mask_bit(bitmask, c, b, t0 + t) : 1);
+                        }
+                        kvo_quantize_group(xs, mem, n, c->bits, &sc, &ze, codes);
+                        for (int t = 0; t < n; ++t) {
+                            if (!mem[t]) continue;
+                            double e = (double)xs[t] - (double)dequant(sc, ze, (uint32_t)codes[t]);
+                            out[has_sink ? 2 : 0] += e * e;
+                            out[has_sink ? 3 : 1] += 1.0;
+                        }
+                    }
+                }
+            } else {
+                for (int t = 0; t < T; ++t) {
+                    int has_sink = mask_bit(bitmask, c, b, t);
+                    if (has_sink && exclude_sinks) continue;
+                    for (int j = 0; j < D / gv; ++j) {
+                        float sc = 0.0f, ze = 0.0f;
+                        for (int e = 0; e < gv; ++e) { xs[e] = half_to_float(base[(int64_t)t * stride_t + j * gv + e]); mem[e] = 1; }
+                        kvo_quantize_group(xs, mem, gv, c->bits, &sc, &ze, codes);
+                        for (int e = 0; e < gv; ++e) {
+                            double er = (double)xs[e] - (double)dequant(sc, ze, (uint32_t)codes[e]);
+                            out[has_sink ? 2 : 0] += er * er;
+                            out[has_sink ? 3 : 1] += 1.0;
+                        }
+                    }
+                }
+            }
+        }
+    free(xs); free(mem); free(codes);
+    return KVO_OK;
+}
+
+/* =====================================================================================================
+ * Static (calibrated) parameters: the scheme of the paper's main comparison (Section 5.1: per-channel keys with
+ * per-token values, static), with sink tokens left out of the calibration as well as of the quantization
+ * (Algorithm 1's remark on calibration; Section 4.1; Appendix C "Dynamic and static quantization").
+ * ===================================================================================================== */
+
+typedef struct {
+    float *k_scale, *k_zero;   /* [Hkv][D]: one pair per key channel, for every token and sequence */
+    float *v_scale, *v_zero;   /* [Hkv][D / v_group]: one pair per value channel group, for every token and sequence */
+} kvo_static_params;
+
+/*
+ * Calibration: "global min-max" (Table 1's caption) over a calibration batch x_k, x_v [B,Hkv,T,D], per key channel
+ * and per value channel group of every KV head, over all sequences and all tokens that are not sink tokens; then
+ * Eq. 10-11.  A range of a single value reproduces itself (scale = |min|, or 1 for 0); no member gives scale = zero = 0.
+ */
+int kvo_calibrate(const kvo_config *c, const uint16_t *k_cal, const uint16_t *v_cal, int32_t T, int64_t stride_b, int64_t stride_h,
+                  int64_t stride_t, const uint32_t *bitmask, kvo_static_params *sp)
+{
+    int rc = check_config(c);
+    if (rc) return rc;
+    if (!k_cal || !v_cal || !bitmask || !sp || T < 0 || T > c->max_seq) return KVO_ERR_BAD_ARG;
+    const int D = c->head_dim, gv = v_group_of(c), ngv = D / gv;
+    const float qmax = (float)((1 << c->bits) - 1);
+    for (int h = 0; h < c->n_kv_heads; ++h)
+        for (int kind = 0; kind < 2; ++kind) {
+            const int ngroups = kind ? ngv : D, width = kind ? gv : 1;
+            for (int j = 0; j < ngroups; ++j) {
+                int any = 0;
+                float mn = 0.0f, mx = 0.0f;
+                for (int b = 0; b < c->batch; ++b)
+                    for (int t = 0; t < T; ++t) {
+                        if (mask_bit(bitmask, c, b, t)) continue;
+                        const uint16_t *row = (kind ? v_cal : k_cal) + b * stride_b + h * stride_h + (int64_t)t * stride_t;
+                        for (int e = 0; e < width; ++e) {
+                            float v = half_to_float(row[j * width + e]);
+                            if (!any) { mn = mx = v; any = 1; }
+                            else { if (v < mn) mn = v; if (v > mx) mx = v; }
+                        }
+                    }
+                float scale = 0.0f, zero = 0.0f;
+                if (any) {
+                    float r = mx - mn;
+                    if (r == 0.0f) scale = (mn == 0.0f) ? 1.0f : fabsf(mn);
+                    else scale = r / qmax;
+                    zero = 0.0f - rintf(mn / scale);
+                }
+                if (kind) { sp->v_scale[h * ngv + j] = scale; sp->v_zero[h * ngv + j] = zero; }
+                else { sp->k_scale[h * D + j] = scale; sp->k_zero[h * D + j] = zero; }
+            }
+        }
+    return KVO_OK;
+}
+
+/* Eq. 8 with fixed parameters: values outside the calibrated range clamp to code 0 or 2^n - 1; scale 0 (a channel
+ * that saw no calibration data) gives code 0. */
+static uint32_t static_code(float x, float scale, float zero, int bits)
+{
+    if (scale == 0.0f) return 0;
+    const float qmax = (float)((1 << bits) - 1);
+    float q = rintf(x / scale) + zero;
+    q = fminf(fmaxf(q, 0.0f), qmax);
+    return (uint32_t)q;
+}
+
+/*
+ * Append (Eq. 6) with static parameters: every token is coded on arrival, keys per channel and values per channel
+ * group with the calibrated pairs (Eq. 8); sink tokens keep exact fp16 rows in the side buffer and code 0.  There is
+ * no key tail and no per-group parameter: cache->k_scale, k_zero, v_scale, v_zero and k_tail are not touched.
+ */
+int kvo_quantize_append_calibrated(const kvo_config *c, kvo_cache *cache, const kvo_static_params *sp, const uint16_t *k_new,
+                                   const uint16_t *v_new, int32_t T, int64_t stride_b, int64_t stride_h, int64_t stride_t)
+{
+    int rc = check_config(c);
+    if (rc) return rc;
+    if (!cache || !sp || !k_new || !v_new || T < 0) return KVO_ERR_BAD_ARG;
+    if (cache->seq_len < 0 || (int64_t)cache->seq_len + T > c->max_seq) return KVO_ERR_SEQ_OVERFLOW;
+    const int D = c->head_dim, gv = v_group_of(c), ngv = D / gv, cap = sink_cap_of(c), Hk = c->n_kv_heads;
+    int bad = 0;
+    for (int64_t unit = 0; unit < (int64_t)c->batch * Hk; ++unit) {
+        const int b = (int)(unit / Hk), h = (int)(unit % Hk);
+        for (int i = 0; i < T; ++i) {
+            int p = cache->seq_len + i;
+            const uint16_t *krow = k_new + b * stride_b + h * stride_h + i * stride_t;
+            const uint16_t *vrow = v_new + b * stride_b + h * stride_h + i * stride_t;
+            int sink = mask_bit(cache->sink_bitmask, c, b, p);
+            if (sink) {
+                int slot = sink_slot(c, cache, b, p);
+                if (slot < 0) { bad = 1; continue; }
+                memcpy(cache->sink_k + (unit * cap + slot) * D, krow, sizeof(uint16_t) * (size_t)D);
+                memcpy(cache->sink_v + (unit * cap + slot) * D, vrow, sizeof(uint16_t) * (size_t)D);
+            }
+            for (int ch = 0; ch < D; ++ch) {
+                uint32_t kc = sink ? 0 : static_code(half_to_float(krow[ch]), sp->k_scale[h * D + ch], sp->k_zero[h * D + ch], c->bits);
+                uint32_t vc = sink ? 0 : static_code(half_to_float(vrow[ch]), sp->v_scale[h * ngv + ch / gv], sp->v_zero[h * ngv + ch / gv], c->bits);
+                k_code_put(cache->k_codes, c, b, h, p, ch, kc);
+                v_code_put(cache->v_codes, c, b, h, p, ch, vc);
+            }
+        }
+    }
+    if (bad) return KVO_ERR_BAD_ARG;
+    cache->seq_len += T;
+    return KVO_OK;
+}
+
+/*
+ * Eq. 3 / Eq. 7 over a cache with static parameters: a sink token's K and V are its fp16 side-buffer rows, every other
+ * token's are scale * (Q - zero) (Eq. 9, binary32) with the calibrated pairs.  binary64 otherwise, as kvo_decode_attention.
+ */
+int kvo_decode_attention_calibrated(const kvo_config *c, const kvo_cache *cache, const kvo_static_params *sp, const uint16_t *q,
+                                    double *out, double *lse)
+{
+    int rc = check_config(c);
+    if (rc) return rc;
+    if (!cache || !sp || !q || !out) return KVO_ERR_BAD_ARG;
+    const int D = c->head_dim, n = cache->seq_len, rep = c->n_q_heads / c->n_kv_heads, gv = v_group_of(c), ngv = D / gv;
+    const int cap = sink_cap_of(c);
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int64_t bh = 0; bh < (int64_t)c->batch * c->n_q_heads; ++bh) {
+        const int b = (int)(bh / c->n_q_heads), hq = (int)(bh % c->n_q_heads), h = hq / rep;
+        const int64_t unit = (int64_t)b * c->n_kv_heads + h;
+        double *s = (double *)malloc(sizeof(double) * (size_t)(n > 0 ? n : 1));
+        double *vrow = (double *)malloc(sizeof(double) * (size_t)D);
+        const uint16_t *qv = q + ((int64_t)b * c->n_q_heads + hq) * D;
+        double *o = out + ((int64_t)b * c->n_q_heads + hq) * D;
+        double mx = -INFINITY;
+        for (int p = 0; p < n; ++p) {
+            int slot = mask_bit(cache->sink_bitmask, c, b, p) ? sink_slot(c, cache, b, p) : -2;
+            double acc = 0.0;
+            for (int ch = 0; ch < D; ++ch) {
+                double kv = slot == -2 ? (double)dequant(sp->k_scale[h * D + ch], sp->k_zero[h * D + ch], k_code_get(cache->k_codes, c, b, h, p, ch))
+                                       : (slot < 0 ? NAN : (double)half_to_float(cache->sink_k[(unit * cap + slot) * D + ch]));
+                acc += (double)half_to_float(qv[ch]) * kv;
+            }
+            s[p] = acc / sqrt((double)D);
+            if (s[p] > mx) mx = s[p];
+        }
+        double den = 0.0;
+        for (int ch = 0; ch < D; ++ch) o[ch] = 0.0;
+        for (int p = 0; p < n; ++p) {
+            int slot = mask_bit(cache->sink_bitmask, c, b, p) ? sink_slot(c, cache, b, p) : -2;
+            for (int ch = 0; ch < D; ++ch)
+                vrow[ch] = slot == -2 ? (double)dequant(sp->v_scale[h * ngv + ch / gv], sp->v_zero[h * ngv + ch / gv], v_code_get(cache->v_codes, c, b, h, p, ch))
+                                      : (slot < 0 ? NAN : (double)half_to_float(cache->sink_v[(unit * cap + slot) * D + ch]));
+            double w = exp(s[p] - mx);
+            den += w;
+            for (int ch = 0; ch < D; ++ch) o[ch] += w * vrow[ch];
+        }
+        for (int ch = 0; ch < D; ++ch) o[ch] = n > 0 ? o[ch] / den : 0.0;
+        if (lse) lse[(int64_t)b * c->n_q_heads + hq] = n > 0 ? mx + log(den) : -INFINITY;
+        free(s); free(vrow);
+    }
+    return KVO_OK;
+}

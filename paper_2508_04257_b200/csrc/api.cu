@@ -116,22 +116,31 @@ extern "C" int kvsink_quantize_append(const kvsink_config *cfg, kvsink_cache *ca
     cudaStream_t st = (cudaStream_t)cuda_stream;
     const int S0 = cache->seq_len, G = p.G;
     const __half *k = (const __half *)k_new, *v = (const __half *)v_new;
-    if (T > 1 && (S0 % G) != 0) return KVSINK_ERR_UNSUPPORTED;
-    if (S0 % G == 0 && T >= G) {
-        const int n_groups = T / G;
-        rc = quantize_groups(p, *cache, k, v, S0, n_groups, stride_b, stride_h, stride_t, true, st);
+    // A chunk that starts inside an open group first completes (or extends) that group token by token; whole groups
+    // that follow take the bulk kernels; what is left goes to the tail token by token.
+    int done = 0;
+    if (S0 % G != 0) {
+        const int head = T < G - S0 % G ? T : G - S0 % G;
+        rc = launch_quantize_tokens(p, *cache, k, v, 0, S0, head, stride_b, stride_h, stride_t, st);
         if (rc) return rc;
-        rc = launch_quantize_tokens(p, *cache, k, v, n_groups * G, S0 + n_groups * G, T - n_groups * G, stride_b, stride_h, stride_t, st);
-        if (rc) return rc;
-    } else {
-        rc = launch_quantize_tokens(p, *cache, k, v, 0, S0, T, stride_b, stride_h, stride_t, st);
-        if (rc) return rc;
-        if ((S0 + T) % G == 0) {
+        if ((S0 + head) % G == 0) {
             // the open group is complete: quantize its keys per channel from the fp16 tail
-            rc = quantize_groups(p, *cache, (const __half *)cache->k_tail, (const __half *)cache->k_tail, S0 + T - G, 1,
-                                        (int64_t)p.Hkv * G * p.D, (int64_t)G * p.D, p.D, false, st);
+            rc = quantize_groups(p, *cache, (const __half *)cache->k_tail, (const __half *)cache->k_tail, S0 + head - G, 1,
+                                 (int64_t)p.Hkv * G * p.D, (int64_t)G * p.D, p.D, false, st);
             if (rc) return rc;
         }
+        done = head;
+    }
+    if (T > done) {   // position S0 + done is the start of a group
+        const int n_groups = (T - done) / G;
+        if (n_groups > 0) {
+            rc = quantize_groups(p, *cache, k + (int64_t)done * stride_t, v + (int64_t)done * stride_t, S0 + done, n_groups, stride_b,
+                                 stride_h, stride_t, true, st);
+            if (rc) return rc;
+        }
+        rc = launch_quantize_tokens(p, *cache, k, v, done + n_groups * G, S0 + done + n_groups * G, T - done - n_groups * G, stride_b,
+                                    stride_h, stride_t, st);
+        if (rc) return rc;
     }
     cache->seq_len = S0 + T;
     return KVSINK_OK;

@@ -44,6 +44,34 @@ def test_appends_across_a_group_boundary():
     assert r["gpu_cache"].seq_len == 98
 
 
+@pytest.mark.parametrize("bits,group,chunks", [(2, 32, (50, 7, 1, 70, 33)), (4, 64, (10, 200, 5, 59, 1, 64)), (3, 64, (63, 1, 64, 65)),
+                                               (2, 128, (100, 300, 28, 84))])
+def test_chunked_prefill(bits, group, chunks):
+    # chunks that start and end inside key groups, complete open groups, and span several groups: every state equals
+    # the oracle's token-by-token cache
+    total = sum(chunks)
+    wl = TINY.scaled(seq=total, group=group, bits=bits, head_dim=128, n_q_heads=4, n_kv_heads=2, batch=2, topk=6, pfn_n=2, seed=31 + bits + group)
+    ocfg, gcfg = configs(wl)
+    H = synth.make_hidden(wl, "cuda")
+    K, V = synth.make_kv(wl, 0, "cuda")
+    gs = kv.SinkSet(gcfg)
+    kv.predict_sinks(gcfg, H, gs)
+    gc = kv.KVCache(gcfg, gs)
+    bm, pos, cnt = oracle.predict_sinks(ocfg, np16(H))
+    oc = oracle.Cache(ocfg, bm, pos, cnt)
+    at = 0
+    for n in chunks:
+        kv.quantize_append(gcfg, gc, K[:, :, at:at + n], V[:, :, at:at + n])
+        oracle.quantize_append(ocfg, oc, np16(K[:, :, at:at + n]), np16(V[:, :, at:at + n]))
+        at += n
+        compare_cache(gc, oc, wl, f"after {at} tokens: ")
+    q = synth.make_query(wl, K)
+    out, _ = kv.decode_attention(gcfg, gc, q)
+    ref, _ = oracle.decode_attention(ocfg, oc, np16(q))
+    assert_close(out.cpu().numpy(), ref, "attention")
+    assert kv.read_status(gc) == 0
+
+
 def test_append_from_an_empty_cache():
     wl = TINY.scaled(seq=0, topk=0, pfn_n=0, group=16, bits=4, batch=1, seed=6)
     ocfg, gcfg = configs(wl, 64)
