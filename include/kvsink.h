@@ -183,6 +183,33 @@ int kvsink_decode_attention(const kvsink_config *cfg, const kvsink_cache *cache,
 int kvsink_decode_attention_static(const kvsink_config *cfg, const kvsink_cache *cache, const void *q, float *out, float *lse,
                                    void *cuda_stream);
 
+/*
+ * Largest magnitude of every hidden channel over all tokens of all sequences: out[c] = max |hidden[b][i][c]| (a NaN
+ * never raises a maximum).  This is the scan from which a model's outlier channels -- the `channels` of kvsink_config --
+ * and the layer where they emerge are read off (Section 3.1; Appendix D, the table of emergence layers and outlier
+ * channels): the few channels whose maximum stands orders of magnitude above the rest.
+ *   hidden   device, fp16, element (b, i, c) at hidden + b*stride_b + i*stride_s + c (strides in elements).
+ *   out      device out, float [d], every entry rewritten.
+ */
+int kvsink_channel_absmax(const void *hidden, int32_t B, int32_t S, int32_t d, int64_t stride_b, int64_t stride_s, float *out,
+                          void *cuda_stream);
+
+/*
+ * Quantization error in the shape of the paper's error table (Section 4.1, Table 1): round-to-nearest asymmetric
+ * quantization (Eq. 8-11) of x, squared error against the dequantised value (Eq. 9), summed separately over the
+ * quantization groups without a sink token and over those with at least one.
+ *   x              device, fp16 [B][Hkv][T][D] with element strides (multiples of 8), 0 <= T <= max_seq.
+ *   per_channel    nonzero: groups of G consecutive tokens of one channel (a last shorter group takes the rest);
+ *                  zero: groups of min(G, D) consecutive channels of one token.
+ *   exclude_sinks  zero: plain quantization, every token takes part in its group's min / max (the table's dynamic rows);
+ *                  nonzero: sink tokens take no part in the statistics and are not quantized or counted (KVSink).
+ *   sink_bitmask   device, uint32 [B][ceil(max_seq/32)].
+ *   out            device out, double [4]: sum of squared errors and element count over groups without a sink token,
+ *                  then the same over groups with one.  Sums are accumulated in binary64 in no fixed order.
+ */
+int kvsink_quant_error(const kvsink_config *cfg, const void *x, int32_t T, int64_t stride_b, int64_t stride_h, int64_t stride_t,
+                       int32_t per_channel, int32_t exclude_sinks, const uint32_t *sink_bitmask, double *out, void *cuda_stream);
+
 /* Copies the device status word to *host_status and waits for the stream (the only call that synchronises). */
 int kvsink_read_status(const kvsink_cache *cache, int32_t *host_status, void *cuda_stream);
 

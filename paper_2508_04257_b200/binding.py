@@ -16,7 +16,8 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _LIB_PATH = os.path.join(_HERE, "libkvsink.so")
 
 EXPORTS = ("kvsink_cache_sizes", "kvsink_predict_sinks", "kvsink_quantize_append", "kvsink_decode_attention",
-           "kvsink_decode_attention_static", "kvsink_read_status", "kvsink_launch_count", "kvsink_strerror")
+           "kvsink_decode_attention_static", "kvsink_channel_absmax", "kvsink_quant_error", "kvsink_read_status",
+           "kvsink_launch_count", "kvsink_strerror")
 STATIC_SCRATCH_BYTES = 4 * 1024 * 1024
 
 
@@ -193,6 +194,32 @@ def decode_attention_static(cfg: Config, cache: KVCache, q: torch.Tensor, out: t
     if rc:
         raise KvsinkError(rc, "kvsink_decode_attention_static")
     return out, lse
+
+
+def channel_absmax(hidden: torch.Tensor, out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """kvsink_channel_absmax: hidden fp16 [B, S, d] on the device (last axis contiguous) -> float32 [d]."""
+    assert hidden.is_cuda and hidden.dtype == torch.float16 and hidden.dim() == 3 and hidden.stride(2) == 1
+    if out is None:
+        out = torch.empty(hidden.shape[2], dtype=torch.float32, device=hidden.device)
+    rc = lib().kvsink_channel_absmax(_ptr(hidden), C.c_int32(hidden.shape[0]), C.c_int32(hidden.shape[1]), C.c_int32(hidden.shape[2]),
+                                     C.c_int64(hidden.stride(0)), C.c_int64(hidden.stride(1)), _ptr(out), _stream())
+    if rc:
+        raise KvsinkError(rc, "kvsink_channel_absmax")
+    return out
+
+
+def quant_error(cfg: Config, x: torch.Tensor, sinks: SinkSet, per_channel: bool, exclude_sinks: bool,
+                out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """kvsink_quant_error: x fp16 [B, Hkv, T, D] on the device -> float64 [4] (sum sq err, count) without / with sink tokens."""
+    assert x.is_cuda and x.dtype == torch.float16 and x.dim() == 4 and x.stride(3) == 1
+    if out is None:
+        out = torch.empty(4, dtype=torch.float64, device=x.device)
+    rc = lib().kvsink_quant_error(C.byref(cfg.c()), _ptr(x), C.c_int32(x.shape[2]), C.c_int64(x.stride(0)), C.c_int64(x.stride(1)),
+                                  C.c_int64(x.stride(2)), C.c_int32(int(per_channel)), C.c_int32(int(exclude_sinks)), _ptr(sinks.bitmask),
+                                  _ptr(out), _stream())
+    if rc:
+        raise KvsinkError(rc, "kvsink_quant_error")
+    return out
 
 
 def launch_count() -> int:

@@ -172,6 +172,26 @@ extern "C" int kvsink_decode_attention_static(const kvsink_config *cfg, const kv
     return launch_decode_static(p, *cache, (const __half *)q, out, lse, (cudaStream_t)cuda_stream);
 }
 
+extern "C" int kvsink_channel_absmax(const void *hidden, int32_t B, int32_t S, int32_t d, int64_t stride_b, int64_t stride_s, float *out,
+                                     void *cuda_stream)
+{
+    if (!out || B < 0 || S < 0 || d < 1 || stride_b < 0) return KVSINK_ERR_BAD_ARG;
+    if ((long long)B * S > 0 && (!hidden || stride_s < d)) return KVSINK_ERR_BAD_ARG;   // no tokens: nothing is read
+    return launch_channel_absmax((const __half *)hidden, B, S, d, stride_b, stride_s, out, (cudaStream_t)cuda_stream);
+}
+
+extern "C" int kvsink_quant_error(const kvsink_config *cfg, const void *x, int32_t T, int64_t stride_b, int64_t stride_h, int64_t stride_t,
+                                  int32_t per_channel, int32_t exclude_sinks, const uint32_t *sink_bitmask, double *out, void *cuda_stream)
+{
+    Params p;
+    int rc = derive(cfg, &p);
+    if (rc) return rc;
+    if (!aligned16(x) || !sink_bitmask || !out || ((uintptr_t)out & 7u) || T < 0 || T > p.max_seq) return KVSINK_ERR_BAD_ARG;
+    if (stride_t < p.D || (stride_t % 8) || (stride_h % 8) || (stride_b % 8) || stride_h < 0 || stride_b < 0) return KVSINK_ERR_BAD_ARG;
+    return launch_quant_error(p, (const __half *)x, T, stride_b, stride_h, stride_t, per_channel != 0, exclude_sinks != 0, sink_bitmask, out,
+                              (cudaStream_t)cuda_stream);
+}
+
 extern "C" int kvsink_read_status(const kvsink_cache *cache, int32_t *host_status, void *cuda_stream)
 {
     if (!cache || !cache->status || !host_status) return KVSINK_ERR_BAD_ARG;

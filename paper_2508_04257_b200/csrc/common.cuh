@@ -147,6 +147,9 @@ int launch_decode_b4(const Params &p, const kvsink_cache &c, const __half *q, fl
 int launch_decode_merge(const float *ws, int nsplit, int D, int n_rows, float *out, float *lse, cudaStream_t st);
 int max_splits(const Params &p);
 int choose_splits(const Params &p, int n_groups);
+int launch_channel_absmax(const __half *hidden, int B, int S, int d, int64_t sb, int64_t ss, float *out, cudaStream_t st);
+int launch_quant_error(const Params &p, const __half *x, int T, int64_t sb, int64_t sh, int64_t stt, bool per_channel, bool exclude_sinks,
+                       const uint32_t *bitmask, double *out, cudaStream_t st);
 size_t decode_workspace_bytes(const Params &p);
 size_t predict_workspace_bytes(const Params &p);
 
