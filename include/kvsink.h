@@ -102,7 +102,8 @@ typedef struct kvsink_sizes {
     int64_t k_tail_halfs, sink_halfs;       /* fp16 elements; sink_halfs for each of sink_k, sink_v */
     int64_t bitmask_words, sink_pos_ints;
     int64_t predict_workspace_bytes;        /* for kvsink_predict_sinks with S == max_seq */
-    int64_t decode_workspace_bytes;         /* for kvsink_decode_attention */
+    int64_t decode_workspace_bytes;         /* for kvsink_decode_attention and kvsink_decode_attention_calibrated */
+    int64_t calibrate_workspace_bytes;      /* for kvsink_calibrate */
     int32_t sink_capacity, v_group, v_groups_per_row, tile_bytes;
 } kvsink_sizes;
 
@@ -182,6 +183,49 @@ int kvsink_decode_attention(const kvsink_config *cfg, const kvsink_cache *cache,
  */
 int kvsink_decode_attention_static(const kvsink_config *cfg, const kvsink_cache *cache, const void *q, float *out, float *lse,
                                    void *cuda_stream);
+
+/*
+ * Static (calibrated) parameters: the scheme of the paper's main comparison -- keys per channel, values per token, static
+ * (Section 5.1) -- with sink tokens left out of the calibration as well as of the quantization (Algorithm 1's remark on
+ * calibration; Section 4.1; Appendix C "Dynamic and static quantization").  One (scale, zero) pair per key channel and one
+ * per value channel group of every KV head serves every token of every sequence.  All four arrays are device memory owned
+ * by the caller: k_scale, k_zero float [Hkv][D]; v_scale, v_zero float [Hkv][D / min(G, D)].
+ */
+typedef struct kvsink_static_params {
+    float *k_scale, *k_zero;
+    float *v_scale, *v_zero;
+} kvsink_static_params;
+
+/*
+ * Calibration: global min / max (the caption of the paper's error table) of every key channel and every value channel
+ * group over a calibration batch, all sequences and all tokens whose mask bit is clear, then Eq. 10-11 (a single value
+ * takes scale = |min|, or 1 for 0; no member at all takes scale = zero = 0).
+ *   k_cal, v_cal  device, fp16 [B][Hkv][T][D] with element strides (multiples of 8), 0 <= T <= max_seq.
+ *   sink_bitmask  device, uint32 [B][ceil(max_seq/32)]: the calibration batch's sink tokens (kvsink_predict_sinks).
+ *   params        the four arrays of *params are rewritten.
+ *   workspace     device scratch of at least kvsink_sizes.calibrate_workspace_bytes, 16-byte aligned.
+ */
+int kvsink_calibrate(const kvsink_config *cfg, const void *k_cal, const void *v_cal, int32_t T, int64_t stride_b, int64_t stride_h,
+                     int64_t stride_t, const uint32_t *sink_bitmask, const kvsink_static_params *params, void *workspace,
+                     size_t workspace_bytes, void *cuda_stream);
+
+/*
+ * kvsink_quantize_append with static parameters (Eq. 6, Eq. 8): every token is coded on arrival, keys per channel and
+ * values per channel group, as clamp(rint(x/scale) + zero, 0, 2^bits - 1) -- values outside the calibrated range clamp, a
+ * pair with scale 0 gives code 0; tokens whose mask bit is set keep exact fp16 rows in the side buffer and code 0.  There is
+ * no key tail and there are no per-group parameters: cache->k_scale, k_zero, v_scale, v_zero and k_tail are not used and
+ * may be null.  Any T >= 0 at any time.  A cache is used with one kind of parameters only.
+ */
+int kvsink_quantize_append_calibrated(const kvsink_config *cfg, kvsink_cache *cache, const kvsink_static_params *params, const void *k_new,
+                                      const void *v_new, int32_t T, int64_t stride_b, int64_t stride_h, int64_t stride_t, void *cuda_stream);
+
+/*
+ * kvsink_decode_attention over a cache written by kvsink_quantize_append_calibrated (Eq. 3, Eq. 7): a sink token's K and V
+ * are its fp16 side-buffer rows, every other token's are scale * (code - zero) with the static pairs.  Head size 128 with
+ * one or two value groups per row; other shapes return KVSINK_ERR_UNSUPPORTED.
+ */
+int kvsink_decode_attention_calibrated(const kvsink_config *cfg, const kvsink_cache *cache, const kvsink_static_params *params, const void *q,
+                                       float *out, float *lse, void *workspace, size_t workspace_bytes, void *cuda_stream);
 
 /*
  * Largest magnitude of every hidden channel over all tokens of all sequences: out[c] = max |hidden[b][i][c]| (a NaN

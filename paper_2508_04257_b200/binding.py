@@ -16,7 +16,8 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _LIB_PATH = os.path.join(_HERE, "libkvsink.so")
 
 EXPORTS = ("kvsink_cache_sizes", "kvsink_predict_sinks", "kvsink_quantize_append", "kvsink_decode_attention",
-           "kvsink_decode_attention_static", "kvsink_channel_absmax", "kvsink_quant_error", "kvsink_read_status",
+           "kvsink_decode_attention_static", "kvsink_calibrate", "kvsink_quantize_append_calibrated",
+           "kvsink_decode_attention_calibrated", "kvsink_channel_absmax", "kvsink_quant_error", "kvsink_read_status",
            "kvsink_launch_count", "kvsink_strerror")
 STATIC_SCRATCH_BYTES = 4 * 1024 * 1024
 
@@ -42,7 +43,7 @@ class _Cache(C.Structure):
 class _Sizes(C.Structure):
     _fields_ = [(n, C.c_int64) for n in ("k_codes_bytes", "v_codes_bytes", "k_param_floats", "v_param_floats",
                                          "k_tail_halfs", "sink_halfs", "bitmask_words", "sink_pos_ints",
-                                         "predict_workspace_bytes", "decode_workspace_bytes")] + \
+                                         "predict_workspace_bytes", "decode_workspace_bytes", "calibrate_workspace_bytes")] + \
                [(n, C.c_int32) for n in ("sink_capacity", "v_group", "v_groups_per_row", "tile_bytes")]
 
 
@@ -193,6 +194,69 @@ def decode_attention_static(cfg: Config, cache: KVCache, q: torch.Tensor, out: t
     rc = lib().kvsink_decode_attention_static(C.byref(cfg.c()), C.byref(cc), _ptr(q), _ptr(out), _ptr(lse), _stream())
     if rc:
         raise KvsinkError(rc, "kvsink_decode_attention_static")
+    return out, lse
+
+
+class _Static(C.Structure):
+    _fields_ = [("k_scale", C.c_void_p), ("k_zero", C.c_void_p), ("v_scale", C.c_void_p), ("v_zero", C.c_void_p)]
+
+
+class StaticParams:
+    """Device buffers of calibrated parameters: keys float32 [Hkv, D], values float32 [Hkv, D / v_group]."""
+
+    def __init__(self, cfg: Config, device="cuda"):
+        ngv = cfg.head_dim // min(cfg.group, cfg.head_dim)
+        z = lambda *shape: torch.zeros(shape, dtype=torch.float32, device=device)
+        self.k_scale, self.k_zero = z(cfg.n_kv_heads, cfg.head_dim), z(cfg.n_kv_heads, cfg.head_dim)
+        self.v_scale, self.v_zero = z(cfg.n_kv_heads, ngv), z(cfg.n_kv_heads, ngv)
+
+    def c(self) -> _Static:
+        return _Static(_ptr(self.k_scale), _ptr(self.k_zero), _ptr(self.v_scale), _ptr(self.v_zero))
+
+
+def calibrate(cfg: Config, k_cal: torch.Tensor, v_cal: torch.Tensor, sinks: SinkSet, params: Optional[StaticParams] = None) -> StaticParams:
+    """kvsink_calibrate: k_cal, v_cal fp16 [B, Hkv, T, D] on the device; sinks = the batch's sink set."""
+    assert k_cal.is_cuda and k_cal.dtype == torch.float16 and k_cal.dim() == 4 and k_cal.stride(3) == 1
+    assert v_cal.shape == k_cal.shape and v_cal.stride() == k_cal.stride() and v_cal.dtype == torch.float16
+    if params is None:
+        params = StaticParams(cfg, k_cal.device)
+    ws = torch.empty(cache_sizes(cfg)["calibrate_workspace_bytes"], dtype=torch.uint8, device=k_cal.device)
+    cs = params.c()
+    rc = lib().kvsink_calibrate(C.byref(cfg.c()), _ptr(k_cal), _ptr(v_cal), C.c_int32(k_cal.shape[2]), C.c_int64(k_cal.stride(0)),
+                                C.c_int64(k_cal.stride(1)), C.c_int64(k_cal.stride(2)), _ptr(sinks.bitmask), C.byref(cs), _ptr(ws),
+                                C.c_size_t(ws.numel()), _stream())
+    if rc:
+        raise KvsinkError(rc, "kvsink_calibrate")
+    return params
+
+
+def quantize_append_calibrated(cfg: Config, cache: KVCache, params: StaticParams, k_new: torch.Tensor, v_new: torch.Tensor) -> None:
+    """kvsink_quantize_append_calibrated: k_new, v_new fp16 [B, Hkv, T, D] on the device with equal strides."""
+    assert k_new.is_cuda and k_new.dtype == torch.float16 and k_new.dim() == 4 and k_new.stride(3) == 1
+    assert v_new.shape == k_new.shape and v_new.stride() == k_new.stride() and v_new.dtype == torch.float16
+    cc, cs = cache.c(), params.c()
+    rc = lib().kvsink_quantize_append_calibrated(C.byref(cfg.c()), C.byref(cc), C.byref(cs), _ptr(k_new), _ptr(v_new), C.c_int32(k_new.shape[2]),
+                                                 C.c_int64(k_new.stride(0)), C.c_int64(k_new.stride(1)), C.c_int64(k_new.stride(2)), _stream())
+    if rc:
+        raise KvsinkError(rc, "kvsink_quantize_append_calibrated")
+    cache.seq_len = cc.seq_len
+
+
+def decode_attention_calibrated(cfg: Config, cache: KVCache, params: StaticParams, q: torch.Tensor, out: Optional[torch.Tensor] = None,
+                                lse: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None, want_lse: bool = True):
+    """kvsink_decode_attention_calibrated: q fp16 [B, Hq, D] contiguous. Returns (out fp32 [B,Hq,D], lse fp32 [B,Hq] or None)."""
+    assert q.is_cuda and q.dtype == torch.float16 and q.is_contiguous()
+    if out is None:
+        out = torch.empty((cfg.batch, cfg.n_q_heads, cfg.head_dim), dtype=torch.float32, device=q.device)
+    if lse is None and want_lse:
+        lse = torch.empty((cfg.batch, cfg.n_q_heads), dtype=torch.float32, device=q.device)
+    if workspace is None:
+        workspace = torch.empty(cache.sizes["decode_workspace_bytes"], dtype=torch.uint8, device=q.device)
+    cc, cs = cache.c(), params.c()
+    rc = lib().kvsink_decode_attention_calibrated(C.byref(cfg.c()), C.byref(cc), C.byref(cs), _ptr(q), _ptr(out), _ptr(lse), _ptr(workspace),
+                                                  C.c_size_t(workspace.numel()), _stream())
+    if rc:
+        raise KvsinkError(rc, "kvsink_decode_attention_calibrated")
     return out, lse
 
 

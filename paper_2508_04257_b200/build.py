@@ -15,7 +15,7 @@ CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(HERE, "_build")
 LIB = os.path.join(HERE, "libkvsink.so")
 HEADER = os.path.join(os.path.dirname(HERE), "include", "kvsink.h")
-SOURCES = ["api.cu", "predict.cu", "quantize.cu", "quantize_groups.cu", "quantize_bulk.cu", "decode.cu", "decode_b2.cu", "decode_b3.cu", "decode_b4.cu", "analysis.cu"]
+SOURCES = ["api.cu", "predict.cu", "quantize.cu", "quantize_groups.cu", "quantize_bulk.cu", "decode.cu", "decode_b2.cu", "decode_b3.cu", "decode_b4.cu", "analysis.cu", "calibrated.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++17", "-lineinfo", "-Xcompiler", "-fPIC"]
 
 

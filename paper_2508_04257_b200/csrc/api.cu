@@ -79,6 +79,7 @@ extern "C" int kvsink_cache_sizes(const kvsink_config *cfg, kvsink_sizes *out)
     out->sink_pos_ints = (int64_t)p.B * p.cap;
     out->predict_workspace_bytes = (int64_t)predict_workspace_bytes(p);
     out->decode_workspace_bytes = (int64_t)decode_workspace_bytes(p);
+    out->calibrate_workspace_bytes = (int64_t)calibrate_workspace_bytes(p);
     out->sink_capacity = p.cap;
     out->v_group = p.Gv;
     out->v_groups_per_row = p.NGv;
@@ -156,7 +157,7 @@ extern "C" int kvsink_decode_attention(const kvsink_config *cfg, const kvsink_ca
     if (rc) return rc;
     if (!aligned16(q) || !aligned16(out)) return KVSINK_ERR_BAD_ARG;
     if (!aligned16(workspace)) return KVSINK_ERR_WORKSPACE;
-    return launch_decode(p, *cache, (const __half *)q, out, lse, workspace, workspace_bytes, (cudaStream_t)cuda_stream);
+    return launch_decode(p, *cache, nullptr, (const __half *)q, out, lse, workspace, workspace_bytes, (cudaStream_t)cuda_stream);
 }
 
 extern "C" int kvsink_decode_attention_static(const kvsink_config *cfg, const kvsink_cache *cache, const void *q, float *out,
@@ -170,6 +171,68 @@ extern "C" int kvsink_decode_attention_static(const kvsink_config *cfg, const kv
     if (rc) return rc;
     if (!aligned16(q) || !aligned16(out)) return KVSINK_ERR_BAD_ARG;
     return launch_decode_static(p, *cache, (const __half *)q, out, lse, (cudaStream_t)cuda_stream);
+}
+
+// A cache used with static parameters: the per-group parameter arrays and the key tail are not used and may be null.
+static int check_cache_calibrated(const kvsink_cache *c, const kvsink_static_params *sp, const Params &p)
+{
+    if (!c || !sp) return KVSINK_ERR_BAD_ARG;
+    if (!aligned16(c->k_codes) || !aligned16(c->v_codes) || !aligned16(c->sink_bitmask) || !c->sink_count || !c->status) return KVSINK_ERR_BAD_ARG;
+    if (p.cap > 0 && (!aligned16(c->sink_k) || !aligned16(c->sink_v) || !c->sink_pos)) return KVSINK_ERR_BAD_ARG;
+    if (!sp->k_scale || !sp->k_zero || !sp->v_scale || !sp->v_zero) return KVSINK_ERR_BAD_ARG;
+    if (c->seq_len < 0 || c->seq_len > p.max_seq) return KVSINK_ERR_BAD_ARG;
+    return KVSINK_OK;
+}
+
+extern "C" int kvsink_calibrate(const kvsink_config *cfg, const void *k_cal, const void *v_cal, int32_t T, int64_t stride_b, int64_t stride_h,
+                                int64_t stride_t, const uint32_t *sink_bitmask, const kvsink_static_params *params, void *workspace,
+                                size_t workspace_bytes, void *cuda_stream)
+{
+    Params p;
+    int rc = derive(cfg, &p);
+    if (rc) return rc;
+    if (!params || !params->k_scale || !params->k_zero || !params->v_scale || !params->v_zero || !sink_bitmask) return KVSINK_ERR_BAD_ARG;
+    if (T < 0 || T > p.max_seq) return KVSINK_ERR_BAD_ARG;
+    if (T > 0 && (!aligned16(k_cal) || !aligned16(v_cal))) return KVSINK_ERR_BAD_ARG;
+    if (stride_t < p.D || (stride_t % 8) || (stride_h % 8) || (stride_b % 8) || stride_h < 0 || stride_b < 0) return KVSINK_ERR_BAD_ARG;
+    if (!aligned16(workspace) || workspace_bytes < calibrate_workspace_bytes(p)) return KVSINK_ERR_WORKSPACE;
+    return launch_calibrate(p, (const __half *)k_cal, (const __half *)v_cal, T, stride_b, stride_h, stride_t, sink_bitmask, *params, workspace,
+                            (cudaStream_t)cuda_stream);
+}
+
+extern "C" int kvsink_quantize_append_calibrated(const kvsink_config *cfg, kvsink_cache *cache, const kvsink_static_params *params,
+                                                 const void *k_new, const void *v_new, int32_t T, int64_t stride_b, int64_t stride_h,
+                                                 int64_t stride_t, void *cuda_stream)
+{
+    Params p;
+    int rc = derive(cfg, &p);
+    if (rc) return rc;
+    rc = check_cache_calibrated(cache, params, p);
+    if (rc) return rc;
+    if (T < 0) return KVSINK_ERR_BAD_ARG;
+    if (T == 0) return KVSINK_OK;
+    if (!aligned16(k_new) || !aligned16(v_new)) return KVSINK_ERR_BAD_ARG;
+    if (stride_t < p.D || (stride_t % 8) || (stride_h % 8) || (stride_b % 8) || stride_h < 0 || stride_b < 0) return KVSINK_ERR_BAD_ARG;
+    if ((int64_t)cache->seq_len + T > p.max_seq) return KVSINK_ERR_SEQ_OVERFLOW;
+    rc = launch_quantize_calibrated(p, *cache, *params, (const __half *)k_new, (const __half *)v_new, cache->seq_len, T, stride_b, stride_h,
+                                    stride_t, (cudaStream_t)cuda_stream);
+    if (rc) return rc;
+    cache->seq_len += T;
+    return KVSINK_OK;
+}
+
+extern "C" int kvsink_decode_attention_calibrated(const kvsink_config *cfg, const kvsink_cache *cache, const kvsink_static_params *params,
+                                                  const void *q, float *out, float *lse, void *workspace, size_t workspace_bytes,
+                                                  void *cuda_stream)
+{
+    Params p;
+    int rc = derive(cfg, &p);
+    if (rc) return rc;
+    rc = check_cache_calibrated(cache, params, p);
+    if (rc) return rc;
+    if (!aligned16(q) || !aligned16(out)) return KVSINK_ERR_BAD_ARG;
+    if (!aligned16(workspace)) return KVSINK_ERR_WORKSPACE;
+    return launch_decode(p, *cache, params, (const __half *)q, out, lse, workspace, workspace_bytes, (cudaStream_t)cuda_stream);
 }
 
 extern "C" int kvsink_channel_absmax(const void *hidden, int32_t B, int32_t S, int32_t d, int64_t stride_b, int64_t stride_s, float *out,

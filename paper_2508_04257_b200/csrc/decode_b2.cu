@@ -3,9 +3,10 @@
 
 namespace kvsink {
 
-int launch_decode_b2(const Params &p, const kvsink_cache &c, const __half *q, float *out, float *lse, float *ws, cudaStream_t st)
+int launch_decode_b2(const Params &p, const kvsink_cache &c, const kvsink_static_params *cal, const __half *q, float *out, float *lse, float *ws,
+                     cudaStream_t st)
 {
-    return launch_decode_bits<2>(p, c, q, out, lse, ws, st);
+    return launch_decode_bits<2>(p, c, cal, q, out, lse, ws, st);
 }
 
 }  // namespace kvsink

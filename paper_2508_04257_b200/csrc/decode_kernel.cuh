@@ -213,9 +213,13 @@ struct DecodePlan {
 // MMAs with the same B operands into accumulators of their own.
 // I8 = 2 (two to four query heads per KV head, 2 and 4 bit): the same with two B operands per word, which hold the upper
 // and the lower byte pair of every head's factors in the pair layout's columns.
-template <int BITS, int D, int NGv, int CT, bool PL, int I8 = 0>
+//
+// CAL (static, calibrated parameters): one (scale, zero) per key channel and per value channel group of the KV head for every
+// token.  There are no token groups: the key B operand is prepared once per block, a ring chunk holds code words only, the
+// stream covers every tile up to the sequence length (tokens beyond it are masked) and there is no fp16 tail.
+template <int BITS, int D, int NGv, int CT, bool PL, int I8 = 0, bool CAL = false>
 __global__ void __launch_bounds__(DEC_THREADS, 4)
-decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__restrict__ out, float *__restrict__ lse,
+decode_kernel(Params p, kvsink_cache c, kvsink_static_params sp, const __half *__restrict__ q, float *__restrict__ out, float *__restrict__ lse,
               float *__restrict__ part_ws, int nsplit, int groups_per_split, int qchunks, int seq_len, int cluster_merge)
 {
     using G_ = Geo<BITS, D>;
@@ -234,7 +238,8 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
     const int split = blockIdx.x, h = blockIdx.y / qchunks, qc = blockIdx.y % qchunks, b = blockIdx.z;
     const int nq = I8 == 1 ? 1 : min(NQMAX, p.rep - 8 * qc), hq0 = h * p.rep + 8 * qc;
     const int64_t unit = (int64_t)b * p.Hkv + h;
-    const int G = p.G, n = seq_len, n_groups = n / G, n_body = n_groups * G;
+    // with static parameters a "group" of the loops below is one ring chunk, and every token belongs to one
+    const int G = CAL ? CT * KVSINK_TILE : p.G, n = seq_len, n_groups = CAL ? (n + G - 1) / G : n / G, n_body = CAL ? n : n_groups * G;
     const int TPG = G / KVSINK_TILE, CPG = TPG / CT;                 // tiles and ring chunks per key group
     const uint32_t *bm = c.sink_bitmask + (size_t)b * p.mask_words;
     const float qscale = LOG2E * rsqrtf((float)D);
@@ -414,11 +419,13 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
         const int slot = iss & (NSLOT - 1);
         const uint32_t dst = ring_s + slot * SLOT_BYTES, bar = cbar + 8 * slot;
         if (lane == 0) {
-            mbar_expect_tx(bar, SLOT_BYTES);
+            mbar_expect_tx(bar, CAL ? 2 * KV_BYTES : SLOT_BYTES);
             bulk_g2s(dst, kc_base + iss_kv, KV_BYTES, bar);
             bulk_g2s(dst + KV_BYTES, vc_base + iss_kv, KV_BYTES, bar);
-            bulk_g2s(dst + 2 * KV_BYTES, (const unsigned char *)vs_base + iss_sz, SZ_BYTES, bar);
-            bulk_g2s(dst + 2 * KV_BYTES + SZ_BYTES, (const unsigned char *)vz_base + iss_sz, SZ_BYTES, bar);
+            if constexpr (!CAL) {
+                bulk_g2s(dst + 2 * KV_BYTES, (const unsigned char *)vs_base + iss_sz, SZ_BYTES, bar);
+                bulk_g2s(dst + 2 * KV_BYTES + SZ_BYTES, (const unsigned char *)vz_base + iss_sz, SZ_BYTES, bar);
+            }
         }
         ++iss;
         iss_kv += KV_BYTES;
@@ -440,8 +447,21 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
         return __all_sync(0xffffffffu, ok);
     };
     if (my_groups > 0) {
-        issue_params(0);
+        if (!CAL) issue_params(0);
         for (int i = 0; i < NSLOT - 1 && iss < n_chunks; ++i) issue_chunk();
+    }
+    // static value parameters of the KV head: the same for every token
+    float cal_sv[NGv], cal_zv[NGv];
+#pragma unroll
+    for (int j = 0; j < NGv; ++j) { cal_sv[j] = cal_zv[j] = 0.f; }
+    if constexpr (CAL) {
+        float mx = 0.f;
+#pragma unroll
+        for (int j = 0; j < NGv; ++j) {
+            cal_sv[j] = sp.v_scale[h * NGv + j]; cal_zv[j] = sp.v_zero[h * NGv + j];
+            mx = fmaxf(mx, fabsf(cal_sv[j]));
+        }
+        fit_value_scale(mx);
     }
     // sink bits of the CT tiles starting at tile T: one 32-bit word covers two tiles
     auto load_mask_words = [&](int T) {
@@ -454,24 +474,39 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
     bool stream_ok = true;
     int ci = 0;                                                      // running chunk index of this warp
 
+    // state of the current key group (with static parameters: of the KV head, set up on the first trip)
+    float bias0 = 0.f, bias1 = 0.f, ks0 = 0.f, ks1 = 0.f;
+    uint32_t need_lo = 0;     // bit m: matrix m also gets the low half of the split factor (warp-uniform)
+    uint32_t bk[NM][2];
+#pragma unroll
+    for (int m = 0; m < NM; ++m) bk[m][0] = bk[m][1] = 0u;
 #pragma unroll 1
     for (int gi = 0; gi < my_groups && stream_ok; ++gi) {
         const int grp = w_begin + gi;
         // ---- B operand of the group: fp16(q * scale * 2^sh) per channel and head (sh puts the largest factor of the
         //      head in [2^13, 2^14)), column half pre-divided by COLF; bias = sum_c of the same rounded factors * zero ----
-        float bias0 = 0.f, bias1 = 0.f, ks0 = 0.f, ks1 = 0.f;
-        uint32_t need_lo = 0;     // bit m: matrix m also gets the low half of the split factor (warp-uniform)
+        if (!CAL || gi == 0) {
+        bias0 = bias1 = ks0 = ks1 = 0.f;
+        need_lo = 0;
         {
-            if (!wait_bar(pbar, (unsigned)gi & 1u)) { stream_ok = false; break; }
-            const float *kp = kp_ring;
             float scv[CPL], zev[CPL];
+            if constexpr (CAL) {
 #pragma unroll
-            for (int e = 0; e < CPL; ++e) {
-                const int ch = I8 ? i8_ch[e] : lane * CPL + e;
-                scv[e] = kp[ch]; zev[e] = kp[D + ch];
+                for (int e = 0; e < CPL; ++e) {
+                    const int ch = I8 ? i8_ch[e] : lane * CPL + e;
+                    scv[e] = sp.k_scale[h * D + ch]; zev[e] = sp.k_zero[h * D + ch];
+                }
+            } else {
+                if (!wait_bar(pbar, (unsigned)gi & 1u)) { stream_ok = false; break; }
+                const float *kp = kp_ring;
+#pragma unroll
+                for (int e = 0; e < CPL; ++e) {
+                    const int ch = I8 ? i8_ch[e] : lane * CPL + e;
+                    scv[e] = kp[ch]; zev[e] = kp[D + ch];
+                }
+                __syncwarp();   // the parameters are in registers: the slot can take the next group's while this one streams
+                if (gi + 1 < my_groups) issue_params(gi + 1);
             }
-            __syncwarp();   // the parameters are in registers: the slot can take the next group's while this one streams
-            if (gi + 1 < my_groups) issue_params(gi + 1);
             if constexpr (I8 == 1) {
                 // limbs of the one head's factors: F = rint(q * scale * 2^sh) with the largest |F| in [2^29, 2^30), cut into
                 // four signed bytes (radix 256): every factor is kept to 2^-30 of the group's largest one (2^-26 where the
@@ -608,7 +643,6 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
             }
             __syncwarp();
         }
-        uint32_t bk[NM][2];
         if constexpr (I8 == 2) {
             // B fragments of the four words, first operand (bk[0..3]) and second (bk[4..7]): column g, slots 4t .. 4t + 3
 #pragma unroll
@@ -634,6 +668,7 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
             const bool col_used = PL ? g < 2 * nq : g < nq;
             bk[m][0] = col_used ? *(const uint32_t *)(Bs + g * BST + 16 * m + 2 * t) : 0u;
             bk[m][1] = col_used ? *(const uint32_t *)(Bs + g * BST + 16 * m + 2 * t + 8) : 0u;
+        }
         }
         }
         const float ks0r = ks0 * R1, ks1r = ks1 * R1;
@@ -775,6 +810,16 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
                     if ((mask16 >> (g + 8)) & 1u) s[k][2] = s[k][3] = -INFINITY;
                 }
             }
+            if constexpr (CAL) {
+                if ((T0 + ST) * KVSINK_TILE > n) {   // the last tiles reach beyond the sequence: those tokens do not exist
+#pragma unroll
+                    for (int k = 0; k < ST; ++k) {
+                        const int tok = (T0 + k) * KVSINK_TILE + g;
+                        if (tok >= n) s[k][0] = s[k][1] = -INFINITY;
+                        if (tok + 8 >= n) s[k][2] = s[k][3] = -INFINITY;
+                    }
+                }
+            }
             // one softmax step for the whole chunk
             {
                 float tm0 = fmaxf(s[0][0], s[0][2]), tm1 = fmaxf(s[0][1], s[0][3]);
@@ -784,7 +829,12 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
             }
             // value scales of this lane's tokens; their maximum bounds the fp16 range needed
             float sv0[ST][NGv], zv0[ST][NGv], sv1[ST][NGv], zv1[ST][NGv];
-            {
+            if constexpr (CAL) {
+#pragma unroll
+                for (int k = 0; k < ST; ++k)
+#pragma unroll
+                    for (int j = 0; j < NGv; ++j) { sv0[k][j] = sv1[k][j] = cal_sv[j]; zv0[k][j] = zv1[k][j] = cal_zv[j]; }
+            } else {
                 float mx = 0.f;
 #pragma unroll
                 for (int k = 0; k < ST; ++k)
@@ -808,7 +858,7 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
     if (!stream_ok && lane == 0) atomicOr(c.status, KVSINK_STATUS_TIMEOUT);
 
     // ---- tokens of the open group: keys from the fp16 tail (last split only) ----
-    if (split == nsplit - 1) {
+    if (!CAL && split == nsplit - 1) {
         const __half *tail = (const __half *)c.k_tail + (size_t)unit * G * D;
         const int T_begin = n_body / KVSINK_TILE, T_end = (n + KVSINK_TILE - 1) / KVSINK_TILE;
         for (int T = T_begin + warp; T < T_end; T += DEC_WARPS) {
@@ -992,15 +1042,18 @@ decode_kernel(Params p, kvsink_cache c, const __half *__restrict__ q, float *__r
 }
 
 // ---- launch: one instantiation per (bits, head size, value groups per row, chunk size, key-side variant) ----
-template <int BITS, int D, int NGV, int CT, bool PL, int I8 = 0>
-static int launch_decode_p(const Params &p, const kvsink_cache &c, const __half *q, float *out, float *lse, float *ws, cudaStream_t st)
+template <int BITS, int D, int NGV, int CT, bool PL, int I8 = 0, bool CAL = false>
+static int launch_decode_p(const Params &p, const kvsink_cache &c, const kvsink_static_params *cal, const __half *q, float *out, float *lse, float *ws,
+                           cudaStream_t st)
 {
-    const int n_groups = c.seq_len / p.G;
+    // the units the sequence is split in: key groups, or ring chunks when the parameters are static
+    const int n_groups = CAL ? (c.seq_len + CT * KVSINK_TILE - 1) / (CT * KVSINK_TILE) : c.seq_len / p.G;
+    const kvsink_static_params sp = CAL ? *cal : kvsink_static_params{nullptr, nullptr, nullptr, nullptr};
     const int nsplit = choose_splits(p, n_groups);
     const int gps = n_groups > 0 ? (n_groups + nsplit - 1) / nsplit : 0;
     const int qchunks = (p.rep + 7) / 8;
     const size_t smem = DecodePlan<BITS, D, NGV, CT, I8 == 1 ? 1 : (PL ? 4 : 8)>::BYTES;
-    auto kern = decode_kernel<BITS, D, NGV, CT, PL, I8>;
+    auto kern = decode_kernel<BITS, D, NGV, CT, PL, I8, CAL>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return KVSINK_ERR_CUDA;
     cudaLaunchAttribute pdl[2];
     pdl[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
@@ -1023,7 +1076,7 @@ static int launch_decode_p(const Params &p, const kvsink_cache &c, const __half 
             pdl[1].val.clusterDim.z = 1;
             cfg.numAttrs = 2;
         }
-        if (cudaLaunchKernelEx(&cfg, kern, p, c, q, out, lse, ws, nsplit, gps, qchunks, (int)c.seq_len, (int)cluster_merge) == cudaSuccess) {
+        if (cudaLaunchKernelEx(&cfg, kern, p, c, sp, q, out, lse, ws, nsplit, gps, qchunks, (int)c.seq_len, (int)cluster_merge) == cudaSuccess) {
             note_launch();
             break;
         }
@@ -1035,45 +1088,51 @@ static int launch_decode_p(const Params &p, const kvsink_cache &c, const __half 
     return KVSINK_OK;
 }
 
-template <int BITS, int D, int NGV, int CT>
-static int launch_decode_c(const Params &p, const kvsink_cache &c, const __half *q, float *out, float *lse, float *ws, cudaStream_t st)
+template <int BITS, int D, int NGV, int CT, bool CAL>
+static int launch_decode_c(const Params &p, const kvsink_cache &c, const kvsink_static_params *cal, const __half *q, float *out, float *lse, float *ws,
+                           cudaStream_t st)
 {
     if constexpr (D == 128)
-        if (p.rep == 1) return launch_decode_p<BITS, D, NGV, CT, true, 1>(p, c, q, out, lse, ws, st);
+        if (p.rep == 1) return launch_decode_p<BITS, D, NGV, CT, true, 1, CAL>(p, c, cal, q, out, lse, ws, st);
     if constexpr (D == 128 && BITS != 3)
-        if (p.rep <= 4) return launch_decode_p<BITS, D, NGV, CT, true, 2>(p, c, q, out, lse, ws, st);
-    if (p.rep <= 4) return launch_decode_p<BITS, D, NGV, CT, true>(p, c, q, out, lse, ws, st);
-    return launch_decode_p<BITS, D, NGV, CT, false>(p, c, q, out, lse, ws, st);
+        if (p.rep <= 4) return launch_decode_p<BITS, D, NGV, CT, true, 2, CAL>(p, c, cal, q, out, lse, ws, st);
+    if (p.rep <= 4) return launch_decode_p<BITS, D, NGV, CT, true, 0, CAL>(p, c, cal, q, out, lse, ws, st);
+    return launch_decode_p<BITS, D, NGV, CT, false, 0, CAL>(p, c, cal, q, out, lse, ws, st);
 }
 
-template <int BITS, int D, int NGV>
-static int launch_decode_n(const Params &p, const kvsink_cache &c, const __half *q, float *out, float *lse, float *ws, cudaStream_t st)
+template <int BITS, int D, int NGV, bool CAL>
+static int launch_decode_n(const Params &p, const kvsink_cache &c, const kvsink_static_params *cal, const __half *q, float *out, float *lse, float *ws,
+                           cudaStream_t st)
 {
     // ring chunks of four tiles where a key group divides into them and two slots of that size stay below ~9 KB per
     // warp, else of two tiles (G a multiple of 32), else of one
     if constexpr (4 * (2 * 128 * (D * BITS / 64) + 2 * 16 * NGV * 4) <= 4800)
-        if ((p.G / KVSINK_TILE) % 4 == 0) return launch_decode_c<BITS, D, NGV, 4>(p, c, q, out, lse, ws, st);
-    if ((p.G / KVSINK_TILE) % 2 == 0) return launch_decode_c<BITS, D, NGV, 2>(p, c, q, out, lse, ws, st);
-    return launch_decode_c<BITS, D, NGV, 1>(p, c, q, out, lse, ws, st);
+        if ((p.G / KVSINK_TILE) % 4 == 0) return launch_decode_c<BITS, D, NGV, 4, CAL>(p, c, cal, q, out, lse, ws, st);
+    if ((p.G / KVSINK_TILE) % 2 == 0) return launch_decode_c<BITS, D, NGV, 2, CAL>(p, c, cal, q, out, lse, ws, st);
+    return launch_decode_c<BITS, D, NGV, 1, CAL>(p, c, cal, q, out, lse, ws, st);
 }
 
-template <int BITS, int D>
-static int launch_decode_t(const Params &p, const kvsink_cache &c, const __half *q, float *out, float *lse, float *ws, cudaStream_t st)
+template <int BITS, int D, bool CAL>
+static int launch_decode_t(const Params &p, const kvsink_cache &c, const kvsink_static_params *cal, const __half *q, float *out, float *lse, float *ws,
+                           cudaStream_t st)
 {
-    if (p.NGv == 1) return launch_decode_n<BITS, D, 1>(p, c, q, out, lse, ws, st);
-    if (p.NGv == 2) return launch_decode_n<BITS, D, 2>(p, c, q, out, lse, ws, st);
-    if (p.NGv == 4) return launch_decode_n<BITS, D, 4>(p, c, q, out, lse, ws, st);
+    if (p.NGv == 1) return launch_decode_n<BITS, D, 1, CAL>(p, c, cal, q, out, lse, ws, st);
+    if (p.NGv == 2) return launch_decode_n<BITS, D, 2, CAL>(p, c, cal, q, out, lse, ws, st);
+    if constexpr (!CAL)
+        if (p.NGv == 4) return launch_decode_n<BITS, D, 4, CAL>(p, c, cal, q, out, lse, ws, st);
     return KVSINK_ERR_UNSUPPORTED;
 }
 
-
-// Dispatch over head size for one code width; each width is compiled in a translation unit of its own.
+// Dispatch over head size for one code width; each width is compiled in a translation unit of its own.  `cal` is null
+// for dynamic parameters; static parameters are built for head size 128 with one or two value groups per row.
 template <int BITS>
-static int launch_decode_bits(const Params &p, const kvsink_cache &c, const __half *q, float *out, float *lse, float *ws, cudaStream_t st)
+static int launch_decode_bits(const Params &p, const kvsink_cache &c, const kvsink_static_params *cal, const __half *q, float *out, float *lse,
+                              float *ws, cudaStream_t st)
 {
-    if (p.D == 128) return launch_decode_t<BITS, 128>(p, c, q, out, lse, ws, st);
+    if (cal) return p.D == 128 ? launch_decode_t<BITS, 128, true>(p, c, cal, q, out, lse, ws, st) : KVSINK_ERR_UNSUPPORTED;
+    if (p.D == 128) return launch_decode_t<BITS, 128, false>(p, c, cal, q, out, lse, ws, st);
     if constexpr (BITS != 3)
-        if (p.D == 64) return launch_decode_t<BITS, 64>(p, c, q, out, lse, ws, st);
+        if (p.D == 64) return launch_decode_t<BITS, 64, false>(p, c, cal, q, out, lse, ws, st);
     return KVSINK_ERR_UNSUPPORTED;
 }
 
