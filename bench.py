@@ -385,6 +385,62 @@ class Bench:
         return ms, int(h2d), int(d2h)
 
 
+def calibrated_record(kv, wl, dev, instances, steps, warmup, peak):
+    """The static-parameter variant of a single-layer workload: calibration on the prompt itself, then per instance
+    quantize_append_calibrated(T=S), one appended token and decode_attention_calibrated (kernel times only)."""
+    cfg = kv.Config(wl.batch, wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.hidden, wl.bits, wl.group, wl.max_seq, wl.topk, wl.pfn_n, wl.channels)
+    L = instances
+    H = synth.make_hidden(wl, dev)
+    KV = [synth.make_kv(wl, l, dev) for l in range(L)]
+    new = [synth.make_new_token(wl, l, 0, dev) for l in range(L)]
+    qs = [synth.make_query(wl, KV[l][0], l) for l in range(L)]
+    sinks = kv.SinkSet(cfg, dev)
+    kv.predict_sinks(cfg, H, sinks)
+    caches = [kv.KVCache(cfg, sinks, dev) for _ in range(L)]
+    params = kv.StaticParams(cfg, dev)
+    outs = [torch.empty((wl.batch, wl.n_q_heads, wl.head_dim), dtype=torch.float32, device=dev) for _ in range(L)]
+    ws_d = torch.empty(kv.cache_sizes(cfg)["decode_workspace_bytes"], dtype=torch.uint8, device=dev)
+    ev = {"calibrate": [], "quantize": [], "decode": []}
+
+    def timed(kind, fn, rec):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        fn()
+        b.record()
+        if rec:
+            ev[kind].append((a, b))
+
+    def quantize_all():
+        for l in range(L):
+            caches[l].seq_len = 0
+            kv.quantize_append_calibrated(cfg, caches[l], params, KV[l][0], KV[l][1])
+
+    def decode_all():
+        for l in range(L):
+            kv.decode_attention_calibrated(cfg, caches[l], params, qs[l], outs[l], None, ws_d, want_lse=False)
+
+    for it in range(warmup + steps):
+        rec = it >= warmup
+        timed("calibrate", lambda: kv.calibrate(cfg, KV[0][0], KV[0][1], sinks, params), rec)
+        timed("quantize", quantize_all, rec)
+        for l in range(L):
+            kv.quantize_append_calibrated(cfg, caches[l], params, new[l][0], new[l][1])
+        timed("decode", decode_all, rec)
+    torch.cuda.synchronize()
+    us = {k: sum(a.elapsed_time(b) for a, b in v) * 1e3 / len(v) / (1 if k == "calibrate" else L) for k, v in ev.items()}
+    units, n = wl.batch * wl.n_kv_heads, wl.seq + 1
+    code_bytes = 2 * units * wl.head_dim * wl.bits // 8
+    qb = 2 * units * wl.seq * wl.head_dim * 2 + code_bytes * wl.seq
+    db = code_bytes * n + wl.batch * n // 8 + units * (wl.topk + wl.pfn_n) * wl.head_dim * 4 + wl.batch * wl.n_q_heads * wl.head_dim * 6
+    cb = 2 * units * wl.seq * wl.head_dim * 2
+    gbs = lambda bytes_, t: bytes_ / (t * 1e-6) / 1e9
+    return {"workload": workload_string(wl) + " (static parameters)", "instances_per_step": L, "calibrate_us": us["calibrate"],
+            "quantize_us": us["quantize"], "decode_us": us["decode"], "device_status": kv.read_status(caches[0]),
+            "calibrate": {"algorithmic_bytes": cb, "GBs": gbs(cb, us["calibrate"]), "frac_of_measured_peak": gbs(cb, us["calibrate"]) / peak},
+            "quantize": {"algorithmic_bytes": qb, "GBs": gbs(qb, us["quantize"]), "frac_of_measured_peak": gbs(qb, us["quantize"]) / peak},
+            "decode": {"algorithmic_bytes": db, "GBs": gbs(db, us["decode"]), "frac_of_measured_peak": gbs(db, us["decode"]) / peak}}
+
+
 def workload_record(b: Bench, ms_step, launches, steps, peak, world, agg):
     wl = b.wl
     us = b.kind_us()
@@ -481,6 +537,11 @@ def run_ours(args):
                         L=b.L, e2e=e2e, clocks=sampler.snapshot(), layered=b.layered)
         per[name] = rec
         del b
+        torch.cuda.empty_cache()
+    if not args.workload:
+        # the next scope row: static (calibrated) parameters on the LLaMA2-7B-shaped layer
+        base = synth.WORKLOADS["llama2_7b_layer"]
+        per["llama2_7b_layer_static"] = calibrated_record(kv, base.scaled(seed=dist_util.rank_seed(base.seed, rank)), dev, args.instances, 20, warmup, peak)
         torch.cuda.empty_cache()
     sampler.finish()
 

@@ -178,6 +178,119 @@ quantize_calibrated_kernel(Params p, kvsink_cache c, kvsink_static_params sp, co
     }
 }
 
+// Eq. 8 with fixed parameters without a division per element: r is the rounded reciprocal of the scale, so x * r is within
+// 2^-22 |x / scale| of the quotient; unless it lies that close to a rounding tie, its nearest integer is that of the IEEE
+// quotient.  Near a tie (fp16 inputs hit exact ties often), for huge quotients and for a reciprocal that is not finite the
+// literal formula is evaluated.
+__device__ __forceinline__ uint32_t code_static_fast(float x, float s, float r, float z, float qmax)
+{
+    const float q = x * r, c = rintf(q);
+    const float room = 0.5f - fabsf(q - c);                    // distance to the nearest tie
+    if (!(room > fabsf(q) * 4.76837158203125e-07f)) return code_static(x, s, z, qmax);
+    return (uint32_t)(int)fminf(fmaxf(c + z, 0.f), qmax);
+}
+
+// Whole fresh tiles (a bulk append that starts on a tile boundary): one warp per 16-token tile.  The warp stages the
+// tile's key and value rows in shared memory and every lane codes exactly the elements of its own pair slots of the packed
+// tiles, so the lane's words come out in the tile's own order and are stored with one 16-byte (or 8-byte) store per plane.
+constexpr int CF_WARPS = 4;
+
+template <int BITS>
+__global__ void __launch_bounds__(32 * CF_WARPS)
+quantize_calibrated_tiles_kernel(Params p, kvsink_cache c, kvsink_static_params sp, const __half *__restrict__ k_src,
+                                 const __half *__restrict__ v_src, int first_token, int n_tiles, int64_t sb, int64_t sh, int64_t stt)
+{
+    constexpr int D = 128, W = D * BITS / 64, NLO = BITS == 3 ? D / 32 : W, NHI = BITS == 3 ? D / 64 : 0;
+    constexpr int ROW = D + 8;                                 // padded row (halves): conflict-free column reads
+    __shared__ __align__(16) __half s_k[CF_WARPS][KVSINK_TILE * ROW], s_v[CF_WARPS][KVSINK_TILE * ROW];
+    __shared__ float4 s_kp[D];                                 // (scale, 1 / scale, zero) of the KV head's key channels
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = lane >> 2, t = lane & 3;
+    const int h = blockIdx.y, b = blockIdx.z;
+    const int64_t unit = (int64_t)b * p.Hkv + h;
+    const float qmax = (float)((1 << BITS) - 1);
+    const uint32_t *bm = c.sink_bitmask + (size_t)b * p.mask_words;
+    pdl_wait();
+    for (int i = tid; i < D; i += 32 * CF_WARPS) {
+        const float sc = sp.k_scale[h * D + i];
+        s_kp[i] = make_float4(sc, sc == 0.f ? 0.f : __frcp_rn(sc), sp.k_zero[h * D + i], 0.f);
+    }
+    __syncthreads();
+    const int ti = blockIdx.x * CF_WARPS + warp;               // tile of this append
+    if (ti >= n_tiles) return;
+    const int tok0 = first_token + ti * KVSINK_TILE, src0 = ti * KVSINK_TILE;
+    __half *mk = s_k[warp], *mv = s_v[warp];
+    for (int i = lane; i < KVSINK_TILE * (D / 8); i += 32) {
+        const int r = i / (D / 8), c8 = i % (D / 8);
+        const int64_t off = b * sb + h * sh + (int64_t)(src0 + r) * stt + c8 * 8;
+        *reinterpret_cast<uint4 *>(mk + r * ROW + c8 * 8) = __ldg(reinterpret_cast<const uint4 *>(k_src + off));
+        *reinterpret_cast<uint4 *>(mv + r * ROW + c8 * 8) = __ldg(reinterpret_cast<const uint4 *>(v_src + off));
+    }
+    const uint32_t mask16 = (bm[tok0 >> 5] >> (tok0 & 31)) & 0xffffu;   // sink bits of the tile's tokens
+    __syncwarp();
+    if (mask16) {   // exact rows to the side buffer at the rank of their position
+        const int count = min(c.sink_count[b], p.cap);
+        for (uint32_t rest = mask16; rest; rest &= rest - 1u) {
+            const int r = __ffs((int)rest) - 1;
+            const int slot = find_slot(c.sink_pos + (size_t)b * p.cap, count, tok0 + r);
+            if (slot < 0) {
+                if (lane == 0) atomicOr(c.status, KVSINK_STATUS_SINK_MISMATCH);
+                continue;
+            }
+            __half *dk = (__half *)c.sink_k + ((size_t)unit * p.cap + slot) * D, *dv = (__half *)c.sink_v + ((size_t)unit * p.cap + slot) * D;
+            if (lane < D / 8) {
+                *reinterpret_cast<uint4 *>(dk + lane * 8) = *reinterpret_cast<const uint4 *>(mk + r * ROW + lane * 8);
+                *reinterpret_cast<uint4 *>(dv + lane * 8) = *reinterpret_cast<const uint4 *>(mv + r * ROW + lane * 8);
+            }
+        }
+    }
+    // codes of pair slot s = 4m + r, half e: keys (token, channel) = (g + 8(r&1), 16m + 8(r>>1) + 2t + e),
+    //                                        values (channel, token) = (16m + g + 8(r&1), 8(r>>1) + 2t + e)
+    uint32_t kw[W], vw[W];
+#pragma unroll
+    for (int i = 0; i < W; ++i) kw[i] = vw[i] = 0u;
+#pragma unroll
+    for (int m = 0; m < D / 16; ++m) {
+        const int vj = (16 * m) / p.Gv;   // value channel group of this matrix (groups are multiples of 16 channels)
+        const float vs = sp.v_scale[h * p.NGv + vj], vz = sp.v_zero[h * p.NGv + vj], vr = vs == 0.f ? 0.f : __frcp_rn(vs);
+#pragma unroll
+        for (int r = 0; r < 4; ++r)
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+                const int s_ = 4 * m + r;
+                const int ktok = g + 8 * (r & 1), kch = 16 * m + 8 * (r >> 1) + 2 * t + e;
+                const int vch = 16 * m + g + 8 * (r & 1), vtok = 8 * (r >> 1) + 2 * t + e;
+                const float4 kp = s_kp[kch];
+                const uint32_t kc = ((mask16 >> ktok) & 1u) || kp.x == 0.f ? 0u : code_static_fast(__half2float(mk[ktok * ROW + kch]), kp.x, kp.y, kp.z, qmax);
+                const uint32_t vc = ((mask16 >> vtok) & 1u) || vs == 0.f ? 0u : code_static_fast(__half2float(mv[vtok * ROW + vch]), vs, vr, vz, qmax);
+                if constexpr (BITS == 2) {
+                    kw[s_ / 8] |= kc << (16 * e + 2 * (s_ % 8)); vw[s_ / 8] |= vc << (16 * e + 2 * (s_ % 8));
+                } else if constexpr (BITS == 4) {
+                    kw[s_ / 4] |= kc << (16 * e + 4 * (s_ % 4)); vw[s_ / 4] |= vc << (16 * e + 4 * (s_ % 4));
+                } else {
+                    const int i = s_ / 8, k = s_ % 8, hb = 16 * e + 4 * (k / 2) + 2 * (1 - (i % 2)) + (k % 2);
+                    kw[i] |= (kc & 3u) << (16 * e + 2 * k); vw[i] |= (vc & 3u) << (16 * e + 2 * k);
+                    kw[NLO + i / 2] |= (kc >> 2) << hb; vw[NLO + i / 2] |= (vc >> 2) << hb;
+                }
+            }
+    }
+    // a section of n words per lane is stored as planes of up to four words per lane
+    const size_t tile_off = (size_t)unit * p.max_seq * p.row_bytes + (size_t)(tok0 / KVSINK_TILE) * p.tile_bytes;
+    uint32_t *ko = (uint32_t *)(c.k_codes + tile_off), *vo = (uint32_t *)(c.v_codes + tile_off);
+    auto store_section = [&](uint32_t *dst, const uint32_t *w, int n) {
+        for (int pl = 0; pl * 4 < n; ++pl) {
+            const int u = n - 4 * pl > 4 ? 4 : n - 4 * pl;
+            uint32_t *d = dst + u * lane;
+            if (u == 4) *reinterpret_cast<uint4 *>(d) = make_uint4(w[4 * pl], w[4 * pl + 1], w[4 * pl + 2], w[4 * pl + 3]);
+            else if (u == 2) *reinterpret_cast<uint2 *>(d) = make_uint2(w[4 * pl], w[4 * pl + 1]);
+            else for (int i = 0; i < u; ++i) d[i] = w[4 * pl + i];
+            dst += 32 * u;
+        }
+    };
+    store_section(ko, kw, NLO);
+    store_section(vo, vw, NLO);
+    if constexpr (BITS == 3) { store_section(ko + 32 * NLO, kw + NLO, NHI); store_section(vo + 32 * NLO, vw + NLO, NHI); }
+}
+
 }  // namespace
 
 size_t calibrate_workspace_bytes(const Params &p) { return (size_t)4 * p.Hkv * p.D * sizeof(int) + 16; }
@@ -201,6 +314,18 @@ int launch_quantize_calibrated(const Params &p, const kvsink_cache &c, const kvs
                                int first_token, int n_tokens, int64_t sb, int64_t sh, int64_t stt, cudaStream_t st)
 {
     if (n_tokens <= 0) return KVSINK_OK;
+    // whole fresh tiles of a head-size-128 cache take the tile kernel, the ragged rest (at most 15 tokens) the general one
+    if (p.D == 128 && first_token % KVSINK_TILE == 0 && n_tokens >= KVSINK_TILE && ((uintptr_t)k_src & 15u) == 0 && ((uintptr_t)v_src & 15u) == 0) {
+        const int n_tiles = n_tokens / KVSINK_TILE;
+        const dim3 grid((n_tiles + CF_WARPS - 1) / CF_WARPS, p.Hkv, p.B);
+        cudaError_t e = p.bits == 2 ? launch_pdl(quantize_calibrated_tiles_kernel<2>, grid, dim3(32 * CF_WARPS), 0, st, p, c, sp, k_src, v_src, first_token, n_tiles, sb, sh, stt)
+                      : p.bits == 3 ? launch_pdl(quantize_calibrated_tiles_kernel<3>, grid, dim3(32 * CF_WARPS), 0, st, p, c, sp, k_src, v_src, first_token, n_tiles, sb, sh, stt)
+                                    : launch_pdl(quantize_calibrated_tiles_kernel<4>, grid, dim3(32 * CF_WARPS), 0, st, p, c, sp, k_src, v_src, first_token, n_tiles, sb, sh, stt);
+        if (e != cudaSuccess) return KVSINK_ERR_CUDA;
+        const int done = n_tiles * KVSINK_TILE;
+        return launch_quantize_calibrated(p, c, sp, k_src + (int64_t)done * stt, v_src + (int64_t)done * stt, first_token + done, n_tokens - done, sb, sh,
+                                          stt, st);
+    }
     const int tiles = (first_token + n_tokens - 1) / KVSINK_TILE - first_token / KVSINK_TILE + 1;
     const dim3 grid(tiles, p.Hkv, p.B);
     return launch_pdl(quantize_calibrated_kernel, grid, dim3(CQ_THREADS), 0, st, p, c, sp, k_src, v_src, first_token, n_tokens, sb, sh, stt) ==
