@@ -28,10 +28,11 @@ extern "C" {
 #define KVSINK_ERR_UNSUPPORTED (-3)  /* a valid request this build has no kernel for */
 #define KVSINK_ERR_WORKSPACE (-4)    /* workspace missing or too small */
 #define KVSINK_ERR_SEQ_OVERFLOW (-5) /* seq_len + T > max_seq */
-#define KVSINK_ERR_SINK_OVERFLOW (-6)
+#define KVSINK_ERR_SINK_MISMATCH (-6) /* kvsink_read_status: status bit KVSINK_STATUS_SINK_MISMATCH is set */
 #define KVSINK_ERR_CUDA (-7)         /* a CUDA runtime call failed (launch, attribute, copy) */
-#define KVSINK_ERR_TIMEOUT (-8)
+#define KVSINK_ERR_TIMEOUT (-8)       /* kvsink_read_status: status bit KVSINK_STATUS_TIMEOUT is set */
 #define KVSINK_ERR_STATIC_SCRATCH (-9) /* kvsink_decode_attention_static: the built-in scratch array is too small */
+#define KVSINK_ERR_BOUNDS (-10)       /* kvsink_read_status: status bit KVSINK_STATUS_BOUNDS is set (debug builds only) */
 
 /* Size of the scratch array built into the library for kvsink_decode_attention_static (4 MiB per GPU). */
 #define KVSINK_STATIC_SCRATCH_BYTES (4 * 1024 * 1024)
@@ -39,6 +40,7 @@ extern "C" {
 /* Bits of the device status word (kvsink_cache.status, read with kvsink_read_status). */
 #define KVSINK_STATUS_SINK_MISMATCH 1 /* a token whose mask bit is set was not found in sink_pos */
 #define KVSINK_STATUS_TIMEOUT 2       /* a bounded wait for a shared-memory bulk copy ran out; the result is invalid */
+#define KVSINK_STATUS_BOUNDS 4        /* a library built with -DKVSINK_DEBUG found an index outside its array and skipped the access */
 
 /* Tokens per packed tile. */
 #define KVSINK_TILE 16
@@ -254,7 +256,9 @@ int kvsink_channel_absmax(const void *hidden, int32_t B, int32_t S, int32_t d, i
 int kvsink_quant_error(const kvsink_config *cfg, const void *x, int32_t T, int64_t stride_b, int64_t stride_h, int64_t stride_t,
                        int32_t per_channel, int32_t exclude_sinks, const uint32_t *sink_bitmask, double *out, void *cuda_stream);
 
-/* Copies the device status word to *host_status and waits for the stream (the only call that synchronises). */
+/* Copies the device status word to *host_status and waits for the stream (the only call that synchronises).  Returns
+ * KVSINK_OK for a zero word, else the error code of the most severe raised bit (TIMEOUT, BOUNDS, SINK_MISMATCH);
+ * *host_status holds the word either way. */
 int kvsink_read_status(const kvsink_cache *cache, int32_t *host_status, void *cuda_stream);
 
 /* Kernel launches the library has made in this process since it was loaded (host counter; every entry point adds the

@@ -13,7 +13,8 @@ from typing import Optional, Sequence
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-_LIB_PATH = os.path.join(_HERE, "libkvsink.so")
+# KVSINK_LIB selects another build of the library (the debug build with index checks, for instance)
+_LIB_PATH = os.environ.get("KVSINK_LIB") or os.path.join(_HERE, "libkvsink.so")
 
 EXPORTS = ("kvsink_cache_sizes", "kvsink_predict_sinks", "kvsink_quantize_append", "kvsink_decode_attention",
            "kvsink_decode_attention_static", "kvsink_calibrate", "kvsink_quantize_append_calibrated",
@@ -295,6 +296,6 @@ def read_status(cache: KVCache) -> int:
     host = C.c_int32(0)
     cc = cache.c()
     rc = lib().kvsink_read_status(C.byref(cc), C.byref(host), _stream())
-    if rc:
+    if rc and not host.value:       # a raised status bit comes back as the word itself
         raise KvsinkError(rc, "kvsink_read_status")
     return int(host.value)

@@ -30,12 +30,18 @@ def _older(target: str, deps) -> bool:
     return any(os.path.getmtime(d) > t for d in deps)
 
 
-def build(force: bool = False, verbose: bool = False, defines=()) -> str:
-    """Compiles what is stale and returns the library's path.  `defines` are extra -D macros (they force a rebuild)."""
+DEBUG_LIB = os.path.join(HERE, "libkvsink_debug.so")
+
+
+def build(force: bool = False, verbose: bool = False, debug: bool = False) -> str:
+    """Compiles what is stale and returns the library's path.  debug=True builds libkvsink_debug.so with -DKVSINK_DEBUG:
+    the same kernels with index checks that raise KVSINK_STATUS_BOUNDS instead of touching memory outside an array."""
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
+    OBJ = os.path.join(HERE, "_build_debug" if debug else "_build")
+    LIB = DEBUG_LIB if debug else globals()["LIB"]
+    defines = ("KVSINK_DEBUG",) if debug else ()
     os.makedirs(OBJ, exist_ok=True)
     hdrs = _headers()
-    force = force or bool(defines)
     jobs = []
     for s in SOURCES:
         src, obj = os.path.join(CSRC, s), os.path.join(OBJ, s[:-3] + ".o")
@@ -73,4 +79,4 @@ def build(force: bool = False, verbose: bool = False, defines=()) -> str:
 
 if __name__ == "__main__":
     import sys
-    print(build(force="-f" in sys.argv, verbose="-v" in sys.argv))
+    print(build(force="-f" in sys.argv, verbose="-v" in sys.argv, debug="--debug" in sys.argv))

@@ -261,6 +261,10 @@ extern "C" int kvsink_read_status(const kvsink_cache *cache, int32_t *host_statu
     cudaStream_t st = (cudaStream_t)cuda_stream;
     if (cudaMemcpyAsync(host_status, cache->status, sizeof(int32_t), cudaMemcpyDeviceToHost, st) != cudaSuccess) return KVSINK_ERR_CUDA;
     if (cudaStreamSynchronize(st) != cudaSuccess) return KVSINK_ERR_CUDA;
+    // the word is delivered in any case; a raised bit is also the call's result
+    if (*host_status & KVSINK_STATUS_TIMEOUT) return KVSINK_ERR_TIMEOUT;
+    if (*host_status & KVSINK_STATUS_BOUNDS) return KVSINK_ERR_BOUNDS;
+    if (*host_status & KVSINK_STATUS_SINK_MISMATCH) return KVSINK_ERR_SINK_MISMATCH;
     return KVSINK_OK;
 }
 
@@ -275,9 +279,10 @@ extern "C" const char *kvsink_strerror(int code)
     case KVSINK_ERR_UNSUPPORTED: return "valid request without a kernel in this build";
     case KVSINK_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
     case KVSINK_ERR_SEQ_OVERFLOW: return "appending would exceed max_seq";
-    case KVSINK_ERR_SINK_OVERFLOW: return "more sink tokens than the side buffer holds";
+    case KVSINK_ERR_SINK_MISMATCH: return "a token whose mask bit is set is missing from the position list (status bit SINK_MISMATCH)";
+    case KVSINK_ERR_BOUNDS: return "a debug build caught an index outside its array (status bit BOUNDS)";
     case KVSINK_ERR_CUDA: return "a CUDA runtime call failed";
-    case KVSINK_ERR_TIMEOUT: return "a bounded device wait ran out";
+    case KVSINK_ERR_TIMEOUT: return "a bounded device wait ran out (status bit TIMEOUT): results of that cache are invalid";
     case KVSINK_ERR_STATIC_SCRATCH:
         return "this configuration needs more split scratch than the library's built-in array holds "
                "(KVSINK_STATIC_SCRATCH_BYTES); use kvsink_decode_attention with a caller workspace";

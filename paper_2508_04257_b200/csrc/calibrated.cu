@@ -130,6 +130,7 @@ quantize_calibrated_kernel(Params p, kvsink_cache c, kvsink_static_params sp, co
     const uint32_t *bm = c.sink_bitmask + (size_t)b * p.mask_words;
     if (tid < KVSINK_TILE) present[tid] = (tile * KVSINK_TILE + tid >= t_lo && tile * KVSINK_TILE + tid < t_hi) ? 1 : 0;
     pdl_wait();
+    if (!in_bounds(first_token >= 0 && first_token + n_tokens <= p.max_seq && (tile + 1) * KVSINK_TILE <= p.max_seq, c.status)) return;
 
     const int cpl = D / 32;   // channels per lane (2 or 4)
     float ks[4], kz[4], vs[4], vz[4];
@@ -218,6 +219,7 @@ quantize_calibrated_tiles_kernel(Params p, kvsink_cache c, kvsink_static_params 
     const int ti = blockIdx.x * CF_WARPS + warp;               // tile of this append
     if (ti >= n_tiles) return;
     const int tok0 = first_token + ti * KVSINK_TILE, src0 = ti * KVSINK_TILE;
+    if (!in_bounds(tok0 >= 0 && tok0 + KVSINK_TILE <= p.max_seq, c.status)) return;
     __half *mk = s_k[warp], *mv = s_v[warp];
     for (int i = lane; i < KVSINK_TILE * (D / 8); i += 32) {
         const int r = i / (D / 8), c8 = i % (D / 8);

@@ -125,6 +125,18 @@ __device__ __forceinline__ float ex2(float x)
     return y;
 }
 
+// Index checks of debug builds (-DKVSINK_DEBUG): a failed check raises KVSINK_STATUS_BOUNDS in the cache's status word and
+// returns false, and the caller skips the guarded work; nothing traps.  Release builds compile the condition away.
+#ifdef KVSINK_DEBUG
+__device__ __forceinline__ bool in_bounds(bool ok, int32_t *status)
+{
+    if (!ok) atomicOr(status, KVSINK_STATUS_BOUNDS);
+    return ok;
+}
+#else
+__device__ __forceinline__ bool in_bounds(bool, int32_t *) { return true; }
+#endif
+
 __device__ __forceinline__ bool mask_bit(const uint32_t *__restrict__ bm, int pos) { return (bm[pos >> 5] >> (pos & 31)) & 1u; }
 
 // Launchers implemented in the kernel translation units; all return a KVSINK_* code.

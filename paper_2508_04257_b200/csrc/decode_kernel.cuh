@@ -417,8 +417,10 @@ decode_kernel(Params p, kvsink_cache c, kvsink_static_params sp, const __half *_
     const uint32_t ring_s = smem_addr(ring), kp_s = smem_addr(kp_ring);
     auto issue_chunk = [&]() {
         const int slot = iss & (NSLOT - 1);
+        // debug builds: the chunk must lie inside the unit's code arrays (a skipped copy ends in the wait's time-out)
+        const bool inside = in_bounds((size_t)iss_kv + KV_BYTES <= (size_t)p.max_seq * p.row_bytes, c.status);
         const uint32_t dst = ring_s + slot * SLOT_BYTES, bar = cbar + 8 * slot;
-        if (lane == 0) {
+        if (lane == 0 && inside) {
             mbar_expect_tx(bar, CAL ? 2 * KV_BYTES : SLOT_BYTES);
             bulk_g2s(dst, kc_base + iss_kv, KV_BYTES, bar);
             bulk_g2s(dst + KV_BYTES, vc_base + iss_kv, KV_BYTES, bar);

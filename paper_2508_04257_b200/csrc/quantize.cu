@@ -17,6 +17,7 @@ quantize_groups_kernel(Params p, kvsink_cache c, const __half *__restrict__ k_sr
 {
     extern __shared__ __align__(16) unsigned char smem[];
     const int D = p.D, G = p.G, RS = D + 8;      // padded row stride in halves
+    if (!in_bounds(first_token >= 0 && first_token + ((int)blockIdx.x + 1) * G <= p.max_seq, c.status)) return;   // every thread of the block alike
     __half *Kt = (__half *)smem;                  // [G][RS]
     __half *Vt = Kt + (size_t)G * RS;             // [G][RS]
     uint8_t *kcode = (uint8_t *)(Vt + (size_t)G * RS);   // [G][D]
@@ -182,6 +183,7 @@ quantize_tokens_kernel(Params p, kvsink_cache c, const __half *__restrict__ k_sr
     const uint32_t *bm = c.sink_bitmask + (size_t)b * p.mask_words;
     if (tid < KVSINK_TILE) present[tid] = (tile * KVSINK_TILE + tid >= t_lo && tile * KVSINK_TILE + tid < t_hi) ? 1 : 0;
     pdl_wait();
+    if (!in_bounds(first_token >= 0 && first_token + n_tokens <= p.max_seq && (tile + 1) * KVSINK_TILE <= p.max_seq, c.status)) return;
 
     const int cpl = D / 32;   // channels per lane (2 or 4)
     for (int pos = t_lo + warp; pos < t_hi; pos += QT_THREADS / 32) {
@@ -281,6 +283,7 @@ append_one_kernel(Params p, kvsink_cache c, const __half *__restrict__ k_src, co
     const int64_t unit = (int64_t)blockIdx.x * QA_WARPS + warp;
     pdl_wait();
     if (unit >= (int64_t)p.B * p.Hkv) return;
+    if (!in_bounds(pos >= 0 && pos < p.max_seq, c.status)) return;
     const int b = (int)(unit / p.Hkv), h = (int)(unit % p.Hkv);
     const float qmax = (float)((1 << p.bits) - 1);
     const int cpl = D / 32;   // channels per lane (2 or 4)

@@ -331,6 +331,7 @@ quantize_bulk_kernel(Params p, kvsink_cache c, const __grid_constant__ CUtensorM
     }
     __syncthreads();   // the only block-wide barrier
     pdl_wait();        // nothing before this line touches global memory
+    if (!in_bounds(sh.first_token >= 0 && (long long)sh.first_token + (long long)sh.n_groups * G <= p.max_seq, c.status)) return;   // every thread alike
     if (smem_addr(smem) & 1023u) {   // the swizzle pattern of the stages assumes 1024-byte alignment
         if (tid == 0) atomicOr(c.status, KVSINK_STATUS_TIMEOUT);
         return;
@@ -607,7 +608,6 @@ quantize_bulk_kernel(Params p, kvsink_cache c, const __grid_constant__ CUtensorM
                     const int u = s * MPS + i;
                     const int m = is_v ? (u & 7) : sub * MT + u / NT;   // matrix of the tile
                     uint32_t pc[4];
-#pragma unroll
                     uint32_t differ[4] = {0u, 0u, 0u, 0u};
 #pragma unroll
                     for (int r = 0; r < 4; ++r) pc[r] = qb_code_pair(a[u][r], k_lo[r >> 1], k_hi[r >> 1], k_magic[r >> 1], differ[r]);

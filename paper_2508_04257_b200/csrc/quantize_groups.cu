@@ -226,6 +226,7 @@ quantize_groups_stream(Params p, kvsink_cache c, const __half *__restrict__ k_sr
     constexpr int TILE_WORDS = 32 * W;
     const float qmax = (float)((1 << BITS) - 1);
     const __half2 H_PINF = __half2half2(__ushort_as_half(0x7C00)), H_NINF = __half2half2(__ushort_as_half(0xFC00));
+    if (!in_bounds(first_token >= 0 && (long long)first_token + (long long)n_groups * G <= p.max_seq, c.status)) return;   // every thread alike
 
     extern __shared__ __align__(128) unsigned char smem[];
     __half *Xbuf = (__half *)smem;                                 // [2][G][D] swizzled 16-byte chunks (double buffer)

@@ -63,6 +63,34 @@ def compare_cache(gc: kv.KVCache, oc: oracle.Cache, wl, what=""):
         assert bits_equal(gt, ot), f"{what}k_tail differs"
 
 
+CANARY, PAD = 0xA5, 256
+
+
+def guard(obj, names, device="cuda"):
+    """Moves the named tensors of a cache / sink set into buffers with PAD canary bytes before and after them."""
+    obj._guards = []
+    for name in names:
+        t = getattr(obj, name)
+        nbytes = t.numel() * t.element_size()
+        buf = torch.full((nbytes + 2 * PAD,), CANARY, dtype=torch.uint8, device=device)
+        mid = buf[PAD:PAD + nbytes].view(t.dtype)
+        mid.copy_(t.reshape(-1))
+        setattr(obj, name, mid.view(t.shape))
+        obj._guards.append((name, buf, nbytes))
+    return obj
+
+
+def check_guards(obj):
+    """No kernel wrote past the ends of a guarded buffer."""
+    for name, buf, nbytes in obj._guards:
+        host = buf.cpu().numpy()
+        assert (host[:PAD] == CANARY).all() and (host[PAD + nbytes:] == CANARY).all(), f"write outside {name}"
+
+
+CACHE_BUFFERS = ("k_codes", "v_codes", "k_scale", "k_zero", "v_scale", "v_zero", "k_tail", "sink_k", "sink_v", "status")
+SINK_BUFFERS = ("bitmask", "pos", "count")
+
+
 def run_both(wl: synth.Workload, appends: int = 0, device="cuda", check=True, H=None, K=None, V=None, max_seq=None):
     """Full path on both sides: predict -> prefill quantize -> `appends` single-token appends -> decode attention."""
     ocfg, gcfg = configs(wl, max_seq)
@@ -70,9 +98,9 @@ def run_both(wl: synth.Workload, appends: int = 0, device="cuda", check=True, H=
     if K is None:
         K, V = synth.make_kv(wl, 0, device)
     # GPU
-    gs = kv.SinkSet(gcfg, device)
+    gs = guard(kv.SinkSet(gcfg, device), SINK_BUFFERS, device)
     kv.predict_sinks(gcfg, H, gs)
-    gc = kv.KVCache(gcfg, gs, device)
+    gc = guard(kv.KVCache(gcfg, gs, device), CACHE_BUFFERS, device)
     kv.quantize_append(gcfg, gc, K, V)
     # oracle
     bm, pos, cnt = oracle.predict_sinks(ocfg, np16(H))
@@ -93,6 +121,8 @@ def run_both(wl: synth.Workload, appends: int = 0, device="cuda", check=True, H=
     ref, ref_lse = oracle.decode_attention(ocfg, oc, np16(q))
     torch.cuda.synchronize()
     assert kv.read_status(gc) == 0
+    check_guards(gs)
+    check_guards(gc)
     err = None
     if check:
         err = assert_close(out.cpu().numpy(), ref, "attention output")
