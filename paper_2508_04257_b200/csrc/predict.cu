@@ -1,5 +1,7 @@
 // Sink-token prediction: per-token outlier score, exact per-sequence top-k with index tie-break,
 // Preserve-First-N, bitmask + ascending position list (Algorithm 1 at the emergence layer; Section 4.3).
+#include <cooperative_groups.h>
+
 #include "common.cuh"
 
 namespace kvsink {
@@ -27,10 +29,14 @@ __global__ void sink_score_listed(const uint16_t *__restrict__ H, int S, int64_t
     pdl_wait();
     if (i >= S) return;
     const uint16_t *row = H + b * sb + i * ss;
+    // the listed channels sit in different sectors of a row: all loads are issued before the first one is used
+    uint16_t v[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) v[j] = j < cl.n ? __ldg(row + cl.c[j]) : (uint16_t)0;
     unsigned best = 0;
-#pragma unroll 1
-    for (int j = 0; j < cl.n; ++j) {
-        unsigned a = magnitude_key(__ldg(row + cl.c[j]));
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        const unsigned a = magnitude_key(v[j]);
         best = a > best ? a : best;
     }
     score[(size_t)b * score_stride + i] = (uint16_t)best;
@@ -202,6 +208,150 @@ sink_select(const uint16_t *__restrict__ score, int score_stride, int S, int k, 
     if (tid == 0) sink_count[b] = run_sel < cap ? run_sel : cap;
 }
 
+// Long sequences: the blocks of one thread-block cluster share a sequence.  Block r owns the tokens
+// [r * slice, (r + 1) * slice), slice a multiple of 4096; the blocks add their histograms up through distributed shared
+// memory (both radix passes), count their keys equal to the k-th largest, and take the ranks of their selected tokens from
+// the counts of the blocks before them, so that the result is the one sink_select gives.
+constexpr int SELC_MAX_STEPS = 8;   // 4096-token steps per block
+
+__global__ void __launch_bounds__(SEL_THREADS)
+sink_select_cluster(const uint16_t *__restrict__ score, int score_stride, int S, int k, int N, int mask_words, int cap, int slice,
+                    uint32_t *__restrict__ bitmask, int32_t *__restrict__ sink_pos, int32_t *__restrict__ sink_count)
+{
+    namespace cg = cooperative_groups;
+    cg::cluster_group cl = cg::this_cluster();
+    __shared__ unsigned hist[256], ghist[256];
+    __shared__ unsigned warp_tot[32];
+    __shared__ int s_hi, s_need, s_lo, s_r, s_neq, s_nsel;
+    const int b = blockIdx.y, tid = threadIdx.x, lane = tid & 31;
+    const int rk = (int)cl.block_rank(), C = (int)cl.num_blocks();
+    const uint16_t *sc = score + (size_t)b * score_stride;
+    const int kk = k < S ? k : S;
+    const int lo = min(S, rk * slice), hi = min(S, lo + slice);
+    pdl_wait();
+    int vstar = 0x10000, r = 0;   // no score exceeds 0x10000: no top-k selection when kk == 0
+    if (tid == 0) { s_neq = 0; s_nsel = 0; }
+    if (kk > 0) {
+        // the cluster's histogram of a key byte: every block sums the blocks' histograms for itself
+        auto global_bin = [&](int need, int *bin_out, int *rest_out) {
+            cl.sync();                                  // every block's histogram is complete
+            if (tid < 256) {
+                unsigned g = 0;
+                for (int j = 0; j < C; ++j) g += cl.map_shared_rank(hist, j)[tid];
+                ghist[tid] = g;
+            }
+            __syncthreads();
+            if (tid < 32) find_bin(ghist, need, bin_out, rest_out);
+            cl.sync();                                  // every block has read every histogram: they may be reused
+        };
+        if (tid < 256) hist[tid] = 0;
+        __syncthreads();
+        for (int i = lo + tid; i < hi; i += SEL_THREADS) atomicAdd(&hist[sc[i] >> 8], 1u);
+        global_bin(kk, &s_hi, &s_need);
+        const int hi_byte = s_hi;
+        if (tid < 256) hist[tid] = 0;
+        __syncthreads();
+        for (int i = lo + tid; i < hi; i += SEL_THREADS) {
+            const unsigned v = sc[i];
+            if ((int)(v >> 8) == hi_byte) atomicAdd(&hist[v & 0xffu], 1u);
+        }
+        global_bin(s_need, &s_lo, &s_r);
+        vstar = (hi_byte << 8) | s_lo;
+        r = s_r;
+    }
+    // keys of this block's steps (TPT consecutive tokens per thread and step), kept in registers for both passes below
+    constexpr int TPT = 4, STEP = SEL_THREADS * TPT;
+    uint2 keys[SELC_MAX_STEPS];
+    int my_eq = 0;
+#pragma unroll
+    for (int st = 0; st < SELC_MAX_STEPS; ++st) {
+        const int i0 = lo + st * STEP + TPT * tid;
+        keys[st] = make_uint2(0xffffffffu, 0xffffffffu);          // 0xffff: no token
+        if (st * STEP < slice && i0 < hi) {
+            if (i0 + TPT <= hi) keys[st] = *reinterpret_cast<const uint2 *>(sc + i0);   // rows are 16-byte aligned, i0 a multiple of 4
+            else {
+                unsigned kq[4];
+                for (int j = 0; j < TPT; ++j) kq[j] = i0 + j < hi ? sc[i0 + j] : 0xffffu;
+                keys[st] = make_uint2(kq[0] | (kq[1] << 16), kq[2] | (kq[3] << 16));
+            }
+            // a token slot beyond the sequence carries 0xffff; a real key equal to it is told apart by its index below
+#pragma unroll
+            for (int j = 0; j < TPT; ++j) {
+                const int key = (int)(((j < 2 ? keys[st].x : keys[st].y) >> (16 * (j & 1))) & 0xffffu);
+                my_eq += (i0 + j < hi) && key == vstar;
+            }
+        }
+    }
+    // keys equal to the k-th largest in the blocks before this one
+    if (my_eq) atomicAdd(&s_neq, my_eq);
+    cl.sync();
+    int run_eq = 0;
+    for (int j = 0; j < rk; ++j) run_eq += *cl.map_shared_rank(&s_neq, j);
+    // ordered pass over the block's tokens: selection bits and local ranks
+    unsigned nib[SELC_MAX_STEPS];
+    int lrank[SELC_MAX_STEPS];
+    int run_sel = 0;
+#pragma unroll
+    for (int st = 0; st < SELC_MAX_STEPS; ++st) {
+        nib[st] = 0; lrank[st] = 0;
+        if (st * STEP < slice && lo + st * STEP < hi) {         // block-uniform
+            const int i0 = lo + st * STEP + TPT * tid;
+            int key[TPT], n_eq = 0;
+#pragma unroll
+            for (int j = 0; j < TPT; ++j) {
+                key[j] = i0 + j < hi ? (int)(((j < 2 ? keys[st].x : keys[st].y) >> (16 * (j & 1))) & 0xffffu) : -1;
+                n_eq += key[j] == vstar;
+            }
+            int tot_eq;
+            int eq_rank = run_eq + block_excl_sum(n_eq, &tot_eq, warp_tot);
+            unsigned nb = 0;
+#pragma unroll
+            for (int j = 0; j < TPT; ++j) {
+                const bool eq = key[j] == vstar;
+                const bool sel = i0 + j < hi && (i0 + j < N || key[j] > vstar || (eq && eq_rank < r));
+                eq_rank += eq;
+                nb |= (unsigned)sel << j;
+            }
+            unsigned word = nb << (4 * (lane & 7));           // eight threads share a mask word
+            word |= __shfl_xor_sync(0xffffffffu, word, 1);
+            word |= __shfl_xor_sync(0xffffffffu, word, 2);
+            word |= __shfl_xor_sync(0xffffffffu, word, 4);
+            if ((lane & 7) == 0 && (i0 >> 5) < mask_words) bitmask[(size_t)b * mask_words + (i0 >> 5)] = word;
+            int tot_sel;
+            lrank[st] = run_sel + block_excl_sum(__popc(nb), &tot_sel, warp_tot);
+            nib[st] = nb;
+            run_eq += tot_eq;
+            run_sel += tot_sel;
+        }
+    }
+    if (tid == 0) s_nsel = run_sel;
+    cl.sync();
+    int base = 0, total = 0;
+    for (int j = 0; j < C; ++j) {
+        const int nj = *cl.map_shared_rank(&s_nsel, j);
+        base += j < rk ? nj : 0;
+        total += nj;
+    }
+#pragma unroll
+    for (int st = 0; st < SELC_MAX_STEPS; ++st) {
+        int rank = base + lrank[st];
+        const int i0 = lo + st * STEP + TPT * tid;
+#pragma unroll
+        for (int j = 0; j < TPT; ++j)
+            if ((nib[st] >> j) & 1u) {
+                if (rank < cap) sink_pos[(size_t)b * cap + rank] = i0 + j;
+                ++rank;
+            }
+    }
+    if (rk == C - 1) {    // mask words beyond the last slice, unused positions, the count
+        const int w0 = (min(S, C * slice) + STEP - 1) / STEP * STEP / 32;   // words the ordered pass has written
+        for (int w = w0 + tid; w < mask_words; w += SEL_THREADS) bitmask[(size_t)b * mask_words + w] = 0u;
+        for (int j = total + tid; j < cap; j += SEL_THREADS) sink_pos[(size_t)b * cap + j] = -1;
+        if (tid == 0) sink_count[b] = total < cap ? total : cap;
+    }
+    cl.sync();   // nobody's shared memory goes away while another block reads it
+}
+
 size_t predict_workspace_bytes(const Params &p)
 {
     size_t stride = ((size_t)p.max_seq + 7) / 8 * 8;
@@ -225,6 +375,32 @@ int launch_predict_sinks(const Params &p, const __half *hidden, int S, int64_t s
             dim3 grid((S + 7) / 8, p.B);
             if (launch_pdl(sink_score_all, grid, dim3(256), 0, st, (const uint16_t *)hidden, S, p.hidden, sb, ss, score, stride) != cudaSuccess)
                 return KVSINK_ERR_CUDA;
+        }
+    }
+    // long sequences: a cluster of 2, 4 or 8 blocks per sequence (slices of at least 8192 tokens, at most 32768)
+    int C = 1;
+    while (C < 8 && S > C * 8192) C *= 2;
+    if (C > 1) {
+        const int step = SEL_THREADS * 4;
+        const int slice = ((S + C - 1) / C + step - 1) / step * step;
+        if (slice <= SELC_MAX_STEPS * step) {
+            cudaLaunchAttribute attr[2];
+            attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+            attr[0].val.programmaticStreamSerializationAllowed = 1;
+            attr[1].id = cudaLaunchAttributeClusterDimension;
+            attr[1].val.clusterDim.x = C; attr[1].val.clusterDim.y = 1; attr[1].val.clusterDim.z = 1;
+            cudaLaunchConfig_t cfg = {};
+            cfg.gridDim = dim3(C, p.B);
+            cfg.blockDim = dim3(SEL_THREADS);
+            cfg.stream = st;
+            cfg.attrs = attr;
+            cfg.numAttrs = 2;
+            if (cudaLaunchKernelEx(&cfg, sink_select_cluster, (const uint16_t *)score, stride, S, p.topk, p.pfn_n, p.mask_words, p.cap, slice,
+                                   bitmask, sink_pos, sink_count) == cudaSuccess) {
+                note_launch();
+                return KVSINK_OK;
+            }
+            (void)cudaGetLastError();   // a cluster that cannot be placed: the one-block kernel below
         }
     }
     return launch_pdl(sink_select, dim3(p.B), dim3(SEL_THREADS), 0, st, (const uint16_t *)score, stride, S, p.topk, p.pfn_n, p.mask_words,

@@ -10,7 +10,7 @@ import oracle
 import paper_2508_04257_b200 as kv
 from paper_2508_04257_b200 import synth
 
-from parity_util import assert_close, bits_equal, compare_cache, configs, np16, run_both
+from parity_util import assert_close, bits_equal, compare_cache, compare_sinks, configs, np16, run_both
 
 pytestmark = pytest.mark.gpu
 TINY = synth.WORKLOADS["tiny"]
@@ -104,6 +104,20 @@ def test_ties_in_the_score_go_to_the_lower_index():
     run_both(wl, H=H)
     wl0 = wl.scaled(channels=())          # no listed channel: maximum over all d
     run_both(wl0, H=H)
+
+
+@pytest.mark.parametrize("seq,topk,pfn", [(40000, 300, 3), (8193, 1, 0), (16384, 0, 5), (70001, 5000, 0), (262144, 17, 1), (300000, 40, 2)])
+def test_long_sequences_with_many_ties(seq, topk, pfn):
+    # sequences long enough for the multi-block selection (and one beyond it): small integer scores, so that the k-th
+    # largest value is shared by thousands of tokens and the index tie-break decides across block boundaries
+    wl = TINY.scaled(seq=seq, topk=topk, pfn_n=pfn, batch=2, hidden=64, channels=(5, 9), seed=seq)
+    ocfg, gcfg = configs(wl)
+    g = torch.Generator("cuda").manual_seed(seq)
+    H = (torch.randint(-6, 7, (wl.batch, wl.seq, wl.hidden), device="cuda", generator=g).half() * 0.5)
+    gs = kv.SinkSet(gcfg)
+    kv.predict_sinks(gcfg, H, gs)
+    bm, pos, cnt = oracle.predict_sinks(ocfg, np16(H))
+    compare_sinks(gs, bm, pos, cnt, topk + pfn)
 
 
 def test_nan_and_infinity_in_the_hidden_state():
