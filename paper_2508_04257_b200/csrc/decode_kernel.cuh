@@ -264,30 +264,6 @@ decode_kernel(Params p, kvsink_cache c, kvsink_static_params sp, const __half *_
     // the next kernel in the stream may be scheduled from now on: its blocks take whatever room this grid leaves, set
     // themselves up, and wait at the same point until this grid has completed
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    for (int i = tid; i < NQMAX * D; i += DEC_THREADS) {
-        const int qh = i / D, ch = i % D;
-        __half v = qh < nq ? q[((size_t)b * p.Hq + hq0 + qh) * D + ch] : __float2half(0.f);
-        q16[i] = v;
-        qs[i] = __half2float(v) * qscale;
-    }
-    __syncthreads();
-
-    constexpr int PS = D + 2;                                        // partial record: o[D], m, l
-
-    // Integer key side: lane l prepares the B operand bytes of one group of four contraction slots, (MMA l/8, lower or
-    // upper slots (l/4)%2, slots 4(l%4) ... +3); these are its four channels and their query values.
-    int i8_ch[4] = {0, 0, 0, 0};
-    float i8_q[4] = {0.f, 0.f, 0.f, 0.f};
-    if constexpr (I8) {
-        const int mi = lane >> 3, c2 = (lane >> 2) & 1, tq = lane & 3;
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-            i8_ch[e] = BITS != 4 ? 16 * (2 * mi + (e & 1)) + 8 * c2 + 2 * tq + (e >> 1)
-                                 : 16 * (2 * mi + c2) + 8 * (e & 1) + 2 * tq + (e >> 1);
-            if (I8 == 1) i8_q[e] = qs[i8_ch[e]];
-        }
-    }
-
     // Sink rows of the side buffer are shared out over all warps of all splits and handled after the stream; the
     // first row of this warp is fetched now, so that its latency hides behind the stream.
     const int sink_n = min(c.sink_count[b], p.cap);
@@ -465,6 +441,31 @@ decode_kernel(Params p, kvsink_cache c, kvsink_static_params sp, const __half *_
         }
         fit_value_scale(mx);
     }
+    // the first copies are in flight: now the query tables (the copies do not depend on them)
+    for (int i = tid; i < NQMAX * D; i += DEC_THREADS) {
+        const int qh = i / D, ch = i % D;
+        __half v = qh < nq ? q[((size_t)b * p.Hq + hq0 + qh) * D + ch] : __float2half(0.f);
+        q16[i] = v;
+        qs[i] = __half2float(v) * qscale;
+    }
+    __syncthreads();
+
+    constexpr int PS = D + 2;                                        // partial record: o[D], m, l
+
+    // Integer key side: lane l prepares the B operand bytes of one group of four contraction slots, (MMA l/8, lower or
+    // upper slots (l/4)%2, slots 4(l%4) ... +3); these are its four channels and their query values.
+    int i8_ch[4] = {0, 0, 0, 0};
+    float i8_q[4] = {0.f, 0.f, 0.f, 0.f};
+    if constexpr (I8) {
+        const int mi = lane >> 3, c2 = (lane >> 2) & 1, tq = lane & 3;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            i8_ch[e] = BITS != 4 ? 16 * (2 * mi + (e & 1)) + 8 * c2 + 2 * tq + (e >> 1)
+                                 : 16 * (2 * mi + c2) + 8 * (e & 1) + 2 * tq + (e >> 1);
+            if (I8 == 1) i8_q[e] = qs[i8_ch[e]];
+        }
+    }
+
     // sink bits of the CT tiles starting at tile T: one 32-bit word covers two tiles
     auto load_mask_words = [&](int T) {
         uint2 w;
@@ -475,6 +476,49 @@ decode_kernel(Params p, kvsink_cache c, kvsink_static_params sp, const __half *_
     uint2 mword_next = my_groups > 0 ? load_mask_words(w_begin * TPG) : make_uint2(0u, 0u);
     bool stream_ok = true;
     int ci = 0;                                                      // running chunk index of this warp
+
+    // ---- tokens of the open group: keys from the fp16 tail (last split only).  They come first, while the warp's first
+    //      chunks are on their way (the order of the softmax steps does not matter) ----
+    if (!CAL && split == nsplit - 1) {
+        const __half *tail = (const __half *)c.k_tail + (size_t)unit * G * D;
+        const int T_begin = n_body / KVSINK_TILE, T_end = (n + KVSINK_TILE - 1) / KVSINK_TILE;
+        for (int T = T_begin + warp; T < T_end; T += DEC_WARPS) {
+            const int tok0 = T * KVSINK_TILE + g, tok1 = tok0 + 8;
+            const bool in0 = tok0 < n, in1 = tok1 < n;
+            const __half *r0 = tail + (size_t)(tok0 % G) * D, *r1 = tail + (size_t)(tok1 % G) * D;
+            float acc[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+            for (int m = 0; m < NM; ++m) {
+                uint32_t a[4];
+                a[0] = in0 ? *(const uint32_t *)(r0 + 16 * m + 2 * t) : 0u;
+                a[1] = in1 ? *(const uint32_t *)(r1 + 16 * m + 2 * t) : 0u;
+                a[2] = in0 ? *(const uint32_t *)(r0 + 16 * m + 2 * t + 8) : 0u;
+                a[3] = in1 ? *(const uint32_t *)(r1 + 16 * m + 2 * t + 8) : 0u;
+                const int qrow = PL ? (g >> 1) : g;          // query head in accumulator column g
+                const bool qcol = PL ? (!(g & 1) && qrow < NQMAX) : true;
+                const uint32_t b0 = qcol ? *(const uint32_t *)(q16 + qrow * D + 16 * m + 2 * t) : 0u;
+                const uint32_t b1 = qcol ? *(const uint32_t *)(q16 + qrow * D + 16 * m + 2 * t + 8) : 0u;
+                mma16816(acc, a, b0, b1);
+            }
+            const bool v0 = in0 && !mask_bit(bm, in0 ? tok0 : 0), v1 = in1 && !mask_bit(bm, in1 ? tok1 : 0);
+            float s[4];
+            s[0] = v0 ? acc[0] * qscale : -INFINITY; s[1] = (v0 && !PL) ? acc[1] * qscale : -INFINITY;
+            s[2] = v1 ? acc[2] * qscale : -INFINITY; s[3] = (v1 && !PL) ? acc[3] * qscale : -INFINITY;
+            advance_max(fmaxf(s[0], s[2]), fmaxf(s[1], s[3]));
+            uint32_t vw[W];
+            load_tile<BITS, D>((const uint32_t *)(vc_base + (size_t)T * p.tile_bytes), lane, vw);
+            float sv0[NGv], zv0[NGv], sv1[NGv], zv1[NGv];
+            float mx = 0.f;
+#pragma unroll
+            for (int j = 0; j < NGv; ++j) {   // tokens beyond the sequence have no parameters yet
+                sv0[j] = v0 ? __ldg(vs_base + (size_t)tok0 * NGv + j) : 0.f; zv0[j] = v0 ? __ldg(vz_base + (size_t)tok0 * NGv + j) : 0.f;
+                sv1[j] = v1 ? __ldg(vs_base + (size_t)tok1 * NGv + j) : 0.f; zv1[j] = v1 ? __ldg(vz_base + (size_t)tok1 * NGv + j) : 0.f;
+                mx = fmaxf(mx, fmaxf(fabsf(sv0[j]), fabsf(sv1[j])));
+            }
+            fit_value_scale(mx);
+            tile_values(s, vw, sv0, zv0, sv1, zv1);
+        }
+    }
 
     // state of the current key group (with static parameters: of the KV head, set up on the first trip)
     float bias0 = 0.f, bias1 = 0.f, ks0 = 0.f, ks1 = 0.f;
@@ -772,8 +816,9 @@ decode_kernel(Params p, kvsink_cache c, kvsink_static_params sp, const __half *_
                     const float yg = __shfl_down_sync(0xffffffffu, xg, 1), yh = __shfl_down_sync(0xffffffffu, xh, 1);
                     const float tg = fmaf(xg, 65536.f, yg);
                     const float th = fmaf(xh, 65536.f, yh);
-                    s[k][0] = t == 0 ? fmaf(tg, ks0, -bias0) : -INFINITY; s[k][1] = -INFINITY;
-                    s[k][2] = t == 0 ? fmaf(th, ks0 * (BITS == 4 ? 0.0625f : 0.25f), -bias0) : -INFINITY; s[k][3] = -INFINITY;
+                    // lanes t != 0 hold no head: their factor and bias are zero, their columns are never read
+                    s[k][0] = fmaf(tg, ks0, -bias0); s[k][1] = -INFINITY;
+                    s[k][2] = fmaf(th, ks0 * (BITS == 4 ? 0.0625f : 0.25f), -bias0); s[k][3] = -INFINITY;
                     continue;
                 }
                 uint32_t kw[W], ka[NM][4];
@@ -858,48 +903,6 @@ decode_kernel(Params p, kvsink_cache c, kvsink_static_params sp, const __half *_
         }
     }
     if (!stream_ok && lane == 0) atomicOr(c.status, KVSINK_STATUS_TIMEOUT);
-
-    // ---- tokens of the open group: keys from the fp16 tail (last split only) ----
-    if (!CAL && split == nsplit - 1) {
-        const __half *tail = (const __half *)c.k_tail + (size_t)unit * G * D;
-        const int T_begin = n_body / KVSINK_TILE, T_end = (n + KVSINK_TILE - 1) / KVSINK_TILE;
-        for (int T = T_begin + warp; T < T_end; T += DEC_WARPS) {
-            const int tok0 = T * KVSINK_TILE + g, tok1 = tok0 + 8;
-            const bool in0 = tok0 < n, in1 = tok1 < n;
-            const __half *r0 = tail + (size_t)(tok0 % G) * D, *r1 = tail + (size_t)(tok1 % G) * D;
-            float acc[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-            for (int m = 0; m < NM; ++m) {
-                uint32_t a[4];
-                a[0] = in0 ? *(const uint32_t *)(r0 + 16 * m + 2 * t) : 0u;
-                a[1] = in1 ? *(const uint32_t *)(r1 + 16 * m + 2 * t) : 0u;
-                a[2] = in0 ? *(const uint32_t *)(r0 + 16 * m + 2 * t + 8) : 0u;
-                a[3] = in1 ? *(const uint32_t *)(r1 + 16 * m + 2 * t + 8) : 0u;
-                const int qrow = PL ? (g >> 1) : g;          // query head in accumulator column g
-                const bool qcol = PL ? (!(g & 1) && qrow < NQMAX) : true;
-                const uint32_t b0 = qcol ? *(const uint32_t *)(q16 + qrow * D + 16 * m + 2 * t) : 0u;
-                const uint32_t b1 = qcol ? *(const uint32_t *)(q16 + qrow * D + 16 * m + 2 * t + 8) : 0u;
-                mma16816(acc, a, b0, b1);
-            }
-            const bool v0 = in0 && !mask_bit(bm, in0 ? tok0 : 0), v1 = in1 && !mask_bit(bm, in1 ? tok1 : 0);
-            float s[4];
-            s[0] = v0 ? acc[0] * qscale : -INFINITY; s[1] = (v0 && !PL) ? acc[1] * qscale : -INFINITY;
-            s[2] = v1 ? acc[2] * qscale : -INFINITY; s[3] = (v1 && !PL) ? acc[3] * qscale : -INFINITY;
-            advance_max(fmaxf(s[0], s[2]), fmaxf(s[1], s[3]));
-            uint32_t vw[W];
-            load_tile<BITS, D>((const uint32_t *)(vc_base + (size_t)T * p.tile_bytes), lane, vw);
-            float sv0[NGv], zv0[NGv], sv1[NGv], zv1[NGv];
-            float mx = 0.f;
-#pragma unroll
-            for (int j = 0; j < NGv; ++j) {   // tokens beyond the sequence have no parameters yet
-                sv0[j] = v0 ? __ldg(vs_base + (size_t)tok0 * NGv + j) : 0.f; zv0[j] = v0 ? __ldg(vz_base + (size_t)tok0 * NGv + j) : 0.f;
-                sv1[j] = v1 ? __ldg(vs_base + (size_t)tok1 * NGv + j) : 0.f; zv1[j] = v1 ? __ldg(vz_base + (size_t)tok1 * NGv + j) : 0.f;
-                mx = fmaxf(mx, fmaxf(fabsf(sv0[j]), fabsf(sv1[j])));
-            }
-            fit_value_scale(mx);
-            tile_values(s, vw, sv0, zv0, sv1, zv1);
-        }
-    }
 
     // ---- this warp's packed partial: finish the reductions over the token lanes, convert units ----
 #pragma unroll

@@ -38,11 +38,13 @@ def test_static_scratch_matches_the_workspace_entry_point_twice_in_a_row():
         lse = torch.full(shape[:2], float("nan"), dtype=torch.float32, device="cuda")
         torch.cuda.synchronize()
         if call == 1:       # the first call has made the one-time address lookup; from now on device memory must not move
-            free_before, allocated_before = torch.cuda.mem_get_info()[0], torch.cuda.memory_allocated()
+            free_before, allocs_before = torch.cuda.mem_get_info()[0], torch.cuda.memory_stats()["allocation.all.allocated"]
         kv.decode_attention_static(cfg, cache, q, out, lse)
         torch.cuda.synchronize()
         if call == 1:
-            assert torch.cuda.mem_get_info()[0] == free_before and torch.cuda.memory_allocated() == allocated_before
+            # no device memory was taken from the driver and no tensor was allocated during the call
+            assert torch.cuda.mem_get_info()[0] >= free_before
+            assert torch.cuda.memory_stats()["allocation.all.allocated"] == allocs_before
         o, r = out.cpu().numpy(), ref.cpu().numpy()
         assert np.all(np.isfinite(o))
         assert np.all(np.abs(o - r) <= ATOL + RTOL * np.abs(r)), f"call {call}: max diff {np.abs(o - r).max():.3e}"
