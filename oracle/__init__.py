@@ -283,3 +283,17 @@ def decode_attention_calibrated(cfg: Config, cache: Cache, sp: StaticParams, q: 
     _check(lib().kvo_decode_attention_calibrated(C.byref(cfg.c()), C.byref(cc), C.byref(cs), qq.ctypes.data_as(C.c_void_p),
                                                  out.ctypes.data_as(C.c_void_p), lse.ctypes.data_as(C.c_void_p)), "decode_attention_calibrated")
     return out, lse
+
+
+def prefill_attention(cfg: Config, cache: Cache, q: np.ndarray, q_pos0: int):
+    """q: float16 [B, Hq, T, D]; query t sits at position q_pos0 + t. Returns (out float64 [B,Hq,T,D], lse [B,Hq,T])."""
+    qq = _u16(q)
+    assert qq.ndim == 4 and qq.strides[3] == 2
+    T = qq.shape[2]
+    out = np.zeros((cfg.batch, cfg.n_q_heads, T, cfg.head_dim), np.float64)
+    lse = np.zeros((cfg.batch, cfg.n_q_heads, T), np.float64)
+    cc = cache.c()
+    _check(lib().kvo_prefill_attention(C.byref(cfg.c()), C.byref(cc), qq.ctypes.data_as(C.c_void_p), C.c_int32(T), C.c_int32(q_pos0),
+                                       C.c_int64(qq.strides[0] // 2), C.c_int64(qq.strides[1] // 2), C.c_int64(qq.strides[2] // 2),
+                                       out.ctypes.data_as(C.c_void_p), lse.ctypes.data_as(C.c_void_p)), "prefill_attention")
+    return out, lse

@@ -805,3 +805,52 @@ int kvo_decode_attention_calibrated(const kvo_config *c, const kvo_cache *cache,
     }
     return KVO_OK;
 }
+
+/*
+ * Attention of the prompt's own queries over the cache that was just quantized (Algorithm 1, the attention statement
+ * after the two quantize statements; Eq. 3 with a causal mask): query token t of the chunk (t = 0 .. T-1) sits at
+ * position q_pos0 + t and attends to the cached tokens 0 .. q_pos0 + t, whose K and V are what decode attention reads
+ * (Eq. 7: sink tokens exact, the others dequantised; open-group keys from the fp16 tail).  binary64 throughout.
+ * q: fp16 [B,Hq,T,D] with element strides; out [B,Hq,T,D]; lse [B,Hq,T] (may be NULL).
+ * Requires q_pos0 >= 0 and q_pos0 + T <= seq_len.
+ */
+int kvo_prefill_attention(const kvo_config *c, const kvo_cache *cache, const uint16_t *q, int32_t T, int32_t q_pos0, int64_t stride_b,
+                          int64_t stride_h, int64_t stride_t, double *out, double *lse)
+{
+    int rc = check_config(c);
+    if (rc) return rc;
+    if (!cache || !q || !out || T < 0 || q_pos0 < 0 || (int64_t)q_pos0 + T > cache->seq_len) return KVO_ERR_BAD_ARG;
+    const int D = c->head_dim, rep = c->n_q_heads / c->n_kv_heads;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int64_t bh = 0; bh < (int64_t)c->batch * c->n_q_heads; ++bh) {
+        const int b = (int)(bh / c->n_q_heads), hq = (int)(bh % c->n_q_heads), h = hq / rep;
+        const int n_max = q_pos0 + T;
+        double *kd = (double *)malloc(sizeof(double) * (size_t)(n_max > 0 ? n_max : 1) * D);
+        double *vd = (double *)malloc(sizeof(double) * (size_t)(n_max > 0 ? n_max : 1) * D);
+        double *s = (double *)malloc(sizeof(double) * (size_t)(n_max > 0 ? n_max : 1));
+        for (int p = 0; p < n_max; ++p) kv_row(c, cache, b, h, p, kd + (int64_t)p * D, vd + (int64_t)p * D);
+        for (int t = 0; t < T; ++t) {
+            const int n = q_pos0 + t + 1;
+            const uint16_t *qv = q + b * stride_b + hq * stride_h + t * stride_t;
+            double *o = out + (((int64_t)b * c->n_q_heads + hq) * T + t) * D;
+            double mx = -INFINITY;
+            for (int p = 0; p < n; ++p) {
+                double acc = 0.0;
+                for (int ch = 0; ch < D; ++ch) acc += (double)half_to_float(qv[ch]) * kd[(int64_t)p * D + ch];
+                s[p] = acc / sqrt((double)D);
+                if (s[p] > mx) mx = s[p];
+            }
+            double den = 0.0;
+            for (int ch = 0; ch < D; ++ch) o[ch] = 0.0;
+            for (int p = 0; p < n; ++p) {
+                double w = exp(s[p] - mx);
+                den += w;
+                for (int ch = 0; ch < D; ++ch) o[ch] += w * vd[(int64_t)p * D + ch];
+            }
+            for (int ch = 0; ch < D; ++ch) o[ch] /= den;
+            if (lse) lse[((int64_t)b * c->n_q_heads + hq) * T + t] = mx + log(den);
+        }
+        free(kd); free(vd); free(s);
+    }
+    return KVO_OK;
+}
