@@ -159,6 +159,20 @@ int kvsink_decode_attention(const kvsink_config *cfg, const kvsink_cache *cache,
                             void *workspace, size_t workspace_bytes, void *cuda_stream);
 
 /*
+ * Attention of a chunk of prompt queries over the cache that holds their own (just quantized) keys and values -- the
+ * attention statement of Algorithm 1, which follows its two quantize statements; Eq. 3 with a causal mask, Eq. 7's split.
+ * Query token t of the chunk (t = 0 .. T-1) sits at position q_pos0 + t and attends to the cached tokens 0 .. q_pos0 + t,
+ * read exactly as kvsink_decode_attention reads them.  Call it after kvsink_quantize_append of the same chunk:
+ * 0 <= q_pos0 and q_pos0 + T <= seq_len.
+ *   q     device, fp16, element (b, hq, t, c) at q + b*stride_b + hq*stride_h + t*stride_t + c (strides in elements,
+ *         multiples of 8).
+ *   out   device out, float [B][Hq][T][D].      lse  device out, float [B][Hq][T] or NULL.
+ * No workspace: every block of eight (query token, query head) rows streams its own prefix of the cache.
+ */
+int kvsink_prefill_attention(const kvsink_config *cfg, const kvsink_cache *cache, const void *q, int32_t T, int32_t q_pos0, int64_t stride_b,
+                             int64_t stride_h, int64_t stride_t, float *out, float *lse, void *cuda_stream);
+
+/*
  * kvsink_decode_attention for callers that cannot allocate device memory.  (No counterpart in the paper: this is
  * a deployment convenience of this library.)
  *

@@ -17,7 +17,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _LIB_PATH = os.environ.get("KVSINK_LIB") or os.path.join(_HERE, "libkvsink.so")
 
 EXPORTS = ("kvsink_cache_sizes", "kvsink_predict_sinks", "kvsink_quantize_append", "kvsink_decode_attention",
-           "kvsink_decode_attention_static", "kvsink_calibrate", "kvsink_quantize_append_calibrated",
+           "kvsink_decode_attention_static", "kvsink_prefill_attention", "kvsink_calibrate", "kvsink_quantize_append_calibrated",
            "kvsink_decode_attention_calibrated", "kvsink_channel_absmax", "kvsink_quant_error", "kvsink_read_status",
            "kvsink_launch_count", "kvsink_strerror")
 STATIC_SCRATCH_BYTES = 4 * 1024 * 1024
@@ -178,6 +178,24 @@ def decode_attention(cfg: Config, cache: KVCache, q: torch.Tensor, out: Optional
                                        C.c_size_t(workspace.numel()), _stream())
     if rc:
         raise KvsinkError(rc, "kvsink_decode_attention")
+    return out, lse
+
+
+def prefill_attention(cfg: Config, cache: KVCache, q: torch.Tensor, q_pos0: int, out: Optional[torch.Tensor] = None,
+                      lse: Optional[torch.Tensor] = None, want_lse: bool = True):
+    """kvsink_prefill_attention: q fp16 [B, Hq, T, D] on the device (last axis contiguous); query t sits at position q_pos0 + t.
+    Returns (out fp32 [B,Hq,T,D], lse fp32 [B,Hq,T] or None)."""
+    assert q.is_cuda and q.dtype == torch.float16 and q.dim() == 4 and q.stride(3) == 1
+    T = q.shape[2]
+    if out is None:
+        out = torch.empty((cfg.batch, cfg.n_q_heads, T, cfg.head_dim), dtype=torch.float32, device=q.device)
+    if lse is None and want_lse:
+        lse = torch.empty((cfg.batch, cfg.n_q_heads, T), dtype=torch.float32, device=q.device)
+    cc = cache.c()
+    rc = lib().kvsink_prefill_attention(C.byref(cfg.c()), C.byref(cc), _ptr(q), C.c_int32(T), C.c_int32(q_pos0), C.c_int64(q.stride(0)),
+                                        C.c_int64(q.stride(1)), C.c_int64(q.stride(2)), _ptr(out), _ptr(lse), _stream())
+    if rc:
+        raise KvsinkError(rc, "kvsink_prefill_attention")
     return out, lse
 
 

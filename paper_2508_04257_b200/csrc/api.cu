@@ -160,6 +160,25 @@ extern "C" int kvsink_decode_attention(const kvsink_config *cfg, const kvsink_ca
     return launch_decode(p, *cache, nullptr, (const __half *)q, out, lse, workspace, workspace_bytes, (cudaStream_t)cuda_stream);
 }
 
+extern "C" int kvsink_prefill_attention(const kvsink_config *cfg, const kvsink_cache *cache, const void *q, int32_t T, int32_t q_pos0,
+                                        int64_t stride_b, int64_t stride_h, int64_t stride_t, float *out, float *lse, void *cuda_stream)
+{
+    Params p;
+    int rc = derive(cfg, &p);
+    if (rc) return rc;
+    rc = check_cache(cache, p);
+    if (rc) return rc;
+    if (T < 0 || q_pos0 < 0 || (int64_t)q_pos0 + T > cache->seq_len) return KVSINK_ERR_BAD_ARG;
+    if (T == 0) return KVSINK_OK;
+    if (!aligned16(q) || !aligned16(out)) return KVSINK_ERR_BAD_ARG;
+    if (stride_t < p.D || (stride_t % 8) || (stride_h % 8) || (stride_b % 8) || stride_h < 0 || stride_b < 0) return KVSINK_ERR_BAD_ARG;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    const __half *qq = (const __half *)q;
+    if (p.bits == 2) return launch_prefill_b2(p, *cache, qq, T, q_pos0, stride_b, stride_h, stride_t, out, lse, st);
+    if (p.bits == 3) return launch_prefill_b3(p, *cache, qq, T, q_pos0, stride_b, stride_h, stride_t, out, lse, st);
+    return launch_prefill_b4(p, *cache, qq, T, q_pos0, stride_b, stride_h, stride_t, out, lse, st);
+}
+
 extern "C" int kvsink_decode_attention_static(const kvsink_config *cfg, const kvsink_cache *cache, const void *q, float *out,
                                               float *lse, void *cuda_stream)
 {

@@ -152,6 +152,12 @@ int launch_quantize_tokens(const Params &p, const kvsink_cache &c, const __half 
                            int first_token, int n_tokens, int64_t sb, int64_t sh, int64_t stt, cudaStream_t st);
 int launch_decode(const Params &p, const kvsink_cache &c, const kvsink_static_params *cal, const __half *q, float *out, float *lse, void *workspace,
                   size_t workspace_bytes, cudaStream_t st);
+int launch_prefill_b2(const Params &p, const kvsink_cache &c, const __half *q, int T, int q_pos0, int64_t sb, int64_t sh, int64_t stt, float *out,
+                      float *lse, cudaStream_t st);
+int launch_prefill_b3(const Params &p, const kvsink_cache &c, const __half *q, int T, int q_pos0, int64_t sb, int64_t sh, int64_t stt, float *out,
+                      float *lse, cudaStream_t st);
+int launch_prefill_b4(const Params &p, const kvsink_cache &c, const __half *q, int T, int q_pos0, int64_t sb, int64_t sh, int64_t stt, float *out,
+                      float *lse, cudaStream_t st);
 int launch_calibrate(const Params &p, const __half *k, const __half *v, int T, int64_t sb, int64_t sh, int64_t stt, const uint32_t *bitmask,
                      const kvsink_static_params &sp, void *workspace, cudaStream_t st);
 int launch_quantize_calibrated(const Params &p, const kvsink_cache &c, const kvsink_static_params &sp, const __half *k_src, const __half *v_src,

@@ -9,4 +9,10 @@ int launch_decode_b4(const Params &p, const kvsink_cache &c, const kvsink_static
     return launch_decode_bits<4>(p, c, cal, q, out, lse, ws, st);
 }
 
+int launch_prefill_b4(const Params &p, const kvsink_cache &c, const __half *q, int T, int q_pos0, int64_t sb, int64_t sh, int64_t stt, float *out,
+                      float *lse, cudaStream_t st)
+{
+    return launch_prefill_bits<4>(p, c, q, T, q_pos0, sb, sh, stt, out, lse, st);
+}
+
 }  // namespace kvsink

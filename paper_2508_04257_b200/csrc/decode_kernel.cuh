@@ -217,10 +217,20 @@ struct DecodePlan {
 // CAL (static, calibrated parameters): one (scale, zero) per key channel and per value channel group of the KV head for every
 // token.  There are no token groups: the key B operand is prepared once per block, a ring chunk holds code words only, the
 // stream covers every tile up to the sequence length (tokens beyond it are masked) and there is no fp16 tail.
-template <int BITS, int D, int NGv, int CT, bool PL, int I8 = 0, bool CAL = false>
+//
+// PRE (attention of a chunk of prompt queries over the cache, Algorithm 1's attention statement): the eight accumulator
+// columns of a block are eight (query token, query head) rows of one KV head, token-major; query token t sits at position
+// q_pos0 + t and sees the cached tokens up to its own position, so every column has its own length limit.  One block streams
+// the cache up to its last row's limit; there are no sequence splits.
+struct PrefillShape {
+    int T, q_pos0;               // queries in the chunk (0: single-token decode), position of the first
+    int64_t q_sb, q_sh, q_st;    // element strides of q [B][Hq][T][D]
+};
+
+template <int BITS, int D, int NGv, int CT, bool PL, int I8 = 0, bool CAL = false, bool PRE = false>
 __global__ void __launch_bounds__(DEC_THREADS, 4)
 decode_kernel(Params p, kvsink_cache c, kvsink_static_params sp, const __half *__restrict__ q, float *__restrict__ out, float *__restrict__ lse,
-              float *__restrict__ part_ws, int nsplit, int groups_per_split, int qchunks, int seq_len, int cluster_merge)
+              float *__restrict__ part_ws, int nsplit, int groups_per_split, int qchunks, int seq_len, int cluster_merge, PrefillShape pre)
 {
     using G_ = Geo<BITS, D>;
     constexpr int NQMAX = I8 == 1 ? 1 : (PL ? 4 : 8);
@@ -235,11 +245,22 @@ decode_kernel(Params p, kvsink_cache c, kvsink_static_params sp, const __half *_
     constexpr float R1 = 1.f / G_::ROWF, C1 = 1.f / G_::COLF;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = __shfl_sync(0xffffffffu, tid >> 5, 0), g = lane >> 2, t = lane & 3;
-    const int split = blockIdx.x, h = blockIdx.y / qchunks, qc = blockIdx.y % qchunks, b = blockIdx.z;
-    const int nq = I8 == 1 ? 1 : min(NQMAX, p.rep - 8 * qc), hq0 = h * p.rep + 8 * qc;
+    static_assert(!PRE || (!PL && I8 == 0 && !CAL), "prompt queries take the eight-column fp16 path");
+    // decode: grid (splits, KV heads x blocks of eight query heads, sequences); prompt queries: grid (row blocks, KV heads, sequences)
+    const int split = PRE ? 0 : blockIdx.x, h = PRE ? blockIdx.y : blockIdx.y / qchunks, qc = PRE ? blockIdx.x : blockIdx.y % qchunks, b = blockIdx.z;
+    const int nq = I8 == 1 ? 1 : (PRE ? min(NQMAX, pre.T * p.rep - 8 * qc) : min(NQMAX, p.rep - 8 * qc)), hq0 = h * p.rep + (PRE ? 0 : 8 * qc);
+    // prompt queries: row i of the block is query token (8 qc + i) / rep, query head (8 qc + i) % rep of this KV head
+    auto row_token = [&](int i) { return (8 * qc + i) / p.rep; };
+    auto row_limit = [&](int i) { return i < nq ? pre.q_pos0 + row_token(i) + 1 : 0; };    // cached tokens the row sees
     const int64_t unit = (int64_t)b * p.Hkv + h;
     // with static parameters a "group" of the loops below is one ring chunk, and every token belongs to one
-    const int G = CAL ? CT * KVSINK_TILE : p.G, n = seq_len, n_groups = CAL ? (n + G - 1) / G : n / G, n_body = CAL ? n : n_groups * G;
+    const int G = CAL ? CT * KVSINK_TILE : p.G;
+    const int n = PRE ? min(seq_len, row_limit(nq - 1)) : seq_len;                        // tokens this block looks at
+    const int n_groups = CAL ? (n + G - 1) / G : (PRE ? min(seq_len / G, (n + G - 1) / G) : n / G);
+    const int n_body = CAL ? n : (seq_len / G) * G;                                       // where the fp16 tail begins
+    // limits of this lane's accumulator columns 2t, 2t+1 and the smallest limit of the block (prompt queries only)
+    const int lim0 = PRE ? row_limit(2 * t) : 0, lim1 = PRE ? row_limit(2 * t + 1) : 0, lim_min = PRE ? row_limit(0) : 0;
+    if (PRE) groups_per_split = n_groups;
     const int TPG = G / KVSINK_TILE, CPG = TPG / CT;                 // tiles and ring chunks per key group
     const uint32_t *bm = c.sink_bitmask + (size_t)b * p.mask_words;
     const float qscale = LOG2E * rsqrtf((float)D);
@@ -444,7 +465,10 @@ decode_kernel(Params p, kvsink_cache c, kvsink_static_params sp, const __half *_
     // the first copies are in flight: now the query tables (the copies do not depend on them)
     for (int i = tid; i < NQMAX * D; i += DEC_THREADS) {
         const int qh = i / D, ch = i % D;
-        __half v = qh < nq ? q[((size_t)b * p.Hq + hq0 + qh) * D + ch] : __float2half(0.f);
+        __half v = __float2half(0.f);
+        if (qh < nq)
+            v = PRE ? q[b * pre.q_sb + (int64_t)(hq0 + (8 * qc + qh) % p.rep) * pre.q_sh + (int64_t)row_token(qh) * pre.q_st + ch]
+                    : q[((size_t)b * p.Hq + hq0 + qh) * D + ch];
         q16[i] = v;
         qs[i] = __half2float(v) * qscale;
     }
@@ -504,6 +528,12 @@ decode_kernel(Params p, kvsink_cache c, kvsink_static_params sp, const __half *_
             float s[4];
             s[0] = v0 ? acc[0] * qscale : -INFINITY; s[1] = (v0 && !PL) ? acc[1] * qscale : -INFINITY;
             s[2] = v1 ? acc[2] * qscale : -INFINITY; s[3] = (v1 && !PL) ? acc[3] * qscale : -INFINITY;
+            if constexpr (PRE) {   // every column sees the tokens up to its own query
+                if (tok0 >= lim0) s[0] = -INFINITY;
+                if (tok0 >= lim1) s[1] = -INFINITY;
+                if (tok1 >= lim0) s[2] = -INFINITY;
+                if (tok1 >= lim1) s[3] = -INFINITY;
+            }
             advance_max(fmaxf(s[0], s[2]), fmaxf(s[1], s[3]));
             uint32_t vw[W];
             load_tile<BITS, D>((const uint32_t *)(vc_base + (size_t)T * p.tile_bytes), lane, vw);
@@ -857,6 +887,18 @@ decode_kernel(Params p, kvsink_cache c, kvsink_static_params sp, const __half *_
                     if ((mask16 >> (g + 8)) & 1u) s[k][2] = s[k][3] = -INFINITY;
                 }
             }
+            if constexpr (PRE) {
+                if ((T0 + ST) * KVSINK_TILE > lim_min) {   // tiles that reach beyond the earliest query of the block
+#pragma unroll
+                    for (int k = 0; k < ST; ++k) {
+                        const int tok = (T0 + k) * KVSINK_TILE + g;
+                        if (tok >= lim0) s[k][0] = -INFINITY;
+                        if (tok >= lim1) s[k][1] = -INFINITY;
+                        if (tok + 8 >= lim0) s[k][2] = -INFINITY;
+                        if (tok + 8 >= lim1) s[k][3] = -INFINITY;
+                    }
+                }
+            }
             if constexpr (CAL) {
                 if ((T0 + ST) * KVSINK_TILE > n) {   // the last tiles reach beyond the sequence: those tokens do not exist
 #pragma unroll
@@ -969,7 +1011,7 @@ decode_kernel(Params p, kvsink_cache c, kvsink_static_params sp, const __half *_
             if (pos < 0 || pos >= n) continue;
 #pragma unroll
             for (int i = 0; i < NQMAX; ++i) {
-                if (i < nq) {
+                if (i < nq && (!PRE || pos < row_limit(i))) {
                     float d = 0.f;
 #pragma unroll
                     for (int e = 0; e < CPL; ++e) d += qs[i * D + lane * CPL + e] * kf[e];
@@ -1007,7 +1049,7 @@ decode_kernel(Params p, kvsink_cache c, kvsink_static_params sp, const __half *_
             acc += pr[ch] * f;
             L += pr[D + 1] * f;
         }
-        const size_t oq = (size_t)b * p.Hq + hq0 + qh;
+        const size_t oq = PRE ? ((size_t)b * p.Hq + hq0 + (8 * qc + qh) % p.rep) * pre.T + row_token(qh) : (size_t)b * p.Hq + hq0 + qh;
         if (nsplit == 1) {
             out[oq * D + ch] = L > 0.f ? acc / L : 0.f;
             if (lse && ch == 0) lse[oq] = L > 0.f ? (M + log2f(L)) * 0.6931471805599453f : -INFINITY;
@@ -1081,7 +1123,7 @@ static int launch_decode_p(const Params &p, const kvsink_cache &c, const kvsink_
             pdl[1].val.clusterDim.z = 1;
             cfg.numAttrs = 2;
         }
-        if (cudaLaunchKernelEx(&cfg, kern, p, c, sp, q, out, lse, ws, nsplit, gps, qchunks, (int)c.seq_len, (int)cluster_merge) == cudaSuccess) {
+        if (cudaLaunchKernelEx(&cfg, kern, p, c, sp, q, out, lse, ws, nsplit, gps, qchunks, (int)c.seq_len, (int)cluster_merge, PrefillShape{0, 0, 0, 0, 0}) == cudaSuccess) {
             note_launch();
             break;
         }
@@ -1091,6 +1133,61 @@ static int launch_decode_p(const Params &p, const kvsink_cache &c, const kvsink_
     }
     if (nsplit > 1 && !cluster_merge) return launch_decode_merge(ws, nsplit, D, p.B * p.Hq, out, lse, st);
     return KVSINK_OK;
+}
+
+// Prompt queries (the eight-column fp16 path): one block per eight (query token, query head) rows of a KV head.
+template <int BITS, int D, int NGV, int CT>
+static int launch_prefill_p(const Params &p, const kvsink_cache &c, const __half *q, const PrefillShape &pre, float *out, float *lse, cudaStream_t st)
+{
+    const size_t smem = DecodePlan<BITS, D, NGV, CT, 8>::BYTES;
+    auto kern = decode_kernel<BITS, D, NGV, CT, false, 0, false, true>;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return KVSINK_ERR_CUDA;
+    const long long blocks = ((long long)pre.T * p.rep + 7) / 8;
+    if (blocks > 0x7fffffffLL) return KVSINK_ERR_UNSUPPORTED;
+    cudaLaunchAttribute pdl[1];
+    pdl[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    pdl[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)blocks, p.Hkv, p.B);
+    cfg.blockDim = dim3(DEC_THREADS);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cfg.attrs = pdl;
+    cfg.numAttrs = 1;
+    const kvsink_static_params none = {nullptr, nullptr, nullptr, nullptr};
+    if (cudaLaunchKernelEx(&cfg, kern, p, c, none, q, out, lse, (float *)nullptr, 1, 0, (int)blocks, (int)c.seq_len, 0, pre) != cudaSuccess)
+        return KVSINK_ERR_CUDA;
+    note_launch();
+    return KVSINK_OK;
+}
+
+template <int BITS, int D, int NGV>
+static int launch_prefill_n(const Params &p, const kvsink_cache &c, const __half *q, const PrefillShape &pre, float *out, float *lse, cudaStream_t st)
+{
+    if constexpr (4 * (2 * 128 * (D * BITS / 64) + 2 * 16 * NGV * 4) <= 4800)
+        if ((p.G / KVSINK_TILE) % 4 == 0) return launch_prefill_p<BITS, D, NGV, 4>(p, c, q, pre, out, lse, st);
+    if ((p.G / KVSINK_TILE) % 2 == 0) return launch_prefill_p<BITS, D, NGV, 2>(p, c, q, pre, out, lse, st);
+    return launch_prefill_p<BITS, D, NGV, 1>(p, c, q, pre, out, lse, st);
+}
+
+template <int BITS, int D>
+static int launch_prefill_t(const Params &p, const kvsink_cache &c, const __half *q, const PrefillShape &pre, float *out, float *lse, cudaStream_t st)
+{
+    if (p.NGv == 1) return launch_prefill_n<BITS, D, 1>(p, c, q, pre, out, lse, st);
+    if (p.NGv == 2) return launch_prefill_n<BITS, D, 2>(p, c, q, pre, out, lse, st);
+    if (p.NGv == 4) return launch_prefill_n<BITS, D, 4>(p, c, q, pre, out, lse, st);
+    return KVSINK_ERR_UNSUPPORTED;
+}
+
+template <int BITS>
+static int launch_prefill_bits(const Params &p, const kvsink_cache &c, const __half *q, int T, int q_pos0, int64_t sb, int64_t sh, int64_t stt,
+                               float *out, float *lse, cudaStream_t st)
+{
+    const PrefillShape pre = {T, q_pos0, sb, sh, stt};
+    if (p.D == 128) return launch_prefill_t<BITS, 128>(p, c, q, pre, out, lse, st);
+    if constexpr (BITS != 3)
+        if (p.D == 64) return launch_prefill_t<BITS, 64>(p, c, q, pre, out, lse, st);
+    return KVSINK_ERR_UNSUPPORTED;
 }
 
 template <int BITS, int D, int NGV, int CT, bool CAL>
