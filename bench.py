@@ -441,6 +441,34 @@ def calibrated_record(kv, wl, dev, instances, steps, warmup, peak):
             "decode": {"algorithmic_bytes": db, "GBs": gbs(db, us["decode"]), "frac_of_measured_peak": gbs(db, us["decode"]) / peak}}
 
 
+def prefill_attention_record(kv, wl, dev, steps, warmup):
+    """Attention of every prompt query over the just-quantized cache of a single-layer workload (kernel time only)."""
+    cfg = kv.Config(wl.batch, wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.hidden, wl.bits, wl.group, wl.max_seq, wl.topk, wl.pfn_n, wl.channels)
+    H = synth.make_hidden(wl, dev)
+    K, V = synth.make_kv(wl, 0, dev)
+    sinks = kv.SinkSet(cfg, dev)
+    kv.predict_sinks(cfg, H, sinks)
+    cache = kv.KVCache(cfg, sinks, dev)
+    kv.quantize_append(cfg, cache, K, V)
+    del H
+    g = torch.Generator(device=dev)
+    g.manual_seed(wl.seed + 77)
+    q = torch.randn((wl.batch, wl.n_q_heads, wl.seq, wl.head_dim), device=dev, generator=g).half()
+    out = torch.empty((wl.batch, wl.n_q_heads, wl.seq, wl.head_dim), dtype=torch.float32, device=dev)
+    for _ in range(warmup):
+        kv.prefill_attention(cfg, cache, q, 0, out, None, want_lse=False)
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    for _ in range(steps):
+        kv.prefill_attention(cfg, cache, q, 0, out, None, want_lse=False)
+    b.record()
+    torch.cuda.synchronize()
+    us = a.elapsed_time(b) * 1e3 / steps
+    flop = 4.0 * wl.batch * wl.n_q_heads * wl.head_dim * wl.seq * (wl.seq + 1) / 2        # QK^T and PV over the causal triangle
+    return {"workload": workload_string(wl) + " (attention of all prompt queries over the quantized cache)", "prefill_attention_us": us,
+            "attention_tflops": flop / (us * 1e-6) / 1e12, "device_status": kv.read_status(cache)}
+
+
 def workload_record(b: Bench, ms_step, launches, steps, peak, world, agg):
     wl = b.wl
     us = b.kind_us()
@@ -542,6 +570,8 @@ def run_ours(args):
         # the next scope row: static (calibrated) parameters on the LLaMA2-7B-shaped layer
         base = synth.WORKLOADS["llama2_7b_layer"]
         per["llama2_7b_layer_static"] = calibrated_record(kv, base.scaled(seed=dist_util.rank_seed(base.seed, rank)), dev, args.instances, 20, warmup, peak)
+        torch.cuda.empty_cache()
+        per["llama2_7b_layer_prefill_attention"] = prefill_attention_record(kv, base.scaled(seed=dist_util.rank_seed(base.seed, rank)), dev, 3, 1)
         torch.cuda.empty_cache()
     sampler.finish()
 

@@ -15,12 +15,19 @@
  *   Eq. 8-11     asymmetric n-bit integer quantization     (Appendix C)
  *   Algorithm 1  prefill with KVSink (sink exclusion, top-k sink prediction) (Appendix G)
  *   Section 4.3  items (1)-(4): top-k on a pre-identified outlier channel, once, at prefill
+ *   Section 4.1  Table 1: quantization error with / without sink tokens; static calibration without them
+ *   Section 5.1, Appendix C  static per-channel-key / per-token-value parameters
+ *   Appendix D   outlier channels (the per-channel magnitude scan)
  *
  * Pins (see tests/test_oracle_*.py): Table 4 memory columns (closed form), |x - x'| <= scale/2,
  * exact rational re-derivation of codes, bit-exact round trip of sink / first-N rows, planted
  * outliers, brute-force sort for top-k, textbook fp64 softmax attention on the dequantised
  * tensors, Eq. 7 log-sum-exp merge identity, and the published m16n8k16 A-fragment ownership
- * table for the physical code order.
+ * table for the physical code order.  The routines at the end of the file (channel scan, error
+ * split of Table 1, static calibration / quantization / attention, prompt attention) are pinned by
+ * tests/test_oracle_analysis.py, test_oracle_static.py and test_oracle_prefill.py: numpy's own
+ * reductions, a group worked by hand, exact rationals with the clamp, the pinned group routine on
+ * numpy's extremes, textbook (causal) attention in numpy, reduction to the pinned decode attention.
  *
  * Parity unpinned: none of the arithmetic.  The physical order of codes inside a 16-token tile is a
  * design choice the paper does not fix; it is pinned only against the published tensor-core
