@@ -100,13 +100,14 @@ class Cache:
     """Host-side cache buffers (numpy, zero-initialised) in the library's layout."""
 
     def __init__(self, cfg: Config, bitmask: Optional[np.ndarray] = None, sink_pos: Optional[np.ndarray] = None,
-                 sink_count: Optional[np.ndarray] = None):
+                 sink_count: Optional[np.ndarray] = None, per_token_keys: bool = False):
         sz = cache_sizes(cfg)
         self.cfg, self.sizes = cfg, sz
         self.k_codes = np.zeros(sz["k_codes_bytes"], np.uint8)
         self.v_codes = np.zeros(sz["v_codes_bytes"], np.uint8)
-        self.k_scale = np.zeros(sz["k_param_floats"], np.float32)
-        self.k_zero = np.zeros(sz["k_param_floats"], np.float32)
+        # per-token keys: the key parameters have the value parameters' shape [units][max_seq][D / v_group]
+        self.k_scale = np.zeros(sz["v_param_floats" if per_token_keys else "k_param_floats"], np.float32)
+        self.k_zero = np.zeros(sz["v_param_floats" if per_token_keys else "k_param_floats"], np.float32)
         self.v_scale = np.zeros(sz["v_param_floats"], np.float32)
         self.v_zero = np.zeros(sz["v_param_floats"], np.float32)
         self.k_tail = np.zeros(sz["k_tail_halfs"], np.uint16)
@@ -296,4 +297,28 @@ def prefill_attention(cfg: Config, cache: Cache, q: np.ndarray, q_pos0: int):
     _check(lib().kvo_prefill_attention(C.byref(cfg.c()), C.byref(cc), qq.ctypes.data_as(C.c_void_p), C.c_int32(T), C.c_int32(q_pos0),
                                        C.c_int64(qq.strides[0] // 2), C.c_int64(qq.strides[1] // 2), C.c_int64(qq.strides[2] // 2),
                                        out.ctypes.data_as(C.c_void_p), lse.ctypes.data_as(C.c_void_p)), "prefill_attention")
+    return out, lse
+
+
+# ---- per-token keys (Section 4.1 "Per-token quantization"; Section 5.1's per-token Key and Value dynamic scheme) ----
+def quantize_append_pertoken(cfg: Config, cache: Cache, k_new: np.ndarray, v_new: np.ndarray) -> None:
+    """Keys and values per token, dynamic; `cache` must have been made with per_token_keys=True."""
+    k, v = _u16(k_new), _u16(v_new)
+    assert k.shape == v.shape and k.strides == v.strides and k.strides[3] == 2
+    assert cache.k_scale.size == cache.sizes["v_param_floats"]
+    cc = cache.c()
+    rc = lib().kvo_quantize_append_pertoken(C.byref(cfg.c()), C.byref(cc), k.ctypes.data_as(C.c_void_p), v.ctypes.data_as(C.c_void_p),
+                                            C.c_int32(k.shape[2]), C.c_int64(k.strides[0] // 2), C.c_int64(k.strides[1] // 2),
+                                            C.c_int64(k.strides[2] // 2))
+    _check(rc, "quantize_append_pertoken")
+    cache.seq_len = cc.seq_len
+
+
+def decode_attention_pertoken(cfg: Config, cache: Cache, q: np.ndarray):
+    qq = np.ascontiguousarray(_u16(q))
+    out = np.zeros((cfg.batch, cfg.n_q_heads, cfg.head_dim), np.float64)
+    lse = np.zeros((cfg.batch, cfg.n_q_heads), np.float64)
+    cc = cache.c()
+    _check(lib().kvo_decode_attention_pertoken(C.byref(cfg.c()), C.byref(cc), qq.ctypes.data_as(C.c_void_p),
+                                               out.ctypes.data_as(C.c_void_p), lse.ctypes.data_as(C.c_void_p)), "decode_attention_pertoken")
     return out, lse

@@ -861,3 +861,107 @@ int kvo_prefill_attention(const kvo_config *c, const kvo_cache *cache, const uin
     }
     return KVO_OK;
 }
+
+/* =====================================================================================================
+ * Per-token keys (Section 4.1 "Per-token quantization"; Section 5.1's "per-token Key and Value dynamic" scheme):
+ * keys are quantized like values -- per token over groups of min(group, D) consecutive channels, parameters computed
+ * on the fly -- so a key is coded on arrival and there is neither a token group nor a tail.  Sink tokens keep exact
+ * rows in the side buffer, code 0 and parameters (0, 0) (Algorithm 1's exclusion).
+ * Cache fields: k_scale, k_zero hold [B*Hkv][max_seq][D / v_group] floats (the value parameters' shape); k_tail is
+ * not used.
+ * ===================================================================================================== */
+int kvo_quantize_append_pertoken(const kvo_config *c, kvo_cache *cache, const uint16_t *k_new, const uint16_t *v_new, int32_t T,
+                                 int64_t stride_b, int64_t stride_h, int64_t stride_t)
+{
+    int rc = check_config(c);
+    if (rc) return rc;
+    if (!cache || !k_new || !v_new || T < 0) return KVO_ERR_BAD_ARG;
+    if (cache->seq_len < 0 || (int64_t)cache->seq_len + T > c->max_seq) return KVO_ERR_SEQ_OVERFLOW;
+    const int D = c->head_dim, gv = v_group_of(c), ngv = D / gv, cap = sink_cap_of(c), Hk = c->n_kv_heads;
+    int bad = 0;
+    float *xs = (float *)malloc(sizeof(float) * (size_t)gv);
+    uint8_t *mem = (uint8_t *)malloc((size_t)gv);
+    int32_t *codes = (int32_t *)malloc(sizeof(int32_t) * (size_t)gv);
+    for (int64_t unit = 0; unit < (int64_t)c->batch * Hk; ++unit) {
+        const int b = (int)(unit / Hk), h = (int)(unit % Hk);
+        for (int i = 0; i < T; ++i) {
+            int p = cache->seq_len + i;
+            const uint16_t *krow = k_new + b * stride_b + h * stride_h + i * stride_t;
+            const uint16_t *vrow = v_new + b * stride_b + h * stride_h + i * stride_t;
+            int sink = mask_bit(cache->sink_bitmask, c, b, p);
+            if (sink) {
+                int slot = sink_slot(c, cache, b, p);
+                if (slot < 0) { bad = 1; continue; }
+                memcpy(cache->sink_k + (unit * cap + slot) * D, krow, sizeof(uint16_t) * (size_t)D);
+                memcpy(cache->sink_v + (unit * cap + slot) * D, vrow, sizeof(uint16_t) * (size_t)D);
+            }
+            for (int kind = 0; kind < 2; ++kind) {
+                const uint16_t *row = kind ? vrow : krow;
+                float *ps = kind ? cache->v_scale : cache->k_scale, *pz = kind ? cache->v_zero : cache->k_zero;
+                for (int j = 0; j < ngv; ++j) {
+                    float sc = 0.0f, ze = 0.0f;
+                    for (int e = 0; e < gv; ++e) { xs[e] = half_to_float(row[j * gv + e]); mem[e] = (uint8_t)!sink; }
+                    kvo_quantize_group(xs, mem, gv, c->bits, &sc, &ze, codes);
+                    ps[(unit * c->max_seq + p) * ngv + j] = sc;
+                    pz[(unit * c->max_seq + p) * ngv + j] = ze;
+                    for (int e = 0; e < gv; ++e) {
+                        if (kind) v_code_put(cache->v_codes, c, b, h, p, j * gv + e, (uint32_t)codes[e]);
+                        else k_code_put(cache->k_codes, c, b, h, p, j * gv + e, (uint32_t)codes[e]);
+                    }
+                }
+            }
+        }
+    }
+    free(xs); free(mem); free(codes);
+    if (bad) return KVO_ERR_BAD_ARG;
+    cache->seq_len += T;
+    return KVO_OK;
+}
+
+/* Eq. 3 / Eq. 7 over a cache with per-token keys: binary64, as kvo_decode_attention. */
+int kvo_decode_attention_pertoken(const kvo_config *c, const kvo_cache *cache, const uint16_t *q, double *out, double *lse)
+{
+    int rc = check_config(c);
+    if (rc) return rc;
+    if (!cache || !q || !out) return KVO_ERR_BAD_ARG;
+    const int D = c->head_dim, n = cache->seq_len, rep = c->n_q_heads / c->n_kv_heads, gv = v_group_of(c), ngv = D / gv;
+    const int cap = sink_cap_of(c);
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int64_t bh = 0; bh < (int64_t)c->batch * c->n_q_heads; ++bh) {
+        const int b = (int)(bh / c->n_q_heads), hq = (int)(bh % c->n_q_heads), h = hq / rep;
+        const int64_t unit = (int64_t)b * c->n_kv_heads + h;
+        double *s = (double *)malloc(sizeof(double) * (size_t)(n > 0 ? n : 1));
+        const uint16_t *qv = q + ((int64_t)b * c->n_q_heads + hq) * D;
+        double *o = out + ((int64_t)b * c->n_q_heads + hq) * D;
+        double mx = -INFINITY;
+        for (int p = 0; p < n; ++p) {
+            int slot = mask_bit(cache->sink_bitmask, c, b, p) ? sink_slot(c, cache, b, p) : -2;
+            double acc = 0.0;
+            for (int ch = 0; ch < D; ++ch) {
+                int64_t pi = (unit * c->max_seq + p) * ngv + ch / gv;
+                double kv = slot == -2 ? (double)dequant(cache->k_scale[pi], cache->k_zero[pi], k_code_get(cache->k_codes, c, b, h, p, ch))
+                                       : (slot < 0 ? NAN : (double)half_to_float(cache->sink_k[(unit * cap + slot) * D + ch]));
+                acc += (double)half_to_float(qv[ch]) * kv;
+            }
+            s[p] = acc / sqrt((double)D);
+            if (s[p] > mx) mx = s[p];
+        }
+        double den = 0.0;
+        for (int ch = 0; ch < D; ++ch) o[ch] = 0.0;
+        for (int p = 0; p < n; ++p) {
+            int slot = mask_bit(cache->sink_bitmask, c, b, p) ? sink_slot(c, cache, b, p) : -2;
+            double w = exp(s[p] - mx);
+            den += w;
+            for (int ch = 0; ch < D; ++ch) {
+                int64_t pi = (unit * c->max_seq + p) * ngv + ch / gv;
+                double vv = slot == -2 ? (double)dequant(cache->v_scale[pi], cache->v_zero[pi], v_code_get(cache->v_codes, c, b, h, p, ch))
+                                       : (slot < 0 ? NAN : (double)half_to_float(cache->sink_v[(unit * cap + slot) * D + ch]));
+                o[ch] += w * vv;
+            }
+        }
+        for (int ch = 0; ch < D; ++ch) o[ch] = n > 0 ? o[ch] / den : 0.0;
+        if (lse) lse[(int64_t)b * c->n_q_heads + hq] = n > 0 ? mx + log(den) : -INFINITY;
+        free(s);
+    }
+    return KVO_OK;
+}
