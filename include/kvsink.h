@@ -104,7 +104,7 @@ typedef struct kvsink_sizes {
     int64_t k_tail_halfs, sink_halfs;       /* fp16 elements; sink_halfs for each of sink_k, sink_v */
     int64_t bitmask_words, sink_pos_ints;
     int64_t predict_workspace_bytes;        /* for kvsink_predict_sinks with S == max_seq */
-    int64_t decode_workspace_bytes;         /* for kvsink_decode_attention and kvsink_decode_attention_calibrated */
+    int64_t decode_workspace_bytes;         /* for kvsink_decode_attention and its _calibrated and _pertoken forms */
     int64_t calibrate_workspace_bytes;      /* for kvsink_calibrate */
     int32_t sink_capacity, v_group, v_groups_per_row, tile_bytes;
 } kvsink_sizes;
@@ -242,6 +242,27 @@ int kvsink_quantize_append_calibrated(const kvsink_config *cfg, kvsink_cache *ca
  */
 int kvsink_decode_attention_calibrated(const kvsink_config *cfg, const kvsink_cache *cache, const kvsink_static_params *params, const void *q,
                                        float *out, float *lse, void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/*
+ * Per-token keys (Section 4.1, "Per-token quantization"; the per-token Key and Value dynamic scheme of Section 5.1's
+ * evaluation with KVQuant's granularities): keys are quantized like values, one (scale, zero) of Eq. 10-11 per token and
+ * channel group of min(G, D) channels.  In a cache used this way k_scale and k_zero are float [u][max_seq][D/Gv] (the
+ * shape of v_scale; kvsink_sizes.v_param_floats floats each) and k_tail is not used and may be null.
+ *
+ * kvsink_quantize_append_pertoken: every token is coded on arrival (any T >= 0 at any time); a token whose mask bit is set
+ * keeps exact fp16 rows in the side buffer, gets code 0 everywhere and scale = zero = 0.  Arguments, strides, ownership
+ * and errors as kvsink_quantize_append.
+ *
+ * kvsink_decode_attention_pertoken: Eq. 3 / Eq. 7 over such a cache; arguments as kvsink_decode_attention.
+ *
+ * Both are built for head size 128, one or two channel groups per row and at most four query heads per KV head (3 bit:
+ * one group and one query head); other shapes return KVSINK_ERR_UNSUPPORTED.  A cache is used with one kind of parameters
+ * only.
+ */
+int kvsink_quantize_append_pertoken(const kvsink_config *cfg, kvsink_cache *cache, const void *k_new, const void *v_new, int32_t T,
+                                    int64_t stride_b, int64_t stride_h, int64_t stride_t, void *cuda_stream);
+int kvsink_decode_attention_pertoken(const kvsink_config *cfg, const kvsink_cache *cache, const void *q, float *out, float *lse,
+                                     void *workspace, size_t workspace_bytes, void *cuda_stream);
 
 /*
  * Largest magnitude of every hidden channel over all tokens of all sequences: out[c] = max |hidden[b][i][c]| (a NaN

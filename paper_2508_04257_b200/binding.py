@@ -18,7 +18,8 @@ _LIB_PATH = os.environ.get("KVSINK_LIB") or os.path.join(_HERE, "libkvsink.so")
 
 EXPORTS = ("kvsink_cache_sizes", "kvsink_predict_sinks", "kvsink_quantize_append", "kvsink_decode_attention",
            "kvsink_decode_attention_static", "kvsink_prefill_attention", "kvsink_calibrate", "kvsink_quantize_append_calibrated",
-           "kvsink_decode_attention_calibrated", "kvsink_channel_absmax", "kvsink_quant_error", "kvsink_read_status",
+           "kvsink_decode_attention_calibrated", "kvsink_quantize_append_pertoken", "kvsink_decode_attention_pertoken",
+           "kvsink_channel_absmax", "kvsink_quant_error", "kvsink_read_status",
            "kvsink_launch_count", "kvsink_strerror")
 STATIC_SCRATCH_BYTES = 4 * 1024 * 1024
 
@@ -116,14 +117,17 @@ class SinkSet:
 
 
 class KVCache:
-    """Device buffers of one layer's cache, zero-filled, in the layout kvsink.h documents."""
+    """Device buffers of one layer's cache, zero-filled, in the layout kvsink.h documents.  With per_token_keys the key
+    parameters take the value parameters' shape (for quantize_append_pertoken / decode_attention_pertoken)."""
 
-    def __init__(self, cfg: Config, sinks: Optional[SinkSet] = None, device="cuda"):
+    def __init__(self, cfg: Config, sinks: Optional[SinkSet] = None, device="cuda", per_token_keys: bool = False):
         sz = cache_sizes(cfg)
         self.cfg, self.sizes = cfg, sz
         z = lambda n, dt: torch.zeros(max(int(n), 1), dtype=dt, device=device)
         self.k_codes, self.v_codes = z(sz["k_codes_bytes"], torch.uint8), z(sz["v_codes_bytes"], torch.uint8)
-        self.k_scale, self.k_zero = z(sz["k_param_floats"], torch.float32), z(sz["k_param_floats"], torch.float32)
+        self.per_token_keys = per_token_keys
+        nkp = sz["v_param_floats"] if per_token_keys else sz["k_param_floats"]
+        self.k_scale, self.k_zero = z(nkp, torch.float32), z(nkp, torch.float32)
         self.v_scale, self.v_zero = z(sz["v_param_floats"], torch.float32), z(sz["v_param_floats"], torch.float32)
         self.k_tail = z(sz["k_tail_halfs"], torch.float16)
         self.sink_k, self.sink_v = z(sz["sink_halfs"], torch.float16), z(sz["sink_halfs"], torch.float16)
@@ -276,6 +280,38 @@ def decode_attention_calibrated(cfg: Config, cache: KVCache, params: StaticParam
                                                   C.c_size_t(workspace.numel()), _stream())
     if rc:
         raise KvsinkError(rc, "kvsink_decode_attention_calibrated")
+    return out, lse
+
+
+def quantize_append_pertoken(cfg: Config, cache: KVCache, k_new: torch.Tensor, v_new: torch.Tensor) -> None:
+    """kvsink_quantize_append_pertoken: k_new, v_new fp16 [B, Hkv, T, D] on the device with equal strides."""
+    assert cache.per_token_keys, "the cache was not sized for per-token key parameters"
+    assert k_new.is_cuda and k_new.dtype == torch.float16 and k_new.dim() == 4 and k_new.stride(3) == 1
+    assert v_new.shape == k_new.shape and v_new.stride() == k_new.stride() and v_new.dtype == torch.float16
+    cc = cache.c()
+    rc = lib().kvsink_quantize_append_pertoken(C.byref(cfg.c()), C.byref(cc), _ptr(k_new), _ptr(v_new), C.c_int32(k_new.shape[2]),
+                                               C.c_int64(k_new.stride(0)), C.c_int64(k_new.stride(1)), C.c_int64(k_new.stride(2)), _stream())
+    if rc:
+        raise KvsinkError(rc, "kvsink_quantize_append_pertoken")
+    cache.seq_len = cc.seq_len
+
+
+def decode_attention_pertoken(cfg: Config, cache: KVCache, q: torch.Tensor, out: Optional[torch.Tensor] = None,
+                              lse: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None, want_lse: bool = True):
+    """kvsink_decode_attention_pertoken: q fp16 [B, Hq, D] contiguous. Returns (out fp32 [B,Hq,D], lse fp32 [B,Hq] or None)."""
+    assert cache.per_token_keys, "the cache was not sized for per-token key parameters"
+    assert q.is_cuda and q.dtype == torch.float16 and q.is_contiguous()
+    if out is None:
+        out = torch.empty((cfg.batch, cfg.n_q_heads, cfg.head_dim), dtype=torch.float32, device=q.device)
+    if lse is None and want_lse:
+        lse = torch.empty((cfg.batch, cfg.n_q_heads), dtype=torch.float32, device=q.device)
+    if workspace is None:
+        workspace = torch.empty(cache.sizes["decode_workspace_bytes"], dtype=torch.uint8, device=q.device)
+    cc = cache.c()
+    rc = lib().kvsink_decode_attention_pertoken(C.byref(cfg.c()), C.byref(cc), _ptr(q), _ptr(out), _ptr(lse), _ptr(workspace),
+                                                C.c_size_t(workspace.numel()), _stream())
+    if rc:
+        raise KvsinkError(rc, "kvsink_decode_attention_pertoken")
     return out, lse
 
 

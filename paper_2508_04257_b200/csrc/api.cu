@@ -157,7 +157,7 @@ extern "C" int kvsink_decode_attention(const kvsink_config *cfg, const kvsink_ca
     if (rc) return rc;
     if (!aligned16(q) || !aligned16(out)) return KVSINK_ERR_BAD_ARG;
     if (!aligned16(workspace)) return KVSINK_ERR_WORKSPACE;
-    return launch_decode(p, *cache, nullptr, (const __half *)q, out, lse, workspace, workspace_bytes, (cudaStream_t)cuda_stream);
+    return launch_decode(p, *cache, nullptr, 0, (const __half *)q, out, lse, workspace, workspace_bytes, (cudaStream_t)cuda_stream);
 }
 
 extern "C" int kvsink_prefill_attention(const kvsink_config *cfg, const kvsink_cache *cache, const void *q, int32_t T, int32_t q_pos0,
@@ -251,7 +251,61 @@ extern "C" int kvsink_decode_attention_calibrated(const kvsink_config *cfg, cons
     if (rc) return rc;
     if (!aligned16(q) || !aligned16(out)) return KVSINK_ERR_BAD_ARG;
     if (!aligned16(workspace)) return KVSINK_ERR_WORKSPACE;
-    return launch_decode(p, *cache, params, (const __half *)q, out, lse, workspace, workspace_bytes, (cudaStream_t)cuda_stream);
+    return launch_decode(p, *cache, params, 1, (const __half *)q, out, lse, workspace, workspace_bytes, (cudaStream_t)cuda_stream);
+}
+
+// A cache with per-token keys: k_scale / k_zero have the value parameters' shape and there is no key tail.
+static int check_cache_pertoken(const kvsink_cache *c, const Params &p)
+{
+    if (!c) return KVSINK_ERR_BAD_ARG;
+    if (!aligned16(c->k_codes) || !aligned16(c->v_codes) || !aligned16(c->sink_bitmask) || !c->sink_count || !c->status) return KVSINK_ERR_BAD_ARG;
+    if (!aligned16(c->k_scale) || !aligned16(c->k_zero) || !aligned16(c->v_scale) || !aligned16(c->v_zero)) return KVSINK_ERR_BAD_ARG;
+    if (p.cap > 0 && (!aligned16(c->sink_k) || !aligned16(c->sink_v) || !c->sink_pos)) return KVSINK_ERR_BAD_ARG;
+    if (c->seq_len < 0 || c->seq_len > p.max_seq) return KVSINK_ERR_BAD_ARG;
+    return KVSINK_OK;
+}
+
+// The shapes the per-token key kernels are built for.
+static bool pertoken_supported(const Params &p)
+{
+    if (p.D != 128 || p.NGv > 2 || p.rep > 4) return false;
+    if (p.bits == 3 && (p.NGv != 1 || p.rep != 1)) return false;
+    return true;
+}
+
+extern "C" int kvsink_quantize_append_pertoken(const kvsink_config *cfg, kvsink_cache *cache, const void *k_new, const void *v_new, int32_t T,
+                                               int64_t stride_b, int64_t stride_h, int64_t stride_t, void *cuda_stream)
+{
+    Params p;
+    int rc = derive(cfg, &p);
+    if (rc) return rc;
+    if (!pertoken_supported(p)) return KVSINK_ERR_UNSUPPORTED;
+    rc = check_cache_pertoken(cache, p);
+    if (rc) return rc;
+    if (T < 0) return KVSINK_ERR_BAD_ARG;
+    if (T == 0) return KVSINK_OK;
+    if (!aligned16(k_new) || !aligned16(v_new)) return KVSINK_ERR_BAD_ARG;
+    if (stride_t < p.D || (stride_t % 8) || (stride_h % 8) || (stride_b % 8) || stride_h < 0 || stride_b < 0) return KVSINK_ERR_BAD_ARG;
+    if ((int64_t)cache->seq_len + T > p.max_seq) return KVSINK_ERR_SEQ_OVERFLOW;
+    rc = launch_quantize_pertoken(p, *cache, (const __half *)k_new, (const __half *)v_new, cache->seq_len, T, stride_b, stride_h, stride_t,
+                                  (cudaStream_t)cuda_stream);
+    if (rc) return rc;
+    cache->seq_len += T;
+    return KVSINK_OK;
+}
+
+extern "C" int kvsink_decode_attention_pertoken(const kvsink_config *cfg, const kvsink_cache *cache, const void *q, float *out, float *lse,
+                                                void *workspace, size_t workspace_bytes, void *cuda_stream)
+{
+    Params p;
+    int rc = derive(cfg, &p);
+    if (rc) return rc;
+    if (!pertoken_supported(p)) return KVSINK_ERR_UNSUPPORTED;
+    rc = check_cache_pertoken(cache, p);
+    if (rc) return rc;
+    if (!aligned16(q) || !aligned16(out)) return KVSINK_ERR_BAD_ARG;
+    if (!aligned16(workspace)) return KVSINK_ERR_WORKSPACE;
+    return launch_decode(p, *cache, nullptr, 2, (const __half *)q, out, lse, workspace, workspace_bytes, (cudaStream_t)cuda_stream);
 }
 
 extern "C" int kvsink_channel_absmax(const void *hidden, int32_t B, int32_t S, int32_t d, int64_t stride_b, int64_t stride_s, float *out,

@@ -5,6 +5,9 @@
 //                 non-sink tokens, then Eq. 10-11
 //   append      : every token is coded on arrival with the fixed pairs (Eq. 8, values outside the calibrated range clamp);
 //                 no key tail, no per-group parameters; sink rows go to the side buffer
+// The same two append kernels serve per-token keys (PT; Section 4.1 "Per-token quantization", Section 5.1's per-token Key and
+// Value dynamic scheme): keys and values alike get one (scale, zero) per token and channel group, computed on arrival from
+// the token's own extremes (Eq. 10-11) and stored in the cache's parameter arrays, sink tokens (0, 0).
 #include "common.cuh"
 #include "tile_words.cuh"
 
@@ -114,6 +117,7 @@ __device__ __forceinline__ uint32_t code_static(float x, float s, float z, float
 // (fields of earlier tokens keep their bits; a tile whose first token arrives is written whole).
 constexpr int CQ_THREADS = 128;
 
+template <bool PT>
 __global__ void __launch_bounds__(CQ_THREADS)
 quantize_calibrated_kernel(Params p, kvsink_cache c, kvsink_static_params sp, const __half *__restrict__ k_src, const __half *__restrict__ v_src,
                            int first_token, int n_tokens, int64_t sb, int64_t sh, int64_t stt)
@@ -136,8 +140,11 @@ quantize_calibrated_kernel(Params p, kvsink_cache c, kvsink_static_params sp, co
     float ks[4], kz[4], vs[4], vz[4];
     for (int e = 0; e < cpl; ++e) {
         const int ch = lane * cpl + e;
-        ks[e] = sp.k_scale[h * D + ch]; kz[e] = sp.k_zero[h * D + ch];
-        vs[e] = sp.v_scale[h * p.NGv + ch / p.Gv]; vz[e] = sp.v_zero[h * p.NGv + ch / p.Gv];
+        ks[e] = kz[e] = vs[e] = vz[e] = 0.f;
+        if constexpr (!PT) {
+            ks[e] = sp.k_scale[h * D + ch]; kz[e] = sp.k_zero[h * D + ch];
+            vs[e] = sp.v_scale[h * p.NGv + ch / p.Gv]; vz[e] = sp.v_zero[h * p.NGv + ch / p.Gv];
+        }
     }
     for (int pos = t_lo + warp; pos < t_hi; pos += CQ_THREADS / 32) {
         const int64_t src = b * sb + h * sh + (int64_t)(pos - first_token) * stt;
@@ -153,6 +160,28 @@ quantize_calibrated_kernel(Params p, kvsink_cache c, kvsink_static_params sp, co
                 __half *dk = (__half *)c.sink_k + ((size_t)unit * p.cap + slot) * D;
                 __half *dv = (__half *)c.sink_v + ((size_t)unit * p.cap + slot) * D;
                 for (int e = 0; e < cpl; ++e) { dk[lane * cpl + e] = kx[e]; dv[lane * cpl + e] = vx[e]; }
+            }
+        }
+        if constexpr (PT) {
+            // the token's own parameters: min / max over the lanes of each channel group, keys and values alike
+            float kmn = __half2float(kx[0]), kmx = kmn, vmn = __half2float(vx[0]), vmx = vmn;
+            for (int e = 1; e < cpl; ++e) {
+                kmn = fminf(kmn, __half2float(kx[e])); kmx = fmaxf(kmx, __half2float(kx[e]));
+                vmn = fminf(vmn, __half2float(vx[e])); vmx = fmaxf(vmx, __half2float(vx[e]));
+            }
+            const int lanes_per_group = p.Gv / cpl;
+            for (int o = 1; o < lanes_per_group; o <<= 1) {
+                kmn = fminf(kmn, __shfl_xor_sync(0xffffffffu, kmn, o)); kmx = fmaxf(kmx, __shfl_xor_sync(0xffffffffu, kmx, o));
+                vmn = fminf(vmn, __shfl_xor_sync(0xffffffffu, vmn, o)); vmx = fmaxf(vmx, __shfl_xor_sync(0xffffffffu, vmx, o));
+            }
+            float s0, z0, s1, z1;
+            group_params(!sink, kmn, kmx, qmax, &s0, &z0);
+            group_params(!sink, vmn, vmx, qmax, &s1, &z1);
+            for (int e = 0; e < cpl; ++e) { ks[e] = s0; kz[e] = z0; vs[e] = s1; vz[e] = z1; }
+            if (lane % lanes_per_group == 0) {
+                const size_t o = ((size_t)unit * p.max_seq + pos) * p.NGv + lane / lanes_per_group;
+                c.k_scale[o] = s0; c.k_zero[o] = z0;
+                c.v_scale[o] = s1; c.v_zero[o] = z1;
             }
         }
         for (int e = 0; e < cpl; ++e) {
@@ -196,7 +225,7 @@ __device__ __forceinline__ uint32_t code_static_fast(float x, float s, float r, 
 // tiles, so the lane's words come out in the tile's own order and are stored with one 16-byte (or 8-byte) store per plane.
 constexpr int CF_WARPS = 4;
 
-template <int BITS>
+template <int BITS, bool PT>
 __global__ void __launch_bounds__(32 * CF_WARPS)
 quantize_calibrated_tiles_kernel(Params p, kvsink_cache c, kvsink_static_params sp, const __half *__restrict__ k_src,
                                  const __half *__restrict__ v_src, int first_token, int n_tiles, int64_t sb, int64_t sh, int64_t stt)
@@ -205,13 +234,14 @@ quantize_calibrated_tiles_kernel(Params p, kvsink_cache c, kvsink_static_params 
     constexpr int ROW = D + 8;                                 // padded row (halves): conflict-free column reads
     __shared__ __align__(16) __half s_k[CF_WARPS][KVSINK_TILE * ROW], s_v[CF_WARPS][KVSINK_TILE * ROW];
     __shared__ float4 s_kp[D];                                 // (scale, 1 / scale, zero) of the KV head's key channels
+    __shared__ float4 s_pt[PT ? CF_WARPS : 1][2][KVSINK_TILE][4];   // per-token keys: the same per (K / V, token, 32-channel block)
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = lane >> 2, t = lane & 3;
     const int h = blockIdx.y, b = blockIdx.z;
     const int64_t unit = (int64_t)b * p.Hkv + h;
     const float qmax = (float)((1 << BITS) - 1);
     const uint32_t *bm = c.sink_bitmask + (size_t)b * p.mask_words;
     pdl_wait();
-    for (int i = tid; i < D; i += 32 * CF_WARPS) {
+    for (int i = tid; i < D && !PT; i += 32 * CF_WARPS) {
         const float sc = sp.k_scale[h * D + i];
         s_kp[i] = make_float4(sc, sc == 0.f ? 0.f : __frcp_rn(sc), sp.k_zero[h * D + i], 0.f);
     }
@@ -245,6 +275,45 @@ quantize_calibrated_tiles_kernel(Params p, kvsink_cache c, kvsink_static_params 
             }
         }
     }
+    if constexpr (PT) {
+        // per-token parameters: lane -> token lane / 2, channels 64 (lane % 2) ... + 63 as two 32-channel blocks, combined to
+        // the channel group (32, 64 or 128 channels) and written to the parameter arrays by the group's first lane
+        const int tk = lane >> 1, hf = lane & 1;
+        const bool sink = (mask16 >> tk) & 1u;
+#pragma unroll
+        for (int kind = 0; kind < 2; ++kind) {
+            const __half *row = (kind ? mv : mk) + tk * ROW + 64 * hf;
+            float mn[2], mx[2];
+#pragma unroll
+            for (int sbk = 0; sbk < 2; ++sbk) {
+                __half2 lo = *reinterpret_cast<const __half2 *>(row + 32 * sbk), hi = lo;
+#pragma unroll
+                for (int i = 1; i < 16; ++i) {
+                    const __half2 x = *reinterpret_cast<const __half2 *>(row + 32 * sbk + 2 * i);
+                    lo = __hmin2(lo, x); hi = __hmax2(hi, x);
+                }
+                mn[sbk] = fminf(__low2float(lo), __high2float(lo)); mx[sbk] = fmaxf(__low2float(hi), __high2float(hi));
+            }
+            if (p.Gv >= 64) { mn[0] = mn[1] = fminf(mn[0], mn[1]); mx[0] = mx[1] = fmaxf(mx[0], mx[1]); }
+            if (p.Gv >= 128) {
+                mn[0] = mn[1] = fminf(mn[0], __shfl_xor_sync(0xffffffffu, mn[0], 1));
+                mx[0] = mx[1] = fmaxf(mx[0], __shfl_xor_sync(0xffffffffu, mx[0], 1));
+            }
+            float *ps = kind ? c.v_scale : c.k_scale, *pz = kind ? c.v_zero : c.k_zero;
+#pragma unroll
+            for (int sbk = 0; sbk < 2; ++sbk) {
+                float sc, ze;
+                group_params(!sink, mn[sbk], mx[sbk], qmax, &sc, &ze);
+                const int ch0 = 64 * hf + 32 * sbk;
+                s_pt[warp][kind][tk][2 * hf + sbk] = make_float4(sc, sc == 0.f ? 0.f : __frcp_rn(sc), ze, 0.f);
+                if (ch0 % p.Gv == 0) {
+                    const size_t o = ((size_t)unit * p.max_seq + tok0 + tk) * p.NGv + ch0 / p.Gv;
+                    ps[o] = sc; pz[o] = ze;
+                }
+            }
+        }
+        __syncwarp();
+    }
     // codes of pair slot s = 4m + r, half e: keys (token, channel) = (g + 8(r&1), 16m + 8(r>>1) + 2t + e),
     //                                        values (channel, token) = (16m + g + 8(r&1), 8(r>>1) + 2t + e)
     uint32_t kw[W], vw[W];
@@ -253,7 +322,8 @@ quantize_calibrated_tiles_kernel(Params p, kvsink_cache c, kvsink_static_params 
 #pragma unroll
     for (int m = 0; m < D / 16; ++m) {
         const int vj = (16 * m) / p.Gv;   // value channel group of this matrix (groups are multiples of 16 channels)
-        const float vs = sp.v_scale[h * p.NGv + vj], vz = sp.v_zero[h * p.NGv + vj], vr = vs == 0.f ? 0.f : __frcp_rn(vs);
+        float vs = 0.f, vz = 0.f, vr = 0.f;
+        if constexpr (!PT) { vs = sp.v_scale[h * p.NGv + vj]; vz = sp.v_zero[h * p.NGv + vj]; vr = vs == 0.f ? 0.f : __frcp_rn(vs); }
 #pragma unroll
         for (int r = 0; r < 4; ++r)
 #pragma unroll
@@ -261,9 +331,10 @@ quantize_calibrated_tiles_kernel(Params p, kvsink_cache c, kvsink_static_params 
                 const int s_ = 4 * m + r;
                 const int ktok = g + 8 * (r & 1), kch = 16 * m + 8 * (r >> 1) + 2 * t + e;
                 const int vch = 16 * m + g + 8 * (r & 1), vtok = 8 * (r >> 1) + 2 * t + e;
-                const float4 kp = s_kp[kch];
+                const float4 kp = PT ? s_pt[PT ? warp : 0][0][ktok][kch >> 5] : s_kp[kch];
+                const float4 vp = PT ? s_pt[PT ? warp : 0][1][vtok][vch >> 5] : make_float4(vs, vr, vz, 0.f);
                 const uint32_t kc = ((mask16 >> ktok) & 1u) || kp.x == 0.f ? 0u : code_static_fast(__half2float(mk[ktok * ROW + kch]), kp.x, kp.y, kp.z, qmax);
-                const uint32_t vc = ((mask16 >> vtok) & 1u) || vs == 0.f ? 0u : code_static_fast(__half2float(mv[vtok * ROW + vch]), vs, vr, vz, qmax);
+                const uint32_t vc = ((mask16 >> vtok) & 1u) || vp.x == 0.f ? 0u : code_static_fast(__half2float(mv[vtok * ROW + vch]), vp.x, vp.y, vp.z, qmax);
                 if constexpr (BITS == 2) {
                     kw[s_ / 8] |= kc << (16 * e + 2 * (s_ % 8)); vw[s_ / 8] |= vc << (16 * e + 2 * (s_ % 8));
                 } else if constexpr (BITS == 4) {
@@ -312,26 +383,39 @@ int launch_calibrate(const Params &p, const __half *k, const __half *v, int T, i
                                                                                                                                 : KVSINK_ERR_CUDA;
 }
 
-int launch_quantize_calibrated(const Params &p, const kvsink_cache &c, const kvsink_static_params &sp, const __half *k_src, const __half *v_src,
-                               int first_token, int n_tokens, int64_t sb, int64_t sh, int64_t stt, cudaStream_t st)
+template <bool PT>
+static int launch_tokens(const Params &p, const kvsink_cache &c, const kvsink_static_params &sp, const __half *k_src, const __half *v_src,
+                         int first_token, int n_tokens, int64_t sb, int64_t sh, int64_t stt, cudaStream_t st)
 {
     if (n_tokens <= 0) return KVSINK_OK;
     // whole fresh tiles of a head-size-128 cache take the tile kernel, the ragged rest (at most 15 tokens) the general one
     if (p.D == 128 && first_token % KVSINK_TILE == 0 && n_tokens >= KVSINK_TILE && ((uintptr_t)k_src & 15u) == 0 && ((uintptr_t)v_src & 15u) == 0) {
         const int n_tiles = n_tokens / KVSINK_TILE;
         const dim3 grid((n_tiles + CF_WARPS - 1) / CF_WARPS, p.Hkv, p.B);
-        cudaError_t e = p.bits == 2 ? launch_pdl(quantize_calibrated_tiles_kernel<2>, grid, dim3(32 * CF_WARPS), 0, st, p, c, sp, k_src, v_src, first_token, n_tiles, sb, sh, stt)
-                      : p.bits == 3 ? launch_pdl(quantize_calibrated_tiles_kernel<3>, grid, dim3(32 * CF_WARPS), 0, st, p, c, sp, k_src, v_src, first_token, n_tiles, sb, sh, stt)
-                                    : launch_pdl(quantize_calibrated_tiles_kernel<4>, grid, dim3(32 * CF_WARPS), 0, st, p, c, sp, k_src, v_src, first_token, n_tiles, sb, sh, stt);
+        cudaError_t e = p.bits == 2 ? launch_pdl(quantize_calibrated_tiles_kernel<2, PT>, grid, dim3(32 * CF_WARPS), 0, st, p, c, sp, k_src, v_src, first_token, n_tiles, sb, sh, stt)
+                      : p.bits == 3 ? launch_pdl(quantize_calibrated_tiles_kernel<3, PT>, grid, dim3(32 * CF_WARPS), 0, st, p, c, sp, k_src, v_src, first_token, n_tiles, sb, sh, stt)
+                                    : launch_pdl(quantize_calibrated_tiles_kernel<4, PT>, grid, dim3(32 * CF_WARPS), 0, st, p, c, sp, k_src, v_src, first_token, n_tiles, sb, sh, stt);
         if (e != cudaSuccess) return KVSINK_ERR_CUDA;
         const int done = n_tiles * KVSINK_TILE;
-        return launch_quantize_calibrated(p, c, sp, k_src + (int64_t)done * stt, v_src + (int64_t)done * stt, first_token + done, n_tokens - done, sb, sh,
-                                          stt, st);
+        return launch_tokens<PT>(p, c, sp, k_src + (int64_t)done * stt, v_src + (int64_t)done * stt, first_token + done, n_tokens - done, sb, sh, stt, st);
     }
     const int tiles = (first_token + n_tokens - 1) / KVSINK_TILE - first_token / KVSINK_TILE + 1;
     const dim3 grid(tiles, p.Hkv, p.B);
-    return launch_pdl(quantize_calibrated_kernel, grid, dim3(CQ_THREADS), 0, st, p, c, sp, k_src, v_src, first_token, n_tokens, sb, sh, stt) ==
+    return launch_pdl(quantize_calibrated_kernel<PT>, grid, dim3(CQ_THREADS), 0, st, p, c, sp, k_src, v_src, first_token, n_tokens, sb, sh, stt) ==
                    cudaSuccess ? KVSINK_OK : KVSINK_ERR_CUDA;
+}
+
+int launch_quantize_calibrated(const Params &p, const kvsink_cache &c, const kvsink_static_params &sp, const __half *k_src, const __half *v_src,
+                               int first_token, int n_tokens, int64_t sb, int64_t sh, int64_t stt, cudaStream_t st)
+{
+    return launch_tokens<false>(p, c, sp, k_src, v_src, first_token, n_tokens, sb, sh, stt, st);
+}
+
+int launch_quantize_pertoken(const Params &p, const kvsink_cache &c, const __half *k_src, const __half *v_src, int first_token, int n_tokens,
+                             int64_t sb, int64_t sh, int64_t stt, cudaStream_t st)
+{
+    const kvsink_static_params none = {nullptr, nullptr, nullptr, nullptr};
+    return launch_tokens<true>(p, c, none, k_src, v_src, first_token, n_tokens, sb, sh, stt, st);
 }
 
 }  // namespace kvsink

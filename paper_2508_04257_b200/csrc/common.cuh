@@ -150,7 +150,7 @@ int launch_quantize_groups_bulk(const Params &p, const kvsink_cache &c, const __
                                 int n_groups, int64_t sb, int64_t sh, int64_t stt, cudaStream_t st);
 int launch_quantize_tokens(const Params &p, const kvsink_cache &c, const __half *k_src, const __half *v_src, int src_offset,
                            int first_token, int n_tokens, int64_t sb, int64_t sh, int64_t stt, cudaStream_t st);
-int launch_decode(const Params &p, const kvsink_cache &c, const kvsink_static_params *cal, const __half *q, float *out, float *lse, void *workspace,
+int launch_decode(const Params &p, const kvsink_cache &c, const kvsink_static_params *cal, int mode, const __half *q, float *out, float *lse, void *workspace,
                   size_t workspace_bytes, cudaStream_t st);
 int launch_prefill_b2(const Params &p, const kvsink_cache &c, const __half *q, int T, int q_pos0, int64_t sb, int64_t sh, int64_t stt, float *out,
                       float *lse, cudaStream_t st);
@@ -162,13 +162,15 @@ int launch_calibrate(const Params &p, const __half *k, const __half *v, int T, i
                      const kvsink_static_params &sp, void *workspace, cudaStream_t st);
 int launch_quantize_calibrated(const Params &p, const kvsink_cache &c, const kvsink_static_params &sp, const __half *k_src, const __half *v_src,
                                int first_token, int n_tokens, int64_t sb, int64_t sh, int64_t stt, cudaStream_t st);
+int launch_quantize_pertoken(const Params &p, const kvsink_cache &c, const __half *k_src, const __half *v_src, int first_token, int n_tokens,
+                             int64_t sb, int64_t sh, int64_t stt, cudaStream_t st);
 size_t calibrate_workspace_bytes(const Params &p);
 int launch_decode_static(const Params &p, const kvsink_cache &c, const __half *q, float *out, float *lse, cudaStream_t st);
-int launch_decode_b2(const Params &p, const kvsink_cache &c, const kvsink_static_params *cal, const __half *q, float *out, float *lse, float *ws,
+int launch_decode_b2(const Params &p, const kvsink_cache &c, const kvsink_static_params *cal, int mode, const __half *q, float *out, float *lse, float *ws,
                      cudaStream_t st);
-int launch_decode_b3(const Params &p, const kvsink_cache &c, const kvsink_static_params *cal, const __half *q, float *out, float *lse, float *ws,
+int launch_decode_b3(const Params &p, const kvsink_cache &c, const kvsink_static_params *cal, int mode, const __half *q, float *out, float *lse, float *ws,
                      cudaStream_t st);
-int launch_decode_b4(const Params &p, const kvsink_cache &c, const kvsink_static_params *cal, const __half *q, float *out, float *lse, float *ws,
+int launch_decode_b4(const Params &p, const kvsink_cache &c, const kvsink_static_params *cal, int mode, const __half *q, float *out, float *lse, float *ws,
                      cudaStream_t st);
 int launch_decode_merge(const float *ws, int nsplit, int D, int n_rows, float *out, float *lse, cudaStream_t st);
 int max_splits(const Params &p);

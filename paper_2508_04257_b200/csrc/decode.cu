@@ -97,14 +97,14 @@ size_t decode_workspace_bytes(const Params &p)
     return (size_t)p.B * p.Hq * max_splits(p) * (p.D + 2) * sizeof(float) + 16;
 }
 
-int launch_decode(const Params &p, const kvsink_cache &c, const kvsink_static_params *cal, const __half *q, float *out, float *lse, void *workspace,
+int launch_decode(const Params &p, const kvsink_cache &c, const kvsink_static_params *cal, int mode, const __half *q, float *out, float *lse, void *workspace,
                   size_t workspace_bytes, cudaStream_t st)
 {
     if (workspace_bytes < decode_workspace_bytes(p)) return KVSINK_ERR_WORKSPACE;
     float *ws = (float *)workspace;
-    if (p.bits == 2) return launch_decode_b2(p, c, cal, q, out, lse, ws, st);
-    if (p.bits == 3) return launch_decode_b3(p, c, cal, q, out, lse, ws, st);
-    if (p.bits == 4) return launch_decode_b4(p, c, cal, q, out, lse, ws, st);
+    if (p.bits == 2) return launch_decode_b2(p, c, cal, mode, q, out, lse, ws, st);
+    if (p.bits == 3) return launch_decode_b3(p, c, cal, mode, q, out, lse, ws, st);
+    if (p.bits == 4) return launch_decode_b4(p, c, cal, mode, q, out, lse, ws, st);
     return KVSINK_ERR_UNSUPPORTED;
 }
 
@@ -133,7 +133,7 @@ int launch_decode_static(const Params &p, const kvsink_cache &c, const __half *q
         g_scratch_known[dev] = true;
     }
     // No clearing is needed: the split kernel writes every partial record the merge kernel reads.
-    return launch_decode(p, c, nullptr, q, out, lse, g_scratch_ptr[dev], (size_t)KVSINK_STATIC_SCRATCH_BYTES, st);
+    return launch_decode(p, c, nullptr, 0, q, out, lse, g_scratch_ptr[dev], (size_t)KVSINK_STATIC_SCRATCH_BYTES, st);
 }
 
 }  // namespace kvsink

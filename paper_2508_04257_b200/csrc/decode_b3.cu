@@ -3,10 +3,10 @@
 
 namespace kvsink {
 
-int launch_decode_b3(const Params &p, const kvsink_cache &c, const kvsink_static_params *cal, const __half *q, float *out, float *lse, float *ws,
+int launch_decode_b3(const Params &p, const kvsink_cache &c, const kvsink_static_params *cal, int mode, const __half *q, float *out, float *lse, float *ws,
                      cudaStream_t st)
 {
-    return launch_decode_bits<3>(p, c, cal, q, out, lse, ws, st);
+    return launch_decode_bits<3>(p, c, cal, mode, q, out, lse, ws, st);
 }
 
 int launch_prefill_b3(const Params &p, const kvsink_cache &c, const __half *q, int T, int q_pos0, int64_t sb, int64_t sh, int64_t stt, float *out,

@@ -181,12 +181,13 @@ constexpr int DEC_WAIT_LIMIT = 1 << 22;   // polls of a full-barrier before a wa
 
 // Shared-memory plan of a decode block, shared by the kernel and the launcher.  CT = tiles per ring chunk, NQMAX = the
 // most query heads a block of this instantiation serves (1 on the integer key side, 4 with the pair layout, else 8).
-template <int BITS, int D, int NGv, int CT, int NQMAX>
+template <int BITS, int D, int NGv, int CT, int NQMAX, bool KTOK = false>
 struct DecodePlan {
     static constexpr int W = D * BITS / 64, TILE_BYTES = 128 * W;
     static constexpr int BST = D + 8;                                   // padded row stride of the key B tables (bank spread)
     static constexpr int KV_BYTES = CT * TILE_BYTES, SZ_BYTES = CT * 16 * NGv * 4;
-    static constexpr int SLOT_BYTES = 2 * KV_BYTES + 2 * SZ_BYTES;      // K words, V words, V scales, V zeros of CT tiles
+    // K words, V words, V scales, V zeros of CT tiles; with per-token keys (KTOK) also the K scales and K zeros
+    static constexpr int SLOT_BYTES = 2 * KV_BYTES + (KTOK ? 4 : 2) * SZ_BYTES;
     static constexpr int NSLOT = (9216 / SLOT_BYTES >= 4) ? 4 : 2;      // power of two
     static constexpr int KP_BYTES = 2 * D * 4;                          // key scale + zero of one group
     static constexpr int WARP_RING = NSLOT * SLOT_BYTES + KP_BYTES;
@@ -218,6 +219,11 @@ struct DecodePlan {
 // token.  There are no token groups: the key B operand is prepared once per block, a ring chunk holds code words only, the
 // stream covers every tile up to the sequence length (tokens beyond it are masked) and there is no fp16 tail.
 //
+// KT (per-token keys, PM = 2): keys carry one (scale, zero) per token and channel group like the values, so the key B operand
+// holds the query alone (prepared once per block) and a token's parameters are applied to its dot products afterwards:
+// score = sum over channel groups j of scale[t][j] * (dot_j - zero[t][j] * sum of the query over group j).  The parameters
+// of a chunk's tokens arrive with the chunk.  Like CAL there are no token groups and no tail.  Integer key side only.
+//
 // PRE (attention of a chunk of prompt queries over the cache, Algorithm 1's attention statement): the eight accumulator
 // columns of a block are eight (query token, query head) rows of one KV head, token-major; query token t sits at position
 // q_pos0 + t and sees the cached tokens up to its own position, so every column has its own length limit.  One block streams
@@ -227,14 +233,14 @@ struct PrefillShape {
     int64_t q_sb, q_sh, q_st;    // element strides of q [B][Hq][T][D]
 };
 
-template <int BITS, int D, int NGv, int CT, bool PL, int I8 = 0, bool CAL = false, bool PRE = false>
+template <int BITS, int D, int NGv, int CT, bool PL, int I8 = 0, int PM = 0, bool PRE = false>
 __global__ void __launch_bounds__(DEC_THREADS, 4)
 decode_kernel(Params p, kvsink_cache c, kvsink_static_params sp, const __half *__restrict__ q, float *__restrict__ out, float *__restrict__ lse,
               float *__restrict__ part_ws, int nsplit, int groups_per_split, int qchunks, int seq_len, int cluster_merge, PrefillShape pre)
 {
     using G_ = Geo<BITS, D>;
     constexpr int NQMAX = I8 == 1 ? 1 : (PL ? 4 : 8);
-    using Plan = DecodePlan<BITS, D, NGv, CT, NQMAX>;
+    using Plan = DecodePlan<BITS, D, NGv, CT, NQMAX, PM == 2>;
     constexpr int NM = G_::NM, W = G_::W, BST = Plan::BST, TILE_WORDS = 32 * W;
     constexpr int NSLOT = Plan::NSLOT, SLOT_BYTES = Plan::SLOT_BYTES, KV_BYTES = Plan::KV_BYTES, SZ_BYTES = Plan::SZ_BYTES;
     constexpr int mpg = (D / NGv) / 16;                              // value matrices per channel group
@@ -245,7 +251,10 @@ decode_kernel(Params p, kvsink_cache c, kvsink_static_params sp, const __half *_
     constexpr float R1 = 1.f / G_::ROWF, C1 = 1.f / G_::COLF;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = __shfl_sync(0xffffffffu, tid >> 5, 0), g = lane >> 2, t = lane & 3;
-    static_assert(!PRE || (!PL && I8 == 0 && !CAL), "prompt queries take the eight-column fp16 path");
+    constexpr bool CAL = PM == 1, KT = PM == 2, FLAT = PM != 0;    // static parameters / per-token keys / either: no token groups
+    constexpr int NGK = KT ? NGv : 1;                              // separate dot products per tile on the key side
+    static_assert(!PRE || (!PL && I8 == 0 && !FLAT), "prompt queries take the eight-column fp16 path");
+    static_assert(!KT || (I8 != 0 && NGv <= 2 && (BITS != 3 || NGv == 1)), "per-token keys: integer key side, one or two channel groups");
     // decode: grid (splits, KV heads x blocks of eight query heads, sequences); prompt queries: grid (row blocks, KV heads, sequences)
     const int split = PRE ? 0 : blockIdx.x, h = PRE ? blockIdx.y : blockIdx.y / qchunks, qc = PRE ? blockIdx.x : blockIdx.y % qchunks, b = blockIdx.z;
     const int nq = I8 == 1 ? 1 : (PRE ? min(NQMAX, pre.T * p.rep - 8 * qc) : min(NQMAX, p.rep - 8 * qc)), hq0 = h * p.rep + (PRE ? 0 : 8 * qc);
@@ -254,10 +263,10 @@ decode_kernel(Params p, kvsink_cache c, kvsink_static_params sp, const __half *_
     auto row_limit = [&](int i) { return i < nq ? pre.q_pos0 + row_token(i) + 1 : 0; };    // cached tokens the row sees
     const int64_t unit = (int64_t)b * p.Hkv + h;
     // with static parameters a "group" of the loops below is one ring chunk, and every token belongs to one
-    const int G = CAL ? CT * KVSINK_TILE : p.G;
+    const int G = FLAT ? CT * KVSINK_TILE : p.G;
     const int n = PRE ? min(seq_len, row_limit(nq - 1)) : seq_len;                        // tokens this block looks at
-    const int n_groups = CAL ? (n + G - 1) / G : (PRE ? min(seq_len / G, (n + G - 1) / G) : n / G);
-    const int n_body = CAL ? n : (seq_len / G) * G;                                       // where the fp16 tail begins
+    const int n_groups = FLAT ? (n + G - 1) / G : (PRE ? min(seq_len / G, (n + G - 1) / G) : n / G);
+    const int n_body = FLAT ? n : (seq_len / G) * G;                                       // where the fp16 tail begins
     // limits of this lane's accumulator columns 2t, 2t+1 and the smallest limit of the block (prompt queries only)
     const int lim0 = PRE ? row_limit(2 * t) : 0, lim1 = PRE ? row_limit(2 * t + 1) : 0, lim_min = PRE ? row_limit(0) : 0;
     if (PRE) groups_per_split = n_groups;
@@ -323,6 +332,8 @@ decode_kernel(Params p, kvsink_cache c, kvsink_static_params sp, const __half *_
     const uint8_t *vc_base = c.v_codes + (size_t)unit * p.max_seq * p.row_bytes;
     const float *vs_base = c.v_scale + (size_t)unit * p.max_seq * NGv;
     const float *vz_base = c.v_zero + (size_t)unit * p.max_seq * NGv;
+    const float *ktok_s_base = c.k_scale + (size_t)unit * p.max_seq * NGv;    // per-token keys: [unit][max_seq][NGv]
+    const float *ktok_z_base = c.k_zero + (size_t)unit * p.max_seq * NGv;
     const float *ks_base = c.k_scale + (size_t)unit * (p.max_seq / G) * D;
     const float *kz_base = c.k_zero + (size_t)unit * (p.max_seq / G) * D;
 
@@ -425,6 +436,10 @@ decode_kernel(Params p, kvsink_cache c, kvsink_static_params sp, const __half *_
                 bulk_g2s(dst + 2 * KV_BYTES, (const unsigned char *)vs_base + iss_sz, SZ_BYTES, bar);
                 bulk_g2s(dst + 2 * KV_BYTES + SZ_BYTES, (const unsigned char *)vz_base + iss_sz, SZ_BYTES, bar);
             }
+            if constexpr (KT) {   // the tokens' key parameters (same shape as the value parameters) follow them in the slot
+                bulk_g2s(dst + 2 * KV_BYTES + 2 * SZ_BYTES, (const unsigned char *)ktok_s_base + iss_sz, SZ_BYTES, bar);
+                bulk_g2s(dst + 2 * KV_BYTES + 3 * SZ_BYTES, (const unsigned char *)ktok_z_base + iss_sz, SZ_BYTES, bar);
+            }
         }
         ++iss;
         iss_kv += KV_BYTES;
@@ -446,7 +461,7 @@ decode_kernel(Params p, kvsink_cache c, kvsink_static_params sp, const __half *_
         return __all_sync(0xffffffffu, ok);
     };
     if (my_groups > 0) {
-        if (!CAL) issue_params(0);
+        if (!FLAT) issue_params(0);
         for (int i = 0; i < NSLOT - 1 && iss < n_chunks; ++i) issue_chunk();
     }
     // static value parameters of the KV head: the same for every token
@@ -503,7 +518,7 @@ decode_kernel(Params p, kvsink_cache c, kvsink_static_params sp, const __half *_
 
     // ---- tokens of the open group: keys from the fp16 tail (last split only).  They come first, while the warp's first
     //      chunks are on their way (the order of the softmax steps does not matter) ----
-    if (!CAL && split == nsplit - 1) {
+    if (!FLAT && split == nsplit - 1) {
         const __half *tail = (const __half *)c.k_tail + (size_t)unit * G * D;
         const int T_begin = n_body / KVSINK_TILE, T_end = (n + KVSINK_TILE - 1) / KVSINK_TILE;
         for (int T = T_begin + warp; T < T_end; T += DEC_WARPS) {
@@ -561,7 +576,7 @@ decode_kernel(Params p, kvsink_cache c, kvsink_static_params sp, const __half *_
         const int grp = w_begin + gi;
         // ---- B operand of the group: fp16(q * scale * 2^sh) per channel and head (sh puts the largest factor of the
         //      head in [2^13, 2^14)), column half pre-divided by COLF; bias = sum_c of the same rounded factors * zero ----
-        if (!CAL || gi == 0) {
+        if (!FLAT || gi == 0) {
         bias0 = bias1 = ks0 = ks1 = 0.f;
         need_lo = 0;
         {
@@ -572,6 +587,10 @@ decode_kernel(Params p, kvsink_cache c, kvsink_static_params sp, const __half *_
                     const int ch = I8 ? i8_ch[e] : lane * CPL + e;
                     scv[e] = sp.k_scale[h * D + ch]; zev[e] = sp.k_zero[h * D + ch];
                 }
+            } else if constexpr (KT) {
+                // the operand is the query itself; with zero = 1 the "zero-point term" below is the sum of the query
+#pragma unroll
+                for (int e = 0; e < CPL; ++e) { scv[e] = 1.f; zev[e] = 1.f; }
             } else {
                 if (!wait_bar(pbar, (unsigned)gi & 1u)) { stream_ok = false; break; }
                 const float *kp = kp_ring;
@@ -614,8 +633,14 @@ decode_kernel(Params p, kvsink_cache c, kvsink_static_params sp, const __half *_
                 tab[4] = __byte_perm(t1, t3, 0x5410);
                 tab[8] = __byte_perm(t0, t2, 0x7632);
                 tab[12] = __byte_perm(t0, t2, 0x5410);
-                bsum = warp_sum(bsum);
-                if (t == 0) { bias0 = bsum; ks0 = pow2i(-sh); }
+                if constexpr (KT && NGv == 2) {
+                    // per-token keys, two channel groups: the query's sum over each (lanes 0-15 hold channels 0-63)
+                    const float b0s = warp_sum(lane < 16 ? bsum : 0.f), b1s = warp_sum(lane < 16 ? 0.f : bsum);
+                    if (t == 0) { bias0 = b0s; bias1 = b1s; ks0 = pow2i(-sh); }
+                } else {
+                    bsum = warp_sum(bsum);
+                    if (t == 0) { bias0 = bsum; ks0 = pow2i(-sh); }
+                }
             } else if constexpr (I8 == 2) {
                 // up to four heads: the same four signed bytes per factor and head, each head with its own power of two.
                 // The two most significant bytes of every head fill the eight columns of one B operand (head h in columns
@@ -645,8 +670,13 @@ decode_kernel(Params p, kvsink_cache c, kvsink_static_params sp, const __half *_
                         const uint32_t t2 = __byte_perm(d[2], d[3], 0x5140), t3 = __byte_perm(d[2], d[3], 0x7362);
                         w3 = __byte_perm(t1, t3, 0x7632); w2 = __byte_perm(t1, t3, 0x5410);
                         w1 = __byte_perm(t0, t2, 0x7632); w0 = __byte_perm(t0, t2, 0x5410);
-                        bsum = warp_sum(bsum);
-                        if (t == hh) { bias0 = bsum; ks0 = pow2i(-sh); }
+                        if constexpr (KT && NGv == 2) {
+                            const float b0s = warp_sum(lane < 16 ? bsum : 0.f), b1s = warp_sum(lane < 16 ? 0.f : bsum);
+                            if (t == hh) { bias0 = b0s; bias1 = b1s; ks0 = pow2i(-sh); }
+                        } else {
+                            bsum = warp_sum(bsum);
+                            if (t == hh) { bias0 = bsum; ks0 = pow2i(-sh); }
+                        }
                     }
                     tab[(2 * hh) * 4] = w3;
                     tab[(2 * hh + 1) * 4] = w2;
@@ -769,6 +799,15 @@ decode_kernel(Params p, kvsink_cache c, kvsink_static_params sp, const __half *_
             const int T0 = grp * TPG + cj * CT + sub * ST;
             const uint32_t mword = ST == 4 ? (mwords.x | mwords.y) : (sub == 0 ? mwords.x : mwords.y);
 
+            // per-token keys: (scale, zero) of the chunk's tokens, token-major, delivered with the chunk
+            const float *kts = ssv0 + 2 * (SZ_BYTES / 4) + sub * ST * 16 * NGv, *ktz = kts + SZ_BYTES / 4;
+            // score of a token from its group dot products d[j] (already in query units): sum_j scale_j * (d_j - zero_j * qsum_j)
+            auto token_score = [&](const float (&d)[NGK], int tok) {
+                float r = 0.f;
+#pragma unroll
+                for (int j = 0; j < NGK; ++j) r = fmaf(kts[tok * NGv + j], fmaf(-ktz[tok * NGv + j], j == 0 ? bias0 : bias1, d[j]), r);
+                return r;
+            };
             // scores of the chunk's tiles
             float s[ST][4];
 #pragma unroll
@@ -776,9 +815,16 @@ decode_kernel(Params p, kvsink_cache c, kvsink_static_params sp, const __half *_
                 if constexpr (I8 == 2) {
                     uint32_t kw[W];
                     load_tile_shared<BITS, D>(kt + k * TILE_WORDS, lane, kw);
-                    int ia[4] = {0, 0, 0, 0}, ib[4] = {0, 0, 0, 0};   // upper / lower byte pair of the heads' sums
+                    // upper / lower byte pair of the heads' sums; per-token keys: one set per channel group (MMA i covers
+                    // channels 32 i ... 32 i + 31)
+                    int ia[NGK][4], ib[NGK][4];
+#pragma unroll
+                    for (int j = 0; j < NGK; ++j)
+#pragma unroll
+                        for (int x = 0; x < 4; ++x) ia[j][x] = ib[j][x] = 0;
 #pragma unroll
                     for (int i = 0; i < 4; ++i) {
+                        const int jg = NGK == 2 ? (i >> 1) : 0;
                         uint32_t a0, a1, a2, a3;
                         if constexpr (BITS != 4) {
                             const uint32_t x = kw[i];
@@ -788,26 +834,42 @@ decode_kernel(Params p, kvsink_cache c, kvsink_static_params sp, const __half *_
                             a0 = x & 0x0f0f0f0fu; a1 = x & 0xf0f0f0f0u; a2 = y & 0x0f0f0f0fu; a3 = y & 0xf0f0f0f0u;
                         }
                         asm volatile("mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-                                     : "+r"(ia[0]), "+r"(ia[1]), "+r"(ia[2]), "+r"(ia[3])
+                                     : "+r"(ia[jg][0]), "+r"(ia[jg][1]), "+r"(ia[jg][2]), "+r"(ia[jg][3])
                                      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(bk[i][0]), "r"(bk[i][1]));
                         asm volatile("mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-                                     : "+r"(ib[0]), "+r"(ib[1]), "+r"(ib[2]), "+r"(ib[3])
+                                     : "+r"(ib[jg][0]), "+r"(ib[jg][1]), "+r"(ib[jg][2]), "+r"(ib[jg][3])
                                      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(bk[4 + i][0]), "r"(bk[4 + i][1]));
                     }
                     // lane t holds head t: bytes 3, 2 of its sum in the first accumulators, bytes 1, 0 in the second
-                    const float tg = fmaf(fmaf((float)ia[0], 256.f, (float)ia[1]), 65536.f, fmaf((float)ib[0], 256.f, (float)ib[1]));
-                    const float th = fmaf(fmaf((float)ia[2], 256.f, (float)ia[3]), 65536.f, fmaf((float)ib[2], 256.f, (float)ib[3]));
-                    s[k][0] = fmaf(tg, ks0, -bias0); s[k][1] = -INFINITY;
-                    s[k][2] = fmaf(th, ks0 * (BITS == 4 ? 0.0625f : 0.25f), -bias0); s[k][3] = -INFINITY;
+                    float tg[NGK], th[NGK];
+#pragma unroll
+                    for (int j = 0; j < NGK; ++j) {
+                        tg[j] = fmaf(fmaf((float)ia[j][0], 256.f, (float)ia[j][1]), 65536.f, fmaf((float)ib[j][0], 256.f, (float)ib[j][1]));
+                        th[j] = fmaf(fmaf((float)ia[j][2], 256.f, (float)ia[j][3]), 65536.f, fmaf((float)ib[j][2], 256.f, (float)ib[j][3]));
+                    }
+                    if constexpr (KT) {
+#pragma unroll
+                        for (int j = 0; j < NGK; ++j) { tg[j] *= ks0; th[j] *= ks0 * (BITS == 4 ? 0.0625f : 0.25f); }
+                        s[k][0] = token_score(tg, k * 16 + g); s[k][1] = -INFINITY;
+                        s[k][2] = token_score(th, k * 16 + g + 8); s[k][3] = -INFINITY;
+                    } else {
+                        s[k][0] = fmaf(tg[0], ks0, -bias0); s[k][1] = -INFINITY;
+                        s[k][2] = fmaf(th[0], ks0 * (BITS == 4 ? 0.0625f : 0.25f), -bias0); s[k][3] = -INFINITY;
+                    }
                     continue;
                 }
                 if constexpr (I8 == 1) {
                     uint32_t kw[W];
                     load_tile_shared<BITS, D>(kt + k * TILE_WORDS, lane, kw);
-                    int ia[4] = {0, 0, 0, 0};
+                    int iag[NGK][4];                                    // per-token keys: one set per channel group
+#pragma unroll
+                    for (int j = 0; j < NGK; ++j)
+#pragma unroll
+                        for (int x = 0; x < 4; ++x) iag[j][x] = 0;
                     int ih0[4] = {0, 0, 0, 0}, ih1[4] = {0, 0, 0, 0};   // 3 bit: the high bits of the even / odd words
 #pragma unroll
                     for (int i = 0; i < 4; ++i) {
+                        int (&ia)[4] = iag[NGK == 2 ? (i >> 1) : 0];
                         uint32_t a0, a1, a2, a3;
                         if constexpr (BITS == 3) {
                             // the second section has the byte structure of the first: the high bits of word i sit at bits
@@ -837,18 +899,30 @@ decode_kernel(Params p, kvsink_cache c, kvsink_static_params sp, const __half *_
                     if constexpr (BITS == 3) {
                         // code = low + 4 * high; in place the high bits weigh 4, 8 (rows g, g + 8) in even words and 1, 2 in
                         // odd ones, the low fields 1, 4: rows g in units of 1, rows g + 8 in units of 4
+                        int (&ia)[4] = iag[0];
                         ia[0] += ih0[0] + 4 * ih1[0]; ia[1] += ih0[1] + 4 * ih1[1];
                         ia[2] += 2 * ih0[2] + 8 * ih1[2]; ia[3] += 2 * ih0[3] + 8 * ih1[3];
                     }
                     // lane t = 0 holds limbs 0, 1 (columns 0, 1), its neighbour limbs 2, 3 (columns 2, 3): each lane combines
                     // its pair (every column sum is below 2^24, exact in binary32), then the pairs combine
-                    const float xg = fmaf((float)ia[0], 256.f, (float)ia[1]), xh = fmaf((float)ia[2], 256.f, (float)ia[3]);
-                    const float yg = __shfl_down_sync(0xffffffffu, xg, 1), yh = __shfl_down_sync(0xffffffffu, xh, 1);
-                    const float tg = fmaf(xg, 65536.f, yg);
-                    const float th = fmaf(xh, 65536.f, yh);
+                    float tg[NGK], th[NGK];
+#pragma unroll
+                    for (int j = 0; j < NGK; ++j) {
+                        const float xg = fmaf((float)iag[j][0], 256.f, (float)iag[j][1]), xh = fmaf((float)iag[j][2], 256.f, (float)iag[j][3]);
+                        const float yg = __shfl_down_sync(0xffffffffu, xg, 1), yh = __shfl_down_sync(0xffffffffu, xh, 1);
+                        tg[j] = fmaf(xg, 65536.f, yg);
+                        th[j] = fmaf(xh, 65536.f, yh);
+                    }
                     // lanes t != 0 hold no head: their factor and bias are zero, their columns are never read
-                    s[k][0] = fmaf(tg, ks0, -bias0); s[k][1] = -INFINITY;
-                    s[k][2] = fmaf(th, ks0 * (BITS == 4 ? 0.0625f : 0.25f), -bias0); s[k][3] = -INFINITY;
+                    if constexpr (KT) {
+#pragma unroll
+                        for (int j = 0; j < NGK; ++j) { tg[j] *= ks0; th[j] *= ks0 * (BITS == 4 ? 0.0625f : 0.25f); }
+                        s[k][0] = token_score(tg, k * 16 + g); s[k][1] = -INFINITY;
+                        s[k][2] = token_score(th, k * 16 + g + 8); s[k][3] = -INFINITY;
+                    } else {
+                        s[k][0] = fmaf(tg[0], ks0, -bias0); s[k][1] = -INFINITY;
+                        s[k][2] = fmaf(th[0], ks0 * (BITS == 4 ? 0.0625f : 0.25f), -bias0); s[k][3] = -INFINITY;
+                    }
                     continue;
                 }
                 uint32_t kw[W], ka[NM][4];
@@ -899,7 +973,7 @@ decode_kernel(Params p, kvsink_cache c, kvsink_static_params sp, const __half *_
                     }
                 }
             }
-            if constexpr (CAL) {
+            if constexpr (FLAT) {
                 if ((T0 + ST) * KVSINK_TILE > n) {   // the last tiles reach beyond the sequence: those tokens do not exist
 #pragma unroll
                     for (int k = 0; k < ST; ++k) {
@@ -931,6 +1005,10 @@ decode_kernel(Params p, kvsink_cache c, kvsink_static_params sp, const __half *_
                     for (int j = 0; j < NGv; ++j) {
                         sv0[k][j] = ssv[(k * 16 + g) * NGv + j]; zv0[k][j] = szv[(k * 16 + g) * NGv + j];
                         sv1[k][j] = ssv[(k * 16 + g + 8) * NGv + j]; zv1[k][j] = szv[(k * 16 + g + 8) * NGv + j];
+                        if constexpr (KT) {   // tokens beyond the sequence: whatever the arrays hold there must not reach the sums
+                            if ((T0 + k) * KVSINK_TILE + g >= n) sv0[k][j] = zv0[k][j] = 0.f;
+                            if ((T0 + k) * KVSINK_TILE + g + 8 >= n) sv1[k][j] = zv1[k][j] = 0.f;
+                        }
                         mx = fmaxf(mx, fmaxf(fabsf(sv0[k][j]), fabsf(sv1[k][j])));
                     }
                 fit_value_scale(mx);
@@ -1089,18 +1167,18 @@ decode_kernel(Params p, kvsink_cache c, kvsink_static_params sp, const __half *_
 }
 
 // ---- launch: one instantiation per (bits, head size, value groups per row, chunk size, key-side variant) ----
-template <int BITS, int D, int NGV, int CT, bool PL, int I8 = 0, bool CAL = false>
+template <int BITS, int D, int NGV, int CT, bool PL, int I8 = 0, int PM = 0>
 static int launch_decode_p(const Params &p, const kvsink_cache &c, const kvsink_static_params *cal, const __half *q, float *out, float *lse, float *ws,
                            cudaStream_t st)
 {
     // the units the sequence is split in: key groups, or ring chunks when the parameters are static
-    const int n_groups = CAL ? (c.seq_len + CT * KVSINK_TILE - 1) / (CT * KVSINK_TILE) : c.seq_len / p.G;
-    const kvsink_static_params sp = CAL ? *cal : kvsink_static_params{nullptr, nullptr, nullptr, nullptr};
+    const int n_groups = PM != 0 ? (c.seq_len + CT * KVSINK_TILE - 1) / (CT * KVSINK_TILE) : c.seq_len / p.G;
+    const kvsink_static_params sp = PM == 1 ? *cal : kvsink_static_params{nullptr, nullptr, nullptr, nullptr};
     const int nsplit = choose_splits(p, n_groups);
     const int gps = n_groups > 0 ? (n_groups + nsplit - 1) / nsplit : 0;
     const int qchunks = (p.rep + 7) / 8;
-    const size_t smem = DecodePlan<BITS, D, NGV, CT, I8 == 1 ? 1 : (PL ? 4 : 8)>::BYTES;
-    auto kern = decode_kernel<BITS, D, NGV, CT, PL, I8, CAL>;
+    const size_t smem = DecodePlan<BITS, D, NGV, CT, I8 == 1 ? 1 : (PL ? 4 : 8), PM == 2>::BYTES;
+    auto kern = decode_kernel<BITS, D, NGV, CT, PL, I8, PM>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return KVSINK_ERR_CUDA;
     cudaLaunchAttribute pdl[2];
     pdl[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
@@ -1140,7 +1218,7 @@ template <int BITS, int D, int NGV, int CT>
 static int launch_prefill_p(const Params &p, const kvsink_cache &c, const __half *q, const PrefillShape &pre, float *out, float *lse, cudaStream_t st)
 {
     const size_t smem = DecodePlan<BITS, D, NGV, CT, 8>::BYTES;
-    auto kern = decode_kernel<BITS, D, NGV, CT, false, 0, false, true>;
+    auto kern = decode_kernel<BITS, D, NGV, CT, false, 0, 0, true>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return KVSINK_ERR_CUDA;
     const long long blocks = ((long long)pre.T * p.rep + 7) / 8;
     if (blocks > 0x7fffffffLL) return KVSINK_ERR_UNSUPPORTED;
@@ -1190,51 +1268,59 @@ static int launch_prefill_bits(const Params &p, const kvsink_cache &c, const __h
     return KVSINK_ERR_UNSUPPORTED;
 }
 
-template <int BITS, int D, int NGV, int CT, bool CAL>
+template <int BITS, int D, int NGV, int CT, int PM>
 static int launch_decode_c(const Params &p, const kvsink_cache &c, const kvsink_static_params *cal, const __half *q, float *out, float *lse, float *ws,
                            cudaStream_t st)
 {
     if constexpr (D == 128)
-        if (p.rep == 1) return launch_decode_p<BITS, D, NGV, CT, true, 1, CAL>(p, c, cal, q, out, lse, ws, st);
+        if (p.rep == 1) return launch_decode_p<BITS, D, NGV, CT, true, 1, PM>(p, c, cal, q, out, lse, ws, st);
     if constexpr (D == 128 && BITS != 3)
-        if (p.rep <= 4) return launch_decode_p<BITS, D, NGV, CT, true, 2, CAL>(p, c, cal, q, out, lse, ws, st);
-    if (p.rep <= 4) return launch_decode_p<BITS, D, NGV, CT, true, 0, CAL>(p, c, cal, q, out, lse, ws, st);
-    return launch_decode_p<BITS, D, NGV, CT, false, 0, CAL>(p, c, cal, q, out, lse, ws, st);
+        if (p.rep <= 4) return launch_decode_p<BITS, D, NGV, CT, true, 2, PM>(p, c, cal, q, out, lse, ws, st);
+    if constexpr (PM == 2) {
+        return KVSINK_ERR_UNSUPPORTED;   // per-token keys run on the integer key side only
+    } else {
+        if (p.rep <= 4) return launch_decode_p<BITS, D, NGV, CT, true, 0, PM>(p, c, cal, q, out, lse, ws, st);
+        return launch_decode_p<BITS, D, NGV, CT, false, 0, PM>(p, c, cal, q, out, lse, ws, st);
+    }
 }
 
-template <int BITS, int D, int NGV, bool CAL>
+template <int BITS, int D, int NGV, int PM>
 static int launch_decode_n(const Params &p, const kvsink_cache &c, const kvsink_static_params *cal, const __half *q, float *out, float *lse, float *ws,
                            cudaStream_t st)
 {
     // ring chunks of four tiles where a key group divides into them and two slots of that size stay below ~9 KB per
     // warp, else of two tiles (G a multiple of 32), else of one
-    if constexpr (4 * (2 * 128 * (D * BITS / 64) + 2 * 16 * NGV * 4) <= 4800)
-        if ((p.G / KVSINK_TILE) % 4 == 0) return launch_decode_c<BITS, D, NGV, 4, CAL>(p, c, cal, q, out, lse, ws, st);
-    if ((p.G / KVSINK_TILE) % 2 == 0) return launch_decode_c<BITS, D, NGV, 2, CAL>(p, c, cal, q, out, lse, ws, st);
-    return launch_decode_c<BITS, D, NGV, 1, CAL>(p, c, cal, q, out, lse, ws, st);
+    if constexpr (4 * (2 * 128 * (D * BITS / 64) + (PM == 2 ? 4 : 2) * 16 * NGV * 4) <= 4800)
+        if ((p.G / KVSINK_TILE) % 4 == 0) return launch_decode_c<BITS, D, NGV, 4, PM>(p, c, cal, q, out, lse, ws, st);
+    if ((p.G / KVSINK_TILE) % 2 == 0) return launch_decode_c<BITS, D, NGV, 2, PM>(p, c, cal, q, out, lse, ws, st);
+    return launch_decode_c<BITS, D, NGV, 1, PM>(p, c, cal, q, out, lse, ws, st);
 }
 
-template <int BITS, int D, bool CAL>
+template <int BITS, int D, int PM>
 static int launch_decode_t(const Params &p, const kvsink_cache &c, const kvsink_static_params *cal, const __half *q, float *out, float *lse, float *ws,
                            cudaStream_t st)
 {
-    if (p.NGv == 1) return launch_decode_n<BITS, D, 1, CAL>(p, c, cal, q, out, lse, ws, st);
-    if (p.NGv == 2) return launch_decode_n<BITS, D, 2, CAL>(p, c, cal, q, out, lse, ws, st);
-    if constexpr (!CAL)
-        if (p.NGv == 4) return launch_decode_n<BITS, D, 4, CAL>(p, c, cal, q, out, lse, ws, st);
+    if (p.NGv == 1) return launch_decode_n<BITS, D, 1, PM>(p, c, cal, q, out, lse, ws, st);
+    if constexpr (PM != 2 || BITS != 3)
+        if (p.NGv == 2) return launch_decode_n<BITS, D, 2, PM>(p, c, cal, q, out, lse, ws, st);
+    if constexpr (PM == 0)
+        if (p.NGv == 4) return launch_decode_n<BITS, D, 4, PM>(p, c, cal, q, out, lse, ws, st);
     return KVSINK_ERR_UNSUPPORTED;
 }
 
-// Dispatch over head size for one code width; each width is compiled in a translation unit of its own.  `cal` is null
-// for dynamic parameters; static parameters are built for head size 128 with one or two value groups per row.
+// Dispatch over head size for one code width; each width is compiled in a translation unit of its own.  mode 0: dynamic
+// per-channel key parameters (`cal` null); 1: static parameters `cal`; 2: per-token key parameters.  Modes 1 and 2 are
+// built for head size 128 with one or two channel groups per row; mode 2 for at most four query heads per KV head
+// (3 bit: one, with one channel group).
 template <int BITS>
-static int launch_decode_bits(const Params &p, const kvsink_cache &c, const kvsink_static_params *cal, const __half *q, float *out, float *lse,
-                              float *ws, cudaStream_t st)
+static int launch_decode_bits(const Params &p, const kvsink_cache &c, const kvsink_static_params *cal, int mode, const __half *q, float *out,
+                              float *lse, float *ws, cudaStream_t st)
 {
-    if (cal) return p.D == 128 ? launch_decode_t<BITS, 128, true>(p, c, cal, q, out, lse, ws, st) : KVSINK_ERR_UNSUPPORTED;
-    if (p.D == 128) return launch_decode_t<BITS, 128, false>(p, c, cal, q, out, lse, ws, st);
+    if (mode == 2) return p.D == 128 ? launch_decode_t<BITS, 128, 2>(p, c, cal, q, out, lse, ws, st) : KVSINK_ERR_UNSUPPORTED;
+    if (mode == 1) return p.D == 128 && cal ? launch_decode_t<BITS, 128, 1>(p, c, cal, q, out, lse, ws, st) : KVSINK_ERR_UNSUPPORTED;
+    if (p.D == 128) return launch_decode_t<BITS, 128, 0>(p, c, cal, q, out, lse, ws, st);
     if constexpr (BITS != 3)
-        if (p.D == 64) return launch_decode_t<BITS, 64, false>(p, c, cal, q, out, lse, ws, st);
+        if (p.D == 64) return launch_decode_t<BITS, 64, 0>(p, c, cal, q, out, lse, ws, st);
     return KVSINK_ERR_UNSUPPORTED;
 }
 
