@@ -441,6 +441,59 @@ def calibrated_record(kv, wl, dev, instances, steps, warmup, peak):
             "decode": {"algorithmic_bytes": db, "GBs": gbs(db, us["decode"]), "frac_of_measured_peak": gbs(db, us["decode"]) / peak}}
 
 
+def pertoken_record(kv, wl, dev, instances, steps, warmup, peak):
+    """The per-token key variant of a single-layer workload: per instance quantize_append_pertoken(T=S), one appended
+    token and decode_attention_pertoken (kernel times only)."""
+    cfg = kv.Config(wl.batch, wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.hidden, wl.bits, wl.group, wl.max_seq, wl.topk, wl.pfn_n, wl.channels)
+    L = instances
+    H = synth.make_hidden(wl, dev)
+    KV = [synth.make_kv(wl, l, dev) for l in range(L)]
+    new = [synth.make_new_token(wl, l, 0, dev) for l in range(L)]
+    qs = [synth.make_query(wl, KV[l][0], l) for l in range(L)]
+    sinks = kv.SinkSet(cfg, dev)
+    kv.predict_sinks(cfg, H, sinks)
+    caches = [kv.KVCache(cfg, sinks, dev, per_token_keys=True) for _ in range(L)]
+    outs = [torch.empty((wl.batch, wl.n_q_heads, wl.head_dim), dtype=torch.float32, device=dev) for _ in range(L)]
+    ws_d = torch.empty(kv.cache_sizes(cfg)["decode_workspace_bytes"], dtype=torch.uint8, device=dev)
+    ev = {"quantize": [], "decode": []}
+
+    def timed(kind, fn, rec):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        fn()
+        b.record()
+        if rec:
+            ev[kind].append((a, b))
+
+    def quantize_all():
+        for l in range(L):
+            caches[l].seq_len = 0
+            kv.quantize_append_pertoken(cfg, caches[l], KV[l][0], KV[l][1])
+
+    def decode_all():
+        for l in range(L):
+            kv.decode_attention_pertoken(cfg, caches[l], qs[l], outs[l], None, ws_d, want_lse=False)
+
+    for it in range(warmup + steps):
+        rec = it >= warmup
+        timed("quantize", quantize_all, rec)
+        for l in range(L):
+            kv.quantize_append_pertoken(cfg, caches[l], new[l][0], new[l][1])
+        timed("decode", decode_all, rec)
+    torch.cuda.synchronize()
+    us = {k: sum(a.elapsed_time(b) for a, b in v) * 1e3 / len(v) / L for k, v in ev.items()}
+    units, n = wl.batch * wl.n_kv_heads, wl.seq + 1
+    ngv = wl.head_dim // min(wl.group, wl.head_dim)
+    tok_bytes = 2 * wl.head_dim * wl.bits // 8 + 4 * 4 * ngv          # codes of K and V, (scale, zero) of both per channel group
+    qb = units * wl.seq * (2 * wl.head_dim * 2 + tok_bytes)
+    db = units * n * tok_bytes + wl.batch * n // 8 + units * (wl.topk + wl.pfn_n) * wl.head_dim * 4 + wl.batch * wl.n_q_heads * wl.head_dim * 6
+    gbs = lambda bytes_, t: bytes_ / (t * 1e-6) / 1e9
+    return {"workload": workload_string(wl) + " (per-token keys)", "instances_per_step": L, "quantize_us": us["quantize"],
+            "decode_us": us["decode"], "device_status": kv.read_status(caches[0]),
+            "quantize": {"algorithmic_bytes": qb, "GBs": gbs(qb, us["quantize"]), "frac_of_measured_peak": gbs(qb, us["quantize"]) / peak},
+            "decode": {"algorithmic_bytes": db, "GBs": gbs(db, us["decode"]), "frac_of_measured_peak": gbs(db, us["decode"]) / peak}}
+
+
 def prefill_attention_record(kv, wl, dev, steps, warmup):
     """Attention of every prompt query over the just-quantized cache of a single-layer workload (kernel time only)."""
     cfg = kv.Config(wl.batch, wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.hidden, wl.bits, wl.group, wl.max_seq, wl.topk, wl.pfn_n, wl.channels)
@@ -567,9 +620,11 @@ def run_ours(args):
         del b
         torch.cuda.empty_cache()
     if not args.workload:
-        # the next scope row: static (calibrated) parameters on the LLaMA2-7B-shaped layer
+        # the next scope rows on the LLaMA2-7B-shaped layer: static (calibrated) parameters, per-token keys, prompt attention
         base = synth.WORKLOADS["llama2_7b_layer"]
         per["llama2_7b_layer_static"] = calibrated_record(kv, base.scaled(seed=dist_util.rank_seed(base.seed, rank)), dev, args.instances, 20, warmup, peak)
+        torch.cuda.empty_cache()
+        per["llama2_7b_layer_pertoken_keys"] = pertoken_record(kv, base.scaled(seed=dist_util.rank_seed(base.seed, rank)), dev, args.instances, 20, warmup, peak)
         torch.cuda.empty_cache()
         per["llama2_7b_layer_prefill_attention"] = prefill_attention_record(kv, base.scaled(seed=dist_util.rank_seed(base.seed, rank)), dev, 3, 1)
         torch.cuda.empty_cache()
