@@ -309,10 +309,15 @@ __device__ __forceinline__ void qb_issue(const CUtensorMap *tm_k, const CUtensor
     }
 }
 
-template <int BITS, int G>
+// MODE 0: dynamic parameters (the statistics of every group are taken here).  MODE 1: static parameters `sp` (one pair per key
+// channel and per value channel group of the KV head): no statistics pass, nothing written to the parameter arrays; the
+// thresholds of the 2-bit coder describe Eq. 8's clamp exactly, so values outside the calibrated range need nothing more.
+template <int BITS, int G, int MODE = 0>
 __global__ void __launch_bounds__(32 * QbGeo<G, BITS>::WARPS, 1)
-quantize_bulk_kernel(Params p, kvsink_cache c, const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v, QbShape sh)
+quantize_bulk_kernel(Params p, kvsink_cache c, const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v, QbShape sh,
+                     kvsink_static_params sp)
 {
+    static_assert(MODE == 0 || BITS == 2, "static parameters: the threshold coder only");
     using Geo = QbGeo<G, BITS>;
     constexpr int D = QB_D, NS = Geo::NS, KPL = Geo::KPL, MT = Geo::MT, NT = Geo::NT, NGv = Geo::NGv, NW = Geo::WARPS;
     constexpr int MPS = 16 / NS;                  // matrices per statistic set
@@ -449,7 +454,9 @@ quantize_bulk_kernel(Params p, kvsink_cache c, const __grid_constant__ CUtensorM
         uint32_t mn[NS][2], mx[NS][2];
 #pragma unroll
         for (int s = 0; s < NS; ++s) { mn[s][0] = mn[s][1] = PINF2; mx[s][0] = mx[s][1] = NINF2; }
-        if (is_v || !has_sink) {
+        if constexpr (MODE == 1) {
+            // static parameters: no statistics
+        } else if (is_v || !has_sink) {
 #pragma unroll
             for (int u = 0; u < 16; ++u) {
                 const int s = u / MPS;
@@ -479,7 +486,7 @@ quantize_bulk_kernel(Params p, kvsink_cache c, const __grid_constant__ CUtensorM
 
         // the other rows of a column live in the lanes that differ in bits 2..4
 #pragma unroll
-        for (int o = 4; o < 32; o <<= 1)
+        for (int o = 4; o < 32 && MODE == 0; o <<= 1)
 #pragma unroll
             for (int s = 0; s < NS; ++s)
 #pragma unroll
@@ -502,14 +509,21 @@ quantize_bulk_kernel(Params p, kvsink_cache c, const __grid_constant__ CUtensorM
             const float fmn = __half2float(__ushort_as_half(lo16)), fmx = __half2float(__ushort_as_half(hi16));
             // values: token of the item (set = tile * NGv + channel group); keys: channel of the item (set = matrix)
             const int idx = 16 * (is_v ? s_ / NGv : s_) + 8 * ab_ + 2 * t4 + e_;
-            const bool member = is_v ? !((mw.w0 >> idx) & 1u) : lo16 != 0x7C00;
+            const bool member = is_v ? !((mw.w0 >> idx) & 1u) : (MODE == 1 || lo16 != 0x7C00);
             float s, z;
-            group_params(member, fmn, fmx, qmax, &s, &z);
-            const size_t ov = ((size_t)unit * p.max_seq + p0 + 32 * sub + idx) * NGv + (s_ % NGv);
-            const size_t ok = ((size_t)unit * (p.max_seq / G) + p0 / G) * D + sub * Geo::KC + idx;
-            float *ps = is_v ? c.v_scale + ov : c.k_scale + ok, *pz = is_v ? c.v_zero + ov : c.k_zero + ok;
-            *ps = s;
-            *pz = z;
+            if constexpr (MODE == 1) {
+                // the pair of this key channel / of this token's value channel group; a sink token's values keep code 0
+                const int pi = is_v ? cur.h * NGv + (s_ % NGv) : cur.h * D + sub * Geo::KC + idx;
+                s = member ? __ldg((is_v ? sp.v_scale : sp.k_scale) + pi) : 0.f;
+                z = member ? __ldg((is_v ? sp.v_zero : sp.k_zero) + pi) : 0.f;
+            } else {
+                group_params(member, fmn, fmx, qmax, &s, &z);
+                const size_t ov = ((size_t)unit * p.max_seq + p0 + 32 * sub + idx) * NGv + (s_ % NGv);
+                const size_t ok = ((size_t)unit * (p.max_seq / G) + p0 / G) * D + sub * Geo::KC + idx;
+                float *ps = is_v ? c.v_scale + ov : c.k_scale + ok, *pz = is_v ? c.v_zero + ov : c.k_zero + ok;
+                *ps = s;
+                *pz = z;
+            }
             const int pos = 8 * (kk >> 1) + 2 * t4 + e_;
             if constexpr (BITS == 2) {
                 const double s_half = 0.5 * (double)s;
@@ -709,9 +723,9 @@ bool make_map(CUtensorMap *tm, const __half *base, const Params &p, int T, int64
               CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int BITS, int G>
-int launch_bulk(const Params &p, const kvsink_cache &c, const __half *k_src, const __half *v_src, int first_token, int n_groups, int64_t sb,
-                int64_t sh, int64_t stt, cudaStream_t st)
+template <int BITS, int G, int MODE = 0>
+int launch_bulk(const Params &p, const kvsink_cache &c, const kvsink_static_params &sp, const __half *k_src, const __half *v_src, int first_token,
+                int n_groups, int64_t sb, int64_t sh, int64_t stt, cudaStream_t st)
 {
     using Geo = QbGeo<G, BITS>;
     CUtensorMap tm_k, tm_v;
@@ -722,7 +736,7 @@ int launch_bulk(const Params &p, const kvsink_cache &c, const __half *k_src, con
     constexpr int NW = Geo::WARPS;
     constexpr size_t smem = (size_t)NW * (QB_STAGE_BYTES + 8 + Geo::SCRATCH);
     static_assert(smem <= 227 * 1024, "stages too large");
-    auto kern = quantize_bulk_kernel<BITS, G>;
+    auto kern = quantize_bulk_kernel<BITS, G, MODE>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return KVSINK_ERR_CUDA;
     QbShape shp;
     shp.first_token = first_token;
@@ -732,7 +746,7 @@ int launch_bulk(const Params &p, const kvsink_cache &c, const __half *k_src, con
     shp.n_items = (unsigned)n_items;
     long blocks = (n_items + NW - 1) / NW;
     if (blocks > 148) blocks = 148;
-    return launch_pdl(kern, dim3((unsigned)blocks), dim3(32 * NW), smem, st, p, c, tm_k, tm_v, shp) == cudaSuccess ? KVSINK_OK : KVSINK_ERR_CUDA;
+    return launch_pdl(kern, dim3((unsigned)blocks), dim3(32 * NW), smem, st, p, c, tm_k, tm_v, shp, sp) == cudaSuccess ? KVSINK_OK : KVSINK_ERR_CUDA;
 }
 
 }  // namespace
@@ -743,11 +757,23 @@ int launch_quantize_groups_bulk(const Params &p, const kvsink_cache &c, const __
                                 int n_groups, int64_t sb, int64_t sh, int64_t stt, cudaStream_t st)
 {
     if (p.D != QB_D || n_groups < 1) return KVSINK_ERR_UNSUPPORTED;
-    if (p.bits == 2 && p.G == 128) return launch_bulk<2, 128>(p, c, k_src, v_src, first_token, n_groups, sb, sh, stt, st);
-    if (p.bits == 2 && p.G == 64) return launch_bulk<2, 64>(p, c, k_src, v_src, first_token, n_groups, sb, sh, stt, st);
-    if (p.bits == 3 && p.G == 64) return launch_bulk<3, 64>(p, c, k_src, v_src, first_token, n_groups, sb, sh, stt, st);
-    if (p.bits == 4 && p.G == 128) return launch_bulk<4, 128>(p, c, k_src, v_src, first_token, n_groups, sb, sh, stt, st);
-    if (p.bits == 4 && p.G == 64) return launch_bulk<4, 64>(p, c, k_src, v_src, first_token, n_groups, sb, sh, stt, st);
+    const kvsink_static_params none = {nullptr, nullptr, nullptr, nullptr};
+    if (p.bits == 2 && p.G == 128) return launch_bulk<2, 128>(p, c, none, k_src, v_src, first_token, n_groups, sb, sh, stt, st);
+    if (p.bits == 2 && p.G == 64) return launch_bulk<2, 64>(p, c, none, k_src, v_src, first_token, n_groups, sb, sh, stt, st);
+    if (p.bits == 3 && p.G == 64) return launch_bulk<3, 64>(p, c, none, k_src, v_src, first_token, n_groups, sb, sh, stt, st);
+    if (p.bits == 4 && p.G == 128) return launch_bulk<4, 128>(p, c, none, k_src, v_src, first_token, n_groups, sb, sh, stt, st);
+    if (p.bits == 4 && p.G == 64) return launch_bulk<4, 64>(p, c, none, k_src, v_src, first_token, n_groups, sb, sh, stt, st);
+    return KVSINK_ERR_UNSUPPORTED;
+}
+
+// The same for static parameters: n_groups spans of G tokens (G only sets the shape of the work items here), the first at a
+// multiple of G.  2 bit only; other shapes return KVSINK_ERR_UNSUPPORTED and the caller uses the tile kernels.
+int launch_quantize_static_bulk(const Params &p, const kvsink_cache &c, const kvsink_static_params &sp, const __half *k_src, const __half *v_src,
+                                int first_token, int n_groups, int64_t sb, int64_t sh, int64_t stt, cudaStream_t st)
+{
+    if (p.D != QB_D || n_groups < 1 || first_token % p.G) return KVSINK_ERR_UNSUPPORTED;
+    if (p.bits == 2 && p.G == 128) return launch_bulk<2, 128, 1>(p, c, sp, k_src, v_src, first_token, n_groups, sb, sh, stt, st);
+    if (p.bits == 2 && p.G == 64) return launch_bulk<2, 64, 1>(p, c, sp, k_src, v_src, first_token, n_groups, sb, sh, stt, st);
     return KVSINK_ERR_UNSUPPORTED;
 }
 

@@ -74,6 +74,15 @@ def test_chunked_appends_and_values_outside_the_calibrated_range():
     _both(wl, chunks=(1, 14, 1, 33, 100, 1, 183), cal_tokens=50)
 
 
+@pytest.mark.parametrize("group", [64, 128])
+def test_two_bit_chunks_through_the_bulk_quantizer_with_values_outside_the_calibrated_range(group):
+    # chunks that start on a multiple of the group size send their whole spans to the bulk kernel, the rest to the tile kernels;
+    # calibrated on 40 tokens only, so later tokens clamp at both ends
+    G = group
+    wl = TINY.scaled(seq=5 * G + 19, group=G, bits=2, head_dim=128, n_q_heads=4, n_kv_heads=2, batch=2, topk=7, pfn_n=2, seed=81 + G)
+    _both(wl, chunks=(G, G + 6, G - 6, 2 * G, 19), cal_tokens=40)
+
+
 def test_many_splits_and_clusters():
     # few units and a long sequence (merge kernel), then many units (cluster merge)
     _both(TINY.scaled(seq=64 * 40 + 5, group=64, bits=2, head_dim=128, n_q_heads=4, n_kv_heads=1, batch=1, topk=20, seed=12))
