@@ -426,6 +426,17 @@ int launch_quantize_pertoken(const Params &p, const kvsink_cache &c, const __hal
                              int64_t sb, int64_t sh, int64_t stt, cudaStream_t st)
 {
     const kvsink_static_params none = {nullptr, nullptr, nullptr, nullptr};
+    // whole G-token spans from a multiple of G go to the bulk quantizer where it has this form (G only shapes its work items)
+    if (n_tokens >= p.G && first_token % p.G == 0) {
+        const int n_groups = n_tokens / p.G;
+        const int rc = launch_quantize_pertoken_bulk(p, c, k_src, v_src, first_token, n_groups, sb, sh, stt, st);
+        if (rc == KVSINK_OK) {
+            const int done = n_groups * p.G;
+            return launch_tokens<true>(p, c, none, k_src + (int64_t)done * stt, v_src + (int64_t)done * stt, first_token + done, n_tokens - done, sb, sh,
+                                       stt, st);
+        }
+        if (rc != KVSINK_ERR_UNSUPPORTED) return rc;
+    }
     return launch_tokens<true>(p, c, none, k_src, v_src, first_token, n_tokens, sb, sh, stt, st);
 }
 

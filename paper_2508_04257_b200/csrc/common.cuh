@@ -164,6 +164,8 @@ int launch_quantize_calibrated(const Params &p, const kvsink_cache &c, const kvs
                                int first_token, int n_tokens, int64_t sb, int64_t sh, int64_t stt, cudaStream_t st);
 int launch_quantize_static_bulk(const Params &p, const kvsink_cache &c, const kvsink_static_params &sp, const __half *k_src, const __half *v_src,
                                 int first_token, int n_groups, int64_t sb, int64_t sh, int64_t stt, cudaStream_t st);
+int launch_quantize_pertoken_bulk(const Params &p, const kvsink_cache &c, const __half *k_src, const __half *v_src, int first_token, int n_groups,
+                                  int64_t sb, int64_t sh, int64_t stt, cudaStream_t st);
 int launch_quantize_pertoken(const Params &p, const kvsink_cache &c, const __half *k_src, const __half *v_src, int first_token, int n_tokens,
                              int64_t sb, int64_t sh, int64_t stt, cudaStream_t st);
 size_t calibrate_workspace_bytes(const Params &p);

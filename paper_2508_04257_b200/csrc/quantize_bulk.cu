@@ -278,14 +278,16 @@ __device__ __forceinline__ QbPos qb_advance(QbPos q, const QbPos &step, int n_gr
 struct QbMask { uint32_t w0, w1, w2, w3; };
 __device__ __forceinline__ uint32_t qb_mask_word(const QbMask &m, int i) { return i == 0 ? m.w0 : (i == 1 ? m.w1 : (i == 2 ? m.w2 : m.w3)); }
 
-template <int G>
+template <int G, bool KSLAB = false>
 __device__ __forceinline__ void qb_load_mask(const Params &p, const kvsink_cache &c, int q_sub, int q_grp, int q_b, int first_token,
                                              QbMask &mw)
 {
     const uint32_t *bm = c.sink_bitmask + (size_t)q_b * p.mask_words;
     const int p0 = first_token + q_grp * G;
     mw.w0 = mw.w1 = mw.w2 = mw.w3 = 0u;
-    if (q_sub < QbGeo<G>::NK) {
+    if (KSLAB && q_sub < QbGeo<G>::NK) {          // per-token keys: a key item is a 32-token slab like a value item
+        mw.w0 = __ldg(bm + ((p0 + 32 * q_sub) >> 5));
+    } else if (q_sub < QbGeo<G>::NK) {
         mw.w0 = __ldg(bm + (p0 >> 5));
         mw.w1 = __ldg(bm + (p0 >> 5) + 1);
         if (G == 128) { mw.w2 = __ldg(bm + (p0 >> 5) + 2); mw.w3 = __ldg(bm + (p0 >> 5) + 3); }
@@ -295,12 +297,16 @@ __device__ __forceinline__ void qb_load_mask(const Params &p, const kvsink_cache
 }
 
 // One stage refill: the bulk copies of item q into `dst`, counted on `bar` (one lane).
-template <int G>
+template <int G, bool KSLAB = false>
 __device__ __forceinline__ void qb_issue(const CUtensorMap *tm_k, const CUtensorMap *tm_v, const QbPos &q, unsigned char *dst, uint64_t *bar)
 {
     using Geo = QbGeo<G>;
     qb_mbar_expect_tx(bar, QB_STAGE_BYTES);
-    if (q.sub < Geo::NK) {
+    if (KSLAB && q.sub < Geo::NK) {               // per-token keys: the key map has the value map's box
+        const int tok = q.grp * G + 32 * q.sub;
+        qb_tma_load(dst, tm_k, 0, tok, q.h, q.b, bar);
+        qb_tma_load(dst + 4096, tm_k, 64, tok, q.h, q.b, bar);
+    } else if (q.sub < Geo::NK) {
         qb_tma_load(dst, tm_k, q.sub * Geo::KC, q.grp * G, q.h, q.b, bar);
     } else {
         const int tok = q.grp * G + 32 * (q.sub - Geo::NK);
@@ -312,12 +318,17 @@ __device__ __forceinline__ void qb_issue(const CUtensorMap *tm_k, const CUtensor
 // MODE 0: dynamic parameters (the statistics of every group are taken here).  MODE 1: static parameters `sp` (one pair per key
 // channel and per value channel group of the KV head): no statistics pass, nothing written to the parameter arrays; the
 // thresholds of the 2-bit coder describe Eq. 8's clamp exactly, so values outside the calibrated range need nothing more.
+// MODE 2: per-token keys.  A key item is a 32-token slab like a value item (both maps have the value map's box) read with the
+// plain ldmatrix, so that the registers are the pair slots of the KEY tiles (rows = tokens): the statistics of a token and
+// channel group run over a row (registers 0, 2 or 1, 3, both halves, the four lanes of a quad), its pair goes to the
+// key parameter arrays in the value parameters' shape, and both elements of a register share one key.
 template <int BITS, int G, int MODE = 0>
 __global__ void __launch_bounds__(32 * QbGeo<G, BITS>::WARPS, 1)
 quantize_bulk_kernel(Params p, kvsink_cache c, const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v, QbShape sh,
                      kvsink_static_params sp)
 {
-    static_assert(MODE == 0 || BITS == 2, "static parameters: the threshold coder only");
+    static_assert(MODE != 1 || BITS == 2, "static parameters: the threshold coder only");
+    static_assert(QbGeo<G, BITS>::NK == QbGeo<G, BITS>::NV, "a group has as many 32-token slabs as 4096-element key items");
     using Geo = QbGeo<G, BITS>;
     constexpr int D = QB_D, NS = Geo::NS, KPL = Geo::KPL, MT = Geo::MT, NT = Geo::NT, NGv = Geo::NGv, NW = Geo::WARPS;
     constexpr int MPS = 16 / NS;                  // matrices per statistic set
@@ -347,6 +358,7 @@ quantize_bulk_kernel(Params p, kvsink_cache c, const __grid_constant__ CUtensorM
     //           matrix 8T + m = tile T x channels [16m, 16m+16): row 16T + rr + 8 (mj >> 1), chunk 2 (m & 3) + (mj & 1)
     //   keys:   KROWB-byte rows of KC channels; matrix NT*mi + T: row 16T + rr + 8 (mj & 1), chunk 2 mi + (mj >> 1)
     const uint32_t lane_v = (uint32_t)((rr + 8 * (mj >> 1)) * 128 + ((((mj & 1) ^ (rr & 1)) | (rr & 6)) << 4));
+    const uint32_t lane_ks = (uint32_t)((rr + 8 * (mj & 1)) * 128 + ((((mj >> 1) ^ (rr & 1)) | (rr & 6)) << 4));   // key slabs (MODE 2): value layout, plain load
     const uint32_t lane_k = Geo::KROWB == 64 ? (uint32_t)((rr + 8 * (mj & 1)) * 64 + ((((mj >> 1) ^ ((rr >> 1) & 1)) | ((rr >> 1) & 2)) << 4))
                                              : (uint32_t)((rr + 8 * (mj & 1)) * 128 + ((((mj >> 1) ^ (rr & 1)) | (rr & 6)) << 4));
 
@@ -365,21 +377,23 @@ quantize_bulk_kernel(Params p, kvsink_cache c, const __grid_constant__ CUtensorM
     QbMask mw;
     mw.w0 = mw.w1 = mw.w2 = mw.w3 = 0u;
     if (id < sh.n_items) {
-        qb_load_mask<G>(p, c, cur.sub, cur.grp, cur.b, sh.first_token, mw);
-        if (lane == 0) qb_issue<G>(&tm_k, &tm_v, cur, my_stage, my_full);
+        qb_load_mask<G, MODE == 2>(p, c, cur.sub, cur.grp, cur.b, sh.first_token, mw);
+        if (lane == 0) qb_issue<G, MODE == 2>(&tm_k, &tm_v, cur, my_stage, my_full);
     }
     unsigned phase = 0;                           // parity of the stage's current use
     for (; id < sh.n_items; id += id_step, phase ^= 1u) {
         // sink bits of the warp's next item, fetched while this one is processed
         QbMask mw_next;
         mw_next.w0 = mw_next.w1 = mw_next.w2 = mw_next.w3 = 0u;
-        if (id + id_step < sh.n_items) qb_load_mask<G>(p, c, nxt.sub, nxt.grp, nxt.b, sh.first_token, mw_next);
+        if (id + id_step < sh.n_items) qb_load_mask<G, MODE == 2>(p, c, nxt.sub, nxt.grp, nxt.b, sh.first_token, mw_next);
         if (!__all_sync(0xffffffffu, qb_wait(my_full, phase))) {
             if (lane == 0) atomicOr(c.status, KVSINK_STATUS_TIMEOUT);
             break;
         }
         const uint32_t stage = smem_addr(my_stage);
         const bool is_v = cur.sub >= Geo::NK;     // warp-uniform
+        const bool kslab = MODE == 2 && !is_v;    // a key item in the slab form
+        const bool slab = is_v || kslab;          // 32 tokens x 128 channels, parameters per token
         const int sub = is_v ? cur.sub - Geo::NK : cur.sub;
         const int64_t unit = (int64_t)cur.b * p.Hkv + cur.h;
         const int p0 = sh.first_token + cur.grp * G;   // first token of the group (multiple of G)
@@ -392,6 +406,12 @@ quantize_bulk_kernel(Params p, kvsink_cache c, const __grid_constant__ CUtensorM
             for (int u = 0; u < 16; ++u) {
                 const int T = u >> 3, m = u & 7;
                 qb_ldmatrix_x4_trans(a[u], ((stage + lane_v) ^ ((m & 3) << 5)) + T * 2048 + (m >> 2) * 4096);
+            }
+        } else if (MODE == 2) {
+#pragma unroll
+            for (int u = 0; u < 16; ++u) {
+                const int T = u >> 3, m = u & 7;
+                qb_ldmatrix_x4(a[u], ((stage + lane_ks) ^ ((m & 3) << 5)) + T * 2048 + (m >> 2) * 4096);
             }
         } else {
 #pragma unroll
@@ -409,7 +429,7 @@ quantize_bulk_kernel(Params p, kvsink_cache c, const __grid_constant__ CUtensorM
             const int count = min(c.sink_count[cur.b], p.cap);
             const int32_t *sp = c.sink_pos + (size_t)cur.b * p.cap;
             __half *side = (__half *)(is_v ? c.sink_v : c.sink_k);
-            const int tok0 = is_v ? p0 + 32 * sub : p0;
+            const int tok0 = slab ? p0 + 32 * sub : p0;
             int slot = -1;                        // rank of the next sink token of the item
 #pragma unroll
             for (int wi = 0; wi < 4; ++wi)
@@ -432,7 +452,7 @@ quantize_bulk_kernel(Params p, kvsink_cache c, const __grid_constant__ CUtensorM
                 __half *dst = side + ((size_t)unit * p.cap + my) * D;
                 uint32_t src;
                 int n16, off;                     // 16-byte chunks of the row held by this item, first channel
-                if (is_v) {
+                if (slab) {
                     src = stage + (lane >> 3) * 4096 + r * 128 + (((lane & 7) ^ (r & 7)) << 4);
                     n16 = 16; off = 0;
                 } else {
@@ -456,6 +476,14 @@ quantize_bulk_kernel(Params p, kvsink_cache c, const __grid_constant__ CUtensorM
         for (int s = 0; s < NS; ++s) { mn[s][0] = mn[s][1] = PINF2; mx[s][0] = mx[s][1] = NINF2; }
         if constexpr (MODE == 1) {
             // static parameters: no statistics
+        } else if (kslab) {
+            // per-token keys: set s = tile x channel group, side 0 = the token of rows g (registers 0, 2), side 1 = that of rows g + 8
+#pragma unroll
+            for (int u = 0; u < 16; ++u) {
+                const int s = u / MPS;
+                mn[s][0] = qb_hmin2(mn[s][0], qb_hmin2(a[u][0], a[u][2])); mx[s][0] = qb_hmax2(mx[s][0], qb_hmax2(a[u][0], a[u][2]));
+                mn[s][1] = qb_hmin2(mn[s][1], qb_hmin2(a[u][1], a[u][3])); mx[s][1] = qb_hmax2(mx[s][1], qb_hmax2(a[u][1], a[u][3]));
+            }
         } else if (is_v || !has_sink) {
 #pragma unroll
             for (int u = 0; u < 16; ++u) {
@@ -482,11 +510,26 @@ quantize_bulk_kernel(Params p, kvsink_cache c, const __grid_constant__ CUtensorM
         // while this one is coded from registers
         const QbPos nn = qb_advance<G>(nxt, step, sh.n_groups, p.Hkv);
         __syncwarp();
-        if (lane == 0 && id + id_step < sh.n_items) qb_issue<G>(&tm_k, &tm_v, nxt, my_stage, my_full);
+        if (lane == 0 && id + id_step < sh.n_items) qb_issue<G, MODE == 2>(&tm_k, &tm_v, nxt, my_stage, my_full);
 
+        if (kslab) {
+            // the other channels of a token row live in the other half of the register and in the other lanes of the quad
+#pragma unroll
+            for (int s = 0; s < NS; ++s)
+#pragma unroll
+                for (int ab = 0; ab < 2; ++ab) {
+                    uint32_t lo2 = qb_hmin2(mn[s][ab], __byte_perm(mn[s][ab], 0u, 0x1032)), hi2 = qb_hmax2(mx[s][ab], __byte_perm(mx[s][ab], 0u, 0x1032));
+#pragma unroll
+                    for (int o = 1; o < 4; o <<= 1) {
+                        lo2 = qb_hmin2(lo2, __shfl_xor_sync(0xffffffffu, lo2, o));
+                        hi2 = qb_hmax2(hi2, __shfl_xor_sync(0xffffffffu, hi2, o));
+                    }
+                    mn[s][ab] = lo2; mx[s][ab] = hi2;
+                }
+        } else {
         // the other rows of a column live in the lanes that differ in bits 2..4
 #pragma unroll
-        for (int o = 4; o < 32 && MODE == 0; o <<= 1)
+        for (int o = 4; o < 32 && MODE != 1; o <<= 1)
 #pragma unroll
             for (int s = 0; s < NS; ++s)
 #pragma unroll
@@ -494,11 +537,14 @@ quantize_bulk_kernel(Params p, kvsink_cache c, const __grid_constant__ CUtensorM
                     mn[s][ab] = qb_hmin2(mn[s][ab], __shfl_xor_sync(0xffffffffu, mn[s][ab], o));
                     mx[s][ab] = qb_hmax2(mx[s][ab], __shfl_xor_sync(0xffffffffu, mx[s][ab], o));
                 }
+        }
 
         // ---- parameters (Eq. 10-11) and thresholds: the eight lanes of a column group share its 4 * NS keys ----
 #pragma unroll
         for (int j = 0; j < KPL; ++j) {
-            const int kk = g + 8 * j, s_ = kk >> 2, ab_ = (kk >> 1) & 1, e_ = kk & 1;
+            // the lane's j-th key.  Per-token keys: lane (g, t) takes the token of tile t >> 1, rows g + 8 (t & 1), channel group j
+            const int kk = g + 8 * j;
+            const int s_ = kslab ? (t4 >> 1) * NGv + j : kk >> 2, ab_ = kslab ? (t4 & 1) : (kk >> 1) & 1, e_ = kslab ? 0 : kk & 1;
             uint32_t smn = 0, smx = 0;
 #pragma unroll
             for (int s = 0; s < NS; ++s)
@@ -508,8 +554,8 @@ quantize_bulk_kernel(Params p, kvsink_cache c, const __grid_constant__ CUtensorM
             const unsigned short lo16 = (unsigned short)(e_ ? smn >> 16 : smn & 0xffffu), hi16 = (unsigned short)(e_ ? smx >> 16 : smx & 0xffffu);
             const float fmn = __half2float(__ushort_as_half(lo16)), fmx = __half2float(__ushort_as_half(hi16));
             // values: token of the item (set = tile * NGv + channel group); keys: channel of the item (set = matrix)
-            const int idx = 16 * (is_v ? s_ / NGv : s_) + 8 * ab_ + 2 * t4 + e_;
-            const bool member = is_v ? !((mw.w0 >> idx) & 1u) : (MODE == 1 || lo16 != 0x7C00);
+            const int idx = kslab ? 16 * (t4 >> 1) + 8 * (t4 & 1) + g : 16 * (is_v ? s_ / NGv : s_) + 8 * ab_ + 2 * t4 + e_;
+            const bool member = slab ? !((mw.w0 >> idx) & 1u) : (MODE == 1 || lo16 != 0x7C00);
             float s, z;
             if constexpr (MODE == 1) {
                 // the pair of this key channel / of this token's value channel group; a sink token's values keep code 0
@@ -520,11 +566,12 @@ quantize_bulk_kernel(Params p, kvsink_cache c, const __grid_constant__ CUtensorM
                 group_params(member, fmn, fmx, qmax, &s, &z);
                 const size_t ov = ((size_t)unit * p.max_seq + p0 + 32 * sub + idx) * NGv + (s_ % NGv);
                 const size_t ok = ((size_t)unit * (p.max_seq / G) + p0 / G) * D + sub * Geo::KC + idx;
-                float *ps = is_v ? c.v_scale + ov : c.k_scale + ok, *pz = is_v ? c.v_zero + ov : c.k_zero + ok;
+                float *ps = is_v ? c.v_scale + ov : c.k_scale + (kslab ? ov : ok), *pz = is_v ? c.v_zero + ov : c.k_zero + (kslab ? ov : ok);
                 *ps = s;
                 *pz = z;
             }
-            const int pos = 8 * (kk >> 1) + 2 * t4 + e_;
+            // place of the key in the warp's table: (set, side) block of eight, then the lane coordinate that owns its elements
+            const int pos = kslab ? 8 * (2 * s_ + ab_) + g : 8 * (kk >> 1) + 2 * t4 + e_;
             if constexpr (BITS == 2) {
                 const double s_half = 0.5 * (double)s;
 #pragma unroll
@@ -533,15 +580,15 @@ quantize_bulk_kernel(Params p, kvsink_cache c, const __grid_constant__ CUtensorM
             } else {
                 const QbCoder cc = qb_make_coder(s, z, fmn, fmx, qmax);
                 QbCoder2 *c2 = coder + (pos >> 1);
-                c2->r_lo[e_] = cc.r_lo;
-                c2->r_hi[e_] = cc.r_hi;
-                c2->magic[e_] = cc.magic;
+                c2->r_lo[pos & 1] = cc.r_lo;
+                c2->r_hi[pos & 1] = cc.r_hi;
+                c2->magic[pos & 1] = cc.magic;
                 sz[pos] = make_float2(s, z);
             }
         }
         __syncwarp();
 
-        const size_t tile0 = (size_t)unit * (p.max_seq / KVSINK_TILE) + p0 / KVSINK_TILE + (is_v ? 2 * sub : 0);
+        const size_t tile0 = (size_t)unit * (p.max_seq / KVSINK_TILE) + p0 / KVSINK_TILE + (slab ? 2 * sub : 0);
         uint8_t *codes = (is_v ? c.v_codes : c.k_codes) + tile0 * Geo::TILE_BYTES;
         if constexpr (BITS == 2) {
             // ---- coding: every register becomes its byte of packed fields (in both halves) ----
@@ -551,26 +598,32 @@ quantize_bulk_kernel(Params p, kvsink_cache c, const __grid_constant__ CUtensorM
             uint32_t bits[16];
 #pragma unroll
             for (int s = 0; s < NS; ++s) {
-                __half2 tq[2][3];
+                // thresholds of the keys of registers 0, 1 (side 0) and 2, 3 (side 1); per-token keys: of registers 0, 2 and 1, 3,
+                // one key for both halves
+                __half2 tq[2][3], tq1[3], tq2[3];
 #pragma unroll
                 for (int ab = 0; ab < 2; ++ab)
 #pragma unroll
-                    for (int l = 0; l < 3; ++l) tq[ab][l] = *reinterpret_cast<const __half2 *>(thr + l * (16 * NS) + 8 * (2 * s + ab) + 2 * t4);
+                    for (int l = 0; l < 3; ++l)
+                        tq[ab][l] = kslab ? __half2half2(thr[l * (16 * NS) + 8 * (2 * s + ab) + g])
+                                          : *reinterpret_cast<const __half2 *>(thr + l * (16 * NS) + 8 * (2 * s + ab) + 2 * t4);
+#pragma unroll
+                for (int l = 0; l < 3; ++l) { tq1[l] = kslab ? tq[1][l] : tq[0][l]; tq2[l] = kslab ? tq[0][l] : tq[1][l]; }
 #pragma unroll
                 for (int i = 0; i < MPS; ++i) {
                     const int u = s * MPS + i;
                     __half2 acc = base;
                     acc = qb_thermo(acc, a[u][0], tq[0], w0);
-                    acc = qb_thermo(acc, a[u][1], tq[0], w1);
-                    acc = qb_thermo(acc, a[u][2], tq[1], w2);
+                    acc = qb_thermo(acc, a[u][1], tq1, w1);
+                    acc = qb_thermo(acc, a[u][2], tq2, w2);
                     acc = qb_thermo(acc, a[u][3], tq[1], w3);
                     bits[u] = *reinterpret_cast<uint32_t *>(&acc);   // 0x6400 | byte in each half
                 }
             }
             __syncwarp();   // the scratch is rewritten by the next item
-            if (has_sink && !is_v) {
-                // sink tokens keep code 0: fields 0, 2 of a byte are row g, fields 1, 3 row g + 8 (value items need
-                // nothing: the thresholds of a sink token are +inf)
+            if (has_sink && !slab) {
+                // sink tokens keep code 0: fields 0, 2 of a byte are row g, fields 1, 3 row g + 8 (items with per-token
+                // parameters need nothing: the thresholds of a sink token are +inf)
 #pragma unroll
                 for (int u = 0; u < 16; ++u) {
                     const int T = u % NT;
@@ -580,7 +633,7 @@ quantize_bulk_kernel(Params p, kvsink_cache c, const __grid_constant__ CUtensorM
                 }
             }
             // ---- packed words: bytes (even matrix lo, odd matrix lo, even matrix hi, odd matrix hi) ----
-            if (is_v) {
+            if (slab) {
 #pragma unroll
                 for (int T = 0; T < 2; ++T) {
                     uint4 w;
@@ -610,31 +663,44 @@ quantize_bulk_kernel(Params p, kvsink_cache c, const __grid_constant__ CUtensorM
                 unsigned long long k_lo[2], k_hi[2], k_magic[2];   // key pairs of this lane's columns (side 0, side 1)
 #pragma unroll
                 for (int q = 0; q < 2; ++q) {
-                    const QbCoder2 *c2 = coder + 4 * (2 * s + q) + t4;
-                    const float4 rr = *reinterpret_cast<const float4 *>(c2->r_lo);
-                    const float2 mm = *reinterpret_cast<const float2 *>(c2->magic);
-                    k_lo[q] = qb_pair(rr.x, rr.y);
-                    k_hi[q] = qb_pair(rr.z, rr.w);
-                    k_magic[q] = qb_pair(mm.x, mm.y);
+                    if (kslab) {                                   // one key (token row g + 8 q) for both elements
+                        const QbCoder2 *c2 = coder + 4 * (2 * s + q) + (g >> 1);
+                        const float rl = c2->r_lo[g & 1], rh = c2->r_hi[g & 1], mg = c2->magic[g & 1];
+                        k_lo[q] = qb_pair(rl, rl);
+                        k_hi[q] = qb_pair(rh, rh);
+                        k_magic[q] = qb_pair(mg, mg);
+                    } else {
+                        const QbCoder2 *c2 = coder + 4 * (2 * s + q) + t4;
+                        const float4 rr = *reinterpret_cast<const float4 *>(c2->r_lo);
+                        const float2 mm = *reinterpret_cast<const float2 *>(c2->magic);
+                        k_lo[q] = qb_pair(rr.x, rr.y);
+                        k_hi[q] = qb_pair(rr.z, rr.w);
+                        k_magic[q] = qb_pair(mm.x, mm.y);
+                    }
                 }
+                // registers 0, 1 take side 0 and 2, 3 side 1; with per-token keys registers 0, 2 take side 0 and 1, 3 side 1
+                const unsigned long long kl[4] = {k_lo[0], kslab ? k_lo[1] : k_lo[0], kslab ? k_lo[0] : k_lo[1], k_lo[1]};
+                const unsigned long long kh[4] = {k_hi[0], kslab ? k_hi[1] : k_hi[0], kslab ? k_hi[0] : k_hi[1], k_hi[1]};
+                const unsigned long long km[4] = {k_magic[0], kslab ? k_magic[1] : k_magic[0], kslab ? k_magic[0] : k_magic[1], k_magic[1]};
 #pragma unroll
                 for (int i = 0; i < MPS; ++i) {
                     const int u = s * MPS + i;
-                    const int m = is_v ? (u & 7) : sub * MT + u / NT;   // matrix of the tile
+                    const int m = slab ? (u & 7) : sub * MT + u / NT;   // matrix of the tile
                     uint32_t pc[4];
                     uint32_t differ[4] = {0u, 0u, 0u, 0u};
 #pragma unroll
-                    for (int r = 0; r < 4; ++r) pc[r] = qb_code_pair(a[u][r], k_lo[r >> 1], k_hi[r >> 1], k_magic[r >> 1], differ[r]);
+                    for (int r = 0; r < 4; ++r) pc[r] = qb_code_pair(a[u][r], kl[r], kh[r], km[r], differ[r]);
                     if (differ[0] | differ[1] | differ[2] | differ[3]) {
                         // a value too close to a rounding tie (fp16 inputs land on exact ties often): redo those registers
 #pragma unroll
                         for (int r = 0; r < 4; ++r)
                             if (differ[r]) {
-                                const float2 z0 = sz[8 * (2 * s + (r >> 1)) + 2 * t4], z1 = sz[8 * (2 * s + (r >> 1)) + 2 * t4 + 1];
+                                const int zi = kslab ? 8 * (2 * s + (r & 1)) + g : 8 * (2 * s + (r >> 1)) + 2 * t4;
+                                const float2 z0 = sz[zi], z1 = sz[kslab ? zi : zi + 1];
                                 pc[r] = qb_code_pair_exact(a[u][r], z0.x, z0.y, z1.x, z1.y, qmax);
                             }
                     }
-                    if (has_sink && !is_v) {   // sink tokens keep code 0: pair slots 0, 2 are row g, slots 1, 3 row g + 8
+                    if (has_sink && !slab) {   // sink tokens keep code 0: pair slots 0, 2 are row g, slots 1, 3 row g + 8
                         const int T = u % NT;
                         const uint32_t m16 = (qb_mask_word(mw, T >> 1) >> (16 * (T & 1))) & 0xffffu;
                         if ((m16 >> g) & 1u) pc[0] = pc[2] = 0;
@@ -646,7 +712,7 @@ quantize_bulk_kernel(Params p, kvsink_cache c, const __grid_constant__ CUtensorM
             __syncwarp();   // the scratch is rewritten by the next item
             // ---- packed words.  4 bit: word m of a lane is matrix m, planes of four words.  3 bit: low section as for
             //      2 bit (word m >> 1, byte m & 1 of each half), high section at 512 bytes (word m >> 2, two per lane) ----
-            if (is_v) {
+            if (slab) {
 #pragma unroll
                 for (int T = 0; T < 2; ++T) {
                     uint8_t *dst = codes + T * Geo::TILE_BYTES;
@@ -730,7 +796,9 @@ int launch_bulk(const Params &p, const kvsink_cache &c, const kvsink_static_para
     using Geo = QbGeo<G, BITS>;
     CUtensorMap tm_k, tm_v;
     const int T = n_groups * G;
-    if (!make_map(&tm_k, k_src, p, T, sb, sh, stt, Geo::KC, G, Geo::KROWB == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B))
+    if (MODE == 2) {
+        if (!make_map(&tm_k, k_src, p, T, sb, sh, stt, 64, 32, CU_TENSOR_MAP_SWIZZLE_128B)) return KVSINK_ERR_UNSUPPORTED;
+    } else if (!make_map(&tm_k, k_src, p, T, sb, sh, stt, Geo::KC, G, Geo::KROWB == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B))
         return KVSINK_ERR_UNSUPPORTED;
     if (!make_map(&tm_v, v_src, p, T, sb, sh, stt, 64, 32, CU_TENSOR_MAP_SWIZZLE_128B)) return KVSINK_ERR_UNSUPPORTED;
     constexpr int NW = Geo::WARPS;
@@ -774,6 +842,21 @@ int launch_quantize_static_bulk(const Params &p, const kvsink_cache &c, const kv
     if (p.D != QB_D || n_groups < 1 || first_token % p.G) return KVSINK_ERR_UNSUPPORTED;
     if (p.bits == 2 && p.G == 128) return launch_bulk<2, 128, 1>(p, c, sp, k_src, v_src, first_token, n_groups, sb, sh, stt, st);
     if (p.bits == 2 && p.G == 64) return launch_bulk<2, 64, 1>(p, c, sp, k_src, v_src, first_token, n_groups, sb, sh, stt, st);
+    return KVSINK_ERR_UNSUPPORTED;
+}
+
+// The same for per-token keys (keys quantized like values; the pairs go to the key parameter arrays in the value parameters' shape).
+// 3 bit has no form here: its bulk items need 64-token spans, which give two channel groups per row, and the decode side of
+// per-token keys takes one group at 3 bit.
+int launch_quantize_pertoken_bulk(const Params &p, const kvsink_cache &c, const __half *k_src, const __half *v_src, int first_token, int n_groups,
+                                  int64_t sb, int64_t sh, int64_t stt, cudaStream_t st)
+{
+    if (p.D != QB_D || n_groups < 1 || first_token % p.G) return KVSINK_ERR_UNSUPPORTED;
+    const kvsink_static_params none = {nullptr, nullptr, nullptr, nullptr};
+    if (p.bits == 2 && p.G == 128) return launch_bulk<2, 128, 2>(p, c, none, k_src, v_src, first_token, n_groups, sb, sh, stt, st);
+    if (p.bits == 2 && p.G == 64) return launch_bulk<2, 64, 2>(p, c, none, k_src, v_src, first_token, n_groups, sb, sh, stt, st);
+    if (p.bits == 4 && p.G == 128) return launch_bulk<4, 128, 2>(p, c, none, k_src, v_src, first_token, n_groups, sb, sh, stt, st);
+    if (p.bits == 4 && p.G == 64) return launch_bulk<4, 64, 2>(p, c, none, k_src, v_src, first_token, n_groups, sb, sh, stt, st);
     return KVSINK_ERR_UNSUPPORTED;
 }
 

@@ -87,6 +87,15 @@ def test_chunked_appends_that_start_and_end_inside_tiles(bits):
     _both(wl, chunks=(1, 14, 1, 33, 100, 1, 183))
 
 
+@pytest.mark.parametrize("bits,group", [(2, 64), (2, 128), (4, 64), (4, 128), (3, 128)])
+def test_chunks_through_the_bulk_quantizer(bits, group):
+    # chunks that start on a multiple of the group size send their whole spans to the bulk kernel, the rest to the tile kernels
+    G = group
+    rep = 1 if bits == 3 else 2
+    wl = TINY.scaled(seq=5 * G + 19, group=G, bits=bits, head_dim=128, n_q_heads=2 * rep, n_kv_heads=2, batch=2, topk=7, pfn_n=2, seed=83 + G + bits)
+    _both(wl, chunks=(G, G + 6, G - 6, 2 * G, 19))
+
+
 @pytest.mark.parametrize("bits,group,seq", [(2, 64, 101), (4, 128, 300), (3, 128, 77)])
 def test_unwritten_cache_memory_never_reaches_a_result(bits, group, seq):
     rep = 1 if bits == 3 else 2
