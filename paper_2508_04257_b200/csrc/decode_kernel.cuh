@@ -1242,9 +1242,13 @@ static int launch_prefill_p(const Params &p, const kvsink_cache &c, const __half
 template <int BITS, int D, int NGV>
 static int launch_prefill_n(const Params &p, const kvsink_cache &c, const __half *q, const PrefillShape &pre, float *out, float *lse, cudaStream_t st)
 {
-    if constexpr (4 * (2 * 128 * (D * BITS / 64) + 2 * 16 * NGV * 4) <= 4800)
+    // several channel groups per row mean G = D / NGV tokens per group: only chunk sizes that divide such a group are built;
+    // four groups per row take one tile per chunk (their parameter registers would spill otherwise)
+    constexpr int TPG_MAX = NGV == 1 ? 4 : D / NGV / KVSINK_TILE;
+    if constexpr (TPG_MAX % 4 == 0 && 4 * (2 * 128 * (D * BITS / 64) + 2 * 16 * NGV * 4) <= 4800)
         if ((p.G / KVSINK_TILE) % 4 == 0) return launch_prefill_p<BITS, D, NGV, 4>(p, c, q, pre, out, lse, st);
-    if ((p.G / KVSINK_TILE) % 2 == 0) return launch_prefill_p<BITS, D, NGV, 2>(p, c, q, pre, out, lse, st);
+    if constexpr (TPG_MAX % 2 == 0 && NGV < 4)
+        if ((p.G / KVSINK_TILE) % 2 == 0) return launch_prefill_p<BITS, D, NGV, 2>(p, c, q, pre, out, lse, st);
     return launch_prefill_p<BITS, D, NGV, 1>(p, c, q, pre, out, lse, st);
 }
 
@@ -1290,9 +1294,13 @@ static int launch_decode_n(const Params &p, const kvsink_cache &c, const kvsink_
 {
     // ring chunks of four tiles where a key group divides into them and two slots of that size stay below ~9 KB per
     // warp, else of two tiles (G a multiple of 32), else of one
-    if constexpr (4 * (2 * 128 * (D * BITS / 64) + (PM == 2 ? 4 : 2) * 16 * NGV * 4) <= 4800)
+    // several channel groups per row mean G = D / NGV tokens per group: only chunk sizes that divide such a group are built;
+    // four groups per row take one tile per chunk (their parameter registers would spill otherwise)
+    constexpr int TPG_MAX = NGV == 1 ? 4 : D / NGV / KVSINK_TILE;
+    if constexpr (TPG_MAX % 4 == 0 && 4 * (2 * 128 * (D * BITS / 64) + (PM == 2 ? 4 : 2) * 16 * NGV * 4) <= 4800)
         if ((p.G / KVSINK_TILE) % 4 == 0) return launch_decode_c<BITS, D, NGV, 4, PM>(p, c, cal, q, out, lse, ws, st);
-    if ((p.G / KVSINK_TILE) % 2 == 0) return launch_decode_c<BITS, D, NGV, 2, PM>(p, c, cal, q, out, lse, ws, st);
+    if constexpr (TPG_MAX % 2 == 0 && NGV < 4)
+        if ((p.G / KVSINK_TILE) % 2 == 0) return launch_decode_c<BITS, D, NGV, 2, PM>(p, c, cal, q, out, lse, ws, st);
     return launch_decode_c<BITS, D, NGV, 1, PM>(p, c, cal, q, out, lse, ws, st);
 }
 

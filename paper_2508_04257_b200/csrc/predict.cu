@@ -123,6 +123,13 @@ __device__ __forceinline__ void find_bin(const unsigned *hist, int need, int *bi
     }
 }
 
+// One more key in a shared-memory histogram.  (Electing one lane per bin with a warp match was measured: slower than the
+// atomics it saves.)
+__device__ __forceinline__ void hist_add(unsigned *hist, unsigned bin, bool valid)
+{
+    if (valid) atomicAdd(&hist[bin], 1u);
+}
+
 // One block per sequence: 2-pass radix select of the k-th largest 16-bit score, then an ordered pass that
 // breaks ties by index, ORs the first N tokens in and emits mask words and ascending positions.
 __global__ void __launch_bounds__(SEL_THREADS)
@@ -140,16 +147,27 @@ sink_select(const uint16_t *__restrict__ score, int score_stride, int S, int k, 
     if (kk > 0) {
         if (tid < 256) hist[tid] = 0;
         __syncthreads();
-        for (int i = tid; i < S; i += SEL_THREADS) atomicAdd(&hist[sc[i] >> 8], 1u);
+        // eight independent loads per thread and trip, so that their latencies overlap
+        constexpr int HB = 8;
+        for (int base = 0; base < S; base += HB * SEL_THREADS) {
+            unsigned v[HB];
+#pragma unroll
+            for (int j = 0; j < HB; ++j) { const int i = base + j * SEL_THREADS + tid; v[j] = i < S ? sc[i] : 0xffffffffu; }
+#pragma unroll
+            for (int j = 0; j < HB; ++j) hist_add(hist, (v[j] >> 8) & 0xffu, v[j] != 0xffffffffu);
+        }
         __syncthreads();
         if (tid < 32) find_bin(hist, kk, &s_hi, &s_need);
         __syncthreads();
         const int hi = s_hi;
         if (tid < 256) hist[tid] = 0;
         __syncthreads();
-        for (int i = tid; i < S; i += SEL_THREADS) {
-            unsigned v = sc[i];
-            if ((int)(v >> 8) == hi) atomicAdd(&hist[v & 0xffu], 1u);
+        for (int base = 0; base < S; base += HB * SEL_THREADS) {
+            unsigned v[HB];
+#pragma unroll
+            for (int j = 0; j < HB; ++j) { const int i = base + j * SEL_THREADS + tid; v[j] = i < S ? sc[i] : 0xffffffffu; }
+#pragma unroll
+            for (int j = 0; j < HB; ++j) hist_add(hist, v[j] & 0xffu, v[j] != 0xffffffffu && (int)(v[j] >> 8) == hi);
         }
         __syncthreads();
         if (tid < 32) find_bin(hist, s_need, &s_lo, &s_r);
@@ -231,6 +249,25 @@ sink_select_cluster(const uint16_t *__restrict__ score, int score_stride, int S,
     pdl_wait();
     int vstar = 0x10000, r = 0;   // no score exceeds 0x10000: no top-k selection when kk == 0
     if (tid == 0) { s_neq = 0; s_nsel = 0; }
+    // keys of this block's steps (TPT consecutive tokens per thread and step), loaded once (all loads in flight together) and
+    // kept in registers for the histograms and both passes below; a token slot beyond the block's slice carries 0xffff,
+    // which no key equals (keys are 15-bit magnitudes)
+    constexpr int TPT = 4, STEP = SEL_THREADS * TPT;
+    uint2 keys[SELC_MAX_STEPS];
+#pragma unroll
+    for (int st = 0; st < SELC_MAX_STEPS; ++st) {
+        const int i0 = lo + st * STEP + TPT * tid;
+        keys[st] = make_uint2(0xffffffffu, 0xffffffffu);
+        if (st * STEP < slice && i0 < hi) {
+            if (i0 + TPT <= hi) keys[st] = *reinterpret_cast<const uint2 *>(sc + i0);   // rows are 16-byte aligned, i0 a multiple of 4
+            else {
+                unsigned kq[4];
+                for (int j = 0; j < TPT; ++j) kq[j] = i0 + j < hi ? sc[i0 + j] : 0xffffu;
+                keys[st] = make_uint2(kq[0] | (kq[1] << 16), kq[2] | (kq[3] << 16));
+            }
+        }
+    }
+    auto key_of = [&](int st, int j) { return ((j < 2 ? keys[st].x : keys[st].y) >> (16 * (j & 1))) & 0xffffu; };
     if (kk > 0) {
         // the cluster's histogram of a key byte: every block sums the blocks' histograms for itself
         auto global_bin = [&](int need, int *bin_out, int *rest_out) {
@@ -246,42 +283,31 @@ sink_select_cluster(const uint16_t *__restrict__ score, int score_stride, int S,
         };
         if (tid < 256) hist[tid] = 0;
         __syncthreads();
-        for (int i = lo + tid; i < hi; i += SEL_THREADS) atomicAdd(&hist[sc[i] >> 8], 1u);
+#pragma unroll
+        for (int st = 0; st < SELC_MAX_STEPS; ++st)
+            if (st * STEP < slice) {                    // block-uniform
+#pragma unroll
+                for (int j = 0; j < TPT; ++j) { const unsigned v = key_of(st, j); hist_add(hist, (v >> 8) & 0xffu, v != 0xffffu); }
+            }
         global_bin(kk, &s_hi, &s_need);
         const int hi_byte = s_hi;
         if (tid < 256) hist[tid] = 0;
         __syncthreads();
-        for (int i = lo + tid; i < hi; i += SEL_THREADS) {
-            const unsigned v = sc[i];
-            if ((int)(v >> 8) == hi_byte) atomicAdd(&hist[v & 0xffu], 1u);
-        }
+#pragma unroll
+        for (int st = 0; st < SELC_MAX_STEPS; ++st)
+            if (st * STEP < slice) {
+#pragma unroll
+                for (int j = 0; j < TPT; ++j) { const unsigned v = key_of(st, j); hist_add(hist, v & 0xffu, v != 0xffffu && (int)(v >> 8) == hi_byte); }
+            }
         global_bin(s_need, &s_lo, &s_r);
         vstar = (hi_byte << 8) | s_lo;
         r = s_r;
     }
-    // keys of this block's steps (TPT consecutive tokens per thread and step), kept in registers for both passes below
-    constexpr int TPT = 4, STEP = SEL_THREADS * TPT;
-    uint2 keys[SELC_MAX_STEPS];
     int my_eq = 0;
 #pragma unroll
-    for (int st = 0; st < SELC_MAX_STEPS; ++st) {
-        const int i0 = lo + st * STEP + TPT * tid;
-        keys[st] = make_uint2(0xffffffffu, 0xffffffffu);          // 0xffff: no token
-        if (st * STEP < slice && i0 < hi) {
-            if (i0 + TPT <= hi) keys[st] = *reinterpret_cast<const uint2 *>(sc + i0);   // rows are 16-byte aligned, i0 a multiple of 4
-            else {
-                unsigned kq[4];
-                for (int j = 0; j < TPT; ++j) kq[j] = i0 + j < hi ? sc[i0 + j] : 0xffffu;
-                keys[st] = make_uint2(kq[0] | (kq[1] << 16), kq[2] | (kq[3] << 16));
-            }
-            // a token slot beyond the sequence carries 0xffff; a real key equal to it is told apart by its index below
+    for (int st = 0; st < SELC_MAX_STEPS; ++st)
 #pragma unroll
-            for (int j = 0; j < TPT; ++j) {
-                const int key = (int)(((j < 2 ? keys[st].x : keys[st].y) >> (16 * (j & 1))) & 0xffffu);
-                my_eq += (i0 + j < hi) && key == vstar;
-            }
-        }
-    }
+        for (int j = 0; j < TPT; ++j) my_eq += (int)key_of(st, j) == vstar;
     // keys equal to the k-th largest in the blocks before this one
     if (my_eq) atomicAdd(&s_neq, my_eq);
     cl.sync();
