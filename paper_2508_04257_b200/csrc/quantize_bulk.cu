@@ -165,6 +165,33 @@ __device__ __forceinline__ QbCoder qb_make_coder(float scale, float zero, float 
     c.magic = QB_MAGIC + (ok ? zero : 0.f);
     return c;
 }
+// Coder for a static pair (Eq. 8 with its clamp, values anywhere in fp16).  The argument is first clamped to fp16 bounds xl, xh
+// whose own codes already saturate (unclamped code of xl <= -1, of xh >= qmax + 1: every value beyond them gets the same
+// clamped code as the bound), which keeps the unclamped integer small enough for a signed 16-bit field; the packed codes are
+// then clamped to [0, qmax] by one two-way 16-bit min/max.  Bounds beyond the fp16 range are infinite (no clamp needed).
+__device__ __forceinline__ QbCoder qb_make_coder_static(float scale, float zero, float qmax, __half *xl, __half *xh)
+{
+    QbCoder c;
+    c.pad = 0.f;
+    *xl = __ushort_as_half((unsigned short)0xFC00);   // -inf
+    *xh = __ushort_as_half((unsigned short)0x7C00);   // +inf
+    if (scale == 0.f) {   // nothing was calibrated, or sink token: code 0
+        c.r_lo = c.r_hi = 0.f;
+        c.magic = QB_MAGIC;
+        return c;
+    }
+    const float r = __frcp_rn(scale);
+    const float lo_real = scale * (-zero - 2.f), hi_real = scale * (qmax - zero + 2.f);
+    *xl = __float2half_rd(lo_real);
+    *xh = __float2half_ru(hi_real);
+    const float reach = fmaxf(fminf(fabsf(lo_real), 65504.f), fminf(fabsf(hi_real), 65504.f));   // largest |argument| after the clamp
+    // NaN in any of these makes the comparison false: exact path
+    const bool ok = reach * r + fabsf(zero) < 30000.f && r < 3.0e38f;
+    c.r_lo = ok ? __fmul_rn(r, 1.f - 2.384185791015625e-07f) : __int_as_float(0x7f800000);
+    c.r_hi = ok ? __fmul_rn(r, 1.f + 2.384185791015625e-07f) : r;
+    c.magic = QB_MAGIC + (ok ? zero : 0.f);
+    return c;
+}
 // The coders of two adjacent keys (the two elements of a half2 register), field by field, so that each field is the
 // operand pair of one packed fp32 FMA.
 struct __align__(16) QbCoder2 {
@@ -239,7 +266,8 @@ struct QbGeo {
     static constexpr int KROWB = 2 * KC;          // bytes per row of a key item in shared memory
     // per warp and for each of the item's 16 * NS keys: three fp16 thresholds (2 bit), or a coder (stored by key pair)
     // and (scale, zero)
-    static constexpr int SCRATCH = BITS == 2 ? 3 * 16 * NS * 2 : 8 * NS * (int)sizeof(QbCoder2) + 16 * NS * (int)sizeof(float2);
+    // (static pairs: also the two fp16 clamp bounds of every key)
+    static constexpr int SCRATCH = BITS == 2 ? 3 * 16 * NS * 2 : 8 * NS * (int)sizeof(QbCoder2) + 16 * NS * (int)sizeof(float2) + 2 * 16 * NS * 2;
     static constexpr int TILE_BYTES = 256 * BITS, ROW_BYTES = 16 * BITS;   // packed tile of 16 tokens x 128 channels
     // warps per block, each with one stage, one mbarrier and its scratch: 20 (96 registers per thread) for the 2-bit
     // coder; 16 (128 registers) for the 3- and 4-bit coder, which spills at 96 and measures 9 % faster this way
@@ -317,7 +345,8 @@ __device__ __forceinline__ void qb_issue(const CUtensorMap *tm_k, const CUtensor
 
 // MODE 0: dynamic parameters (the statistics of every group are taken here).  MODE 1: static parameters `sp` (one pair per key
 // channel and per value channel group of the KV head): no statistics pass, nothing written to the parameter arrays; the
-// thresholds of the 2-bit coder describe Eq. 8's clamp exactly, so values outside the calibrated range need nothing more.
+// thresholds of the 2-bit coder describe Eq. 8's clamp exactly, so values outside the calibrated range need nothing more;
+// the 3- and 4-bit coder clamps (qb_make_coder_static).
 // MODE 2: per-token keys.  A key item is a 32-token slab like a value item (both maps have the value map's box) read with the
 // plain ldmatrix, so that the registers are the pair slots of the KEY tiles (rows = tokens): the statistics of a token and
 // channel group run over a row (registers 0, 2 or 1, 3, both halves, the four lanes of a quad), its pair goes to the
@@ -327,7 +356,6 @@ __global__ void __launch_bounds__(32 * QbGeo<G, BITS>::WARPS, 1)
 quantize_bulk_kernel(Params p, kvsink_cache c, const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v, QbShape sh,
                      kvsink_static_params sp)
 {
-    static_assert(MODE != 1 || BITS == 2, "static parameters: the threshold coder only");
     static_assert(QbGeo<G, BITS>::NK == QbGeo<G, BITS>::NV, "a group has as many 32-token slabs as 4096-element key items");
     using Geo = QbGeo<G, BITS>;
     constexpr int D = QB_D, NS = Geo::NS, KPL = Geo::KPL, MT = Geo::MT, NT = Geo::NT, NGv = Geo::NGv, NW = Geo::WARPS;
@@ -365,6 +393,7 @@ quantize_bulk_kernel(Params p, kvsink_cache c, const __grid_constant__ CUtensorM
     __half *thr = (__half *)(scratch + (size_t)warp * Geo::SCRATCH);            // 2 bit: [3][16 * NS] thresholds
     QbCoder2 *coder = (QbCoder2 *)(scratch + (size_t)warp * Geo::SCRATCH);      // 3, 4 bit: [8 * NS] coders of key pairs ...
     float2 *sz = (float2 *)(coder + 8 * NS);                                   // ... and [16 * NS] (scale, zero)
+    __half *xl_tab = (__half *)(sz + 16 * NS), *xh_tab = xl_tab + 16 * NS;      // ... and (static pairs) [16 * NS] lower / upper clamp bounds
     unsigned char *my_stage = stages + (size_t)warp * QB_STAGE_BYTES;
     uint64_t *my_full = full + warp;
 
@@ -578,7 +607,15 @@ quantize_bulk_kernel(Params p, kvsink_cache c, const __grid_constant__ CUtensorM
                 for (int l = 0; l < 3; ++l)
                     thr[l * (16 * NS) + pos] = __ushort_as_half((unsigned short)qb_threshold(s, s_half, z, (float)(l + 1), qmax));
             } else {
-                const QbCoder cc = qb_make_coder(s, z, fmn, fmx, qmax);
+                QbCoder cc;
+                if constexpr (MODE == 1) {
+                    __half xl, xh;
+                    cc = qb_make_coder_static(s, z, qmax, &xl, &xh);
+                    xl_tab[pos] = xl;
+                    xh_tab[pos] = xh;
+                } else {
+                    cc = qb_make_coder(s, z, fmn, fmx, qmax);
+                }
                 QbCoder2 *c2 = coder + (pos >> 1);
                 c2->r_lo[pos & 1] = cc.r_lo;
                 c2->r_hi[pos & 1] = cc.r_hi;
@@ -682,6 +719,14 @@ quantize_bulk_kernel(Params p, kvsink_cache c, const __grid_constant__ CUtensorM
                 const unsigned long long kl[4] = {k_lo[0], kslab ? k_lo[1] : k_lo[0], kslab ? k_lo[0] : k_lo[1], k_lo[1]};
                 const unsigned long long kh[4] = {k_hi[0], kslab ? k_hi[1] : k_hi[0], kslab ? k_hi[0] : k_hi[1], k_hi[1]};
                 const unsigned long long km[4] = {k_magic[0], kslab ? k_magic[1] : k_magic[0], kslab ? k_magic[0] : k_magic[1], k_magic[1]};
+                uint32_t xl2[2] = {0u, 0u}, xh2[2] = {0u, 0u};   // static pairs: clamp bounds of the two keys of side 0 / side 1
+                if constexpr (MODE == 1) {
+#pragma unroll
+                    for (int q = 0; q < 2; ++q) {
+                        xl2[q] = *reinterpret_cast<const uint32_t *>(xl_tab + 8 * (2 * s + q) + 2 * t4);
+                        xh2[q] = *reinterpret_cast<const uint32_t *>(xh_tab + 8 * (2 * s + q) + 2 * t4);
+                    }
+                }
 #pragma unroll
                 for (int i = 0; i < MPS; ++i) {
                     const int u = s * MPS + i;
@@ -689,7 +734,11 @@ quantize_bulk_kernel(Params p, kvsink_cache c, const __grid_constant__ CUtensorM
                     uint32_t pc[4];
                     uint32_t differ[4] = {0u, 0u, 0u, 0u};
 #pragma unroll
-                    for (int r = 0; r < 4; ++r) pc[r] = qb_code_pair(a[u][r], kl[r], kh[r], km[r], differ[r]);
+                    for (int r = 0; r < 4; ++r) {
+                        uint32_t x2 = a[u][r];
+                        if constexpr (MODE == 1) x2 = qb_hmin2(qb_hmax2(x2, xl2[r >> 1]), xh2[r >> 1]);
+                        pc[r] = qb_code_pair(x2, kl[r], kh[r], km[r], differ[r]);
+                    }
                     if (differ[0] | differ[1] | differ[2] | differ[3]) {
                         // a value too close to a rounding tie (fp16 inputs land on exact ties often): redo those registers
 #pragma unroll
@@ -699,6 +748,11 @@ quantize_bulk_kernel(Params p, kvsink_cache c, const __grid_constant__ CUtensorM
                                 const float2 z0 = sz[zi], z1 = sz[kslab ? zi : zi + 1];
                                 pc[r] = qb_code_pair_exact(a[u][r], z0.x, z0.y, z1.x, z1.y, qmax);
                             }
+                    }
+                    if constexpr (MODE == 1) {   // Eq. 8's clamp on both 16-bit fields (an exact redo is inside the range already)
+                        const uint32_t q2 = (uint32_t)((1 << BITS) - 1) * 0x00010001u;
+#pragma unroll
+                        for (int r = 0; r < 4; ++r) pc[r] = __vimin_s16x2_relu(pc[r], q2);
                     }
                     if (has_sink && !slab) {   // sink tokens keep code 0: pair slots 0, 2 are row g, slots 1, 3 row g + 8
                         const int T = u % NT;
@@ -835,13 +889,16 @@ int launch_quantize_groups_bulk(const Params &p, const kvsink_cache &c, const __
 }
 
 // The same for static parameters: n_groups spans of G tokens (G only sets the shape of the work items here), the first at a
-// multiple of G.  2 bit only; other shapes return KVSINK_ERR_UNSUPPORTED and the caller uses the tile kernels.
+// multiple of G.  Shapes without a bulk kernel return KVSINK_ERR_UNSUPPORTED and the caller uses the tile kernels.
 int launch_quantize_static_bulk(const Params &p, const kvsink_cache &c, const kvsink_static_params &sp, const __half *k_src, const __half *v_src,
                                 int first_token, int n_groups, int64_t sb, int64_t sh, int64_t stt, cudaStream_t st)
 {
     if (p.D != QB_D || n_groups < 1 || first_token % p.G) return KVSINK_ERR_UNSUPPORTED;
     if (p.bits == 2 && p.G == 128) return launch_bulk<2, 128, 1>(p, c, sp, k_src, v_src, first_token, n_groups, sb, sh, stt, st);
     if (p.bits == 2 && p.G == 64) return launch_bulk<2, 64, 1>(p, c, sp, k_src, v_src, first_token, n_groups, sb, sh, stt, st);
+    if (p.bits == 3 && p.G == 64) return launch_bulk<3, 64, 1>(p, c, sp, k_src, v_src, first_token, n_groups, sb, sh, stt, st);
+    if (p.bits == 4 && p.G == 128) return launch_bulk<4, 128, 1>(p, c, sp, k_src, v_src, first_token, n_groups, sb, sh, stt, st);
+    if (p.bits == 4 && p.G == 64) return launch_bulk<4, 64, 1>(p, c, sp, k_src, v_src, first_token, n_groups, sb, sh, stt, st);
     return KVSINK_ERR_UNSUPPORTED;
 }
 

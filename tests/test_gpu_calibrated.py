@@ -74,13 +74,48 @@ def test_chunked_appends_and_values_outside_the_calibrated_range():
     _both(wl, chunks=(1, 14, 1, 33, 100, 1, 183), cal_tokens=50)
 
 
-@pytest.mark.parametrize("group", [64, 128])
-def test_two_bit_chunks_through_the_bulk_quantizer_with_values_outside_the_calibrated_range(group):
+@pytest.mark.parametrize("bits,group", [(2, 64), (2, 128), (3, 64), (4, 64), (4, 128)])
+@pytest.mark.parametrize("cal_tokens", [40, 3])
+def test_chunks_through_the_bulk_quantizer_with_values_outside_the_calibrated_range(bits, group, cal_tokens):
     # chunks that start on a multiple of the group size send their whole spans to the bulk kernel, the rest to the tile kernels;
-    # calibrated on 40 tokens only, so later tokens clamp at both ends
+    # calibrated on a few tokens only, so later tokens clamp at both ends (three tokens: most of them do)
     G = group
-    wl = TINY.scaled(seq=5 * G + 19, group=G, bits=2, head_dim=128, n_q_heads=4, n_kv_heads=2, batch=2, topk=7, pfn_n=2, seed=81 + G)
-    _both(wl, chunks=(G, G + 6, G - 6, 2 * G, 19), cal_tokens=40)
+    wl = TINY.scaled(seq=5 * G + 19, group=G, bits=bits, head_dim=128, n_q_heads=4, n_kv_heads=2, batch=2, topk=7, pfn_n=2, seed=81 + G + bits)
+    _both(wl, chunks=(G, G + 6, G - 6, 2 * G, 19), cal_tokens=cal_tokens)
+
+
+def test_static_pairs_that_force_the_literal_formula():
+    # hand-made pairs: a tiny scale with a huge zero-point (the fast coder declines), scale 0, and a scale so large that every
+    # value codes to the zero-point; the codes must still be the oracle's bit for bit
+    wl = TINY.scaled(seq=256, group=64, bits=4, head_dim=128, n_q_heads=2, n_kv_heads=2, batch=1, topk=3, pfn_n=1, seed=5)
+    ocfg, gcfg = configs(wl)
+    H = synth.make_hidden(wl, "cuda")
+    K, V = synth.make_kv(wl, 0, "cuda")
+    gs = kv.SinkSet(gcfg)
+    kv.predict_sinks(gcfg, H, gs)
+    bm, pos, cnt = oracle.predict_sinks(ocfg, np16(H))
+    gp, op = kv.StaticParams(gcfg), oracle.StaticParams(ocfg)
+    rng = np.random.default_rng(11)
+    ks = rng.uniform(0.05, 0.5, size=(2, 128)).astype(np.float32)
+    kz = np.rint(rng.uniform(0, 15, size=(2, 128))).astype(np.float32)
+    ks[:, 0] = 1e-6; kz[:, 0] = 5e6          # |zero| far beyond the fast coder's range
+    ks[:, 1] = 0.0; kz[:, 1] = 0.0           # never calibrated
+    ks[:, 2] = 1e4; kz[:, 2] = 7.0           # every value rounds to 0: code 7
+    ks[:, 3] = 3e-4; kz[:, 3] = 40000.0      # integer part beyond 16 bits: literal formula
+    ks[:, 4] = 2e-3; kz[:, 4] = -29990.0     # just inside the fast coder's range
+    vs = np.array([[0.3, 1e-5]] * 2, np.float32)
+    vz = np.array([[8.0, -70000.0]] * 2, np.float32)
+    for name, arr in (("k_scale", ks), ("k_zero", kz), ("v_scale", vs), ("v_zero", vz)):
+        getattr(gp, name).copy_(torch.from_numpy(arr))
+        getattr(op, name)[...] = arr.reshape(getattr(op, name).shape)
+    gc, oc = kv.KVCache(gcfg, gs), oracle.Cache(ocfg, bm, pos, cnt)
+    kv.quantize_append_calibrated(gcfg, gc, gp, K, V)
+    oracle.quantize_append_calibrated(ocfg, oc, op, np16(K), np16(V))
+    torch.cuda.synchronize()
+    per, nb = wl.max_seq * wl.head_dim * wl.bits // 8, wl.seq * wl.head_dim * wl.bits // 8
+    for name in ("k_codes", "v_codes"):
+        assert bits_equal(getattr(gc, name).cpu().numpy().reshape(-1, per)[:, :nb], getattr(oc, name).reshape(-1, per)[:, :nb]), name
+    assert kv.read_status(gc) == 0
 
 
 def test_many_splits_and_clusters():
