@@ -177,6 +177,12 @@ int launch_decode_b3(const Params &p, const kvsink_cache &c, const kvsink_static
 int launch_decode_b4(const Params &p, const kvsink_cache &c, const kvsink_static_params *cal, int mode, const __half *q, float *out, float *lse, float *ws,
                      cudaStream_t st);
 int launch_decode_merge(const float *ws, int nsplit, int D, int n_rows, float *out, float *lse, cudaStream_t st);
+// Query heads of one KV head that one decode block serves, and the blocks per KV head that makes.  Up to four heads share a
+// block; five to eight share one on the eight-column fp16 path, except at 2 and 3 bit with head size 128, where they go four
+// at a time to the integer key side (2 bit) or to the fp16 pair layout (3 bit): the eight-column path has no residual
+// columns, and with few bits and large zero-points its error comes close to, at 2 bit beyond, the attention tolerance.
+inline int decode_heads_per_block(const Params &p) { return p.rep <= 4 ? 4 : (p.D == 128 && p.bits <= 3 ? 4 : 8); }
+inline int decode_qchunks(const Params &p) { return (p.rep + decode_heads_per_block(p) - 1) / decode_heads_per_block(p); }
 int max_splits(const Params &p);
 int choose_splits(const Params &p, int n_groups);
 int launch_channel_absmax(const __half *hidden, int B, int S, int d, int64_t sb, int64_t ss, float *out, cudaStream_t st);

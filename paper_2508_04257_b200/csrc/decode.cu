@@ -67,7 +67,7 @@ constexpr int DEC_SLOTS = 148 * 4;   // resident blocks the split heuristic plan
 
 int max_splits(const Params &p)
 {
-    const int qchunks = (p.rep + 7) / 8;
+    const int qchunks = decode_qchunks(p);
     const long units = (long)p.B * p.Hkv * qchunks;
     long ns = (2L * DEC_SLOTS + units - 1) / units;
     const long mg = p.max_seq / p.G;
@@ -77,7 +77,7 @@ int max_splits(const Params &p)
 
 int choose_splits(const Params &p, int n_groups)
 {
-    const int qchunks = (p.rep + 7) / 8;
+    const int qchunks = decode_qchunks(p);
     const long units = (long)p.B * p.Hkv * qchunks;
     const int ns_max = max_splits(p) < n_groups ? max_splits(p) : (n_groups > 0 ? n_groups : 1);
     int best = 1;

@@ -257,7 +257,7 @@ decode_kernel(Params p, kvsink_cache c, kvsink_static_params sp, const __half *_
     static_assert(!KT || (I8 != 0 && NGv <= 2 && (BITS != 3 || NGv == 1)), "per-token keys: integer key side, one or two channel groups");
     // decode: grid (splits, KV heads x blocks of eight query heads, sequences); prompt queries: grid (row blocks, KV heads, sequences)
     const int split = PRE ? 0 : blockIdx.x, h = PRE ? blockIdx.y : blockIdx.y / qchunks, qc = PRE ? blockIdx.x : blockIdx.y % qchunks, b = blockIdx.z;
-    const int nq = I8 == 1 ? 1 : (PRE ? min(NQMAX, pre.T * p.rep - 8 * qc) : min(NQMAX, p.rep - 8 * qc)), hq0 = h * p.rep + (PRE ? 0 : 8 * qc);
+    const int nq = I8 == 1 ? 1 : (PRE ? min(NQMAX, pre.T * p.rep - 8 * qc) : min(NQMAX, p.rep - NQMAX * qc)), hq0 = h * p.rep + (PRE ? 0 : NQMAX * qc);
     // prompt queries: row i of the block is query token (8 qc + i) / rep, query head (8 qc + i) % rep of this KV head
     auto row_token = [&](int i) { return (8 * qc + i) / p.rep; };
     auto row_limit = [&](int i) { return i < nq ? pre.q_pos0 + row_token(i) + 1 : 0; };    // cached tokens the row sees
@@ -1176,7 +1176,8 @@ static int launch_decode_p(const Params &p, const kvsink_cache &c, const kvsink_
     const kvsink_static_params sp = PM == 1 ? *cal : kvsink_static_params{nullptr, nullptr, nullptr, nullptr};
     const int nsplit = choose_splits(p, n_groups);
     const int gps = n_groups > 0 ? (n_groups + nsplit - 1) / nsplit : 0;
-    const int qchunks = (p.rep + 7) / 8;
+    const int qchunks = decode_qchunks(p);      // blocks per KV head; each serves up to NQMAX query heads
+    if (qchunks * (I8 == 1 ? 1 : (PL ? 4 : 8)) < p.rep) return KVSINK_ERR_UNSUPPORTED;
     const size_t smem = DecodePlan<BITS, D, NGV, CT, I8 == 1 ? 1 : (PL ? 4 : 8), PM == 2>::BYTES;
     auto kern = decode_kernel<BITS, D, NGV, CT, PL, I8, PM>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return KVSINK_ERR_CUDA;
@@ -1279,11 +1280,11 @@ static int launch_decode_c(const Params &p, const kvsink_cache &c, const kvsink_
     if constexpr (D == 128)
         if (p.rep == 1) return launch_decode_p<BITS, D, NGV, CT, true, 1, PM>(p, c, cal, q, out, lse, ws, st);
     if constexpr (D == 128 && BITS != 3)
-        if (p.rep <= 4) return launch_decode_p<BITS, D, NGV, CT, true, 2, PM>(p, c, cal, q, out, lse, ws, st);
+        if (decode_heads_per_block(p) == 4) return launch_decode_p<BITS, D, NGV, CT, true, 2, PM>(p, c, cal, q, out, lse, ws, st);
     if constexpr (PM == 2) {
         return KVSINK_ERR_UNSUPPORTED;   // per-token keys run on the integer key side only
     } else {
-        if (p.rep <= 4) return launch_decode_p<BITS, D, NGV, CT, true, 0, PM>(p, c, cal, q, out, lse, ws, st);
+        if (decode_heads_per_block(p) == 4) return launch_decode_p<BITS, D, NGV, CT, true, 0, PM>(p, c, cal, q, out, lse, ws, st);
         return launch_decode_p<BITS, D, NGV, CT, false, 0, PM>(p, c, cal, q, out, lse, ws, st);
     }
 }

@@ -153,10 +153,10 @@ def test_constant_groups_negative_zero_and_extremes():
 
 
 @pytest.mark.parametrize("seed", range(6))
-@pytest.mark.parametrize("hq,hkv", [(2, 2), (8, 2)])
+@pytest.mark.parametrize("hq,hkv", [(2, 2), (8, 2), (16, 2)])
 @pytest.mark.parametrize("bits", [2, 3, 4])
 def test_wide_factor_range(bits, hq, hkv, seed):
-    # head_dim 128, one and four query heads per KV head: channels whose q * scale differ by several orders of magnitude
+    # head_dim 128; one, four and eight query heads per KV head (the three key-side paths): channels whose q * scale differ by several orders of magnitude
     # (one 300 times louder, one 1000 times quieter than the rest), large zero-points (a ramp far from zero, and seeded
     # noise of 0.01 around -40, |zero| ~ 1e4), constant and zero channels
     wl = TINY.scaled(seq=160, group=32, bits=bits, head_dim=128, batch=2, n_q_heads=hq, n_kv_heads=hkv, seed=500 + seed)

@@ -53,8 +53,9 @@ def test_static_scratch_matches_the_workspace_entry_point_twice_in_a_row():
 
 
 def test_static_scratch_refuses_what_does_not_fit():
-    # 64 units x up to 19 splits x 64 query heads x 130 floats > 4 MiB: refused on the host, before any launch
-    cfg = kv.Config(8, 64, 8, 128, 4096, 2, 128, 32768, 4, 1, (1,))
+    # 64 units (4 bit: eight query heads share a block) x up to 19 splits x 64 query heads x 130 floats > 4 MiB: refused on the
+    # host, before any launch
+    cfg = kv.Config(8, 64, 8, 128, 4096, 4, 128, 32768, 4, 1, (1,))
     assert kv.cache_sizes(cfg)["decode_workspace_bytes"] > binding.STATIC_SCRATCH_BYTES
     cache = binding._Cache()
     rc = binding.lib().kvsink_decode_attention_static(C.byref(cfg.c()), C.byref(cache), None, None, None, None)
