@@ -178,10 +178,10 @@ int launch_decode_b4(const Params &p, const kvsink_cache &c, const kvsink_static
                      cudaStream_t st);
 int launch_decode_merge(const float *ws, int nsplit, int D, int n_rows, float *out, float *lse, cudaStream_t st);
 // Query heads of one KV head that one decode block serves, and the blocks per KV head that makes.  Up to four heads share a
-// block; five to eight share one on the eight-column fp16 path, except at 2 and 3 bit with head size 128, where they go four
-// at a time to the integer key side (2 bit) or to the fp16 pair layout (3 bit): the eight-column path has no residual
-// columns, and with few bits and large zero-points its error comes close to, at 2 bit beyond, the attention tolerance.
-inline int decode_heads_per_block(const Params &p) { return p.rep <= 4 ? 4 : (p.D == 128 && p.bits <= 3 ? 4 : 8); }
+// block.  Five to eight share one where a path with eight columns exists: the integer key side with two operand tables (2 and
+// 4 bit, head size 128) or the eight-column fp16 path (head size 64); at 3 bit with head size 128 they go four at a time to
+// the fp16 pair layout, whose residual columns the eight-column fp16 path lacks.
+inline int decode_heads_per_block(const Params &p) { return p.rep <= 4 ? 4 : (p.D == 128 && p.bits == 3 ? 4 : 8); }
 inline int decode_qchunks(const Params &p) { return (p.rep + decode_heads_per_block(p) - 1) / decode_heads_per_block(p); }
 int max_splits(const Params &p);
 int choose_splits(const Params &p, int n_groups);

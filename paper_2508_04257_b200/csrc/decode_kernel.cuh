@@ -214,6 +214,10 @@ struct DecodePlan {
 // MMAs with the same B operands into accumulators of their own.
 // I8 = 2 (two to four query heads per KV head, 2 and 4 bit): the same with two B operands per word, which hold the upper
 // and the lower byte pair of every head's factors in the pair layout's columns.
+// I8 = 3 (five to eight rows: query heads, or the rows of a block of prompt queries; 2 and 4 bit): two operand tables of the
+// I8 = 2 kind, one for the even rows and one for the odd rows, multiplied with the same masked words, so that lane t finds
+// rows 2t and 2t+1 in its accumulators: the two columns it owns on the (eight-column, fp16) value side.  The key sums are
+// exact integers, which the fp16 key side cannot offer when one channel is far louder than the rest.
 //
 // CAL (static, calibrated parameters): one (scale, zero) per key channel and per value channel group of the KV head for every
 // token.  There are no token groups: the key B operand is prepared once per block, a ring chunk holds code words only, the
@@ -253,7 +257,8 @@ decode_kernel(Params p, kvsink_cache c, kvsink_static_params sp, const __half *_
     const int tid = threadIdx.x, lane = tid & 31, warp = __shfl_sync(0xffffffffu, tid >> 5, 0), g = lane >> 2, t = lane & 3;
     constexpr bool CAL = PM == 1, KT = PM == 2, FLAT = PM != 0;    // static parameters / per-token keys / either: no token groups
     constexpr int NGK = KT ? NGv : 1;                              // separate dot products per tile on the key side
-    static_assert(!PRE || (!PL && I8 == 0 && !FLAT), "prompt queries take the eight-column fp16 path");
+    static_assert(!PRE || (!PL && (I8 == 0 || I8 == 3) && !FLAT), "prompt queries take an eight-column path");
+    static_assert(I8 != 3 || (!PL && !KT && D == 128 && BITS != 3), "eight rows on the integer key side: 2 and 4 bit, head size 128");
     static_assert(!KT || (I8 != 0 && NGv <= 2 && (BITS != 3 || NGv == 1)), "per-token keys: integer key side, one or two channel groups");
     // decode: grid (splits, KV heads x blocks of eight query heads, sequences); prompt queries: grid (row blocks, KV heads, sequences)
     const int split = PRE ? 0 : blockIdx.x, h = PRE ? blockIdx.y : blockIdx.y / qchunks, qc = PRE ? blockIdx.x : blockIdx.y % qchunks, b = blockIdx.z;
@@ -641,21 +646,25 @@ decode_kernel(Params p, kvsink_cache c, kvsink_static_params sp, const __half *_
                     bsum = warp_sum(bsum);
                     if (t == 0) { bias0 = bsum; ks0 = pow2i(-sh); }
                 }
-            } else if constexpr (I8 == 2) {
+            } else if constexpr (I8 >= 2) {
                 // up to four heads: the same four signed bytes per factor and head, each head with its own power of two.
                 // The two most significant bytes of every head fill the eight columns of one B operand (head h in columns
                 // 2h, 2h+1), the two less significant ones those of a second: lane t then finds both halves of head t's sum
                 // in its own accumulators.  Table [MMA][lower / upper slots][operand][column][t] in 32-bit words.
+                // I8 = 3 (five to eight rows): two such tables, the first for the even rows and the second for the odd rows, so
+                // that lane t finds rows 2t and 2t+1 -- the two columns it owns on the value side -- in its accumulators.
+                constexpr int NROW = I8 == 3 ? 8 : 4;
                 const bool upper = BITS != 4 && (lane & 4) != 0;
-                uint32_t *tab = reinterpret_cast<uint32_t *>(Bs) + (lane >> 2) * 64 + (lane & 3);
 #pragma unroll
-                for (int hh = 0; hh < 4; ++hh) {
+                for (int row = 0; row < NROW; ++row) {
+                    const int hh = I8 == 3 ? row >> 1 : row, set = I8 == 3 ? row & 1 : 0;
+                    uint32_t *tab = reinterpret_cast<uint32_t *>(Bs) + set * 512 + (lane >> 2) * 64 + (lane & 3);
                     uint32_t w3 = 0u, w2 = 0u, w1 = 0u, w0 = 0u;
-                    if (hh < nq) {
+                    if (row < nq) {
                         float v[4], amax = 0.f, bsum = 0.f;
 #pragma unroll
                         for (int e = 0; e < 4; ++e) {
-                            v[e] = qs[hh * D + i8_ch[e]] * scv[e];
+                            v[e] = qs[row * D + i8_ch[e]] * scv[e];
                             amax = fmaxf(amax, fabsf(v[e]));
                             bsum = fmaf(v[e], zev[e], bsum);
                         }
@@ -675,7 +684,9 @@ decode_kernel(Params p, kvsink_cache c, kvsink_static_params sp, const __half *_
                             if (t == hh) { bias0 = b0s; bias1 = b1s; ks0 = pow2i(-sh); }
                         } else {
                             bsum = warp_sum(bsum);
-                            if (t == hh) { bias0 = bsum; ks0 = pow2i(-sh); }
+                            if (t == hh) {
+                                if (set == 0) { bias0 = bsum; ks0 = pow2i(-sh); } else { bias1 = bsum; ks1 = pow2i(-sh); }
+                            }
                         }
                     }
                     tab[(2 * hh) * 4] = w3;
@@ -749,7 +760,8 @@ decode_kernel(Params p, kvsink_cache c, kvsink_static_params sp, const __half *_
             }
             __syncwarp();
         }
-        if constexpr (I8 == 2) {
+        if constexpr (I8 >= 2) {
+            // (I8 = 3: those of the even rows; the odd rows' are read from the table tile by tile)
             // B fragments of the four words, first operand (bk[0..3]) and second (bk[4..7]): column g, slots 4t .. 4t + 3
 #pragma unroll
             for (int i = 0; i < 4; ++i)
@@ -812,12 +824,13 @@ decode_kernel(Params p, kvsink_cache c, kvsink_static_params sp, const __half *_
             float s[ST][4];
 #pragma unroll
             for (int k = 0; k < ST; ++k) {
-                if constexpr (I8 == 2) {
+                if constexpr (I8 >= 2) {
                     uint32_t kw[W];
                     load_tile_shared<BITS, D>(kt + k * TILE_WORDS, lane, kw);
                     // upper / lower byte pair of the heads' sums; per-token keys: one set per channel group (MMA i covers
                     // channels 32 i ... 32 i + 31)
                     int ia[NGK][4], ib[NGK][4];
+                    int ic[4] = {0, 0, 0, 0}, id[4] = {0, 0, 0, 0};   // I8 = 3: the same for the odd rows
 #pragma unroll
                     for (int j = 0; j < NGK; ++j)
 #pragma unroll
@@ -839,6 +852,16 @@ decode_kernel(Params p, kvsink_cache c, kvsink_static_params sp, const __half *_
                         asm volatile("mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
                                      : "+r"(ib[jg][0]), "+r"(ib[jg][1]), "+r"(ib[jg][2]), "+r"(ib[jg][3])
                                      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(bk[4 + i][0]), "r"(bk[4 + i][1]));
+                        if constexpr (I8 == 3) {   // the odd rows' operands from the second table, the same masked words
+                            const uint32_t *e0 = reinterpret_cast<const uint32_t *>(Bs) + 512 + (i * 2) * 64 + g * 4 + t;
+                            const uint32_t c00 = e0[0], c01 = e0[64], c10 = e0[32], c11 = e0[96];
+                            asm volatile("mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                                         : "+r"(ic[0]), "+r"(ic[1]), "+r"(ic[2]), "+r"(ic[3])
+                                         : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(c00), "r"(c01));
+                            asm volatile("mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                                         : "+r"(id[0]), "+r"(id[1]), "+r"(id[2]), "+r"(id[3])
+                                         : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(c10), "r"(c11));
+                        }
                     }
                     // lane t holds head t: bytes 3, 2 of its sum in the first accumulators, bytes 1, 0 in the second
                     float tg[NGK], th[NGK];
@@ -852,6 +875,12 @@ decode_kernel(Params p, kvsink_cache c, kvsink_static_params sp, const __half *_
                         for (int j = 0; j < NGK; ++j) { tg[j] *= ks0; th[j] *= ks0 * (BITS == 4 ? 0.0625f : 0.25f); }
                         s[k][0] = token_score(tg, k * 16 + g); s[k][1] = -INFINITY;
                         s[k][2] = token_score(th, k * 16 + g + 8); s[k][3] = -INFINITY;
+                    } else if constexpr (I8 == 3) {   // rows 2t (even table) and 2t + 1 (odd table): this lane's two columns
+                        const float ug = fmaf(fmaf((float)ic[0], 256.f, (float)ic[1]), 65536.f, fmaf((float)id[0], 256.f, (float)id[1]));
+                        const float uh = fmaf(fmaf((float)ic[2], 256.f, (float)ic[3]), 65536.f, fmaf((float)id[2], 256.f, (float)id[3]));
+                        s[k][0] = fmaf(tg[0], ks0, -bias0); s[k][1] = fmaf(ug, ks1, -bias1);
+                        s[k][2] = fmaf(th[0], ks0 * (BITS == 4 ? 0.0625f : 0.25f), -bias0);
+                        s[k][3] = fmaf(uh, ks1 * (BITS == 4 ? 0.0625f : 0.25f), -bias1);
                     } else {
                         s[k][0] = fmaf(tg[0], ks0, -bias0); s[k][1] = -INFINITY;
                         s[k][2] = fmaf(th[0], ks0 * (BITS == 4 ? 0.0625f : 0.25f), -bias0); s[k][3] = -INFINITY;
@@ -1219,7 +1248,7 @@ template <int BITS, int D, int NGV, int CT>
 static int launch_prefill_p(const Params &p, const kvsink_cache &c, const __half *q, const PrefillShape &pre, float *out, float *lse, cudaStream_t st)
 {
     const size_t smem = DecodePlan<BITS, D, NGV, CT, 8>::BYTES;
-    auto kern = decode_kernel<BITS, D, NGV, CT, false, 0, 0, true>;
+    auto kern = decode_kernel<BITS, D, NGV, CT, false, (D == 128 && BITS != 3) ? 3 : 0, 0, true>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return KVSINK_ERR_CUDA;
     const long long blocks = ((long long)pre.T * p.rep + 7) / 8;
     if (blocks > 0x7fffffffLL) return KVSINK_ERR_UNSUPPORTED;
@@ -1279,8 +1308,10 @@ static int launch_decode_c(const Params &p, const kvsink_cache &c, const kvsink_
 {
     if constexpr (D == 128)
         if (p.rep == 1) return launch_decode_p<BITS, D, NGV, CT, true, 1, PM>(p, c, cal, q, out, lse, ws, st);
-    if constexpr (D == 128 && BITS != 3)
-        if (decode_heads_per_block(p) == 4) return launch_decode_p<BITS, D, NGV, CT, true, 2, PM>(p, c, cal, q, out, lse, ws, st);
+    if constexpr (D == 128 && BITS != 3) {
+        if (p.rep <= 4) return launch_decode_p<BITS, D, NGV, CT, true, 2, PM>(p, c, cal, q, out, lse, ws, st);
+        if constexpr (PM != 2) return launch_decode_p<BITS, D, NGV, CT, false, 3, PM>(p, c, cal, q, out, lse, ws, st);
+    }
     if constexpr (PM == 2) {
         return KVSINK_ERR_UNSUPPORTED;   // per-token keys run on the integer key side only
     } else {

@@ -65,3 +65,37 @@ def test_queries_beyond_the_cache_are_refused():
     with pytest.raises(kv.KvsinkError) as e:
         kv.prefill_attention(gcfg, gc, q, 18)
     assert e.value.code == -1
+
+
+@pytest.mark.parametrize("seed", range(3))
+@pytest.mark.parametrize("hq,hkv", [(2, 2), (8, 2)])
+@pytest.mark.parametrize("bits", [2, 4])
+def test_keys_with_a_wide_factor_range(bits, hq, hkv, seed):
+    # the decode test's family of keys (a channel 300 times louder and one 1000 times quieter than the rest, ramps and noise far
+    # from zero, constant channels) under N(0,1) queries at every position: 2 and 4 bit take the integer key side, whose sums
+    # are exact whatever the spread of the factors
+    wl = TINY.scaled(seq=160, group=32, bits=bits, head_dim=128, batch=2, n_q_heads=hq, n_kv_heads=hkv, seed=500 + seed)
+    ocfg, gcfg = configs(wl)
+    H = synth.make_hidden(wl, "cuda")
+    K, V = synth.make_kv(wl, 0, "cuda")
+    g = torch.Generator("cuda").manual_seed(seed)
+    K[:, :, :, 3] = 2.5
+    K[:, :, :, 4] = 0.0
+    K[:, :, :, 6] *= 300.0
+    K[:, :, :, 70] *= 1e-3
+    K[:, :, :, 8] = 300.0 + torch.arange(160, device="cuda").half() * 0.25
+    K[:, :, :, 100] = -40.0 + torch.randn(160, device="cuda", generator=g).half() * 0.01
+    gs = kv.SinkSet(gcfg)
+    kv.predict_sinks(gcfg, H, gs)
+    bm, pos, cnt = oracle.predict_sinks(ocfg, np16(H))
+    gc, oc = kv.KVCache(gcfg, gs), oracle.Cache(ocfg, bm, pos, cnt)
+    kv.quantize_append(gcfg, gc, K, V)
+    oracle.quantize_append(ocfg, oc, np16(K), np16(V))
+    gq = torch.Generator("cuda").manual_seed(seed + 100)
+    q = torch.randn((2, hq, 160, 128), device="cuda", generator=gq).half()
+    out, lse = kv.prefill_attention(gcfg, gc, q, 0)
+    ref, ref_lse = oracle.prefill_attention(ocfg, oc, np16(q), 0)
+    torch.cuda.synchronize()
+    assert kv.read_status(gc) == 0
+    assert_close(out.cpu().numpy(), ref, "prompt attention")
+    assert np.abs(lse.cpu().numpy() - ref_lse).max() <= 2e-3 + 1e-3 * np.abs(ref_lse).max()
