@@ -555,6 +555,25 @@ quantize_bulk_kernel(Params p, kvsink_cache c, const __grid_constant__ CUtensorM
                     }
                     mn[s][ab] = lo2; mx[s][ab] = hi2;
                 }
+        } else if (NS == 4 && MODE != 1) {
+            // The other rows of a column live in the lanes that differ in bits 2..4.  Eight (set, side) pairs for the eight
+            // lanes of a column group: each exchange halves what a lane carries (it keeps the half its own bit names and sends
+            // the other), so that lane g ends with the extremes of pair g alone -- both of its keys, one per half
+            uint32_t vn[8], vx[8];
+#pragma unroll
+            for (int c8 = 0; c8 < 8; ++c8) { vn[c8] = mn[(c8 >> 1) % NS][c8 & 1]; vx[c8] = mx[(c8 >> 1) % NS][c8 & 1]; }
+#pragma unroll
+            for (int w = 4; w >= 1; w >>= 1) {
+                const bool up = (lane & (4 * w)) != 0;     // bit 4, 3, 2 of the lane = bit 2, 1, 0 of g
+#pragma unroll
+                for (int i = 0; i < w; ++i) {
+                    const uint32_t sn = up ? vn[i] : vn[w + i], kn = up ? vn[w + i] : vn[i];
+                    const uint32_t sx = up ? vx[i] : vx[w + i], kx = up ? vx[w + i] : vx[i];
+                    vn[i] = qb_hmin2(kn, __shfl_xor_sync(0xffffffffu, sn, 4 * w));
+                    vx[i] = qb_hmax2(kx, __shfl_xor_sync(0xffffffffu, sx, 4 * w));
+                }
+            }
+            mn[0][0] = vn[0]; mx[0][0] = vx[0];
         } else {
         // the other rows of a column live in the lanes that differ in bits 2..4
 #pragma unroll
@@ -572,14 +591,20 @@ quantize_bulk_kernel(Params p, kvsink_cache c, const __grid_constant__ CUtensorM
 #pragma unroll
         for (int j = 0; j < KPL; ++j) {
             // the lane's j-th key.  Per-token keys: lane (g, t) takes the token of tile t >> 1, rows g + 8 (t & 1), channel group j
-            const int kk = g + 8 * j;
+            // With eight (set, side) pairs (NS = 4) the exchange above left lane g with pair g: its keys are the two halves.
+            const bool scat = NS == 4 && MODE != 1 && !kslab;
+            const int kk = scat ? 2 * g + j : g + 8 * j;
             const int s_ = kslab ? (t4 >> 1) * NGv + j : kk >> 2, ab_ = kslab ? (t4 & 1) : (kk >> 1) & 1, e_ = kslab ? 0 : kk & 1;
             uint32_t smn = 0, smx = 0;
+            if (scat) {
+                smn = mn[0][0]; smx = mx[0][0];
+            } else {
 #pragma unroll
-            for (int s = 0; s < NS; ++s)
+                for (int s = 0; s < NS; ++s)
 #pragma unroll
-                for (int ab = 0; ab < 2; ++ab)
-                    if (s_ == s && ab_ == ab) { smn = mn[s][ab]; smx = mx[s][ab]; }
+                    for (int ab = 0; ab < 2; ++ab)
+                        if (s_ == s && ab_ == ab) { smn = mn[s][ab]; smx = mx[s][ab]; }
+            }
             const unsigned short lo16 = (unsigned short)(e_ ? smn >> 16 : smn & 0xffffu), hi16 = (unsigned short)(e_ ? smx >> 16 : smx & 0xffffu);
             const float fmn = __half2float(__ushort_as_half(lo16)), fmx = __half2float(__ushort_as_half(hi16));
             // values: token of the item (set = tile * NGv + channel group); keys: channel of the item (set = matrix)
