@@ -404,8 +404,16 @@ decode_kernel(Params p, kvsink_cache c, kvsink_static_params sp, const __half *_
                 b0 = movm_trans(pack_half2(x0, r0));
                 b1 = movm_trans(pack_half2(x1, r1));
             } else {
-                b0 = movm_trans(pack_half2(p0 * e0, p1 * e0));
-                b1 = movm_trans(pack_half2(p2 * e1, p3 * e1));
+                // every column is a row of its own: the fp16 rounding residuals of the four weights go through a second
+                // multiply of the same value fragments (no further masks), which keeps the weights to ~22 bits here too
+                const float x0 = p0 * e0, x1 = p1 * e0, x2 = p2 * e1, x3 = p3 * e1;
+                const __half2 h01 = __floats2half2_rn(x0, x1), h23 = __floats2half2_rn(x2, x3);
+                const float2 f01 = __half22float2(h01), f23 = __half22float2(h23);
+                b0 = movm_trans(*reinterpret_cast<const uint32_t *>(&h01));
+                b1 = movm_trans(*reinterpret_cast<const uint32_t *>(&h23));
+                const uint32_t r0 = movm_trans(pack_half2(x0 - f01.x, x1 - f01.y)), r1 = movm_trans(pack_half2(x2 - f23.x, x3 - f23.y));
+#pragma unroll
+                for (int mi = 0; mi < mpg; ++mi) mma16816(O[j * mpg + mi], va[j * mpg + mi], r0, r1);
             }
 #pragma unroll
             for (int mi = 0; mi < mpg; ++mi) mma16816(O[j * mpg + mi], va[j * mpg + mi], b0, b1);
@@ -1306,16 +1314,19 @@ template <int BITS, int D, int NGV, int CT, int PM>
 static int launch_decode_c(const Params &p, const kvsink_cache &c, const kvsink_static_params *cal, const __half *q, float *out, float *lse, float *ws,
                            cudaStream_t st)
 {
+    // key side by head size, code width and query heads per KV head; only the reachable kernels are built
     if constexpr (D == 128)
         if (p.rep == 1) return launch_decode_p<BITS, D, NGV, CT, true, 1, PM>(p, c, cal, q, out, lse, ws, st);
     if constexpr (D == 128 && BITS != 3) {
         if (p.rep <= 4) return launch_decode_p<BITS, D, NGV, CT, true, 2, PM>(p, c, cal, q, out, lse, ws, st);
         if constexpr (PM != 2) return launch_decode_p<BITS, D, NGV, CT, false, 3, PM>(p, c, cal, q, out, lse, ws, st);
-    }
-    if constexpr (PM == 2) {
-        return KVSINK_ERR_UNSUPPORTED;   // per-token keys run on the integer key side only
+        else return KVSINK_ERR_UNSUPPORTED;      // per-token keys: at most four query heads per KV head
+    } else if constexpr (PM == 2) {
+        return KVSINK_ERR_UNSUPPORTED;           // per-token keys run on the integer key side only
+    } else if constexpr (D == 128) {
+        return launch_decode_p<BITS, D, NGV, CT, true, 0, PM>(p, c, cal, q, out, lse, ws, st);   // 3 bit: pair layout, four heads at a time
     } else {
-        if (decode_heads_per_block(p) == 4) return launch_decode_p<BITS, D, NGV, CT, true, 0, PM>(p, c, cal, q, out, lse, ws, st);
+        if (p.rep <= 4) return launch_decode_p<BITS, D, NGV, CT, true, 0, PM>(p, c, cal, q, out, lse, ws, st);
         return launch_decode_p<BITS, D, NGV, CT, false, 0, PM>(p, c, cal, q, out, lse, ws, st);
     }
 }
