@@ -69,11 +69,11 @@ def test_queries_beyond_the_cache_are_refused():
 
 @pytest.mark.parametrize("seed", range(3))
 @pytest.mark.parametrize("hq,hkv", [(2, 2), (8, 2)])
-@pytest.mark.parametrize("bits", [2, 4])
+@pytest.mark.parametrize("bits", [2, 3, 4])
 def test_keys_with_a_wide_factor_range(bits, hq, hkv, seed):
     # the decode test's family of keys (a channel 300 times louder and one 1000 times quieter than the rest, ramps and noise far
     # from zero, constant channels) under N(0,1) queries at every position: 2 and 4 bit take the integer key side, whose sums
-    # are exact whatever the spread of the factors
+    # are exact whatever the spread of the factors; 3 bit stays on the fp16 key side (worst case 0.8 of the tolerance here)
     wl = TINY.scaled(seq=160, group=32, bits=bits, head_dim=128, batch=2, n_q_heads=hq, n_kv_heads=hkv, seed=500 + seed)
     ocfg, gcfg = configs(wl)
     H = synth.make_hidden(wl, "cuda")
