@@ -1340,7 +1340,7 @@ static int launch_decode_n(const Params &p, const kvsink_cache &c, const kvsink_
     // several channel groups per row mean G = D / NGV tokens per group: only chunk sizes that divide such a group are built;
     // four groups per row take one tile per chunk (their parameter registers would spill otherwise)
     constexpr int TPG_MAX = NGV == 1 ? 4 : D / NGV / KVSINK_TILE;
-    if constexpr (TPG_MAX % 4 == 0 && 4 * (2 * 128 * (D * BITS / 64) + (PM == 2 ? 4 : 2) * 16 * NGV * 4) <= 4800)
+    if constexpr (TPG_MAX % 4 == 0 && 4 * (2 * 128 * (D * BITS / 64) + (PM == 2 ? 4 : 2) * 16 * NGV * 4) <= (PM == 2 ? 5200 : 4800))
         if ((p.G / KVSINK_TILE) % 4 == 0) return launch_decode_c<BITS, D, NGV, 4, PM>(p, c, cal, q, out, lse, ws, st);
     if constexpr (TPG_MAX % 2 == 0 && NGV < 4)
         if ((p.G / KVSINK_TILE) % 2 == 0) return launch_decode_c<BITS, D, NGV, 2, PM>(p, c, cal, q, out, lse, ws, st);
